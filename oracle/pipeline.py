@@ -1,0 +1,127 @@
+"""Stage-by-stage compositions of the oracle: attention block (Fig. 1(b)) and a
+ViT encoder layer with fp32 LayerNorm / GELU islands between integerized linears.
+
+TEST INFRASTRUCTURE ONLY (see oracle/__init__.py).  Every function returns a
+dict holding all intermediate stages so a checker can compare stage by stage.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+import oracle as vo
+
+
+def softmax_scale(s_q, s_k, head_dim: int) -> np.float32:
+    """c = s_q s_k / sqrt(d), fp64 then one rounding (the scale `s` of Eq. 3)."""
+    return np.float32(float(s_q) * float(s_k) / math.sqrt(head_dim))
+
+
+def inv_step(s) -> np.ndarray:
+    return (1.0 / np.asarray(s, dtype=np.float64)).astype(np.float32)
+
+
+def fold(s_x, s_w, bias, s_out):
+    """Eq. 2 folding: alpha = s_x s_w/s_out, beta = b/s_out (fp64, one rounding each)."""
+    s_w64 = np.asarray(s_w, dtype=np.float64)
+    s_out64 = np.broadcast_to(np.asarray(s_out, dtype=np.float64), s_w64.shape)
+    alpha = (float(s_x) * s_w64 / s_out64).astype(np.float32)
+    beta = np.zeros_like(alpha) if bias is None else (np.asarray(bias, np.float64) / s_out64).astype(np.float32)
+    return alpha, beta
+
+
+def split_heads(codes, batch: int, tokens: int, heads: int, head_dim: int, col0: int):
+    """[batch*tokens, *] code matrix -> [batch*heads, tokens, head_dim] slabs starting at column col0."""
+    out = np.empty((batch * heads, tokens, head_dim), dtype=np.int16)
+    for b in range(batch):
+        for h in range(heads):
+            out[b * heads + h] = codes[b * tokens:(b + 1) * tokens, col0 + h * head_dim: col0 + (h + 1) * head_dim]
+    return out
+
+
+def merge_heads(slabs, batch: int, tokens: int, heads: int, head_dim: int):
+    out = np.empty((batch * tokens, heads * head_dim), dtype=slabs.dtype)
+    for b in range(batch):
+        for h in range(heads):
+            out[b * tokens:(b + 1) * tokens, h * head_dim:(h + 1) * head_dim] = slabs[b * heads + h]
+    return out
+
+
+def attention_block(x_codes, s_x, prm: dict, batch: int, tokens: int, heads: int, bits: int, head_dim: int = 64,
+                    proj: str = "dequant", residual=None, wq: dict | None = None) -> dict:
+    """Integerized self-attention: QKV linear -> Q K^T -> softmax -> quantize -> P V -> proj.
+
+    proj: "dequant" (fp32 output, optional residual) or "requant" (codes at step prm["s_out"]).
+    wq: optional pre-quantized weight codes {"w_qkv", "w_proj"}.
+    """
+    D = heads * head_dim
+    st: dict = {}
+    wq = wq or {}
+    w_qkv = wq.get("w_qkv")
+    if w_qkv is None:
+        w_qkv = vo.quantize(prm["w_qkv"], 0.0, bits, True, row_steps=prm["s_w_qkv"])
+    w_proj = wq.get("w_proj")
+    if w_proj is None:
+        w_proj = vo.quantize(prm["w_proj"], 0.0, bits, True, row_steps=prm["s_w_proj"])
+    st["w_qkv_codes"], st["w_proj_codes"] = w_qkv, w_proj
+
+    # QKV linear, requantized to three per-tensor steps (one per segment of the output channels)
+    s_seg = np.concatenate([np.full(D, prm["s_q"]), np.full(D, prm["s_k"]), np.full(D, prm["s_v"])]).astype(np.float32)
+    a_qkv, b_qkv = fold(s_x, prm["s_w_qkv"], prm["b_qkv"], s_seg)
+    st["alpha_qkv"], st["beta_qkv"] = a_qkv, b_qkv
+    st["acc_qkv"] = vo.matmul_i32(x_codes, w_qkv)
+    st["qkv_codes"] = vo.epilogue_requant(st["acc_qkv"], a_qkv, b_qkv, bits, True)
+
+    q = split_heads(st["qkv_codes"], batch, tokens, heads, head_dim, 0)
+    k = split_heads(st["qkv_codes"], batch, tokens, heads, head_dim, D)
+    v = split_heads(st["qkv_codes"], batch, tokens, heads, head_dim, 2 * D)
+    st["S"] = vo.qk(q, k)
+    c = softmax_scale(prm["s_q"], prm["s_k"], head_dim)
+    st["c"] = c
+    n = batch * heads
+    p, pc, plo, phi = vo.softmax_quantize(st["S"].reshape(n * tokens, tokens), c, prm["s_p"], bits)
+    st["p"], st["p_codes"] = p.reshape(n, tokens, tokens), pc.reshape(n, tokens, tokens)
+    st["p_lo"], st["p_hi"] = plo.reshape(n, tokens, tokens), phi.reshape(n, tokens, tokens)
+
+    st["acc_o"] = vo.pv(st["p_codes"], v)
+    a_o, b_o = fold(prm["s_p"], np.full(head_dim, prm["s_v"], np.float32), None, prm["s_o"])
+    st["alpha_o"] = a_o
+    o_slabs = vo.epilogue_requant(st["acc_o"].reshape(n * tokens, head_dim), a_o, b_o, bits, True)
+    st["o_codes"] = merge_heads(o_slabs.reshape(n, tokens, head_dim), batch, tokens, heads, head_dim)
+
+    st["acc_proj"] = vo.matmul_i32(st["o_codes"], w_proj)
+    if proj == "dequant":
+        st["out"] = vo.epilogue_dequant(st["acc_proj"], prm["s_o"], prm["s_w_proj"], prm["b_proj"], residual)
+    else:
+        a_p, b_p = fold(prm["s_o"], prm["s_w_proj"], prm["b_proj"], prm["s_out"])
+        st["alpha_proj"], st["beta_proj"] = a_p, b_p
+        st["out_codes"] = vo.epilogue_requant(st["acc_proj"], a_p, b_p, bits, True)
+    return st
+
+
+def encoder_layer(x, prm: dict, batch: int, tokens: int, heads: int, bits: int, head_dim: int = 64,
+                  eps: float = 1e-6) -> dict:
+    """LN1 -> quantize -> attention (+residual) -> LN2 -> quantize -> fc1 -> GELU -> quantize -> fc2 (+residual)."""
+    st: dict = {}
+    y1, tol1 = vo.layernorm(x, prm["ln1_g"], prm["ln1_b"], eps)
+    st["ln1"], st["ln1_tol"] = y1, tol1
+    st["x1_codes"], st["x1_lo"], st["x1_hi"] = vo.quantize_band(y1, tol1, prm["s_ln"], bits, True)
+    att = attention_block(st["x1_codes"], prm["s_ln"], prm, batch, tokens, heads, bits, head_dim, "dequant", x)
+    st["attn"] = att
+    h = att["out"]
+    st["h"] = h
+    y2, tol2 = vo.layernorm(h, prm["ln2_g"], prm["ln2_b"], eps)
+    st["ln2"], st["ln2_tol"] = y2, tol2
+    st["x2_codes"], st["x2_lo"], st["x2_hi"] = vo.quantize_band(y2, tol2, prm["s_ln"], bits, True)
+    w_fc1 = vo.quantize(prm["w_fc1"], 0.0, bits, True, row_steps=prm["s_w_fc1"])
+    w_fc2 = vo.quantize(prm["w_fc2"], 0.0, bits, True, row_steps=prm["s_w_fc2"])
+    st["w_fc1_codes"], st["w_fc2_codes"] = w_fc1, w_fc2
+    st["acc_fc1"] = vo.matmul_i32(st["x2_codes"], w_fc1)
+    inv_g = inv_step(np.full(w_fc1.shape[0], prm["s_g"], np.float32))
+    st["inv_s_g"] = inv_g
+    st["g_codes"], st["g_lo"], st["g_hi"] = vo.epilogue_gelu_requant(st["acc_fc1"], prm["s_ln"], prm["s_w_fc1"],
+                                                                     prm["b_fc1"], inv_g, bits, False)
+    st["acc_fc2"] = vo.matmul_i32(st["g_codes"], w_fc2)
+    st["out"] = vo.epilogue_dequant(st["acc_fc2"], prm["s_g"], prm["s_w_fc2"], prm["b_fc2"], h)
+    return st

@@ -1,0 +1,472 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (CPU only).
+
+Each test compares an oracle function with something that is not the oracle:
+values the paper prints, exact rational arithmetic, brute force in Python
+integers, closed forms, or a library routine for a special case.
+"""
+import itertools
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle as vo
+import synth_inputs as si
+from oracle import pipeline as vp
+
+
+# ---------------------------------------------------------------------------
+# helpers that do not use the oracle
+# ---------------------------------------------------------------------------
+
+def f32_from_fraction(fr: Fraction) -> np.float32:
+    """Exact round-to-nearest-even of a rational to fp32 (normal range only)."""
+    if fr == 0:
+        return np.float32(0.0)
+    sign = -1 if fr < 0 else 1
+    fr = abs(fr)
+    e = math.floor(math.log2(fr))
+    while Fraction(2) ** e > fr:
+        e -= 1
+    while Fraction(2) ** (e + 1) <= fr:
+        e += 1
+    scaled = fr / Fraction(2) ** (e - 23)          # in [2^23, 2^24)
+    n = scaled.numerator // scaled.denominator
+    rem = scaled - n
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and n % 2 == 1):
+        n += 1
+    return np.float32(sign * float(n) * 2.0 ** (e - 23))
+
+
+def comparator_code(x: float, step: float, bits: int, signed: bool) -> int:
+    """Code = lowest level + number of thresholds (k-1/2)*step strictly exceeded (Section IV-B)."""
+    qn, qp = si.code_range(bits, signed)
+    return qn + sum(1 for k in range(qn + 1, qp + 1) if Fraction(x) > (Fraction(k) - Fraction(1, 2)) * Fraction(step))
+
+
+# ---------------------------------------------------------------------------
+# quantizer
+# ---------------------------------------------------------------------------
+
+def test_three_bit_ladder_from_paper(golden_dir):
+    rows = [l.split() for l in (golden_dir / "ladder_3bit.txt").read_text().splitlines() if l and l[0] != "#"]
+    assert len(rows) == 7
+    for step in (0.25, 1.0, 0.0078125):
+        for b, below, above in rows:
+            thr = float(b) * step
+            eps = step / 64.0
+            x = np.array([[thr - eps, thr + eps]], dtype=np.float32)
+            q = vo.quantize(x, step, 3, True)
+            assert q.tolist() == [[int(below), int(above)]]
+    # outside the ladder: clamp to the end levels
+    q = vo.quantize(np.array([[-100.0, 100.0]], np.float32), 0.25, 3, True)
+    assert q.tolist() == [[-4, 3]]
+
+
+@pytest.mark.parametrize("bits,signed", [(2, True), (3, True), (4, True), (8, True), (2, False), (4, False), (8, False)])
+def test_quantizer_equals_comparator_count_off_ties(bits, signed):
+    step = 0.125
+    x = si.normal(11 + bits, (1, 4096), 0.0, step * (1 << bits) / 3.0)
+    q = vo.quantize(x, step, bits, signed)[0]
+    for xi, qi in zip(x[0, :600], q[:600]):
+        assert comparator_code(float(xi), step, bits, signed) == int(qi)
+
+
+@pytest.mark.parametrize("bits,signed", [(2, True), (3, True), (4, True), (8, True), (4, False), (8, False)])
+def test_quantizer_ties_to_even_and_idempotent(bits, signed):
+    qn, qp = si.code_range(bits, signed)
+    step = 0.5
+    ks = np.arange(qn, qp + 1)
+    # exact representable points: codes reproduce themselves
+    x = (ks * step).astype(np.float32)[None, :]
+    assert vo.quantize(x, step, bits, signed)[0].tolist() == ks.tolist()
+    # exact ties (k + 1/2)*step go to the even neighbour (then clamp)
+    ties = ((ks[:-1] + 0.5) * step).astype(np.float32)[None, :]
+    want = [int(k if k % 2 == 0 else k + 1) for k in ks[:-1]]
+    assert vo.quantize(ties, step, bits, signed)[0].tolist() == want
+
+
+def test_quantizer_per_row_steps_and_true_division():
+    # 0.3 is not a power of two: x/s and x*(1/s) differ for some x; the oracle must divide.
+    s = np.float32(0.3)
+    inv = np.float32(1.0) / s
+    xs = np.arange(1, 200001, dtype=np.float32) * np.float32(0.05)
+    div = np.rint(xs / s)
+    mul = np.rint(xs * inv)
+    differ = np.nonzero(div != mul)[0]
+    assert differ.size > 0
+    x = xs[differ[:64]][None, :]
+    q = vo.quantize(x, s, 8, False)
+    assert q[0].tolist() == np.clip(div[differ[:64]], 0, 255).astype(int).tolist()
+    # per-row steps: row m uses steps[m]
+    xr = np.array([[1.0, 2.0, 3.0], [1.0, 2.0, 3.0]], np.float32)
+    q = vo.quantize(xr, 0.0, 4, True, row_steps=np.array([1.0, 0.5], np.float32))
+    assert q.tolist() == [[1, 2, 3], [2, 4, 6]]
+
+
+# ---------------------------------------------------------------------------
+# packed format
+# ---------------------------------------------------------------------------
+
+def test_pack_hand_computed_bytes():
+    # 4-bit: element 0 in the low nibble; -1 -> 0xF, -8 -> 0x8
+    assert vo.pack(np.array([[1, -1, -8, 7]], np.int16), 4)[0, :2].tolist() == [0xF1, 0x78]
+    # 3-bit codes live in 4-bit containers, sign-extended
+    assert vo.pack(np.array([[-4, 3]], np.int16), 3)[0, :1].tolist() == [0x3C]
+    # 2-bit: four per byte, element i at bit 2*i;  [1,-1,-2,0] -> 01 | 11<<2 | 10<<4 | 00<<6 = 0x2D
+    assert vo.pack(np.array([[1, -1, -2, 0]], np.int16), 2)[0, :1].tolist() == [0x2D]
+    # 8-bit: plain bytes
+    assert vo.pack(np.array([[-128, 127, 255 - 256]], np.int16), 8)[0, :3].tolist() == [0x80, 0x7F, 0xFF]
+    # pitch is a multiple of 16 and the tail is zero
+    pk = vo.pack(np.full((1, 5), -1, np.int16), 4)
+    assert pk.shape == (1, 16) and pk[0, 3:].tolist() == [0] * 13 and pk[0, 2] == 0x0F
+
+
+@pytest.mark.parametrize("bits,signed", [(2, True), (2, False), (3, True), (3, False), (4, True), (4, False), (8, True), (8, False)])
+def test_pack_roundtrip_all_values_all_residues(bits, signed):
+    qn, qp = si.code_range(bits, signed)
+    vals = np.arange(qn, qp + 1)
+    for cols in range(1, 34):
+        q = np.array([[vals[(i * 7 + r) % len(vals)] for i in range(cols)] for r in range(len(vals))], np.int16)
+        pk = vo.pack(q, bits)
+        assert pk.shape[1] % 16 == 0
+        assert np.array_equal(vo.unpack(pk, cols, bits, signed), q)
+
+
+# ---------------------------------------------------------------------------
+# integer contraction (Eq. 1)
+# ---------------------------------------------------------------------------
+
+def test_contraction_brute_force_every_two_bit_code():
+    vals = [-2, -1, 0, 1]
+    # every pair of 2-element rows over all 2-bit codes: 16 x 16 dot products, checked with Python ints
+    rows = np.array(list(itertools.product(vals, repeat=2)), np.int16)
+    acc = vo.matmul_i32(rows, rows)
+    for i, a in enumerate(rows):
+        for j, b in enumerate(rows):
+            assert int(acc[i, j]) == int(a[0]) * int(b[0]) + int(a[1]) * int(b[1])
+
+
+def test_contraction_rectangular_against_python_ints():
+    # M, N, K all different: a transposed operand or swapped index cannot pass
+    a = (si.splitmix64(5, 3 * 7) % np.uint64(16)).astype(np.int64).reshape(3, 7) - 8
+    b = (si.splitmix64(6, 5 * 7) % np.uint64(16)).astype(np.int64).reshape(5, 7) - 8
+    acc = vo.matmul_i32(a, b)
+    assert acc.shape == (3, 5)
+    for m in range(3):
+        for n in range(5):
+            assert int(acc[m, n]) == sum(int(a[m, k]) * int(b[n, k]) for k in range(7))
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+def test_contraction_closed_forms(bits):
+    qn, qp = si.code_range(bits, True)
+    K = 193
+    a = np.full((2, K), qp, np.int16)
+    a[1] = qn
+    b = np.full((3, K), qn, np.int16)
+    b[1] = qp
+    b[2] = 0
+    b[2, 17] = 1                      # one-hot picks a[:, 17]
+    acc = vo.matmul_i32(a, b)
+    assert acc.tolist() == [[K * qp * qn, K * qp * qp, qp], [K * qn * qn, K * qn * qp, qn]]
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+def test_reordering_identity_against_fp64_dequantized_matmul(bits):
+    """(s_x q_x)(s_w q_w)^T + b  ==  [q_x q_w^T] s_x diag(s_w) + b  (Eq. 1, Eq. 2)."""
+    M, N, K = 13, 11, 96
+    x = si.normal(21, (M, K))
+    w = si.normal(22, (N, K), 0.0, 0.02)
+    bias = si.normal(23, (N,), 0.0, 0.01)
+    s_x = si.lsq_step(x, bits, True)
+    s_w = si.lsq_step_rows(w, bits)
+    qx = vo.quantize(x, s_x, bits, True)
+    qw = vo.quantize(w, 0.0, bits, True, row_steps=s_w)
+    y = vo.epilogue_dequant(vo.matmul_i32(qx, qw), s_x, s_w, bias)
+    xd = qx.astype(np.float64) * float(s_x)
+    wd = qw.astype(np.float64) * s_w.astype(np.float64)[:, None]
+    ref = xd @ wd.T + bias.astype(np.float64)
+    mag = np.abs(xd) @ np.abs(wd).T + np.abs(bias.astype(np.float64))
+    assert np.all(np.abs(y.astype(np.float64) - ref) <= 2.0 ** -22 * mag)
+    assert np.abs(ref).max() > 0.05      # the comparison is not vacuous
+
+
+def test_overflow_bound_and_int64_edge():
+    # the declared-range bound
+    assert vo.overflow_bound(4096, 4, True, 4, True) == 4096 * 8 * 8
+    assert vo.overflow_bound(768, 4, False, 4, True) == 768 * 15 * 8
+    assert vo.overflow_bound(100, 8, False, 8, True) == 100 * 255 * 128
+    # 8-bit at the edge: K*128*128 reaches 2^31 at K = 131072; one less still fits
+    K = 131072
+    assert vo.overflow_bound(K, 8, True, 8, True) == 2 ** 31
+    a = np.full((1, K), -128, np.int16)
+    acc64 = vo.matmul_i64(a, a)
+    assert int(acc64[0, 0]) == 2 ** 31                  # needs more than int32
+    assert vo.overflow_bound(K - 1, 8, True, 8, True) < 2 ** 31
+    acc32 = vo.matmul_i32(a[:, :K - 1], a[:, :K - 1])
+    assert int(acc32[0, 0]) == (K - 1) * 16384 == int(vo.matmul_i64(a[:, :K - 1], a[:, :K - 1])[0, 0])
+
+
+# ---------------------------------------------------------------------------
+# epilogues (Eq. 2)
+# ---------------------------------------------------------------------------
+
+def test_dequant_epilogue_is_one_fused_multiply_add_exact_rational():
+    acc = np.array([[3, -7, 12345, 16777215, -491520]], np.int32)
+    s_x = np.float32(0.3)
+    s_w = np.array([0.01, 0.7, 1.1e-3, 3.3e-5, 0.123], np.float32)
+    bias = np.array([-0.009, 4.9, -13.58, 1e-4, 60457.0], np.float32)
+    y = vo.epilogue_dequant(acc, s_x, s_w, bias)
+    for n in range(5):
+        sc = f32_from_fraction(Fraction(float(s_x)) * Fraction(float(s_w[n])))
+        want = f32_from_fraction(Fraction(int(acc[0, n])) * Fraction(float(sc)) + Fraction(float(bias[n])))
+        assert y[0, n] == want
+    # a case where multiply-then-add rounds differently from the fused form must follow the fused form
+    found = False
+    for a in range(1, 4000):
+        sc = np.float32(0.1)
+        b = -np.float32(np.float32(a) * sc)
+        fused = f32_from_fraction(Fraction(a) * Fraction(float(sc)) + Fraction(float(b)))
+        if fused != np.float32(np.float32(a) * sc + b):
+            out = vo.epilogue_dequant(np.array([[a]], np.int32), np.float32(1.0), np.array([sc], np.float32),
+                                      np.array([b], np.float32))
+            assert out[0, 0] == fused
+            found = True
+            break
+    assert found
+
+
+def test_dequant_residual_is_a_second_rounded_add():
+    acc = np.array([[5, -3]], np.int32)
+    s_w = np.array([0.1, 0.2], np.float32)
+    bias = np.array([0.3, 0.4], np.float32)
+    res = np.array([[1e-3, 7.0]], np.float32)
+    y = vo.epilogue_dequant(acc, np.float32(0.7), s_w, bias, res)
+    for n in range(2):
+        sc = f32_from_fraction(Fraction(float(np.float32(0.7))) * Fraction(float(s_w[n])))
+        v = f32_from_fraction(Fraction(int(acc[0, n])) * Fraction(float(sc)) + Fraction(float(bias[n])))
+        assert y[0, n] == f32_from_fraction(Fraction(float(v)) + Fraction(float(res[0, n])))
+
+
+def test_requant_epilogue_exact_cases_and_clamp():
+    # alpha, beta powers of two: fmaf is exact, result known by hand
+    acc = np.array([[8, 9, 10, 11, 12, -100, 100, 0]], np.int32)
+    alpha = np.full(8, 0.25, np.float32)
+    beta = np.full(8, 0.25, np.float32)
+    # values 2.25 2.5 2.75 3.0 3.25 -24.75 25.25 0.25 -> rint (ties even) 2 2 3 3 3 -25 25 0 -> clamp [-8,7]
+    assert vo.epilogue_requant(acc, alpha, beta, 4, True)[0].tolist() == [2, 2, 3, 3, 3, -8, 7, 0]
+    assert vo.epilogue_requant(acc, alpha, beta, 4, False)[0].tolist() == [2, 2, 3, 3, 3, 0, 15, 0]
+
+
+def test_folded_requant_equals_quantized_dequant_off_ties():
+    """Eq. 2: [acc + b/(s_x s_w)] s_x s_w / s_out  vs quantizing the dequantized output."""
+    M, N, K = 64, 48, 192
+    qx = vo.quantize(si.normal(31, (M, K)), 0.6, 4, True)
+    w = si.normal(32, (N, K), 0.0, 0.02)
+    s_w = si.lsq_step_rows(w, 4)
+    qw = vo.quantize(w, 0.0, 4, True, row_steps=s_w)
+    bias = si.normal(33, (N,), 0.0, 0.01)
+    acc = vo.matmul_i32(qx, qw)
+    s_out = np.float32(0.1)
+    alpha, beta = vp.fold(np.float32(0.6), s_w, bias, s_out)
+    folded = vo.epilogue_requant(acc, alpha, beta, 4, True)
+    exact = acc.astype(np.float64) * 0.6000000238418579 * s_w.astype(np.float64) + bias.astype(np.float64)
+    u = exact / float(s_out)
+    want = np.clip(np.rint(u), -8, 7)
+    near_tie = np.abs(u - np.floor(u) - 0.5) < 1e-5
+    assert np.array_equal(folded[~near_tie], want[~near_tie].astype(np.int16))
+    assert np.all(np.abs(folded - want) <= 1)
+    assert (~near_tie).mean() > 0.999
+    assert len(np.unique(folded)) >= 12
+
+
+def test_gelu_against_erf_definition_and_identities():
+    y = np.linspace(-6, 6, 2401).astype(np.float32)
+    acc = np.arange(2401, dtype=np.int32)[None, :]
+    # use acc*0 + bias = y so that the activation input is exactly y
+    g = vo.epilogue_dequant(acc * 0, np.float32(1.0), np.ones(2401, np.float32), y, None, act=1)[0]
+    ref = np.array([0.5 * float(v) * (1.0 + math.erf(float(v) / math.sqrt(2.0))) for v in y])
+    assert np.all(np.abs(g.astype(np.float64) - ref) <= np.abs(ref) * 2.0 ** -23 + 1e-45)
+    assert g[1200] == 0.0 and y[1200] == 0.0
+    assert g[-1] == y[-1]                                   # Phi(6) rounds to 1 in fp32
+    sym = g.astype(np.float64) - g[::-1].astype(np.float64)  # GELU(y) - GELU(-y) = y
+    assert np.all(np.abs(sym - y.astype(np.float64)) <= 2.0 ** -22 * np.abs(y) + 1e-30)
+
+
+def test_gelu_requant_band_brackets_code():
+    M, N = 8, 512
+    acc = (si.splitmix64(41, M * N) % np.uint64(4001)).astype(np.int64).reshape(M, N) - 2000
+    s_w = np.full(N, 1e-3, np.float32)
+    bias = si.normal(42, (N,), 0.0, 0.01)
+    inv_s = np.full(N, np.float32(1.0 / 0.05), np.float32)
+    q, lo, hi = vo.epilogue_gelu_requant(acc.astype(np.int32), np.float32(0.6), s_w, bias, inv_s, 4, False)
+    assert np.all(lo <= q) and np.all(q <= hi) and np.all(hi - lo <= 1)
+    assert (hi != lo).mean() < 1e-3
+    # independent evaluation of the code in fp64 agrees wherever the band is a single code
+    yy = acc.astype(np.float64) * float(np.float32(np.float64(np.float32(0.6)) * np.float64(np.float32(1e-3)))) + bias.astype(np.float64)
+    gg = 0.5 * yy * (1.0 + np.vectorize(math.erf)(yy / math.sqrt(2.0)))
+    want = np.clip(np.rint(gg * float(inv_s[0])), 0, 15)
+    u = gg * float(inv_s[0])
+    safe = (np.abs(u - np.floor(u) - 0.5) > 1e-4)
+    assert np.array_equal(q[safe], want[safe].astype(np.int16))
+    assert q.max() == 15 and q.min() == 0
+
+
+# ---------------------------------------------------------------------------
+# softmax (Eq. 3)
+# ---------------------------------------------------------------------------
+
+def test_softmax_rows_sum_to_one_and_closed_forms():
+    T = 197
+    S = (si.splitmix64(51, 8 * T) % np.uint64(1201)).astype(np.int64).reshape(8, T) - 600
+    S[1] = 37                                   # all-equal row -> 1/T
+    p, q, lo, hi = vo.softmax_quantize(S, np.float32(0.01), np.float32(0.0026), 4)
+    assert np.all(np.abs(p.astype(np.float64).sum(1) - 1.0) <= T * 2.0 ** -24)
+    assert np.all(p[1] == np.float32(1.0 / T))
+    assert np.all(p >= 0)
+    # two-element row: logistic closed form
+    for d in (0, 1, 5, -40, 300):
+        p2, *_ = vo.softmax_quantize(np.array([[d, 0]], np.int32), np.float32(0.125), np.float32(0.07), 4)
+        t = float(np.float32(d) * np.float32(0.125))
+        want = 1.0 / (1.0 + math.exp(-t))
+        assert abs(float(p2[0, 0]) - want) <= 2.0 ** -24 * want
+        other = 1.0 / (1.0 + math.exp(t))
+        assert abs(float(p2[0, 1]) - other) <= 2.0 ** -24 * other
+    # against a straightforward numpy fp64 softmax
+    t = (S.astype(np.float32) * np.float32(0.01)).astype(np.float64)
+    e = np.exp(t - t.max(1, keepdims=True))
+    ref = e / e.sum(1, keepdims=True)
+    assert np.all(np.abs(p.astype(np.float64) - ref) <= 2.0 ** -24 * ref + 1e-45)
+
+
+def test_softmax_shift_invariance_with_power_of_two_scale():
+    T = 64
+    S = (si.splitmix64(52, 4 * T) % np.uint64(257)).astype(np.int64).reshape(4, T) - 128
+    c = np.float32(2.0 ** -5)                     # exact products: adding k to S adds k*c to t exactly
+    p0, q0, *_ = vo.softmax_quantize(S, c, np.float32(0.004), 4)
+    p1, q1, *_ = vo.softmax_quantize(S + 1000, c, np.float32(0.004), 4)
+    assert np.array_equal(p0, p1) and np.array_equal(q0, q1)
+
+
+def test_softmax_codes_decided_in_fp32_and_band():
+    T = 197
+    S = (si.splitmix64(53, 32 * T) % np.uint64(801)).astype(np.int64).reshape(32, T) - 400
+    s_p = np.float32(2.0 / (T * math.sqrt(15.0)))
+    p, q, lo, hi = vo.softmax_quantize(S, np.float32(0.02), s_p, 4)
+    want = np.clip(np.rint(p / s_p), 0, 15).astype(np.int16)      # numpy fp32 division, ties-to-even
+    assert np.array_equal(q, want)
+    assert np.all(lo <= q) and np.all(q <= hi) and np.all(hi - lo <= 1)
+    assert (hi != lo).mean() < 1e-3
+    assert q.max() == 15 and (q == 0).any()
+    # unsigned range (probabilities are never negative): 2-bit gives 0..3
+    _, q2, *_ = vo.softmax_quantize(S, np.float32(0.02), s_p, 2)
+    assert q2.min() == 0 and q2.max() == 3
+
+
+def test_qk_and_pv_orientation():
+    n, T, d = 2, 5, 3
+    Q = (si.splitmix64(61, n * T * d) % np.uint64(16)).astype(np.int64).reshape(n, T, d) - 8
+    K = (si.splitmix64(62, n * T * d) % np.uint64(16)).astype(np.int64).reshape(n, T, d) - 8
+    V = (si.splitmix64(63, n * T * d) % np.uint64(16)).astype(np.int64).reshape(n, T, d) - 8
+    P = (si.splitmix64(64, n * T * T) % np.uint64(16)).astype(np.int64).reshape(n, T, T)
+    S = vo.qk(Q, K)
+    O = vo.pv(P, V)
+    for p_ in range(n):
+        assert np.array_equal(S[p_], Q[p_] @ K[p_].T)      # numpy int64 matmul
+        assert np.array_equal(O[p_], P[p_] @ V[p_])
+
+
+# ---------------------------------------------------------------------------
+# LayerNorm glue and Eq. 5
+# ---------------------------------------------------------------------------
+
+def test_layernorm_against_running_statistics_of_eq5_and_numpy():
+    x = si.normal(71, (6, 768), 0.3, 2.0)
+    g = si.normal(72, (768,), 1.0, 0.02)
+    b = si.normal(73, (768,), 0.0, 0.02)
+    y, tol = vo.layernorm(x, g, b, 1e-6)
+    for m in range(6):
+        mu, m2 = vo.running_stats(x[m])
+        xd = x[m].astype(np.float64)
+        assert abs(mu - xd.mean()) < 1e-12 and abs(m2 / 768 - xd.var()) < 1e-10
+        ref = (xd - mu) / math.sqrt(m2 / 768 + 1e-6) * g + b
+        assert np.all(np.abs(y[m] - ref) <= 2.0 ** -23 * np.abs(ref) + 1e-12)
+    ones = np.ones(768, np.float32)
+    y0, _ = vo.layernorm(x, ones, 0 * ones, 0.0)
+    assert np.all(np.abs(y0.mean(1)) < 1e-6) and np.all(np.abs(y0.astype(np.float64).var(1) - 1.0) < 1e-5)
+    assert np.all(tol > 0) and tol.max() < 1e-4
+
+
+def test_running_stats_small_case_by_hand():
+    # x = 1, 2, 4: mu = 7/3, M2 = sum (x-mu)^2 = 42/9
+    mu, m2 = vo.running_stats(np.array([1.0, 2.0, 4.0], np.float32))
+    assert abs(mu - 7.0 / 3.0) < 1e-15 and abs(m2 - 42.0 / 9.0) < 1e-14
+
+
+# ---------------------------------------------------------------------------
+# op counts (Table I) and the composed block
+# ---------------------------------------------------------------------------
+
+def test_table1_counts(golden_dir):
+    rows = {l.split()[0]: l.split()[1:] for l in (golden_dir / "table1_counts.txt").read_text().splitlines()
+            if l and l[0] != "#"}
+    c = si.head_mac_counts(198, 384, 64)
+    assert c["linear_pe"] == int(rows["linear"][0]) and round(c["linear_mac"] / 1e6, 2) == float(rows["linear"][1])
+    assert c["layernorm_pe"] == int(rows["layernorm"][0])
+    assert round(c["layernorm_mac"] / 1e6, 2) == float(rows["layernorm"][1])
+    assert c["delay"] == int(rows["delay"][0])
+    assert c["matmul_qk_pe"] == int(rows["matmul_qk"][0])
+    assert round(c["matmul_qk_mac"] / 1e6, 2) == float(rows["matmul_qk"][1])
+    assert c["matmul_pv_pe"] == int(rows["matmul_pv"][0])
+    assert round(c["matmul_pv_mac"] / 1e6, 2) == float(rows["matmul_pv"][1])
+    m = si.mac_counts(197, 768, 12, 64, 3072)
+    assert abs(m["total"] / 1e6 - 1453.95) < 0.01
+
+
+@pytest.mark.parametrize("w_std", [0.02, 0.12])
+def test_attention_block_matches_dequantize_first_datapath(w_std):
+    """Fig. 1: the integerized datapath (b) equals the dequantize-first datapath (a) given the same codes."""
+    cfg = si.VIT_TINY_BLOCK.with_(w_std=w_std)
+    prm = si.layer_parameters(cfg)
+    x = si.activations(cfg)
+    s_x = si.lsq_step(x, cfg.bits, True)
+    xq = vo.quantize(x, s_x, cfg.bits, True)
+    st = vp.attention_block(xq, s_x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits)
+    D, T, H = cfg.dim, cfg.tokens, cfg.heads
+    # (a): dequantize codes, float matmuls
+    xd = xq.astype(np.float64) * float(s_x)
+    wd = st["w_qkv_codes"].astype(np.float64) * prm["s_w_qkv"].astype(np.float64)[:, None]
+    qkv = xd @ wd.T + prm["b_qkv"].astype(np.float64)
+    seg = np.concatenate([np.full(D, prm["s_q"]), np.full(D, prm["s_k"]), np.full(D, prm["s_v"])]).astype(np.float64)
+    u = qkv / seg
+    codes = np.clip(np.rint(u), -8, 7)
+    safe = np.abs(u - np.floor(u) - 0.5) > 1e-4
+    assert np.array_equal(st["qkv_codes"][safe], codes[safe].astype(np.int16))
+    assert st["qkv_codes"].shape == (T, 3 * D)
+    # attention for head 1 from the oracle's own codes, in floats
+    h = 1
+    qd = st["qkv_codes"][:, h * 64:(h + 1) * 64].astype(np.float64) * float(prm["s_q"])
+    kd = st["qkv_codes"][:, D + h * 64: D + (h + 1) * 64].astype(np.float64) * float(prm["s_k"])
+    vd = st["qkv_codes"][:, 2 * D + h * 64: 2 * D + (h + 1) * 64].astype(np.float64) * float(prm["s_v"])
+    logits = qd @ kd.T / 8.0
+    e = np.exp(logits - logits.max(1, keepdims=True))
+    pr = e / e.sum(1, keepdims=True)
+    assert np.all(np.abs(st["p"][h] - pr) <= 4e-6 * pr + 1e-12)
+    pd = st["p_codes"][h].astype(np.float64) * float(prm["s_p"])
+    od = pd @ vd
+    uo = od / float(prm["s_o"])
+    want_o = np.clip(np.rint(uo), -8, 7)
+    safe_o = np.abs(uo - np.floor(uo) - 0.5) > 1e-4
+    got_o = st["o_codes"][:, h * 64:(h + 1) * 64]
+    assert np.array_equal(got_o[safe_o], want_o[safe_o].astype(np.int16))
+    assert len(np.unique(got_o)) >= 6
+    if w_std > 0.1:                      # peaked attention rows: the whole unsigned range is used
+        assert len(np.unique(st["p_codes"])) == 16
+    # projection output: dequantized float path
+    o_all = st["o_codes"].astype(np.float64) * float(prm["s_o"])
+    wp = st["w_proj_codes"].astype(np.float64) * prm["s_w_proj"].astype(np.float64)[:, None]
+    ref = o_all @ wp.T + prm["b_proj"].astype(np.float64)
+    mag = np.abs(o_all) @ np.abs(wp).T + np.abs(prm["b_proj"].astype(np.float64))
+    assert np.all(np.abs(st["out"] - ref) <= 2.0 ** -22 * mag)
