@@ -1,0 +1,206 @@
+/* vitint - integerized ViT matmul path for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The library implements the operand-reordered ("integerized") linear layer and
+ * attention matmuls of Lin & Shah, "Low-Bit Integerization of Vision
+ * Transformers using Operand Reordering for Efficient Hardware": low-bit codes
+ * are contracted as integers into int32 accumulators and every step size is
+ * applied once, after the contraction (Section III, Eq. 1-3).
+ *
+ * General rules for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller; the library
+ *     allocates no device memory and keeps no reference after the call returns.
+ *     Descriptor structs (vitint_codes, vitint_epilogue, ...) are HOST structs.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work
+ *     is enqueued asynchronously on it; results are ready when the stream
+ *     reaches that point.
+ *   - Return value: VITINT_OK or a negative vitint_status.  Argument errors are
+ *     detected on the host before anything is launched.  No exceptions cross
+ *     the boundary.
+ *   - Kernels never spin without bound: a wait that exceeds its limit makes the
+ *     kernel record VITINT_ERR_TIMEOUT in a device status word and return; read
+ *     it with vitint_device_status().
+ *
+ * Packed code format (vitint_codes)
+ *   Row-major.  b-bit codes (b = 2, 3, 4, 8) live in containers of c = 2, 4, 4, 8
+ *   bits.  Element i of a row occupies bits [c*(i mod 8/c), +c) of byte
+ *   i / (8/c) (little-endian inside the byte).  Signed codes are two's
+ *   complement sign-extended to the container; signed range
+ *   [-2^(b-1), 2^(b-1)-1], unsigned [0, 2^b-1] (the 3-bit comparator ladder
+ *   -3.5D ... 2.5D of Section IV-B gives levels -4..3).  `data` and
+ *   `pitch_bytes` are multiples of 16; bytes between the last code of a row and
+ *   the pitch are ZERO (producers in this library write them as zero, and they
+ *   may enter contractions).
+ */
+#ifndef VITINT_H_
+#define VITINT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    VITINT_OK = 0,
+    VITINT_ERR_INVALID_ARG = -1,    /* null pointer, non-positive size, bad enum, non-finite or non-positive step */
+    VITINT_ERR_UNSUPPORTED = -2,    /* a shape or format this build has no kernel for */
+    VITINT_ERR_ALIGNMENT = -3,      /* pointer or pitch not aligned as documented */
+    VITINT_ERR_OVERFLOW_BOUND = -4, /* K * max|q_x| * max|q_w| >= 2^31 for the declared formats */
+    VITINT_ERR_WORKSPACE = -5,      /* workspace missing, misaligned or too small */
+    VITINT_ERR_CUDA = -6,           /* a CUDA runtime / driver call failed */
+    VITINT_ERR_TIMEOUT = -7         /* a bounded device-side wait gave up (device status word) */
+} vitint_status;
+
+typedef struct {
+    void* data;          /* device, 16-byte aligned */
+    int64_t rows, cols;  /* logical code counts */
+    int64_t pitch_bytes; /* multiple of 16, >= ceil(cols*c/8) */
+    int32_t bits;        /* 2, 3, 4 or 8 */
+    int32_t is_signed;   /* 0 / 1 */
+} vitint_codes;
+
+typedef enum {
+    VITINT_EPI_ACC_I32 = 0,     /* raw int32 accumulators */
+    VITINT_EPI_DEQUANT_F32 = 1, /* y = fma(float(acc), s_x*s_w[n], b[n]) [GELU] [+ residual] */
+    VITINT_EPI_REQUANT = 2      /* codes at the next layer's step */
+} vitint_epi_mode;
+
+/* Epilogue applied to the int32 accumulators (Eq. 2: the "equivalent bias" and
+ * "post-scaling factor" moved behind the contraction; Section IV-B: operand
+ * scales "absorbed within the quantizer").
+ *   DEQUANT_F32: sc[n] = fl32(x_step * w_step[n]); y = fmaf((float)acc, sc[n], bias[n] or 0);
+ *                act == 1 applies GELU(y) = y*Phi(y) in fp32; then, if residual != NULL,
+ *                y += residual[m*ld_res + n] as one more rounded add.  fp32 output.
+ *   REQUANT, act == 0: q = clamp(rint(fmaf((float)acc, alpha[n], beta[n]))) with the
+ *                folded alpha = s_x s_w / s_out, beta = b / s_out supplied by the caller.
+ *   REQUANT, act == 1: y as in DEQUANT, g = GELU(y), q = clamp(rint(g * inv_out_step[n])).
+ * Rounding is to nearest, ties to even; the clamp range follows out_bits/out_signed.
+ * alpha, beta, inv_out_step: device arrays of N floats. */
+typedef struct {
+    int32_t mode;               /* vitint_epi_mode */
+    int32_t act;                /* 0 none, 1 GELU */
+    const float* residual;      /* DEQUANT only, or NULL */
+    int64_t ld_res;             /* elements */
+    const float* alpha;         /* REQUANT, act 0 */
+    const float* beta;          /* REQUANT, act 0 */
+    const float* inv_out_step;  /* REQUANT, act 1 */
+    int32_t out_bits;           /* REQUANT: 2, 3, 4, 8 */
+    int32_t out_signed;
+} vitint_epilogue;
+
+const char* vitint_status_string(int status);
+int vitint_version(void);
+
+/* Reads (and clears) the device status word of the current device; synchronizes
+ * the device.  Returns VITINT_OK, VITINT_ERR_TIMEOUT or VITINT_ERR_CUDA. */
+int vitint_device_status(void);
+
+/* Bytes a packed row of `cols` b-bit codes needs, rounded up to 16. */
+int64_t vitint_packed_pitch(int64_t cols, int32_t bits);
+
+/* a1. Quantize and pack (Section IV-B comparator quantizer, round-to-nearest-even):
+ *   q[m][k] = clamp(rint(x[m*ldx + k] / s_m)), s_m = row_steps[m] if row_steps != NULL
+ *   (per-output-channel weight steps, Eq. 1's Delta_W) else `step` (the single input
+ *   step of Eq. 2).  One IEEE fp32 division per element.
+ *   x: device fp32 [rows, ldx] (ldx >= cols, elements).  out: descriptor whose data,
+ *   rows (== rows), cols (== cols), pitch_bytes, bits, is_signed are set by the caller;
+ *   the whole pitch of every row is written (padding as zero).
+ *   Errors: INVALID_ARG (sizes, step <= 0 or not finite when row_steps == NULL, bits),
+ *   ALIGNMENT (out->data or pitch not multiples of 16). */
+int vitint_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, float step, const float* row_steps,
+                    const vitint_codes* out, void* stream);
+
+/* a2 + a3. Integerized linear layer (Eq. 1-2): acc[m][n] = sum_k q_x[m][k] * q_w[n][k]
+ *   in int32, then the epilogue above.
+ *   x: codes [M, K];  w: codes [N, K] (one row per output channel);  w_step: device [N]
+ *   (DEQUANT and GELU epilogues; may be NULL for ACC_I32 / plain REQUANT);  bias: device
+ *   [N] or NULL.  out / ld_out: int32* and elements (ACC_I32), float* and elements
+ *   (DEQUANT_F32), packed bytes and pitch in bytes (REQUANT; 16-byte aligned, the row
+ *   padding up to ld_out is written as zero).
+ *   Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED, OVERFLOW_BOUND (K*max|q_x|*max|q_w| >= 2^31
+ *   over the declared code ranges), CUDA. */
+int vitint_linear(const vitint_codes* x, float x_step, const vitint_codes* w, const float* w_step,
+                  const float* bias, const vitint_epilogue* epi, void* out, int64_t ld_out, void* stream);
+
+/* Strided set of [tokens, head_dim] code slabs inside a larger code matrix (the Q, K
+ * or V part of a QKV activation).  Slab (image b, head h) starts at
+ * data + b*image_stride_bytes + h*head_stride_bytes; rows are pitch_bytes apart.
+ * head_dim is 64.  All three byte quantities are multiples of 16. */
+typedef struct {
+    const void* data;
+    int64_t pitch_bytes, image_stride_bytes, head_stride_bytes;
+    int32_t bits, is_signed;
+} vitint_slabs;
+
+/* a4. S[p][i][j] = sum_c Q_p[i][c] * K_p[j][c] for every problem p = b*heads + h
+ *   (Eq. 3 before the scale).  s_out: int32, problem p at s_out + p*tokens*ld_s, row i at
+ *   + i*ld_s (ld_s >= tokens, elements). */
+int vitint_qk(const vitint_slabs* q, const vitint_slabs* k, int32_t batch, int32_t heads, int32_t tokens,
+              int32_t* s_out, int64_t ld_s, void* stream);
+
+/* a5. Scale + row softmax + quantize (Eq. 3): t_j = fl32((float)S_j * c), p = softmax_j(t)
+ *   in fp32 with <= 2 ulp error, q_j = clamp(rint(p_j / p_step), 0, 2^bits - 1) decided in
+ *   fp32 (one IEEE division).  s: int32 [rows, ld_s];  p_out: unsigned codes [rows, cols]
+ *   (padding written as zero);  p_f32: optional fp32 probabilities [rows, ld_p] or NULL.
+ *   cols <= 1024. */
+int vitint_softmax_quantize(const int32_t* s, int64_t rows, int32_t cols, int64_t ld_s, float c, float p_step,
+                            const vitint_codes* p_out, float* p_f32, int64_t ld_p, void* stream);
+
+/* a6. O[p][i][c] = sum_j P_p[i][j] * V_p[j][c] (Section IV-B, W_attn V), then the epilogue
+ *   with s_x*s_w[n] replaced by p_step*v_step (bias NULL; alpha/beta/inv_out_step, when
+ *   used, are indexed by the output column h*64 + c).
+ *   p: codes with rows = batch*heads*tokens (problem p owns rows p*tokens ...), cols = tokens.
+ *   out: [batch*tokens, heads*64] matrix (int32 / fp32 elements, or packed with ld_out = pitch
+ *   bytes); problem (b, h) writes rows b*tokens + i, columns h*64 + c. */
+int vitint_pv(const vitint_codes* p, const vitint_slabs* v, int32_t batch, int32_t heads, int32_t tokens,
+              float p_step, float v_step, const vitint_epilogue* epi, void* out, int64_t ld_out, void* stream);
+
+/* a7. Integerized self-attention block (Fig. 1(b)):
+ *   QKV linear (requantized with per-channel alpha_qkv/beta_qkv, i.e. three per-tensor
+ *   steps q_step, k_step, v_step laid out per output channel) -> Q K^T -> scale, softmax,
+ *   quantize to unsigned p_bits at p_step -> P V -> requantize with alpha_o/beta_o to
+ *   signed o codes -> output projection with proj_epi.
+ *   x: codes [batch*tokens, D], D = heads*64.  w_qkv: codes [3D, D]; w_proj: codes [D, D].
+ *   alpha_qkv, beta_qkv: device [3D];  alpha_o: device [D], beta_o: device [D] or NULL.
+ *   w_proj_step, b_proj: device [D] as in vitint_linear (x_step of the projection = o_step).
+ *   out / ld_out as in vitint_linear for proj_epi.mode.
+ *   dbg_qkv / dbg_p / dbg_o: optional descriptors (data may point anywhere suitably sized)
+ *   that receive copies of the intermediate codes: QKV [M, 3D], P [batch*heads*tokens, tokens],
+ *   O [M, D]; NULL to skip.
+ *   workspace: device scratch of at least vitint_attention_block_workspace_bytes(...) bytes,
+ *   256-byte aligned; contents are undefined afterwards. */
+typedef struct {
+    int32_t batch, tokens, heads;
+    int32_t bits;                 /* activation / weight code width of the block */
+    vitint_codes w_qkv;
+    const float* alpha_qkv;
+    const float* beta_qkv;
+    float q_step, k_step, v_step, p_step, o_step;
+    int32_t p_bits;
+    const float* alpha_o;
+    const float* beta_o;
+    vitint_codes w_proj;
+    const float* w_proj_step;
+    const float* b_proj;
+    vitint_epilogue proj_epi;
+} vitint_attention_desc;
+
+size_t vitint_attention_block_workspace_bytes(const vitint_attention_desc* d);
+
+int vitint_attention_block(const vitint_codes* x, const vitint_attention_desc* d, void* out, int64_t ld_out,
+                           const vitint_codes* dbg_qkv, const vitint_codes* dbg_p, const vitint_codes* dbg_o,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* Glue between integerized linears (the full-precision LayerNorm island of Fig. 1(b)):
+ *   y = (x - mean)/sqrt(var + eps) * gamma + beta per row in fp32 (biased variance), then
+ *   the a1 quantizer with `step`.  out: codes [rows, cols];  y_f32: optional fp32 copy of y
+ *   [rows, ld_y] or NULL.  cols <= 4096 and a multiple of 4. */
+int vitint_layernorm_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, const float* gamma,
+                              const float* beta, float eps, float step, const vitint_codes* out, float* y_f32,
+                              int64_t ld_y, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VITINT_H_ */

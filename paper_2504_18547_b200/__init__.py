@@ -1,0 +1,12 @@
+"""vitint: integerized ViT matmul path for NVIDIA B200 (thin ctypes binding over libvitint.so).
+
+Every function here only marshals arguments: all arithmetic of the path runs in the CUDA
+kernels of the C-ABI library declared in include/vitint.h.  PyTorch supplies device memory
+and streams.  There is no CPU fallback: a missing library raises at import of the binding.
+"""
+from .binding import (  # noqa: F401
+    Codes, Epilogue, Slabs, AttentionWeights, VitintError, fold_requant, lib, packed_pitch,
+    vitint_attention_block, vitint_attention_block_workspace_bytes, vitint_device_status,
+    vitint_layernorm_quantize, vitint_linear, vitint_pv, vitint_qk, vitint_quantize,
+    vitint_softmax_quantize, vitint_status_string, vitint_version, EPI_ACC_I32, EPI_DEQUANT_F32, EPI_REQUANT,
+)

@@ -1,0 +1,659 @@
+// a2/a3/a4/a6: integer GEMM  acc[m][n] = sum_k A[m][k] * B[n][k]  on the 5th-generation
+// tensor cores (tcgen05, kind::i8, int32 accumulators in TMEM) with the fused
+// post-contraction epilogue of Eq. 2.
+//
+// One persistent CTA per SM walks 128 x BN output tiles.  Warp roles:
+//   warps 0-3  epilogue: tcgen05.ld of their 32 TMEM lanes, rescale / bias / GELU /
+//              requantize / pack, global stores (warp w owns TMEM lanes 32w..32w+31);
+//   warp  4    TMA producer: packed low-bit tiles of A and B -> shared memory ring;
+//   warp  5    MMA issuer (one thread) and owner of the TMEM allocation;
+//   warps 6-9  unpack: packed codes -> int8 operand tiles in the shared-memory layout
+//              the tensor core expects (128-byte swizzle, K contiguous; or 64-byte
+//              swizzle, N contiguous, for the V operand of P*V).
+// The accumulator is double buffered in TMEM so the epilogue of tile i overlaps the
+// MMAs of tile i+1.
+//
+// Sign handling without sign extension: a signed c-bit code q is placed in the HIGH
+// bits of its byte, i.e. the int8 value is q * 2^(8-c).  The contraction then yields
+// acc * 2^shift exactly and the epilogue shifts it back (host checks that the scaled
+// sum still fits in int32).  Unsigned codes are placed in the low bits unscaled.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace vitint {
+
+namespace {
+
+constexpr int BM = 128;   // rows per tile (= TMEM lanes)
+constexpr int BK = 128;   // int8 elements per K block (= one 128-byte swizzle row)
+constexpr int EPI_WARPS = 4;
+constexpr int UNPACK_WARPS = 4;
+constexpr int WARP_TMA = 4, WARP_MMA = 5, WARP_UNPACK0 = 6;
+constexpr int NUM_THREADS = (WARP_UNPACK0 + UNPACK_WARPS) * 32;
+constexpr int MAX_STAGES = 6;
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000ll;   // about one second
+
+struct GemmParams {
+    int M, N, K;
+    int bn, m_tiles, n_tiles, n_inner, total_tiles, k_blocks;
+    int ca, cb, a_signed, b_signed, shift, b_mn_major;
+    int ns_i, ns_p;
+    uint32_t ia_bytes, ib_bytes, pa_bytes, pb_bytes, tmem_cols;
+    int mode, act, out_c;
+    float out_qn, out_qp, x_step;
+    void* out;
+    long long ld_out, row_off_outer, row_off_inner, col_off_inner;
+    const float* col_a;
+    const float* col_b;
+    const float* inv_s;
+    const float* residual;
+    long long ld_res;
+};
+
+struct Bars {
+    uint64_t p_full[MAX_STAGES], p_empty[MAX_STAGES], i_full[MAX_STAGES], i_empty[MAX_STAGES];
+    uint64_t acc_full[2], acc_empty[2];
+};
+
+// Bounded wait.  Gives up after WAIT_LIMIT_CYCLES or as soon as another thread of the CTA
+// has given up; the first to give up records the timeout in the device status word.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t spin = 1;; ++spin) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((spin & 127u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(&g_device_status, (int)VITINT_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+// 8 four-bit codes of one word -> 8 bytes in natural order.
+__device__ __forceinline__ void unpack4(uint32_t w, int sgn, uint32_t& o0, uint32_t& o1) {
+    uint32_t lo, hi;
+    if (sgn) { lo = (w << 4) & 0xF0F0F0F0u; hi = w & 0xF0F0F0F0u; }
+    else     { lo = w & 0x0F0F0F0Fu;        hi = (w >> 4) & 0x0F0F0F0Fu; }
+    o0 = __byte_perm(lo, hi, 0x5140);
+    o1 = __byte_perm(lo, hi, 0x7362);
+}
+// 16 two-bit codes of one word -> 16 bytes in natural order.
+__device__ __forceinline__ uint4 unpack2(uint32_t w, int sgn) {
+    uint32_t p0, p1, p2, p3;
+    if (sgn) {
+        p0 = (w << 6) & 0xC0C0C0C0u; p1 = (w << 4) & 0xC0C0C0C0u; p2 = (w << 2) & 0xC0C0C0C0u; p3 = w & 0xC0C0C0C0u;
+    } else {
+        p0 = w & 0x03030303u; p1 = (w >> 2) & 0x03030303u; p2 = (w >> 4) & 0x03030303u; p3 = (w >> 6) & 0x03030303u;
+    }
+    const uint32_t a = __byte_perm(p0, p1, 0x5140), b = __byte_perm(p2, p3, 0x5140);
+    const uint32_t c = __byte_perm(p0, p1, 0x7362), d = __byte_perm(p2, p3, 0x7362);
+    return make_uint4(__byte_perm(a, b, 0x5410), __byte_perm(a, b, 0x7632), __byte_perm(c, d, 0x5410),
+                      __byte_perm(c, d, 0x7632));
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// Expands one 16-byte chunk of packed codes and stores the resulting 8/C chunks of int8.
+// out_addr(oc) gives the shared-memory address of output chunk oc (0-based within the
+// 16-byte input chunk's span).
+template <typename AddrFn>
+__device__ __forceinline__ void expand_chunk(uint4 in, int c, int sgn, AddrFn out_addr) {
+    if (c == 4) {
+        uint4 o0, o1;
+        unpack4(in.x, sgn, o0.x, o0.y);
+        unpack4(in.y, sgn, o0.z, o0.w);
+        unpack4(in.z, sgn, o1.x, o1.y);
+        unpack4(in.w, sgn, o1.z, o1.w);
+        sts128(out_addr(0), o0);
+        sts128(out_addr(1), o1);
+    } else if (c == 2) {
+        sts128(out_addr(0), unpack2(in.x, sgn));
+        sts128(out_addr(1), unpack2(in.y, sgn));
+        sts128(out_addr(2), unpack2(in.z, sgn));
+        sts128(out_addr(3), unpack2(in.w, sgn));
+    } else {
+        sts128(out_addr(0), in);
+    }
+}
+
+__device__ __forceinline__ void tile_coords(const GemmParams& P, int tile, int& m_tile, int& n_tile, int& inner,
+                                            int& outer) {
+    const int per_problem = P.m_tiles * P.n_tiles;
+    const int prob = tile / per_problem;
+    const int rem = tile - prob * per_problem;
+    m_tile = rem / P.n_tiles;
+    n_tile = rem - m_tile * P.n_tiles;
+    outer = prob / P.n_inner;
+    inner = prob - outer * P.n_inner;
+}
+
+// Epilogue of one row x 32 columns: accumulators v[] (scaled by 2^shift) -> output.
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32_t (&v)[32], long long orow,
+                                               long long colbase, int n0) {
+    const int out_words = P.out_c;   // 32 codes = 4*out_c bytes = out_c words
+    const bool full = n0 + 32 <= P.N;
+    if (P.mode == VITINT_EPI_ACC_I32) {
+        int32_t* o = (int32_t*)P.out + orow * P.ld_out + colbase + n0;
+        if (full && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                reinterpret_cast<int4*>(o)[i] = make_int4((int)v[4 * i] >> P.shift, (int)v[4 * i + 1] >> P.shift,
+                                                          (int)v[4 * i + 2] >> P.shift, (int)v[4 * i + 3] >> P.shift);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (n0 + i < P.N) o[i] = (int)v[i] >> P.shift;
+        }
+        return;
+    }
+    // fp32 value per column
+    float y[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const bool valid = n0 + i < P.N;
+        const long long cidx = colbase + n0 + i;
+        const float f = (float)((int)v[i] >> P.shift);
+        float val = 0.0f;
+        if (valid) {
+            if (P.mode == VITINT_EPI_REQUANT && P.act == 0) {
+                val = fmaf(f, __ldg(P.col_a + cidx), P.col_b ? __ldg(P.col_b + cidx) : 0.0f);
+            } else {
+                const float sc = P.col_a ? __fmul_rn(P.x_step, __ldg(P.col_a + cidx)) : P.x_step;
+                val = fmaf(f, sc, P.col_b ? __ldg(P.col_b + cidx) : 0.0f);
+                if (P.act == 1) val = gelu_f32(val);
+                if (P.mode == VITINT_EPI_REQUANT) val = val * __ldg(P.inv_s + cidx);
+                else if (P.residual) val = val + __ldg(P.residual + orow * P.ld_res + cidx);
+            }
+        }
+        y[i] = val;
+    }
+    if (P.mode == VITINT_EPI_DEQUANT_F32) {
+        float* o = (float*)P.out + orow * P.ld_out + colbase + n0;
+        if (full && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                reinterpret_cast<float4*>(o)[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (n0 + i < P.N) o[i] = y[i];
+        }
+        return;
+    }
+    // REQUANT: 32 codes -> out_c words
+    uint32_t wds[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const uint32_t mask = (1u << P.out_c) - 1u;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const uint32_t code = (n0 + i < P.N) ? ((uint32_t)round_clamp(y[i], P.out_qn, P.out_qp) & mask) : 0u;
+        // static word index for each container width keeps wds[] in registers
+        if (P.out_c == 4) wds[i >> 3] |= code << (4 * (i & 7));
+        else if (P.out_c == 2) wds[i >> 4] |= code << (2 * (i & 15));
+        else wds[i >> 2] |= code << (8 * (i & 3));
+    }
+    const long long byte0 = ((colbase + n0) * P.out_c) >> 3;
+    uint8_t* o = (uint8_t*)P.out + orow * P.ld_out + byte0;
+    if (P.out_c == 4 && byte0 + 16 <= P.ld_out) {
+        *reinterpret_cast<uint4*>(o) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (k < out_words && byte0 + 4 * k + 4 <= P.ld_out) reinterpret_cast<uint32_t*>(o)[k] = wds[k];
+    }
+    // row padding behind the last chunk of the last column tile
+    if (P.col_off_inner == 0 && n0 + 32 >= P.N) {
+        for (long long off = byte0 + 4 * out_words; off + 4 <= P.ld_out; off += 4)
+            *reinterpret_cast<uint32_t*>((uint8_t*)P.out + orow * P.ld_out + off) = 0u;
+    }
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ GemmParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ Bars bars;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+    const uint32_t stage_i = P.ia_bytes + P.ib_bytes, stage_p = P.pa_bytes + P.pb_bytes;
+    const uint32_t packed_base = smem_base + (uint32_t)P.ns_i * stage_i;
+    volatile int* abort_ptr = &abort_flag;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < MAX_STAGES; ++s) {
+            ptx::mbar_init(ptx::smem_addr(&bars.p_full[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&bars.p_empty[s]), UNPACK_WARPS);
+            ptx::mbar_init(ptx::smem_addr(&bars.i_full[s]), UNPACK_WARPS);
+            ptx::mbar_init(ptx::smem_addr(&bars.i_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(ptx::smem_addr(&bars.acc_full[b]), 1);
+            ptx::mbar_init(ptx::smem_addr(&bars.acc_empty[b]), EPI_WARPS);
+        }
+        ptx::fence_mbar_init();
+        ptx::fence_proxy_async_smem();
+    }
+    if (warp == WARP_MMA) {
+        ptx::tmem_alloc(ptx::smem_addr(&tmem_base_slot), P.tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    if (warp == WARP_TMA && lane == 0) {
+        ptx::prefetch_tensormap(&map_a);
+        ptx::prefetch_tensormap(&map_b);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    const uint32_t acc_stride = P.tmem_cols >> 1;
+
+    if (warp == WARP_TMA) {
+        // ------------------------------ TMA producer -------------------------------
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+                int m_tile, n_tile, inner, outer;
+                tile_coords(P, tile, m_tile, n_tile, inner, outer);
+                for (int kb = 0; kb < P.k_blocks; ++kb, ++it) {
+                    const int s = it % P.ns_p;
+                    const uint32_t ph = (uint32_t)(it / P.ns_p) & 1u;
+                    if (!mbar_wait(ptx::smem_addr(&bars.p_empty[s]), ph ^ 1u, abort_ptr)) { ok = false; break; }
+                    const uint32_t full = ptx::smem_addr(&bars.p_full[s]);
+                    ptx::mbar_arrive_expect_tx(full, stage_p);
+                    const uint32_t dst = packed_base + (uint32_t)s * stage_p;
+                    ptx::tma_load_4d(dst, &map_a, full, kb * 16 * P.ca, m_tile * BM, inner, outer);
+                    if (P.b_mn_major)
+                        ptx::tma_load_4d(dst + P.pa_bytes, &map_b, full, 0, kb * BK, inner, outer);
+                    else
+                        ptx::tma_load_4d(dst + P.pa_bytes, &map_b, full, kb * 16 * P.cb, n_tile * P.bn, inner, outer);
+                }
+            }
+            if (!ok) {
+                // give the copies still in flight a bounded chance to land before the CTA exits
+                for (int j = (it > P.ns_p ? it - P.ns_p : 0); j < it; ++j) {
+                    const uint32_t bar = ptx::smem_addr(&bars.p_full[j % P.ns_p]);
+                    const uint32_t ph = (uint32_t)(j / P.ns_p) & 1u;
+                    for (int spin = 0; spin < (1 << 20) && !ptx::mbar_try_wait(bar, ph); ++spin) {}
+                }
+            }
+        }
+    } else if (warp == WARP_MMA) {
+        // ------------------------------- MMA issuer --------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = ptx::idesc_i8(BM, P.bn, P.a_signed, P.b_signed, P.b_mn_major);
+            int it = 0, tl = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++tl) {
+                const int buf = tl & 1;
+                const uint32_t acc_ph = (uint32_t)(tl >> 1) & 1u;
+                if (!mbar_wait(ptx::smem_addr(&bars.acc_empty[buf]), acc_ph ^ 1u, abort_ptr)) { ok = false; break; }
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * acc_stride;
+                for (int kb = 0; kb < P.k_blocks; ++kb, ++it) {
+                    const int s = it % P.ns_i;
+                    const uint32_t ph = (uint32_t)(it / P.ns_i) & 1u;
+                    if (!mbar_wait(ptx::smem_addr(&bars.i_full[s]), ph, abort_ptr)) { ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t a_addr = smem_base + (uint32_t)s * stage_i;
+                    const uint32_t b_addr = a_addr + P.ia_bytes;
+                    const uint64_t a_desc = ptx::smem_desc(a_addr, 16, 1024, ptx::SWIZZLE_128B);
+                    const uint64_t b_desc = P.b_mn_major ? ptx::smem_desc(b_addr, 16, 512, ptx::SWIZZLE_64B)
+                                                         : ptx::smem_desc(b_addr, 16, 1024, ptx::SWIZZLE_128B);
+                    const int k_left = P.K - kb * BK;
+                    const int k_steps = k_left >= BK ? BK / 32 : (k_left + 31) / 32;
+                    for (int k = 0; k < k_steps; ++k) {
+                        // 32 int8 of K per MMA: 32 bytes along a swizzled row, or four 8-row
+                        // groups (4 * 512 bytes) when K is the slow axis of the B tile
+                        const uint64_t a_k = a_desc + (uint64_t)(k * 2);
+                        const uint64_t b_k = b_desc + (uint64_t)(P.b_mn_major ? k * 128 : k * 2);
+                        ptx::mma_i8(d_tmem, a_k, b_k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    ptx::mma_commit(ptx::smem_addr(&bars.i_empty[s]));
+                }
+                if (ok) ptx::mma_commit(ptx::smem_addr(&bars.acc_full[buf]));
+            }
+        }
+    } else if (warp >= WARP_UNPACK0) {
+        // --------------------------------- unpack ----------------------------------
+        const int tid_u = threadIdx.x - WARP_UNPACK0 * 32;
+        constexpr int NU = UNPACK_WARPS * 32;
+        const int la = P.ca == 2 ? 1 : (P.ca == 4 ? 2 : 3);        // log2(chunks per packed A row)
+        const int lb = P.cb == 2 ? 1 : (P.cb == 4 ? 2 : 3);
+        const int ea = 8 / P.ca, eb = 8 / P.cb;                    // int8 chunks per packed chunk
+        const int chunks_a = BM << la;
+        const int chunks_b = P.b_mn_major ? (BK << lb) >> 1 : P.bn << lb;
+        int it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+            for (int kb = 0; kb < P.k_blocks; ++kb, ++it) {
+                const int sp = it % P.ns_p, si = it % P.ns_i;
+                const uint32_t php = (uint32_t)(it / P.ns_p) & 1u, phi = (uint32_t)(it / P.ns_i) & 1u;
+                bool w = mbar_wait(ptx::smem_addr(&bars.p_full[sp]), php, abort_ptr);
+                w = w && mbar_wait(ptx::smem_addr(&bars.i_empty[si]), phi ^ 1u, abort_ptr);
+                if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+                ptx::tc_fence_after();
+                const uint32_t pa = packed_base + (uint32_t)sp * stage_p, pb = pa + P.pa_bytes;
+                const uint32_t ia = smem_base + (uint32_t)si * stage_i, ib = ia + P.ia_bytes;
+                for (int q = tid_u; q < chunks_a; q += NU) {
+                    const int r = q >> la, j = q & ((1 << la) - 1);
+                    const uint32_t row = ia + (uint32_t)r * 128u;
+                    const int oc0 = j * ea, sw = r & 7;
+                    expand_chunk(lds128(pa + (uint32_t)q * 16u), P.ca, P.a_signed,
+                                 [&](int e) { return row + (uint32_t)(((oc0 + e) ^ sw) << 4); });
+                }
+                if (!P.b_mn_major) {
+                    for (int q = tid_u; q < chunks_b; q += NU) {
+                        const int r = q >> lb, j = q & ((1 << lb) - 1);
+                        const uint32_t row = ib + (uint32_t)r * 128u;
+                        const int oc0 = j * eb, sw = r & 7;
+                        expand_chunk(lds128(pb + (uint32_t)q * 16u), P.cb, P.b_signed,
+                                     [&](int e) { return row + (uint32_t)(((oc0 + e) ^ sw) << 4); });
+                    }
+                } else {
+                    // B tile = 128 rows of K, 64 codes of N each: rows of 64 int8, 64-byte swizzle
+                    const int lh = lb - 1;                         // log2(packed chunks per row)
+                    for (int q = tid_u; q < chunks_b; q += NU) {
+                        const int r = q >> lh, h = q & ((1 << lh) - 1);
+                        const uint32_t row = ib + (uint32_t)(r >> 3) * 512u + (uint32_t)(r & 7) * 64u;
+                        const int oc0 = h * eb, sw = (r >> 1) & 3;
+                        expand_chunk(lds128(pb + (uint32_t)q * 16u), P.cb, P.b_signed,
+                                     [&](int e) { return row + (uint32_t)(((oc0 + e) ^ sw) << 4); });
+                    }
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    ptx::mbar_arrive(ptx::smem_addr(&bars.i_full[si]));
+                    ptx::mbar_arrive(ptx::smem_addr(&bars.p_empty[sp]));
+                }
+            }
+        }
+    } else {
+        // -------------------------------- epilogue ---------------------------------
+        const int q4 = warp;   // TMEM lane quarter
+        int tl = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++tl) {
+            int m_tile, n_tile, inner, outer;
+            tile_coords(P, tile, m_tile, n_tile, inner, outer);
+            const int buf = tl & 1;
+            const uint32_t acc_ph = (uint32_t)(tl >> 1) & 1u;
+            const bool w = mbar_wait(ptx::smem_addr(&bars.acc_full[buf]), acc_ph, abort_ptr);
+            if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+            ptx::tc_fence_after();
+            const int row_in_problem = m_tile * BM + q4 * 32 + lane;
+            const bool row_ok = row_in_problem < P.M;
+            const long long orow = (long long)outer * P.row_off_outer + (long long)inner * P.row_off_inner + row_in_problem;
+            const long long colbase = (long long)inner * P.col_off_inner;
+            const uint32_t t_row = tmem_base + (uint32_t)buf * acc_stride + ((uint32_t)(q4 * 32) << 16);
+            for (int chunk = 0; chunk * 32 < P.bn; ++chunk) {
+                const int n0 = n_tile * P.bn + chunk * 32;
+                if (n0 >= P.N) break;
+                uint32_t v[32];
+                ptx::tmem_ld32(t_row + (uint32_t)(chunk * 32), v);
+                ptx::tmem_ld_wait();
+                if (row_ok) epilogue_chunk(P, v, orow, colbase, n0);
+                __syncwarp();
+            }
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&bars.acc_empty[buf]));
+        }
+    }
+
+    // ---------------------------------- teardown -----------------------------------
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == WARP_MMA) {
+        ptx::tc_fence_after();
+        __syncwarp();
+        ptx::tmem_dealloc(tmem_base, P.tmem_cols);
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// 4-D byte tensor (inner bytes, rows, inner problems, outer problems); out-of-range reads give zero.
+int make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t d3, uint64_t s1,
+             uint64_t s2, uint64_t s3, uint32_t box0, uint32_t box1) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return VITINT_ERR_CUDA;
+    cuuint64_t dims[4] = {d0, d1, d2, d3};
+    cuuint64_t strides[3] = {s1, s2, s3};
+    cuuint32_t box[4] = {box0, box1, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? VITINT_OK : VITINT_ERR_CUDA;
+}
+
+struct Operand {
+    const void* data;
+    int bits, is_signed;
+    uint64_t row_bytes;   // valid bytes of one row (inner extent of the tensor map)
+    uint64_t rows;        // rows per problem
+    uint64_t pitch, inner_stride, outer_stride;
+};
+
+int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 1;
+    }
+    return n;
+}
+
+}  // namespace
+
+// Batched NT integer GEMM launcher shared by the linear layer, Q K^T and P V.
+int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_inner, int n_outer, int b_mn_major,
+                GemmParams P, cudaStream_t st) {
+    const int ca = container_bits(A.bits), cb = container_bits(B.bits);
+    P.M = M; P.N = N; P.K = K;
+    P.ca = ca; P.cb = cb; P.a_signed = A.is_signed; P.b_signed = B.is_signed; P.b_mn_major = b_mn_major;
+    P.shift = (A.is_signed ? 8 - ca : 0) + (B.is_signed ? 8 - cb : 0);
+    // exact int32 contraction, also after the power-of-two operand scaling
+    const long long bound = (long long)K * max_abs_code(A.bits, A.is_signed) * max_abs_code(B.bits, B.is_signed);
+    if (bound >= (1ll << 31)) return VITINT_ERR_OVERFLOW_BOUND;
+    if ((bound << P.shift) >= (1ll << 31)) return VITINT_ERR_UNSUPPORTED;
+    int bn = N >= 256 ? 256 : ((N + 15) / 16) * 16;
+    if (b_mn_major) { if (N != 64) return VITINT_ERR_UNSUPPORTED; bn = 64; }
+    P.bn = bn;
+    P.m_tiles = (M + BM - 1) / BM;
+    P.n_tiles = (N + bn - 1) / bn;
+    P.n_inner = n_inner;
+    const long long tiles = (long long)P.m_tiles * P.n_tiles * n_inner * n_outer;
+    if (tiles <= 0 || tiles > 0x7fffffffll) return VITINT_ERR_UNSUPPORTED;
+    P.total_tiles = (int)tiles;
+    P.k_blocks = (K + BK - 1) / BK;
+    P.ia_bytes = BM * BK;
+    P.ib_bytes = b_mn_major ? BK * 64 : (uint32_t)bn * BK;
+    P.pa_bytes = BM * 16 * ca;
+    P.pb_bytes = b_mn_major ? BK * 8 * cb : (uint32_t)bn * 16 * cb;
+    const uint32_t per_stage = P.ia_bytes + P.ib_bytes + P.pa_bytes + P.pb_bytes;
+    int ns = (int)((220u * 1024u) / per_stage);
+    if (ns > 4) ns = 4;
+    if (ns < 2) return VITINT_ERR_UNSUPPORTED;
+    P.ns_i = P.ns_p = ns;
+    uint32_t cols = 32;
+    while (cols < 2u * (uint32_t)((bn + 31) / 32 * 32)) cols <<= 1;
+    P.tmem_cols = cols;
+
+    CUtensorMap map_a, map_b;
+    if (int rc = make_map(&map_a, A.data, A.row_bytes, A.rows, (uint64_t)n_inner, (uint64_t)n_outer, A.pitch,
+                          A.inner_stride, A.outer_stride, 16u * ca, BM))
+        return rc;
+    if (b_mn_major) {
+        if (int rc = make_map(&map_b, B.data, B.row_bytes, B.rows, (uint64_t)n_inner, (uint64_t)n_outer, B.pitch,
+                              B.inner_stride, B.outer_stride, 8u * cb, BK))
+            return rc;
+    } else {
+        if (int rc = make_map(&map_b, B.data, B.row_bytes, B.rows, (uint64_t)n_inner, (uint64_t)n_outer, B.pitch,
+                              B.inner_stride, B.outer_stride, 16u * cb, (uint32_t)bn))
+            return rc;
+    }
+    // at least ~120 KB so that two CTAs never share an SM (and its tensor memory)
+    size_t smem = (size_t)ns * per_stage + 1024;
+    if (smem < 120 * 1024) smem = 120 * 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) !=
+            cudaSuccess)
+            return VITINT_ERR_CUDA;
+        attr_set = true;
+    }
+    int grid = sm_count();
+    if (grid > P.total_tiles) grid = P.total_tiles;
+    gemm_i8_kernel<<<grid, NUM_THREADS, smem, st>>>(map_a, map_b, P);
+    return cuda_status(cudaGetLastError());
+}
+
+static int fill_epilogue(GemmParams& P, const vitint_epilogue* epi, float x_step, const float* w_step,
+                         const float* bias, void* out, int64_t ld_out, int64_t n_cols_total) {
+    if (!epi || !out) return VITINT_ERR_INVALID_ARG;
+    P.mode = epi->mode; P.act = epi->act; P.out = out; P.ld_out = ld_out;
+    P.x_step = x_step; P.col_a = nullptr; P.col_b = nullptr; P.inv_s = nullptr; P.residual = nullptr; P.ld_res = 0;
+    P.out_c = 4; P.out_qn = 0; P.out_qp = 0;
+    if (epi->act != 0 && epi->act != 1) return VITINT_ERR_INVALID_ARG;
+    switch (epi->mode) {
+        case VITINT_EPI_ACC_I32:
+            if (epi->act) return VITINT_ERR_INVALID_ARG;
+            if (ld_out < n_cols_total || (reinterpret_cast<uintptr_t>(out) & 3u)) return VITINT_ERR_INVALID_ARG;
+            break;
+        case VITINT_EPI_DEQUANT_F32:
+            if (ld_out < n_cols_total || (reinterpret_cast<uintptr_t>(out) & 3u)) return VITINT_ERR_INVALID_ARG;
+            if (!(x_step > 0.0f && x_step < INFINITY)) return VITINT_ERR_INVALID_ARG;
+            P.col_a = w_step; P.col_b = bias; P.residual = epi->residual; P.ld_res = epi->ld_res;
+            if (epi->residual && epi->ld_res < n_cols_total) return VITINT_ERR_INVALID_ARG;
+            break;
+        case VITINT_EPI_REQUANT: {
+            if (!valid_bits(epi->out_bits)) return VITINT_ERR_INVALID_ARG;
+            if (!aligned16(out) || ld_out % 16 != 0) return VITINT_ERR_ALIGNMENT;
+            if (ld_out < row_bytes(n_cols_total, epi->out_bits)) return VITINT_ERR_INVALID_ARG;
+            int qn, qp;
+            code_range(epi->out_bits, epi->out_signed, &qn, &qp);
+            P.out_c = container_bits(epi->out_bits); P.out_qn = (float)qn; P.out_qp = (float)qp;
+            if (epi->act == 0) {
+                if (!epi->alpha) return VITINT_ERR_INVALID_ARG;
+                P.col_a = epi->alpha; P.col_b = epi->beta;
+            } else {
+                if (!epi->inv_out_step || !(x_step > 0.0f && x_step < INFINITY)) return VITINT_ERR_INVALID_ARG;
+                P.col_a = w_step; P.col_b = bias; P.inv_s = epi->inv_out_step;
+            }
+            break;
+        }
+        default:
+            return VITINT_ERR_INVALID_ARG;
+    }
+    return VITINT_OK;
+}
+
+static int check_slabs(const vitint_slabs* s) {
+    if (!s || !s->data) return VITINT_ERR_INVALID_ARG;
+    if (!valid_bits(s->bits)) return VITINT_ERR_INVALID_ARG;
+    if (!aligned16(s->data) || s->pitch_bytes % 16 || s->image_stride_bytes % 16 || s->head_stride_bytes % 16)
+        return VITINT_ERR_ALIGNMENT;
+    if (s->pitch_bytes < row_bytes(64, s->bits) || s->image_stride_bytes <= 0 || s->head_stride_bytes <= 0)
+        return VITINT_ERR_INVALID_ARG;
+    return VITINT_OK;
+}
+
+}  // namespace vitint
+
+using namespace vitint;
+
+extern "C" int vitint_linear(const vitint_codes* x, float x_step, const vitint_codes* w, const float* w_step,
+                             const float* bias, const vitint_epilogue* epi, void* out, int64_t ld_out, void* stream) {
+    if (int rc = check_codes(x)) return rc;
+    if (int rc = check_codes(w)) return rc;
+    if (x->cols != w->cols) return VITINT_ERR_INVALID_ARG;
+    if (x->rows > 0x7fffffff || w->rows > 0x7fffffff || x->cols > 0x7fffffff) return VITINT_ERR_UNSUPPORTED;
+    GemmParams P{};
+    if (int rc = fill_epilogue(P, epi, x_step, w_step, bias, out, ld_out, w->rows)) return rc;
+    if ((epi->mode == VITINT_EPI_DEQUANT_F32 || (epi->mode == VITINT_EPI_REQUANT && epi->act == 1)) && !w_step)
+        return VITINT_ERR_INVALID_ARG;
+    P.row_off_outer = 0; P.row_off_inner = 0; P.col_off_inner = 0;
+    Operand A{x->data, x->bits, x->is_signed, (uint64_t)row_bytes(x->cols, x->bits), (uint64_t)x->rows,
+              (uint64_t)x->pitch_bytes, (uint64_t)x->pitch_bytes * (uint64_t)x->rows,
+              (uint64_t)x->pitch_bytes * (uint64_t)x->rows};
+    Operand B{w->data, w->bits, w->is_signed, (uint64_t)row_bytes(w->cols, w->bits), (uint64_t)w->rows,
+              (uint64_t)w->pitch_bytes, (uint64_t)w->pitch_bytes * (uint64_t)w->rows,
+              (uint64_t)w->pitch_bytes * (uint64_t)w->rows};
+    return launch_gemm(A, B, (int)x->rows, (int)w->rows, (int)x->cols, 1, 1, 0, P, (cudaStream_t)stream);
+}
+
+extern "C" int vitint_qk(const vitint_slabs* q, const vitint_slabs* k, int32_t batch, int32_t heads, int32_t tokens,
+                         int32_t* s_out, int64_t ld_s, void* stream) {
+    if (int rc = check_slabs(q)) return rc;
+    if (int rc = check_slabs(k)) return rc;
+    if (batch <= 0 || heads <= 0 || tokens <= 0 || !s_out || ld_s < tokens) return VITINT_ERR_INVALID_ARG;
+    if (tokens > 256) return VITINT_ERR_UNSUPPORTED;   // one column tile per problem in this kernel
+    GemmParams P{};
+    vitint_epilogue epi{};
+    epi.mode = VITINT_EPI_ACC_I32;
+    if (int rc = fill_epilogue(P, &epi, 1.0f, nullptr, nullptr, s_out, ld_s, tokens)) return rc;
+    P.row_off_outer = (long long)heads * tokens; P.row_off_inner = tokens; P.col_off_inner = 0;
+    Operand A{q->data, q->bits, q->is_signed, (uint64_t)row_bytes(64, q->bits), (uint64_t)tokens,
+              (uint64_t)q->pitch_bytes, (uint64_t)q->head_stride_bytes, (uint64_t)q->image_stride_bytes};
+    Operand B{k->data, k->bits, k->is_signed, (uint64_t)row_bytes(64, k->bits), (uint64_t)tokens,
+              (uint64_t)k->pitch_bytes, (uint64_t)k->head_stride_bytes, (uint64_t)k->image_stride_bytes};
+    return launch_gemm(A, B, tokens, tokens, 64, heads, batch, 0, P, (cudaStream_t)stream);
+}
+
+extern "C" int vitint_pv(const vitint_codes* p, const vitint_slabs* v, int32_t batch, int32_t heads, int32_t tokens,
+                         float p_step, float v_step, const vitint_epilogue* epi, void* out, int64_t ld_out,
+                         void* stream) {
+    if (int rc = check_codes(p)) return rc;
+    if (int rc = check_slabs(v)) return rc;
+    if (batch <= 0 || heads <= 0 || tokens <= 0) return VITINT_ERR_INVALID_ARG;
+    if (p->rows != (int64_t)batch * heads * tokens || p->cols != tokens) return VITINT_ERR_INVALID_ARG;
+    if (!(p_step > 0.0f && p_step < INFINITY) || !(v_step > 0.0f && v_step < INFINITY)) return VITINT_ERR_INVALID_ARG;
+    GemmParams P{};
+    // the scale product s_P * s_V takes the place of s_x * s_w[n]
+    if (int rc = fill_epilogue(P, epi, p_step * v_step, nullptr, nullptr, out, ld_out,
+                               (int64_t)heads * 64))
+        return rc;
+    if (epi->mode == VITINT_EPI_REQUANT && epi->act == 1) return VITINT_ERR_UNSUPPORTED;
+    P.row_off_outer = tokens; P.row_off_inner = 0; P.col_off_inner = 64;
+    Operand A{p->data, p->bits, p->is_signed, (uint64_t)row_bytes(tokens, p->bits), (uint64_t)tokens,
+              (uint64_t)p->pitch_bytes, (uint64_t)p->pitch_bytes * tokens, (uint64_t)p->pitch_bytes * tokens * heads};
+    Operand B{v->data, v->bits, v->is_signed, (uint64_t)row_bytes(64, v->bits), (uint64_t)tokens,
+              (uint64_t)v->pitch_bytes, (uint64_t)v->head_stride_bytes, (uint64_t)v->image_stride_bytes};
+    return launch_gemm(A, B, tokens, 64, tokens, heads, batch, 1, P, (cudaStream_t)stream);
+}

@@ -1,0 +1,201 @@
+// a1: quantize + pack, and the LayerNorm + quantize glue.  Both are streaming,
+// HBM-bound kernels: 4 + c/8 bytes per element (c = container bits).
+#include "common.cuh"
+
+namespace vitint {
+
+// One thread produces one 32-bit word of packed output = 32/C consecutive codes.
+// Threads of a warp cover consecutive words of one row, so a warp reads
+// 32 * (32/C) * 4 contiguous bytes and writes 128 contiguous bytes.
+template <int C>
+__global__ void __launch_bounds__(256)
+quantize_pack_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, int64_t ldx, float step,
+                     const float* __restrict__ row_steps, uint8_t* __restrict__ out, int64_t pitch,
+                     int words_per_row, float qn, float qp, int vec_ok) {
+    constexpr int E = 32 / C;  // codes per word
+    const int w = blockIdx.x * blockDim.x + threadIdx.x;
+    if (w >= words_per_row) return;
+    const int64_t col0 = (int64_t)w * E;
+    for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows;
+         row += (int64_t)gridDim.y * blockDim.y) {
+        const float s = row_steps ? row_steps[row] : step;
+        const float* xr = x + row * ldx + col0;
+        float v[E];
+        if (vec_ok && col0 + E <= cols) {
+#pragma unroll
+            for (int i = 0; i < E / 4; ++i) {
+                const float4 f = __ldg(reinterpret_cast<const float4*>(xr) + i);
+                v[4 * i + 0] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < E; ++i) v[i] = (col0 + i < cols) ? __ldg(xr + i) : 0.0f;
+        }
+        uint32_t word = 0;
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+            const int q = round_clamp(__fdiv_rn(v[i], s), qn, qp);
+            word |= ((uint32_t)q & ((1u << C) - 1u)) << (C * i);
+        }
+        *reinterpret_cast<uint32_t*>(out + row * pitch + (int64_t)w * 4) = word;
+    }
+}
+
+// One warp per row; the row stays in registers between the statistics and the
+// normalisation.  Lane l owns float4 number v*32 + l of the row, v < NV.
+// Sums run in fp64 so that the result stays inside a few fp32 ulp of the exact
+// normalisation even when |mean| >> sigma.
+template <int C, int NV>
+__global__ void __launch_bounds__(256)
+layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, int64_t ldx,
+                          const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float step,
+                          uint8_t* __restrict__ out, int64_t pitch, float* __restrict__ y_out, int64_t ld_y,
+                          float qn, float qp) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const float* xr = x + row * ldx;
+    float4 f[NV];
+    double sum = 0.0;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int col = (v * 32 + lane) * 4;
+        f[v] = (col < cols) ? __ldg(reinterpret_cast<const float4*>(xr + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        sum += ((double)f[v].x + (double)f[v].y) + ((double)f[v].z + (double)f[v].w);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const double mean = sum / (double)cols;
+    double m2 = 0.0;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int col = (v * 32 + lane) * 4;
+        if (col < cols) {
+            f[v].x = (float)((double)f[v].x - mean);
+            f[v].y = (float)((double)f[v].y - mean);
+            f[v].z = (float)((double)f[v].z - mean);
+            f[v].w = (float)((double)f[v].w - mean);
+            m2 += ((double)f[v].x * f[v].x + (double)f[v].y * f[v].y) +
+                  ((double)f[v].z * f[v].z + (double)f[v].w * f[v].w);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
+    const float rstd = (float)(1.0 / sqrt(m2 / (double)cols + (double)eps));
+
+    constexpr int LANES_PER_WORD = 8 / C;          // 4 codes per lane per v -> 4*C bits
+    const int words_per_row = (int)(pitch >> 2);
+    const int nv_out = (words_per_row * LANES_PER_WORD + 31) / 32;   // v range that covers the pitch
+    for (int v = 0; v < nv_out; ++v) {
+        uint32_t bits = 0;
+        const int col = (v * 32 + lane) * 4;
+        if (v < NV && col < cols) {
+            const float4 g = __ldg(reinterpret_cast<const float4*>(gamma + col));
+            const float4 b = __ldg(reinterpret_cast<const float4*>(beta + col));
+            // static indexing of f[] keeps it in registers
+            float4 d = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < NV; ++u) if (u == v) d = f[u];
+            float4 y;
+            y.x = fmaf(d.x * rstd, g.x, b.x);
+            y.y = fmaf(d.y * rstd, g.y, b.y);
+            y.z = fmaf(d.z * rstd, g.z, b.z);
+            y.w = fmaf(d.w * rstd, g.w, b.w);
+            if (y_out) *reinterpret_cast<float4*>(y_out + row * ld_y + col) = y;
+            const uint32_t m = (1u << C) - 1u;
+            bits = ((uint32_t)round_clamp(__fdiv_rn(y.x, step), qn, qp) & m) |
+                   (((uint32_t)round_clamp(__fdiv_rn(y.y, step), qn, qp) & m) << C) |
+                   (((uint32_t)round_clamp(__fdiv_rn(y.z, step), qn, qp) & m) << (2 * C)) |
+                   (((uint32_t)round_clamp(__fdiv_rn(y.w, step), qn, qp) & m) << (3 * C));
+        }
+        // gather 8/C neighbouring lanes into one 32-bit word
+        if (C == 4) {
+            bits |= __shfl_xor_sync(0xffffffffu, bits, 1) << 16;
+        } else if (C == 2) {
+            bits |= __shfl_xor_sync(0xffffffffu, bits, 1) << 8;
+            bits |= __shfl_xor_sync(0xffffffffu, bits, 2) << 16;
+        }
+        const int word = (v * 32 + lane) / LANES_PER_WORD;
+        if ((lane % LANES_PER_WORD) == 0 && word < words_per_row)
+            *reinterpret_cast<uint32_t*>(out + row * pitch + (int64_t)word * 4) = bits;
+    }
+}
+
+template <int C>
+static int launch_ln(int nv, const float* x, int64_t rows, int cols, int64_t ldx, const float* gamma,
+                     const float* beta, float eps, float step, uint8_t* out, int64_t pitch, float* y, int64_t ld_y,
+                     float qn, float qp, cudaStream_t st) {
+    const int warps = 8;
+    dim3 grid((unsigned)((rows + warps - 1) / warps)), block(32 * warps);
+#define VITINT_LN_CASE(NVV)                                                                                     \
+    case NVV:                                                                                                   \
+        layernorm_quantize_kernel<C, NVV><<<grid, block, 0, st>>>(x, rows, cols, ldx, gamma, beta, eps, step,   \
+                                                                  out, pitch, y, ld_y, qn, qp);                 \
+        break;
+    switch (nv) {
+        VITINT_LN_CASE(1) VITINT_LN_CASE(2) VITINT_LN_CASE(3) VITINT_LN_CASE(4) VITINT_LN_CASE(6)
+        VITINT_LN_CASE(8) VITINT_LN_CASE(12) VITINT_LN_CASE(16)
+        default: return VITINT_ERR_UNSUPPORTED;
+    }
+#undef VITINT_LN_CASE
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace vitint
+
+using namespace vitint;
+
+extern "C" int vitint_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, float step,
+                               const float* row_steps, const vitint_codes* out, void* stream) {
+    if (!x || !out) return VITINT_ERR_INVALID_ARG;
+    if (int rc = check_codes(out)) return rc;
+    if (rows <= 0 || cols <= 0 || ldx < cols || out->rows != rows || out->cols != cols) return VITINT_ERR_INVALID_ARG;
+    if (!row_steps && !(step > 0.0f && step < INFINITY)) return VITINT_ERR_INVALID_ARG;
+    const int c = container_bits(out->bits);
+    int qn, qp;
+    code_range(out->bits, out->is_signed, &qn, &qp);
+    const int words = (int)(out->pitch_bytes / 4);
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(x) & 15u) == 0 && (ldx % 4) == 0) ? 1 : 0;
+    int bx = 32;
+    while (bx < 128 && bx < words) bx *= 2;
+    const int by = 256 / bx;
+    dim3 block(bx, by);
+    int64_t gy = (rows + by - 1) / by;
+    if (gy > 16384) gy = 16384;
+    dim3 grid((words + bx - 1) / bx, (unsigned)gy);
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* o = (uint8_t*)out->data;
+    if (c == 2)
+        quantize_pack_kernel<2><<<grid, block, 0, st>>>(x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
+                                                        words, (float)qn, (float)qp, vec_ok);
+    else if (c == 4)
+        quantize_pack_kernel<4><<<grid, block, 0, st>>>(x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
+                                                        words, (float)qn, (float)qp, vec_ok);
+    else
+        quantize_pack_kernel<8><<<grid, block, 0, st>>>(x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
+                                                        words, (float)qn, (float)qp, vec_ok);
+    return cuda_status(cudaGetLastError());
+}
+
+extern "C" int vitint_layernorm_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, const float* gamma,
+                                         const float* beta, float eps, float step, const vitint_codes* out,
+                                         float* y_f32, int64_t ld_y, void* stream) {
+    if (!x || !gamma || !beta || !out) return VITINT_ERR_INVALID_ARG;
+    if (int rc = check_codes(out)) return rc;
+    if (rows <= 0 || cols <= 0 || ldx < cols || out->rows != rows || out->cols != cols) return VITINT_ERR_INVALID_ARG;
+    if (!(step > 0.0f && step < INFINITY) || !(eps >= 0.0f)) return VITINT_ERR_INVALID_ARG;
+    if (cols % 4 != 0 || cols > 2048) return VITINT_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(gamma) || !aligned16(beta) || ldx % 4 != 0) return VITINT_ERR_ALIGNMENT;
+    if (y_f32 && (!aligned16(y_f32) || ld_y % 4 != 0 || ld_y < cols)) return VITINT_ERR_ALIGNMENT;
+    const int c = container_bits(out->bits);
+    int qn, qp;
+    code_range(out->bits, out->is_signed, &qn, &qp);
+    int nv = (int)((cols + 127) / 128);
+    const int sizes[] = {1, 2, 3, 4, 6, 8, 12, 16};
+    for (int s : sizes) if (s >= nv) { nv = s; break; }
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* o = (uint8_t*)out->data;
+    if (c == 2) return launch_ln<2>(nv, x, rows, (int)cols, ldx, gamma, beta, eps, step, o, out->pitch_bytes, y_f32, ld_y, (float)qn, (float)qp, st);
+    if (c == 4) return launch_ln<4>(nv, x, rows, (int)cols, ldx, gamma, beta, eps, step, o, out->pitch_bytes, y_f32, ld_y, (float)qn, (float)qp, st);
+    return launch_ln<8>(nv, x, rows, (int)cols, ldx, gamma, beta, eps, step, o, out->pitch_bytes, y_f32, ld_y, (float)qn, (float)qp, st);
+}

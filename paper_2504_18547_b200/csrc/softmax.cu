@@ -1,0 +1,169 @@
+// a5: scale + row softmax + quantize (Eq. 3), one warp per row.
+//
+// HBM-bound: 4 bytes read and c/8 bytes written per element.  The row lives in
+// registers (lane l owns columns 256*k + 8*l .. +7 of chunk k); the maximum and
+// the normaliser are reduced with warp shuffles.
+//
+// Accuracy target: probabilities within 2 ulp of the exactly rounded softmax.
+//   * t_j - max is formed exactly in fp64 (a rounded fp32 difference would already
+//     cost |t_j - max| * 2^-24 of relative error after the exponential);
+//   * exp(d) = 2^k * exp(r), k = rint(d*log2 e), r = d - k*ln2 reduced in fp64, then a
+//     degree-7 Taylor polynomial in fp32 on |r| <= ln2/2 (truncation < 0.1 ulp);
+//   * the normaliser is accumulated in fp64 and applied as one fp64 multiply.
+#include "common.cuh"
+
+namespace vitint {
+
+__device__ __forceinline__ float exp_reduced(double d) {
+    // d <= 0.  Below -200 the result is far under the smallest denormal.
+    d = fmax(d, -200.0);
+    const float kf = rintf((float)d * 1.44269504088896340736f);
+    const double r = fma(-(double)kf, 0.693147180559945309417, d);
+    const float rf = (float)r;
+    float p = 1.0f / 5040.0f;
+    p = fmaf(p, rf, 1.0f / 720.0f);
+    p = fmaf(p, rf, 1.0f / 120.0f);
+    p = fmaf(p, rf, 1.0f / 24.0f);
+    p = fmaf(p, rf, 1.0f / 6.0f);
+    p = fmaf(p, rf, 0.5f);
+    p = fmaf(p, rf, 1.0f);
+    p = fmaf(p, rf, 1.0f);
+    // 2^k in two exact factors so that k down to -252 stays representable
+    const int k = (int)kf;
+    const int k1 = k >> 1, k2 = k - k1;
+    return p * __int_as_float((k1 + 127) << 23) * __int_as_float((k2 + 127) << 23);
+}
+
+template <int C, int NCH>
+__global__ void __launch_bounds__(256)
+softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, int64_t ld_s, float c, float p_step,
+                        uint8_t* __restrict__ out, int64_t pitch, float* __restrict__ p_out, int64_t ld_p, float qp,
+                        int vec_in, int vec_p) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int32_t* sr = s + row * ld_s;
+
+    float t[NCH][8];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < NCH; ++k) {
+        const int col = k * 256 + lane * 8;
+        if (vec_in && col + 8 <= cols) {
+            const int4 a = __ldg(reinterpret_cast<const int4*>(sr + col));
+            const int4 b = __ldg(reinterpret_cast<const int4*>(sr + col) + 1);
+            t[k][0] = (float)a.x * c; t[k][1] = (float)a.y * c; t[k][2] = (float)a.z * c; t[k][3] = (float)a.w * c;
+            t[k][4] = (float)b.x * c; t[k][5] = (float)b.y * c; t[k][6] = (float)b.z * c; t[k][7] = (float)b.w * c;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) t[k][i] = (col + i < cols) ? (float)__ldg(sr + col + i) * c : -INFINITY;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mx = fmaxf(mx, t[k][i]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+
+    const double mxd = (double)mx;
+    double z = 0.0;
+#pragma unroll
+    for (int k = 0; k < NCH; ++k) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int col = k * 256 + lane * 8 + i;
+            const float e = (col < cols) ? exp_reduced((double)t[k][i] - mxd) : 0.0f;
+            t[k][i] = e;
+            z += (double)e;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    const double rz = 1.0 / z;
+
+    constexpr uint32_t MASK = (1u << C) - 1u;
+    const int chunk_bytes = 32 * C;                                   // 256 codes
+    const int n_out_chunks = (int)((pitch + chunk_bytes - 1) / chunk_bytes);
+    for (int k = 0; k < n_out_chunks; ++k) {
+        uint32_t w0 = 0, w1 = 0;
+        if (k < NCH) {
+            float p[8];
+#pragma unroll
+            for (int u = 0; u < NCH; ++u)
+                if (u == k) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) p[i] = (float)((double)t[u][i] * rz);
+                }
+            const int col = k * 256 + lane * 8;
+            if (p_out && col < cols) {
+                float* pr = p_out + row * ld_p + col;
+                if (vec_p && col + 8 <= cols) {
+                    reinterpret_cast<float4*>(pr)[0] = make_float4(p[0], p[1], p[2], p[3]);
+                    reinterpret_cast<float4*>(pr)[1] = make_float4(p[4], p[5], p[6], p[7]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) if (col + i < cols) pr[i] = p[i];
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t q = (col + i < cols) ? (uint32_t)round_clamp(__fdiv_rn(p[i], p_step), 0.0f, qp) : 0u;
+                if (C == 8) { if (i < 4) w0 |= q << (8 * i); else w1 |= q << (8 * (i - 4)); }
+                else w0 |= (q & MASK) << (C * i);
+            }
+        }
+        uint8_t* orow = out + row * pitch;
+        const int64_t off = (int64_t)k * chunk_bytes + lane * C;       // this lane's C bytes
+        if (C == 8) {
+            if (off + 8 <= pitch) *reinterpret_cast<uint2*>(orow + off) = make_uint2(w0, w1);
+        } else if (C == 4) {
+            if (off + 4 <= pitch) *reinterpret_cast<uint32_t*>(orow + off) = w0;
+        } else {
+            w0 |= __shfl_xor_sync(0xffffffffu, w0, 1) << 16;
+            if ((lane & 1) == 0 && off + 4 <= pitch) *reinterpret_cast<uint32_t*>(orow + off) = w0;
+        }
+    }
+}
+
+template <int C>
+static int launch_softmax(int nch, const int32_t* s, int64_t rows, int cols, int64_t ld_s, float c, float p_step,
+                          uint8_t* out, int64_t pitch, float* p, int64_t ld_p, float qp, int vec_in, int vec_p,
+                          cudaStream_t st) {
+    const int warps = 8;
+    dim3 grid((unsigned)((rows + warps - 1) / warps)), block(32 * warps);
+    switch (nch) {
+        case 1: softmax_quantize_kernel<C, 1><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
+        case 2: softmax_quantize_kernel<C, 2><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
+        case 3: softmax_quantize_kernel<C, 3><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
+        case 4: softmax_quantize_kernel<C, 4><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
+        default: return VITINT_ERR_UNSUPPORTED;
+    }
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace vitint
+
+using namespace vitint;
+
+extern "C" int vitint_softmax_quantize(const int32_t* s, int64_t rows, int32_t cols, int64_t ld_s, float c,
+                                       float p_step, const vitint_codes* p_out, float* p_f32, int64_t ld_p,
+                                       void* stream) {
+    if (!s || !p_out) return VITINT_ERR_INVALID_ARG;
+    if (int rc = check_codes(p_out)) return rc;
+    if (rows <= 0 || cols <= 0 || ld_s < cols || p_out->rows != rows || p_out->cols != cols || p_out->is_signed)
+        return VITINT_ERR_INVALID_ARG;
+    if (!(p_step > 0.0f && p_step < INFINITY) || !(c == c) || fabsf(c) == INFINITY) return VITINT_ERR_INVALID_ARG;
+    if (p_f32 && ld_p < cols) return VITINT_ERR_INVALID_ARG;
+    if (cols > 1024) return VITINT_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(s) & 3u) != 0) return VITINT_ERR_ALIGNMENT;
+    const int cb = container_bits(p_out->bits);
+    int qn, qp;
+    code_range(p_out->bits, 0, &qn, &qp);
+    const int nch = (cols + 255) / 256;
+    const int vec_in = (aligned16(s) && ld_s % 4 == 0) ? 1 : 0;
+    const int vec_p = (p_f32 && aligned16(p_f32) && ld_p % 4 == 0) ? 1 : 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* o = (uint8_t*)p_out->data;
+    if (cb == 2) return launch_softmax<2>(nch, s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
+    if (cb == 4) return launch_softmax<4>(nch, s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
+    return launch_softmax<8>(nch, s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
+}

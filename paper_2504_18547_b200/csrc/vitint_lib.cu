@@ -1,0 +1,6 @@
+// The whole library as one translation unit (one device status word, no device linking).
+#include "api.cu"
+#include "quantize.cu"
+#include "softmax.cu"
+#include "gemm.cu"
+#include "attention.cu"

@@ -1,0 +1,328 @@
+"""GPU parity: every C-ABI entry point against the CPU oracle on the same seeded inputs.
+
+Bar: bit-exact for int32 accumulators, a1 codes and requantized codes; bit-exact fp32 for
+the dequantizing epilogue (both sides run the same IEEE operation sequence); <= 2 ulp for
+softmax probabilities, with codes inside the oracle's band of codes reachable within that
+tolerance; GELU within 2^-21*|y|; LayerNorm within the oracle's per-element tolerance.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as vo
+import synth_inputs as si
+from oracle import pipeline as vp
+
+pytestmark = pytest.mark.gpu
+
+vt = pytest.importorskip("paper_2504_18547_b200")
+from gpu_util import dev, from_codes, padding_is_zero, rand_codes, to_codes, ulp_diff  # noqa: E402
+
+
+@pytest.fixture(autouse=True)
+def _device_status_clean():
+    yield
+    assert vt.vitint_device_status() == 0, "a device-side wait timed out"
+
+
+# ---------------------------------------------------------------------------
+# a1
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("bits,signed", [(2, True), (3, True), (4, True), (8, True), (2, False), (4, False), (8, False)])
+@pytest.mark.parametrize("rows,cols", [(197, 192), (3, 1), (130, 333), (64, 3072)])
+def test_quantize_matches_oracle(bits, signed, rows, cols):
+    x = si.normal(100 + bits + rows, (rows, cols), 0.1, 1.3)
+    step = si.lsq_step(x, bits, signed)
+    got = vt.vitint_quantize(dev(x), float(step), bits, signed)
+    assert np.array_equal(from_codes(got), vo.quantize(x, step, bits, signed))
+    assert np.array_equal(got.data.cpu().numpy(), vo.pack(vo.quantize(x, step, bits, signed), bits))
+    assert padding_is_zero(got)
+
+
+def test_quantize_row_steps_strided_input_and_ties():
+    rows, cols = 70, 200
+    w = si.normal(7, (rows, cols + 8), 0.0, 0.02)
+    steps = si.lsq_step_rows(w[:, :cols], 4)
+    xw = dev(w)[:, :cols]                      # ldx = cols + 8, rows not 16-byte aligned views
+    got = vt.vitint_quantize(xw, 0.0, 4, True, row_steps=dev(steps))
+    assert np.array_equal(from_codes(got), vo.quantize(w[:, :cols], 0.0, 4, True, row_steps=steps))
+    # exact ties and clamps
+    ks = np.arange(-12, 12, dtype=np.float32)
+    t = ((ks + 0.5) * 0.25).astype(np.float32)[None, :]
+    got = vt.vitint_quantize(dev(t), 0.25, 4, True)
+    assert np.array_equal(from_codes(got), vo.quantize(t, 0.25, 4, True))
+
+
+# ---------------------------------------------------------------------------
+# a2 + a3
+# ---------------------------------------------------------------------------
+
+LIN_SHAPES = [(197, 192, 576), (300, 320, 100), (128, 128, 256), (1, 64, 16), (515, 1000, 264), (260, 3072, 80)]
+
+
+@pytest.mark.parametrize("M,K,N", LIN_SHAPES)
+@pytest.mark.parametrize("bits,xs", [(4, True), (2, True), (3, True), (8, True), (4, False), (8, False), (2, False)])
+def test_linear_accumulators_bit_exact(M, K, N, bits, xs):
+    qx = rand_codes(1, (M, K), bits, xs)
+    qw = rand_codes(2, (N, K), bits, True)
+    acc = vt.vitint_linear(to_codes(qx, bits, xs), 1.0, to_codes(qw, bits, True), None, None,
+                           vt.Epilogue(mode=vt.EPI_ACC_I32))
+    assert np.array_equal(acc.cpu().numpy(), vo.matmul_i32(qx, qw))
+
+
+def test_linear_extreme_codes_closed_form():
+    # all-minimum x all-minimum at K = 4096: the largest magnitude the 4-bit path can produce
+    M, K, N = 130, 4096, 48
+    qx = np.full((M, K), -8, np.int16)
+    qw = np.full((N, K), -8, np.int16)
+    qw[1] = 7
+    acc = vt.vitint_linear(to_codes(qx, 4, True), 1.0, to_codes(qw, 4, True), None, None,
+                           vt.Epilogue(mode=vt.EPI_ACC_I32)).cpu().numpy()
+    assert np.all(acc[:, 0] == 64 * K) and np.all(acc[:, 1] == -56 * K)
+
+
+def test_linear_mixed_widths():
+    M, K, N = 200, 256, 96
+    qx = rand_codes(3, (M, K), 8, False)
+    qw = rand_codes(4, (N, K), 4, True)
+    acc = vt.vitint_linear(to_codes(qx, 8, False), 1.0, to_codes(qw, 4, True), None, None,
+                           vt.Epilogue(mode=vt.EPI_ACC_I32))
+    assert np.array_equal(acc.cpu().numpy(), vo.matmul_i32(qx, qw))
+
+
+@pytest.mark.parametrize("M,K,N", [(197, 192, 576), (300, 320, 100)])
+def test_linear_dequant_bias_residual_bit_exact(M, K, N):
+    qx = rand_codes(5, (M, K), 4, True)
+    qw = rand_codes(6, (N, K), 4, True)
+    s_w = (np.abs(si.normal(8, (N,), 0.0, 0.01)) + 1e-3).astype(np.float32)
+    bias = si.normal(9, (N,), 0.0, 0.01)
+    res = si.normal(10, (M, N))
+    acc = vo.matmul_i32(qx, qw)
+    for b_, r_ in ((None, None), (bias, None), (bias, res)):
+        epi = vt.Epilogue(mode=vt.EPI_DEQUANT_F32, residual=dev(r_))
+        y = vt.vitint_linear(to_codes(qx, 4, True), 0.37, to_codes(qw, 4, True), dev(s_w), dev(b_), epi)
+        want = vo.epilogue_dequant(acc, np.float32(0.37), s_w, b_, r_)
+        assert np.array_equal(y.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("out_bits,out_signed", [(4, True), (2, True), (3, True), (8, True), (4, False), (8, False)])
+@pytest.mark.parametrize("M,K,N", [(197, 192, 576), (300, 320, 100), (140, 128, 33)])
+def test_linear_requant_bit_exact(M, K, N, out_bits, out_signed):
+    qx = rand_codes(11, (M, K), 4, True)
+    qw = rand_codes(12, (N, K), 4, True)
+    s_w = (np.abs(si.normal(13, (N,), 0.0, 0.01)) + 1e-3).astype(np.float32)
+    bias = si.normal(14, (N,), 0.0, 0.05)
+    qp = si.code_range(out_bits, out_signed)[1]
+    alpha, beta = vp.fold(0.5, s_w, bias, 0.5 * 0.011 * 8 * math.sqrt(K) * 4 / qp)
+    a2, b2 = vt.fold_requant(0.5, s_w, bias, 0.5 * 0.011 * 8 * math.sqrt(K) * 4 / qp)
+    assert np.array_equal(alpha, a2) and np.array_equal(beta, b2)
+    epi = vt.Epilogue(mode=vt.EPI_REQUANT, alpha=dev(alpha), beta=dev(beta), out_bits=out_bits, out_signed=out_signed)
+    got = vt.vitint_linear(to_codes(qx, 4, True), 1.0, to_codes(qw, 4, True), None, None, epi)
+    want = vo.epilogue_requant(vo.matmul_i32(qx, qw), alpha, beta, out_bits, out_signed)
+    assert np.array_equal(from_codes(got), want)
+    assert padding_is_zero(got)
+    assert len(np.unique(want)) >= min(4, qp)
+
+
+def test_linear_gelu_dequant_and_requant():
+    M, K, N = 197, 192, 320
+    qx = rand_codes(15, (M, K), 4, True)
+    qw = rand_codes(16, (N, K), 4, True)
+    s_w = (np.abs(si.normal(17, (N,), 0.0, 0.004)) + 5e-4).astype(np.float32)
+    bias = si.normal(18, (N,), 0.0, 0.05)
+    acc = vo.matmul_i32(qx, qw)
+    x, w = to_codes(qx, 4, True), to_codes(qw, 4, True)
+    y = vt.vitint_linear(x, 0.6, w, dev(s_w), dev(bias), vt.Epilogue(mode=vt.EPI_DEQUANT_F32, act=1)).cpu().numpy()
+    pre = vo.epilogue_dequant(acc, np.float32(0.6), s_w, bias)
+    want = vo.epilogue_dequant(acc, np.float32(0.6), s_w, bias, None, act=1)
+    assert np.all(np.abs(y.astype(np.float64) - want) <= vo.GELU_TOL_REL * np.abs(pre) + 1e-30)
+    inv_s = vp.inv_step(np.full(N, 0.04, np.float32))
+    epi = vt.Epilogue(mode=vt.EPI_REQUANT, act=1, inv_out_step=dev(inv_s), out_bits=4, out_signed=False)
+    got = from_codes(vt.vitint_linear(x, 0.6, w, dev(s_w), dev(bias), epi))
+    q, lo, hi = vo.epilogue_gelu_requant(acc, np.float32(0.6), s_w, bias, inv_s, 4, False)
+    assert np.all(got >= lo) and np.all(got <= hi)
+    assert (got != q).mean() < 1e-3 and len(np.unique(q)) == 16
+
+
+# ---------------------------------------------------------------------------
+# a4, a5, a6
+# ---------------------------------------------------------------------------
+
+def _qkv_codes(batch, tokens, heads, bits, seed):
+    D = heads * 64
+    return rand_codes(seed, (batch * tokens, 3 * D), bits, True)
+
+
+@pytest.mark.parametrize("bits", [4, 2, 8])
+@pytest.mark.parametrize("batch,tokens,heads", [(1, 197, 3), (3, 197, 2), (2, 50, 1), (1, 256, 2)])
+def test_qk_bit_exact(batch, tokens, heads, bits):
+    D = heads * 64
+    qkv = _qkv_codes(batch, tokens, heads, bits, 21)
+    c = to_codes(qkv, bits, True)
+    S = vt.vitint_qk(vt.Slabs.of_qkv(c, tokens, D, 0), vt.Slabs.of_qkv(c, tokens, D, 1), batch, heads, tokens)
+    want = vo.qk(vp.split_heads(qkv, batch, tokens, heads, 64, 0), vp.split_heads(qkv, batch, tokens, heads, 64, D))
+    assert np.array_equal(S.cpu().numpy()[:, :, :tokens], want)
+
+
+@pytest.mark.parametrize("bits", [4, 2, 8])
+@pytest.mark.parametrize("batch,tokens,heads", [(1, 197, 3), (3, 197, 2), (2, 50, 1), (1, 256, 2)])
+def test_pv_bit_exact(batch, tokens, heads, bits):
+    D = heads * 64
+    qkv = _qkv_codes(batch, tokens, heads, bits, 22)
+    P = rand_codes(23, (batch * heads * tokens, tokens), bits, False)
+    c = to_codes(qkv, bits, True)
+    O = vt.vitint_pv(to_codes(P, bits, False), vt.Slabs.of_qkv(c, tokens, D, 2), batch, heads, tokens, 1.0, 1.0,
+                     vt.Epilogue(mode=vt.EPI_ACC_I32))
+    v = vp.split_heads(qkv, batch, tokens, heads, 64, 2 * D)
+    want = vp.merge_heads(vo.pv(P.reshape(batch * heads, tokens, tokens), v), batch, tokens, heads, 64)
+    assert np.array_equal(O.cpu().numpy(), want)
+
+
+def test_pv_requant_and_dequant_epilogues():
+    batch, tokens, heads, bits = 2, 197, 3, 4
+    D = heads * 64
+    qkv = _qkv_codes(batch, tokens, heads, bits, 24)
+    P = rand_codes(25, (batch * heads * tokens, tokens), bits, False)
+    c = to_codes(qkv, bits, True)
+    v = vp.split_heads(qkv, batch, tokens, heads, 64, 2 * D)
+    acc = vp.merge_heads(vo.pv(P.reshape(batch * heads, tokens, tokens), v), batch, tokens, heads, 64)
+    s_p, s_v, s_o = np.float32(0.0026), np.float32(0.17), np.float32(0.31)
+    alpha, beta = vp.fold(s_p, np.full(D, s_v, np.float32), None, s_o)
+    epi = vt.Epilogue(mode=vt.EPI_REQUANT, alpha=dev(alpha), out_bits=4, out_signed=True)
+    got = vt.vitint_pv(to_codes(P, bits, False), vt.Slabs.of_qkv(c, tokens, D, 2), batch, heads, tokens, s_p, s_v, epi)
+    want = vo.epilogue_requant(acc, alpha, beta, 4, True)
+    assert np.array_equal(from_codes(got), want) and len(np.unique(want)) >= 8
+    y = vt.vitint_pv(to_codes(P, bits, False), vt.Slabs.of_qkv(c, tokens, D, 2), batch, heads, tokens, s_p, s_v,
+                     vt.Epilogue(mode=vt.EPI_DEQUANT_F32))
+    sc = np.float32(s_p * s_v)
+    wanty = vo.epilogue_dequant(acc, sc, np.ones(D, np.float32), None)
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), wanty.view(np.uint32))
+
+
+@pytest.mark.parametrize("bits", [4, 2, 3, 8])
+@pytest.mark.parametrize("rows,cols,ld", [(591, 197, 200), (64, 197, 197), (33, 50, 52), (40, 577, 580), (24, 785, 785), (9, 1, 4)])
+def test_softmax_quantize_within_two_ulp_and_band(rows, cols, ld, bits):
+    S = np.zeros((rows, ld), np.int32)
+    S[:, :cols] = (si.splitmix64(31 + cols, rows * cols) % np.uint64(1401)).astype(np.int64).reshape(rows, cols) - 700
+    S[0, :cols] = 5                                     # uniform row
+    if cols > 3:
+        S[1, :cols] = -700
+        S[1, 2] = 700                                   # one dominant entry, the rest underflow
+    c = np.float32(0.0211)
+    s_p = np.float32(2.0 / (cols * math.sqrt(si.code_range(bits, False)[1])))
+    got, p = vt.vitint_softmax_quantize(dev(S), cols, c, s_p, bits, want_p=True)
+    p_ref, q, lo, hi = vo.softmax_quantize(S[:, :cols], c, s_p, bits)
+    p = p.cpu().numpy()
+    normal = p_ref >= 2.0 ** -126
+    assert ulp_diff(p[normal], p_ref[normal]).max() <= 2
+    assert np.all(np.abs(p[~normal].astype(np.float64) - p_ref[~normal]) <= 2.0 ** -126)
+    g = from_codes(got)
+    assert np.all(g >= lo) and np.all(g <= hi)
+    assert (g != q).mean() < 1e-3
+    assert padding_is_zero(got)
+
+
+def test_softmax_error_statistics_on_attention_like_rows():
+    rows, cols = 4096, 197
+    S = (si.splitmix64(77, rows * cols) % np.uint64(257)).astype(np.int64).reshape(rows, cols) - 128
+    c = np.float32(0.0035)
+    got, p = vt.vitint_softmax_quantize(dev(S.astype(np.int32)), cols, c, 0.00262, 4, want_p=True)
+    p_ref, q, lo, hi = vo.softmax_quantize(S, c, np.float32(0.00262), 4)
+    d = ulp_diff(p.cpu().numpy(), p_ref)
+    assert d.max() <= 2 and d.mean() < 0.6
+    g = from_codes(got)
+    assert np.all(g >= lo) and np.all(g <= hi)
+
+
+# ---------------------------------------------------------------------------
+# glue
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("cols", [192, 384, 768, 1024, 100])
+@pytest.mark.parametrize("bits", [4, 2, 8])
+def test_layernorm_quantize(cols, bits):
+    rows = 197
+    x = si.normal(41 + cols, (rows, cols), 3.0, 2.0)
+    x[5] += 100.0                                   # |mean| >> sigma
+    g = si.normal(42, (cols,), 1.0, 0.02)
+    b = si.normal(43, (cols,), 0.0, 0.02)
+    step = si.gaussian_lsq_step(1.0, bits)
+    got, y = vt.vitint_layernorm_quantize(dev(x), dev(g), dev(b), 1e-6, step, bits, True, want_y=True)
+    y_ref, tol = vo.layernorm(x, g, b, 1e-6)
+    assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - y_ref) <= tol)
+    q, lo, hi = vo.quantize_band(y_ref, tol, step, bits, True)
+    gq = from_codes(got)
+    assert np.all(gq >= lo) and np.all(gq <= hi) and (gq != q).mean() < 1e-3
+    assert padding_is_zero(got)
+
+
+# ---------------------------------------------------------------------------
+# a7: composed block, staged
+# ---------------------------------------------------------------------------
+
+def _attention_weights(cfg, prm, st, proj_epi):
+    D = cfg.dim
+    return vt.AttentionWeights(
+        batch=cfg.batch, tokens=cfg.tokens, heads=cfg.heads, bits=cfg.bits,
+        w_qkv=to_codes(st["w_qkv_codes"], cfg.bits, True), alpha_qkv=dev(st["alpha_qkv"]), beta_qkv=dev(st["beta_qkv"]),
+        q_step=float(prm["s_q"]), k_step=float(prm["s_k"]), v_step=float(prm["s_v"]), p_step=float(prm["s_p"]),
+        o_step=float(prm["s_o"]), p_bits=cfg.bits, alpha_o=dev(np.tile(st["alpha_o"], cfg.heads)), beta_o=None,
+        w_proj=to_codes(st["w_proj_codes"], cfg.bits, True), w_proj_step=dev(prm["s_w_proj"]),
+        b_proj=dev(prm["b_proj"]), proj_epi=proj_epi)
+
+
+@pytest.mark.parametrize("cfg", [si.VIT_TINY_BLOCK, si.VIT_TINY_BLOCK.with_(w_std=0.12, seed_index=11),
+                                 si.VIT_SMALL_BLOCK.with_(batch=3)], ids=["tiny", "tiny_peaked", "small_b3"])
+def test_attention_block_staged(cfg):
+    prm = si.layer_parameters(cfg)
+    x = si.activations(cfg)
+    s_x = si.lsq_step(x, cfg.bits, True)
+    xq = vo.quantize(x, s_x, cfg.bits, True)
+    st = vp.attention_block(xq, s_x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits, proj="dequant")
+    aw = _attention_weights(cfg, prm, st, vt.Epilogue(mode=vt.EPI_DEQUANT_F32))
+    M, D, T, H = cfg.rows, cfg.dim, cfg.tokens, cfg.heads
+    dq = vt.Codes.empty(M, 3 * D, cfg.bits, True)
+    dp = vt.Codes.empty(cfg.batch * H * T, T, cfg.bits, False)
+    do = vt.Codes.empty(M, D, cfg.bits, True)
+    xg = vt.vitint_quantize(dev(x), float(s_x), cfg.bits, True)
+    out = vt.vitint_attention_block(xg, aw, dbg_qkv=dq, dbg_p=dp, dbg_o=do).cpu().numpy()
+    # stage 1: QKV codes are unique
+    assert np.array_equal(from_codes(dq), st["qkv_codes"])
+    # stage 2: P codes inside the band; rows (image, head, token) holding an off-centre code are marked
+    gp = from_codes(dp).reshape(cfg.batch * H, T, T)
+    assert np.all(gp >= st["p_lo"]) and np.all(gp <= st["p_hi"])
+    flipped = (gp != st["p_codes"]).any(axis=2)                        # [B*H, T]
+    assert flipped.mean() < 0.02
+    # stage 3: O codes exact wherever the P row agreed
+    go = from_codes(do)
+    o_ok = np.ones((M, D), bool)
+    for b in range(cfg.batch):
+        for h in range(H):
+            o_ok[b * T:(b + 1) * T, h * 64:(h + 1) * 64] = ~flipped[b * H + h][:, None]
+    assert np.array_equal(go[o_ok], st["o_codes"][o_ok])
+    assert np.all(np.abs(go.astype(int) - st["o_codes"]) <= 1)
+    # stage 4: projection bit-exact on token rows whose O codes all agreed
+    rows_ok = (go == st["o_codes"]).all(axis=1)
+    assert rows_ok.mean() > 0.9
+    assert np.array_equal(out[rows_ok].view(np.uint32), st["out"][rows_ok].view(np.uint32))
+
+
+def test_attention_block_requant_output():
+    cfg = si.VIT_SMALL_BLOCK.with_(batch=2)
+    prm = si.layer_parameters(cfg)
+    x = si.activations(cfg)
+    s_x = si.lsq_step(x, cfg.bits, True)
+    xq = vo.quantize(x, s_x, cfg.bits, True)
+    st = vp.attention_block(xq, s_x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits, proj="requant")
+    epi = vt.Epilogue(mode=vt.EPI_REQUANT, alpha=dev(st["alpha_proj"]), beta=dev(st["beta_proj"]), out_bits=cfg.bits,
+                      out_signed=True)
+    aw = _attention_weights(cfg, prm, st, epi)
+    do = vt.Codes.empty(cfg.rows, cfg.dim, cfg.bits, True)
+    out = vt.vitint_attention_block(to_codes(xq, cfg.bits, True), aw, dbg_o=do)
+    rows_ok = (from_codes(do) == st["o_codes"]).all(axis=1)
+    assert rows_ok.mean() > 0.9
+    assert np.array_equal(from_codes(out)[rows_ok], st["out_codes"][rows_ok])
+    assert len(np.unique(st["out_codes"])) >= 8
