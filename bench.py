@@ -1,0 +1,305 @@
+"""Benchmark of the integerized ViT-Base encoder layer (batch 128, 197 tokens, 4-bit W/A).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--bits 4]
+
+One step = one pass of the whole hot path over one batch of synthetic activations:
+LayerNorm+quantize -> QKV linear -> Q K^T -> scale+softmax+quantize -> P V -> projection ->
+LayerNorm+quantize -> fc1 (GELU, requantize) -> fc2.  Prints ONE JSON line (rank 0).
+
+value      effective TOPS (2 x true multiply-accumulates of the six integer contractions per
+           second), inputs resident in HBM, whole job over all ranks (ranks hold disjoint images).
+e2e        same metric through the same calls with the step's fp32 input copied from pinned host
+           memory and the fp32 output copied back inside the timed region.
+roofline   the integer GEMM kernel: achieved TOPS over its launches inside the timed region
+           (CUDA events around each call) against the int8 tensor peak.
+cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import synth_inputs as si  # noqa: E402
+
+INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor throughput ratio on B200 (4.5 : 2.25 PFLOP/s)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+N_INPUT_BUFFERS = 4           # 4 x 77.5 MB of fp32 activations > 126 MB of L2
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        mhz = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for r in self.rows if len(r) >= 6 for n, v in zip(names, r[2:6]) if v.lower() == "active"})
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(mhz)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """MAX all-reduce of a scalar (identity for a single process)."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def layer_ops(cfg: si.BlockConfig, batch: int) -> int:
+    return 2 * batch * si.mac_counts(cfg.tokens, cfg.dim, cfg.heads, 64, cfg.mlp_dim)["total"]
+
+
+# ---------------------------------------------------------------------------
+# reference arm: the CPU oracle
+# ---------------------------------------------------------------------------
+
+def run_reference(args, cfg):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import oracle as vo
+    from oracle import pipeline as vp
+    prm = si.layer_parameters(cfg)
+    sample = args.ref_images
+    x = si.activations(cfg, batch=sample)
+    for _ in range(args.warmup):
+        vp.encoder_layer(x[:cfg.tokens], prm, 1, cfg.tokens, cfg.heads, cfg.bits)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        vp.encoder_layer(x, prm, sample, cfg.tokens, cfg.heads, cfg.bits)
+    dt = (time.perf_counter() - t0) / args.steps
+    tops = layer_ops(cfg, sample) / dt / 1e12
+    line = {
+        "impl": "reference", "metric": "integerized ViT-B block effective TOPS", "value": tops, "unit": "TOPS",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "images_per_s": sample / dt,
+        "config": {"workload": cfg.name, "bits": cfg.bits, "batch": cfg.batch, "tokens": cfg.tokens, "dim": cfg.dim,
+                   "heads": cfg.heads, "mlp_dim": cfg.mlp_dim, "l2": "n/a (CPU)"},
+        "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": vo.get_threads(), "kind": "oracle",
+                         "sample": f"{sample} of {cfg.batch} images per step, whole encoder layer"},
+        "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2504_18547_b200 as vt
+    from paper_2504_18547_b200.encoder import GEMM_STAGES, STAGES, EncoderLayer
+
+    rank, local_rank, world = dist_env()
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    prm = si.layer_parameters(cfg)
+    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, device)
+    M, D = cfg.rows, cfg.dim
+    # each rank owns a disjoint range of images (weak scaling, no exchange on the data path)
+    first = rank * cfg.batch
+    host_x = [torch.from_numpy(si.activations(cfg, batch=cfg.batch, first_image=first + i * cfg.batch * world)
+                               ).pin_memory() for i in range(N_INPUT_BUFFERS)]
+    xs = [h.to(device) for h in host_x]
+    out = torch.empty((M, D), dtype=torch.float32, device=device)
+    host_out = torch.empty((M, D), dtype=torch.float32).pin_memory()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        layer.forward(xs[i % N_INPUT_BUFFERS], out)
+    barrier()
+    if vt.vitint_device_status() != 0:
+        raise RuntimeError("device-side timeout during warm-up")
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+
+    # ---- device-resident timing: K steps, stage events inside ------------------------
+    barrier()
+    ev_steps = []
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(args.steps):
+        ev = []
+        layer.forward(xs[i % N_INPUT_BUFFERS], out, events=ev)
+        ev_steps.append(ev)
+    t_end.record()
+    barrier()
+    ms_total = max_over_ranks(t_start.elapsed_time(t_end), world, device)
+    clocks = sampler.stop() if rank == 0 else None
+
+    stage_ms = {s: 0.0 for s in STAGES}
+    for ev in ev_steps:
+        for j, s in enumerate(STAGES):
+            stage_ms[s] += ev[j].elapsed_time(ev[j + 1])
+    stage_ms = {s: v / args.steps for s, v in stage_ms.items()}
+
+    # ---- end to end: host -> device, step, device -> host, every step -----------------
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    x_dev = torch.empty_like(xs[0])
+    t0.record()
+    for i in range(args.steps):
+        x_dev.copy_(host_x[i % N_INPUT_BUFFERS], non_blocking=True)
+        layer.forward(x_dev, out)
+        host_out.copy_(out, non_blocking=True)
+    t1.record()
+    barrier()
+    ms_e2e = max_over_ranks(t0.elapsed_time(t1), world, device)
+    if vt.vitint_device_status() != 0:
+        raise RuntimeError("device-side timeout during the timed region")
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    ops_step = layer_ops(cfg, cfg.batch)
+    ms_step = ms_total / args.steps
+    tops = world * ops_step / (ms_step * 1e-3) / 1e12
+    e2e_tops = world * ops_step / (ms_e2e / args.steps * 1e-3) / 1e12
+
+    sops = layer.stage_ops()
+    gemm_ms = sum(stage_ms[s] for s in GEMM_STAGES)
+    gemm_ops = sum(sops[s] for s in GEMM_STAGES)
+    int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+    achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
+    sbytes = layer.stage_bytes()
+    kernels = {}
+    for s in STAGES:
+        k = {"ms": round(stage_ms[s], 4)}
+        if s in sops:
+            k["tops"] = round(sops[s] / (stage_ms[s] * 1e-3) / 1e12, 1)
+            k["frac_int8_peak"] = round(k["tops"] / int8_peak, 4)
+        if s in sbytes:
+            k["gbs"] = round(sbytes[s] / (stage_ms[s] * 1e-3) / 1e9, 1)
+            k["frac_hbm_peak"] = round(k["gbs"] / peaks["hbm_gbs"], 4)
+        kernels[s] = k
+
+    # ---- CPU oracle on a bounded sample (rank 0, single-GPU runs only) -----------------
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle as vo
+        from oracle import pipeline as vp
+        sample = args.ref_images
+        xs_cpu = si.activations(cfg, batch=sample)
+        t0c = time.perf_counter()
+        vp.encoder_layer(xs_cpu, prm, sample, cfg.tokens, cfg.heads, cfg.bits)
+        dtc = time.perf_counter() - t0c
+        cpu = {"value": layer_ops(cfg, sample) / dtc / 1e12, "unit": "TOPS", "cores": vo.get_threads(),
+               "kind": "oracle", "sample": f"{sample} of {cfg.batch} images, whole encoder layer, {dtc:.1f} s"}
+
+    line = {
+        "metric": "integerized ViT-B block effective TOPS", "value": tops, "unit": "TOPS", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "images_per_s": world * cfg.batch / (ms_step * 1e-3),
+        "config": {"workload": cfg.name, "bits": cfg.bits, "batch_per_gpu": cfg.batch, "tokens": cfg.tokens,
+                   "dim": cfg.dim, "heads": cfg.heads, "mlp_dim": cfg.mlp_dim,
+                   "l2": f"inputs rotate over {N_INPUT_BUFFERS} buffers of {M * D * 4 / 1e6:.1f} MB (> 126 MB L2)"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_tops, "unit": "TOPS", "h2d_bytes_per_step": M * D * 4, "d2h_bytes_per_step": M * D * 4,
+                "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": len(STAGES) * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel (6 launches per step)", "achieved": achieved,
+                     "peak": int8_peak, "unit": "TOPS", "frac": achieved / int8_peak, "traffic": None,
+                     "peak_source": f"{peaks['source']} sustained bf16 cuBLAS x {INT8_OVER_BF16:g} (nominal int8:bf16)",
+                     "frac_of_nominal_4500": achieved / 4500.0},
+        "kernels": kernels,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--bits", type=int, default=4, choices=[2, 3, 4])
+    ap.add_argument("--batch", type=int, default=None, help="images per GPU (default: the configuration's 128)")
+    ap.add_argument("--ref-images", type=int, default=None, help="images per step of the CPU oracle")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = si.VIT_BASE_LAYER.with_(bits=args.bits)
+    if args.batch:
+        cfg = cfg.with_(batch=args.batch, name=f"vit_base_layer_b{args.batch}")
+    if args.ref_images is None:
+        args.ref_images = 64 if args.impl == "ours" else 8
+    args.ref_images = min(args.ref_images, cfg.batch)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

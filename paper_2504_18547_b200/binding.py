@@ -109,6 +109,11 @@ def _ptr(t):
     return None if t is None else t.data_ptr()
 
 
+def _ld(t) -> int:
+    """Leading dimension in elements of a 2-D tensor (a single row reports its width)."""
+    return int(t.stride(0)) if t.shape[0] > 1 else max(int(t.stride(0)), int(t.shape[-1]))
+
+
 @dataclass
 class Codes:
     """Packed low-bit codes on the device: a uint8 tensor [rows, pitch] plus the logical shape."""
@@ -148,7 +153,7 @@ class Epilogue:
     out_signed: bool = True
 
     def desc(self) -> _Epilogue:
-        ld_res = int(self.residual.stride(0)) if self.residual is not None else 0
+        ld_res = _ld(self.residual) if self.residual is not None else 0
         return _Epilogue(self.mode, self.act, _ptr(self.residual), ld_res, _ptr(self.alpha), _ptr(self.beta),
                          _ptr(self.inv_out_step), self.out_bits, int(self.out_signed))
 
@@ -194,7 +199,7 @@ def vitint_quantize(x: torch.Tensor, step: float, bits: int, signed: bool, row_s
     rows, cols = x.shape
     out = Codes.empty(rows, cols, bits, signed, x.device) if out is None else out
     d = out.desc()
-    _check(lib().vitint_quantize(x.data_ptr(), rows, cols, x.stride(0), float(step), _ptr(row_steps), byref(d),
+    _check(lib().vitint_quantize(x.data_ptr(), rows, cols, _ld(x), float(step), _ptr(row_steps), byref(d),
                                  _stream()), "vitint_quantize")
     return out
 
@@ -210,7 +215,7 @@ def _alloc_out(epi: Epilogue, rows: int, cols: int, device):
 def _out_ptr_ld(out):
     if isinstance(out, Codes):
         return out.data.data_ptr(), out.pitch
-    return out.data_ptr(), int(out.stride(0))
+    return out.data_ptr(), _ld(out)
 
 
 def vitint_linear(x: Codes, x_step: float, w: Codes, w_step: torch.Tensor | None, bias: torch.Tensor | None,
@@ -236,7 +241,7 @@ def vitint_qk(q: Slabs, k: Slabs, batch: int, heads: int, tokens: int, out: torc
 def vitint_softmax_quantize(s: torch.Tensor, cols: int, c: float, p_step: float, bits: int,
                             want_p: bool = False, out: Codes | None = None):
     """s: int32 [rows, ld_s] (only the first `cols` columns of each row are read)."""
-    rows, ld_s = s.shape[0], int(s.stride(0))
+    rows, ld_s = s.shape[0], _ld(s)
     out = Codes.empty(rows, cols, bits, False, s.device) if out is None else out
     p = torch.empty((rows, cols), dtype=torch.float32, device=s.device) if want_p else None
     d = out.desc()
@@ -311,7 +316,7 @@ def vitint_layernorm_quantize(x: torch.Tensor, gamma: torch.Tensor, beta: torch.
     out = Codes.empty(rows, cols, bits, signed, x.device) if out is None else out
     y = torch.empty((rows, cols), dtype=torch.float32, device=x.device) if want_y else None
     d = out.desc()
-    _check(lib().vitint_layernorm_quantize(x.data_ptr(), rows, cols, x.stride(0), gamma.data_ptr(), beta.data_ptr(),
+    _check(lib().vitint_layernorm_quantize(x.data_ptr(), rows, cols, _ld(x), gamma.data_ptr(), beta.data_ptr(),
                                            float(eps), float(step), byref(d), _ptr(y), cols if want_y else 0,
                                            _stream()), "vitint_layernorm_quantize")
     return (out, y) if want_y else out

@@ -1,0 +1,110 @@
+"""Integerized ViT encoder layer as a fixed sequence of C-ABI calls with preallocated buffers.
+
+LayerNorm+quantize -> QKV linear -> Q K^T -> softmax+quantize -> P V -> projection (+residual)
+-> LayerNorm+quantize -> fc1 (GELU, requantize) -> fc2 (+residual).  This module only owns
+device buffers and marshals arguments; every step runs in the library's kernels.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+STAGES = ("ln1_quant", "qkv_linear", "qk", "softmax_quant", "pv", "proj_linear", "ln2_quant", "fc1_linear",
+          "fc2_linear")
+GEMM_STAGES = ("qkv_linear", "qk", "pv", "proj_linear", "fc1_linear", "fc2_linear")
+
+
+def _dev(a, device):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+class EncoderLayer:
+    def __init__(self, batch: int, tokens: int, heads: int, mlp_dim: int, bits: int, prm: dict, device="cuda",
+                 eps: float = 1e-6):
+        self.batch, self.tokens, self.heads, self.bits, self.eps = batch, tokens, heads, bits, eps
+        self.dim = D = heads * 64
+        self.mlp_dim = F = mlp_dim
+        self.rows = M = batch * tokens
+        self.device = device
+        d = lambda a: _dev(a, device)
+        f = lambda k: float(prm[k])
+        self.s_ln, self.s_q, self.s_k, self.s_v = f("s_ln"), f("s_q"), f("s_k"), f("s_v")
+        self.s_p, self.s_o, self.s_g = f("s_p"), f("s_o"), f("s_g")
+        self.ln1_g, self.ln1_b, self.ln2_g, self.ln2_b = d(prm["ln1_g"]), d(prm["ln1_b"]), d(prm["ln2_g"]), d(prm["ln2_b"])
+        # weights: quantized once by the library's own quantizer (per-output-channel steps)
+        self.w = {}
+        for name in ("qkv", "proj", "fc1", "fc2"):
+            self.w[name] = B.vitint_quantize(d(prm[f"w_{name}"]), 0.0, bits, True, row_steps=d(prm[f"s_w_{name}"]))
+        self.s_w = {n: d(prm[f"s_w_{n}"]) for n in ("proj", "fc1", "fc2")}
+        self.bias = {n: d(prm[f"b_{n}"]) for n in ("proj", "fc1", "fc2")}
+        seg = np.concatenate([np.full(D, prm["s_q"]), np.full(D, prm["s_k"]), np.full(D, prm["s_v"])]).astype(np.float32)
+        a, b = B.fold_requant(prm["s_ln"], prm["s_w_qkv"], prm["b_qkv"], seg)
+        self.alpha_qkv, self.beta_qkv = d(a), d(b)
+        a, _ = B.fold_requant(prm["s_p"], np.full(D, prm["s_v"], np.float32), None, prm["s_o"])
+        self.alpha_o = d(a)
+        self.inv_s_g = d((1.0 / np.full(F, prm["s_g"], np.float64)).astype(np.float32))
+        self.c = float(np.float32(float(prm["s_q"]) * float(prm["s_k"]) / 8.0))
+        # activations
+        self.x1 = B.Codes.empty(M, D, bits, True, device)
+        self.qkv = B.Codes.empty(M, 3 * D, bits, True, device)
+        self.ld_s = (tokens + 3) // 4 * 4
+        self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
+        self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
+        self.O = B.Codes.empty(M, D, bits, True, device)
+        self.h = torch.empty((M, D), dtype=torch.float32, device=device)
+        self.x2 = B.Codes.empty(M, D, bits, True, device)
+        self.g = B.Codes.empty(M, F, bits, False, device)
+        self.slabs = [B.Slabs.of_qkv(self.qkv, tokens, D, i) for i in range(3)]
+        self.epi_qkv = B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_qkv, beta=self.beta_qkv, out_bits=bits,
+                                  out_signed=True)
+        self.epi_o = B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_o, out_bits=bits, out_signed=True)
+        self.epi_fc1 = B.Epilogue(mode=B.EPI_REQUANT, act=1, inv_out_step=self.inv_s_g, out_bits=bits, out_signed=False)
+
+    def forward(self, x: torch.Tensor, out: torch.Tensor, events: list | None = None) -> torch.Tensor:
+        """x, out: fp32 [batch*tokens, dim] on the device.  `events`, when given, receives
+        len(STAGES)+1 recorded CUDA events bracketing the stages."""
+        def mark():
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record()
+                events.append(e)
+        b, t, h = self.batch, self.tokens, self.heads
+        mark()
+        B.vitint_layernorm_quantize(x, self.ln1_g, self.ln1_b, self.eps, self.s_ln, self.bits, True, out=self.x1)
+        mark()
+        B.vitint_linear(self.x1, self.s_ln, self.w["qkv"], None, None, self.epi_qkv, out=self.qkv)
+        mark()
+        B.vitint_qk(self.slabs[0], self.slabs[1], b, h, t, out=self.S, ld_s=self.ld_s)
+        mark()
+        B.vitint_softmax_quantize(self.S, t, self.c, self.s_p, self.bits, out=self.P)
+        mark()
+        B.vitint_pv(self.P, self.slabs[2], b, h, t, self.s_p, self.s_v, self.epi_o, out=self.O)
+        mark()
+        B.vitint_linear(self.O, self.s_o, self.w["proj"], self.s_w["proj"], self.bias["proj"],
+                        B.Epilogue(mode=B.EPI_DEQUANT_F32, residual=x), out=self.h)
+        mark()
+        B.vitint_layernorm_quantize(self.h, self.ln2_g, self.ln2_b, self.eps, self.s_ln, self.bits, True, out=self.x2)
+        mark()
+        B.vitint_linear(self.x2, self.s_ln, self.w["fc1"], self.s_w["fc1"], self.bias["fc1"], self.epi_fc1, out=self.g)
+        mark()
+        B.vitint_linear(self.g, self.s_g, self.w["fc2"], self.s_w["fc2"], self.bias["fc2"],
+                        B.Epilogue(mode=B.EPI_DEQUANT_F32, residual=self.h), out=out)
+        mark()
+        return out
+
+    def stage_ops(self) -> dict:
+        """Integer operations (2 per multiply-accumulate, true shapes) of each contraction."""
+        M, D, F, T = self.rows, self.dim, self.mlp_dim, self.tokens
+        n = self.batch * self.heads
+        return {"qkv_linear": 2 * M * D * 3 * D, "qk": 2 * n * T * T * 64, "pv": 2 * n * T * T * 64,
+                "proj_linear": 2 * M * D * D, "fc1_linear": 2 * M * D * F, "fc2_linear": 2 * M * F * D}
+
+    def stage_bytes(self) -> dict:
+        """Algorithmic HBM bytes of the streaming stages (4 + c/8 per element)."""
+        c = 4 if self.bits == 3 else self.bits
+        M, D, T = self.rows, self.dim, self.tokens
+        n = self.batch * self.heads * T
+        return {"ln1_quant": M * D * 4 + M * D * c // 8, "ln2_quant": M * D * 4 + M * D * c // 8,
+                "softmax_quant": n * T * 4 + n * ((T * c + 7) // 8)}

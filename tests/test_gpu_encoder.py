@@ -1,0 +1,78 @@
+"""GPU parity of the whole integerized ViT-Base encoder layer, stage by stage.
+
+Stages downstream of an fp32 island (LayerNorm, softmax, GELU) may legitimately differ by one
+code on near-ties.  Each stage is therefore compared on exactly those images / token rows whose
+upstream codes were identical on both sides; there the comparison is bit-exact (or inside the
+oracle's band for the stage's own fp32 decision).  The excluded fraction must stay small.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as vo
+import synth_inputs as si
+from oracle import pipeline as vp
+
+pytestmark = pytest.mark.gpu
+vt = pytest.importorskip("paper_2504_18547_b200")
+from gpu_util import dev, from_codes  # noqa: E402
+
+
+@pytest.mark.parametrize("bits", [4, 3, 2])
+def test_encoder_layer_staged(bits):
+    from paper_2504_18547_b200.encoder import EncoderLayer
+    cfg = si.VIT_BASE_LAYER.with_(batch=3, bits=bits)
+    prm = si.layer_parameters(cfg)
+    x = si.activations(cfg)
+    st = vp.encoder_layer(x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits)
+    att = st["attn"]
+    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm)
+    out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
+    layer.forward(dev(x), out)
+    assert vt.vitint_device_status() == 0
+    T, H, B, D = cfg.tokens, cfg.heads, cfg.batch, cfg.dim
+    # weights quantized by the library equal the oracle's
+    assert np.array_equal(from_codes(layer.w["qkv"]), att["w_qkv_codes"])
+    assert np.array_equal(from_codes(layer.w["fc2"]), st["w_fc2_codes"])
+
+    x1 = from_codes(layer.x1)
+    assert np.all(x1 >= st["x1_lo"]) and np.all(x1 <= st["x1_hi"])
+    img_ok = np.array([(x1[b * T:(b + 1) * T] == st["x1_codes"][b * T:(b + 1) * T]).all() for b in range(B)])
+    assert img_ok.sum() >= 2
+    rows_img = np.repeat(img_ok, T)
+
+    qkv = from_codes(layer.qkv)
+    assert np.array_equal(qkv[rows_img], att["qkv_codes"][rows_img])
+
+    P = from_codes(layer.P).reshape(B * H, T, T)
+    prob_ok = np.repeat(img_ok, H)
+    assert np.all(P[prob_ok] >= att["p_lo"][prob_ok]) and np.all(P[prob_ok] <= att["p_hi"][prob_ok])
+    p_row_ok = (P == att["p_codes"]).all(axis=2) & prob_ok[:, None]           # [B*H, T]
+    assert p_row_ok[prob_ok].mean() > 0.97
+
+    O = from_codes(layer.O)
+    tok_ok = np.ones(B * T, bool)
+    for b in range(B):
+        for h in range(H):
+            sel = p_row_ok[b * H + h]
+            blk = slice(b * T, (b + 1) * T)
+            assert np.array_equal(O[blk, h * 64:(h + 1) * 64][sel], att["o_codes"][blk, h * 64:(h + 1) * 64][sel])
+            tok_ok[blk] &= sel
+    assert tok_ok.mean() > 0.5
+
+    hh = layer.h.cpu().numpy()
+    assert np.array_equal(hh[tok_ok].view(np.uint32), st["h"][tok_ok].view(np.uint32))
+
+    x2 = from_codes(layer.x2)
+    assert np.all(x2[tok_ok] >= st["x2_lo"][tok_ok]) and np.all(x2[tok_ok] <= st["x2_hi"][tok_ok])
+    tok_ok2 = tok_ok & (x2 == st["x2_codes"]).all(axis=1)
+
+    g = from_codes(layer.g)
+    assert np.all(g[tok_ok2] >= st["g_lo"][tok_ok2]) and np.all(g[tok_ok2] <= st["g_hi"][tok_ok2])
+    tok_ok3 = tok_ok2 & (g == st["g_codes"]).all(axis=1)
+    assert tok_ok3.mean() > 0.4
+
+    o = out.cpu().numpy()
+    assert np.array_equal(o[tok_ok3].view(np.uint32), st["out"][tok_ok3].view(np.uint32))
+    # everything else stays close: one code flip moves an output by a few steps at most
+    assert np.abs(o - st["out"]).max() < 0.5
