@@ -111,6 +111,13 @@ int64_t vitint_packed_pitch(int64_t cols, int32_t bits);
 int vitint_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, float step, const float* row_steps,
                     const vitint_codes* out, void* stream);
 
+/* Re-stores b-bit codes in 8-bit containers (same values, same signedness): out->bits must be 8,
+ *   rows/cols equal to the input's.  Weights widened once this way let vitint_linear feed the
+ *   tensor cores straight from the TMA copy, with no in-kernel unpacking of that operand; the
+ *   value range of the codes is unchanged, so Eq. 1's integer contraction is the same.
+ *   Errors: INVALID_ARG, ALIGNMENT. */
+int vitint_widen(const vitint_codes* in, const vitint_codes* out, void* stream);
+
 /* a2 + a3. Integerized linear layer (Eq. 1-2): acc[m][n] = sum_k q_x[m][k] * q_w[n][k]
  *   in int32, then the epilogue above.
  *   x: codes [M, K];  w: codes [N, K] (one row per output channel);  w_step: device [N]

@@ -62,6 +62,7 @@ def lib():
         L.vitint_packed_pitch.restype = c_int64
         L.vitint_packed_pitch.argtypes = [c_int64, c_int32]
         L.vitint_quantize.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_float, c_void_p, POINTER(_Codes), c_void_p]
+        L.vitint_widen.argtypes = [POINTER(_Codes), POINTER(_Codes), c_void_p]
         L.vitint_linear.argtypes = [POINTER(_Codes), c_float, POINTER(_Codes), c_void_p, c_void_p, POINTER(_Epilogue),
                                     c_void_p, c_int64, c_void_p]
         L.vitint_qk.argtypes = [POINTER(_Slabs), POINTER(_Slabs), c_int32, c_int32, c_int32, c_void_p, c_int64, c_void_p]
@@ -201,6 +202,14 @@ def vitint_quantize(x: torch.Tensor, step: float, bits: int, signed: bool, row_s
     d = out.desc()
     _check(lib().vitint_quantize(x.data_ptr(), rows, cols, _ld(x), float(step), _ptr(row_steps), byref(d),
                                  _stream()), "vitint_quantize")
+    return out
+
+
+def vitint_widen(x: Codes, out: Codes | None = None) -> Codes:
+    """The same codes in 8-bit containers (used once for weights)."""
+    out = Codes.empty(x.rows, x.cols, 8, x.signed, x.data.device) if out is None else out
+    di, do = x.desc(), out.desc()
+    _check(lib().vitint_widen(byref(di), byref(do), _stream()), "vitint_widen")
     return out
 
 

@@ -3,9 +3,11 @@
 // post-contraction epilogue of Eq. 2.
 //
 // One persistent CTA per SM walks 128 x BN output tiles.  Warp roles:
-//   warps 0-3  epilogue: tcgen05.ld of their 32 TMEM lanes, rescale / bias / GELU /
-//              requantize / pack, global stores (warp w owns TMEM lanes 32w..32w+31);
-//   warp  4    TMA producer: packed low-bit tiles of A and B -> shared memory ring;
+//   warps 0-3  epilogue: stage the tile's per-column scale / bias in shared memory,
+//              tcgen05.ld of their 32 TMEM lanes, rescale / bias / GELU / requantize /
+//              pack, global stores (warp w owns TMEM lanes 32w..32w+31);
+//   warp  4    TMA producer: packed low-bit tiles -> shared-memory ring; operands that are
+//              already 8-bit go straight into the swizzled int8 operand ring;
 //   warp  5    MMA issuer (one thread) and owner of the TMEM allocation;
 //   warps 6-9  unpack: packed codes -> int8 operand tiles in the shared-memory layout
 //              the tensor core expects (128-byte swizzle, K contiguous; or 64-byte
@@ -15,8 +17,9 @@
 //
 // Sign handling without sign extension: a signed c-bit code q is placed in the HIGH
 // bits of its byte, i.e. the int8 value is q * 2^(8-c).  The contraction then yields
-// acc * 2^shift exactly and the epilogue shifts it back (host checks that the scaled
-// sum still fits in int32).  Unsigned codes are placed in the low bits unscaled.
+// acc * 2^shift exactly (host checks that the scaled sum still fits in int32); the
+// epilogue folds 2^-shift into the per-column multiplier, which is exact in binary
+// floating point, or shifts the integer back when raw accumulators are requested.
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -30,16 +33,20 @@ constexpr int EPI_WARPS = 4;
 constexpr int UNPACK_WARPS = 4;
 constexpr int WARP_TMA = 4, WARP_MMA = 5, WARP_UNPACK0 = 6;
 constexpr int NUM_THREADS = (WARP_UNPACK0 + UNPACK_WARPS) * 32;
-constexpr int MAX_STAGES = 6;
+constexpr int MAX_STAGES = 8;
+constexpr int MAX_BN = 256;
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000ll;   // about one second
+
+enum EpiKind { EK_ACC = 0, EK_DEQUANT = 1, EK_DEQUANT_GELU = 2, EK_REQUANT = 3, EK_REQUANT_GELU = 4 };
 
 struct GemmParams {
     int M, N, K;
     int bn, m_tiles, n_tiles, n_inner, total_tiles, k_blocks;
     int ca, cb, a_signed, b_signed, shift, b_mn_major;
+    int a_direct, b_direct;            // operand already int8: TMA writes the operand ring itself
     int ns_i, ns_p;
     uint32_t ia_bytes, ib_bytes, pa_bytes, pb_bytes, tmem_cols;
-    int mode, act, out_c;
+    int kind, out_c;
     float out_qn, out_qp, x_step;
     void* out;
     long long ld_out, row_off_outer, row_off_inner, col_off_inner;
@@ -52,7 +59,11 @@ struct GemmParams {
 
 struct Bars {
     uint64_t p_full[MAX_STAGES], p_empty[MAX_STAGES], i_full[MAX_STAGES], i_empty[MAX_STAGES];
-    uint64_t acc_full[2], acc_empty[2];
+    uint64_t acc_full[2], acc_empty[2], epi_sync;
+};
+
+struct EpiParams {                      // per-column epilogue parameters of the two tiles in flight
+    float a[2][MAX_BN], b[2][MAX_BN], q[2][MAX_BN];
 };
 
 // Bounded wait.  Gives up after WAIT_LIMIT_CYCLES or as soon as another thread of the CTA
@@ -74,17 +85,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 }
 
 // 8 four-bit codes of one word -> 8 bytes in natural order.
-__device__ __forceinline__ void unpack4(uint32_t w, int sgn, uint32_t& o0, uint32_t& o1) {
+template <int SGN>
+__device__ __forceinline__ void unpack4(uint32_t w, uint32_t& o0, uint32_t& o1) {
     uint32_t lo, hi;
-    if (sgn) { lo = (w << 4) & 0xF0F0F0F0u; hi = w & 0xF0F0F0F0u; }
+    if (SGN) { lo = (w << 4) & 0xF0F0F0F0u; hi = w & 0xF0F0F0F0u; }
     else     { lo = w & 0x0F0F0F0Fu;        hi = (w >> 4) & 0x0F0F0F0Fu; }
     o0 = __byte_perm(lo, hi, 0x5140);
     o1 = __byte_perm(lo, hi, 0x7362);
 }
 // 16 two-bit codes of one word -> 16 bytes in natural order.
-__device__ __forceinline__ uint4 unpack2(uint32_t w, int sgn) {
+template <int SGN>
+__device__ __forceinline__ uint4 unpack2(uint32_t w) {
     uint32_t p0, p1, p2, p3;
-    if (sgn) {
+    if (SGN) {
         p0 = (w << 6) & 0xC0C0C0C0u; p1 = (w << 4) & 0xC0C0C0C0u; p2 = (w << 2) & 0xC0C0C0C0u; p3 = w & 0xC0C0C0C0u;
     } else {
         p0 = w & 0x03030303u; p1 = (w >> 2) & 0x03030303u; p2 = (w >> 4) & 0x03030303u; p3 = (w >> 6) & 0x03030303u;
@@ -95,37 +108,67 @@ __device__ __forceinline__ uint4 unpack2(uint32_t w, int sgn) {
                       __byte_perm(c, d, 0x7632));
 }
 
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
-                 : "memory");
+// One 16-byte chunk of packed codes -> 8/C chunks of int8 written at dst[oc ^ sw], oc = oc0 .. oc0 + 8/C - 1.
+// `row` points at the first chunk slot of the destination row; `sw` is the row's swizzle mask.
+template <int C, int SGN>
+__device__ __forceinline__ void expand_chunk(uint4 in, uint8_t* row, int oc0, int sw) {
+    if (C == 4) {
+        uint4 o0, o1;
+        unpack4<SGN>(in.x, o0.x, o0.y);
+        unpack4<SGN>(in.y, o0.z, o0.w);
+        unpack4<SGN>(in.z, o1.x, o1.y);
+        unpack4<SGN>(in.w, o1.z, o1.w);
+        *reinterpret_cast<uint4*>(row + ((oc0 ^ sw) << 4)) = o0;
+        *reinterpret_cast<uint4*>(row + (((oc0 + 1) ^ sw) << 4)) = o1;
+    } else if (C == 2) {
+        *reinterpret_cast<uint4*>(row + ((oc0 ^ sw) << 4)) = unpack2<SGN>(in.x);
+        *reinterpret_cast<uint4*>(row + (((oc0 + 1) ^ sw) << 4)) = unpack2<SGN>(in.y);
+        *reinterpret_cast<uint4*>(row + (((oc0 + 2) ^ sw) << 4)) = unpack2<SGN>(in.z);
+        *reinterpret_cast<uint4*>(row + (((oc0 + 3) ^ sw) << 4)) = unpack2<SGN>(in.w);
+    } else {
+        *reinterpret_cast<uint4*>(row + ((oc0 ^ sw) << 4)) = in;
+    }
 }
 
-// Expands one 16-byte chunk of packed codes and stores the resulting 8/C chunks of int8.
-// out_addr(oc) gives the shared-memory address of output chunk oc (0-based within the
-// 16-byte input chunk's span).
-template <typename AddrFn>
-__device__ __forceinline__ void expand_chunk(uint4 in, int c, int sgn, AddrFn out_addr) {
-    if (c == 4) {
-        uint4 o0, o1;
-        unpack4(in.x, sgn, o0.x, o0.y);
-        unpack4(in.y, sgn, o0.z, o0.w);
-        unpack4(in.z, sgn, o1.x, o1.y);
-        unpack4(in.w, sgn, o1.z, o1.w);
-        sts128(out_addr(0), o0);
-        sts128(out_addr(1), o1);
-    } else if (c == 2) {
-        sts128(out_addr(0), unpack2(in.x, sgn));
-        sts128(out_addr(1), unpack2(in.y, sgn));
-        sts128(out_addr(2), unpack2(in.z, sgn));
-        sts128(out_addr(3), unpack2(in.w, sgn));
-    } else {
-        sts128(out_addr(0), in);
+// K-contiguous operand tile: `rows` rows of 16*C packed bytes -> rows of 128 int8, 128-byte swizzle.
+template <int C, int SGN>
+__device__ __forceinline__ void unpack_k_major(const uint8_t* src, uint8_t* dst, int rows, int tid, int nthreads) {
+    constexpr int LC = C == 2 ? 1 : (C == 4 ? 2 : 3);   // log2(packed chunks per row)
+    constexpr int E = 8 / C;
+    const int chunks = rows << LC;
+#pragma unroll 2
+    for (int q = tid; q < chunks; q += nthreads) {
+        const int r = q >> LC, j = q & ((1 << LC) - 1);
+        const uint4 in = *reinterpret_cast<const uint4*>(src + (size_t)q * 16);
+        expand_chunk<C, SGN>(in, dst + r * 128, j * E, r & 7);
     }
+}
+// N-contiguous B tile (the V operand): 128 rows of K, 64 codes each -> rows of 64 int8 grouped
+// by 8 rows (512 bytes), 64-byte swizzle.
+template <int C, int SGN>
+__device__ __forceinline__ void unpack_mn_major(const uint8_t* src, uint8_t* dst, int tid, int nthreads) {
+    constexpr int LH = C == 2 ? 0 : (C == 4 ? 1 : 2);   // log2(packed chunks per 64-code row)
+    constexpr int E = 8 / C;
+    const int chunks = BK << LH;
+#pragma unroll 2
+    for (int q = tid; q < chunks; q += nthreads) {
+        const int r = q >> LH, h = q & ((1 << LH) - 1);
+        const uint4 in = *reinterpret_cast<const uint4*>(src + (size_t)q * 16);
+        expand_chunk<C, SGN>(in, dst + (r >> 3) * 512 + (r & 7) * 64, h * E, (r >> 1) & 3);
+    }
+}
+
+template <int SGN>
+__device__ __forceinline__ void unpack_k_major_c(int c, const uint8_t* src, uint8_t* dst, int rows, int tid, int nt) {
+    if (c == 4) unpack_k_major<4, SGN>(src, dst, rows, tid, nt);
+    else if (c == 2) unpack_k_major<2, SGN>(src, dst, rows, tid, nt);
+    else unpack_k_major<8, SGN>(src, dst, rows, tid, nt);
+}
+template <int SGN>
+__device__ __forceinline__ void unpack_mn_major_c(int c, const uint8_t* src, uint8_t* dst, int tid, int nt) {
+    if (c == 4) unpack_mn_major<4, SGN>(src, dst, tid, nt);
+    else if (c == 2) unpack_mn_major<2, SGN>(src, dst, tid, nt);
+    else unpack_mn_major<8, SGN>(src, dst, tid, nt);
 }
 
 __device__ __forceinline__ void tile_coords(const GemmParams& P, int tile, int& m_tile, int& n_tile, int& inner,
@@ -139,68 +182,95 @@ __device__ __forceinline__ void tile_coords(const GemmParams& P, int tile, int& 
     inner = prob - outer * P.n_inner;
 }
 
-// Epilogue of one row x 32 columns: accumulators v[] (scaled by 2^shift) -> output.
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32_t (&v)[32], long long orow,
-                                               long long colbase, int n0) {
-    const int out_words = P.out_c;   // 32 codes = 4*out_c bytes = out_c words
-    const bool full = n0 + 32 <= P.N;
-    if (P.mode == VITINT_EPI_ACC_I32) {
+// Barrier among the 128 epilogue threads, bounded like every other wait (an mbarrier with one
+// phase per tile instead of bar.sync, which could not give up).
+__device__ __forceinline__ bool epi_barrier(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    ptx::mbar_arrive(bar);
+    return mbar_wait(bar, parity, abort_flag);
+}
+
+// Epilogue of one row x 32 columns.  v[]: accumulators scaled by 2^shift; pa/pb/pq: the 32
+// columns' parameters in shared memory (multiplier already carries 2^-shift).
+// FULL: all 32 columns exist and 16-byte vector accesses are legal.
+template <int KIND, bool FULL>
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32_t (&v)[32], const float* pa,
+                                               const float* pb, const float* pq, long long orow, long long colbase,
+                                               int n0) {
+    const int nvalid = FULL ? 32 : (P.N - n0 < 32 ? P.N - n0 : 32);
+    if (KIND == EK_ACC) {
         int32_t* o = (int32_t*)P.out + orow * P.ld_out + colbase + n0;
-        if (full && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
+        if (FULL) {
 #pragma unroll
             for (int i = 0; i < 8; ++i)
                 reinterpret_cast<int4*>(o)[i] = make_int4((int)v[4 * i] >> P.shift, (int)v[4 * i + 1] >> P.shift,
                                                           (int)v[4 * i + 2] >> P.shift, (int)v[4 * i + 3] >> P.shift);
         } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) if (n0 + i < P.N) o[i] = (int)v[i] >> P.shift;
+            for (int i = 0; i < 32; ++i) if (i < nvalid) o[i] = (int)v[i] >> P.shift;
         }
         return;
     }
-    // fp32 value per column
     float y[32];
+    // residual first: independent 16-byte loads in flight while the arithmetic runs
+    float res[32];
+    const bool has_res = (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU) && P.residual != nullptr;
+    if (has_res) {
+        const float* r = P.residual + orow * P.ld_res + colbase + n0;
+        if (FULL && ((reinterpret_cast<uintptr_t>(r) & 15u) == 0)) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        const bool valid = n0 + i < P.N;
-        const long long cidx = colbase + n0 + i;
-        const float f = (float)((int)v[i] >> P.shift);
-        float val = 0.0f;
-        if (valid) {
-            if (P.mode == VITINT_EPI_REQUANT && P.act == 0) {
-                val = fmaf(f, __ldg(P.col_a + cidx), P.col_b ? __ldg(P.col_b + cidx) : 0.0f);
-            } else {
-                const float sc = P.col_a ? __fmul_rn(P.x_step, __ldg(P.col_a + cidx)) : P.x_step;
-                val = fmaf(f, sc, P.col_b ? __ldg(P.col_b + cidx) : 0.0f);
-                if (P.act == 1) val = gelu_f32(val);
-                if (P.mode == VITINT_EPI_REQUANT) val = val * __ldg(P.inv_s + cidx);
-                else if (P.residual) val = val + __ldg(P.residual + orow * P.ld_res + cidx);
+            for (int i = 0; i < 8; ++i) {
+                const float4 t = __ldg(reinterpret_cast<const float4*>(r) + i);
+                res[4 * i] = t.x; res[4 * i + 1] = t.y; res[4 * i + 2] = t.z; res[4 * i + 3] = t.w;
             }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) res[i] = (i < nvalid) ? __ldg(r + i) : 0.0f;
         }
-        y[i] = val;
     }
-    if (P.mode == VITINT_EPI_DEQUANT_F32) {
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4) {
+        const float4 a4 = *reinterpret_cast<const float4*>(pa + 4 * i4);
+        const float4 b4 = *reinterpret_cast<const float4*>(pb + 4 * i4);
+        const float aa[4] = {a4.x, a4.y, a4.z, a4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w};
+        float qq[4] = {0.f, 0.f, 0.f, 0.f};
+        if (KIND == EK_REQUANT_GELU) {
+            const float4 q4 = *reinterpret_cast<const float4*>(pq + 4 * i4);
+            qq[0] = q4.x; qq[1] = q4.y; qq[2] = q4.z; qq[3] = q4.w;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = 4 * i4 + j;
+            float val = fmaf((float)(int)v[i], aa[j], bb[j]);
+            if (KIND == EK_DEQUANT_GELU || KIND == EK_REQUANT_GELU) val = gelu_f32(val);
+            if (KIND == EK_REQUANT_GELU) val = val * qq[j];
+            if (has_res) val = val + res[i];
+            y[i] = val;
+        }
+    }
+    if (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU) {
         float* o = (float*)P.out + orow * P.ld_out + colbase + n0;
-        if (full && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
+        if (FULL && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
 #pragma unroll
             for (int i = 0; i < 8; ++i)
                 reinterpret_cast<float4*>(o)[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
         } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) if (n0 + i < P.N) o[i] = y[i];
+            for (int i = 0; i < 32; ++i) if (i < nvalid) o[i] = y[i];
         }
         return;
     }
-    // REQUANT: 32 codes -> out_c words
+    // REQUANT: 32 codes -> out_c 32-bit words
     uint32_t wds[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     const uint32_t mask = (1u << P.out_c) - 1u;
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-        const uint32_t code = (n0 + i < P.N) ? ((uint32_t)round_clamp(y[i], P.out_qn, P.out_qp) & mask) : 0u;
+        const uint32_t code = (FULL || i < nvalid) ? ((uint32_t)round_clamp(y[i], P.out_qn, P.out_qp) & mask) : 0u;
         // static word index for each container width keeps wds[] in registers
         if (P.out_c == 4) wds[i >> 3] |= code << (4 * (i & 7));
         else if (P.out_c == 2) wds[i >> 4] |= code << (2 * (i & 15));
         else wds[i >> 2] |= code << (8 * (i & 3));
     }
+    const int out_words = P.out_c;   // 32 codes = 4*out_c bytes
     const long long byte0 = ((colbase + n0) * P.out_c) >> 3;
     uint8_t* o = (uint8_t*)P.out + orow * P.ld_out + byte0;
     if (P.out_c == 4 && byte0 + 16 <= P.ld_out) {
@@ -211,9 +281,30 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
             if (k < out_words && byte0 + 4 * k + 4 <= P.ld_out) reinterpret_cast<uint32_t*>(o)[k] = wds[k];
     }
     // row padding behind the last chunk of the last column tile
-    if (P.col_off_inner == 0 && n0 + 32 >= P.N) {
-        for (long long off = byte0 + 4 * out_words; off + 4 <= P.ld_out; off += 4)
-            *reinterpret_cast<uint32_t*>((uint8_t*)P.out + orow * P.ld_out + off) = 0u;
+    if (!FULL || (P.col_off_inner == 0 && n0 + 32 >= P.N)) {
+        if (P.col_off_inner == 0)
+            for (long long off = byte0 + 4 * out_words; off + 4 <= P.ld_out; off += 4)
+                *reinterpret_cast<uint32_t*>((uint8_t*)P.out + orow * P.ld_out + off) = 0u;
+    }
+}
+
+template <int KIND>
+__device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiParams& ep, int buf, uint32_t t_row,
+                                              bool row_ok, long long orow, long long colbase, int n_tile) {
+    for (int chunk = 0; chunk * 32 < P.bn; ++chunk) {
+        const int n0 = n_tile * P.bn + chunk * 32;
+        if (n0 >= P.N) break;
+        uint32_t v[32];
+        ptx::tmem_ld32(t_row + (uint32_t)(chunk * 32), v);
+        ptx::tmem_ld_wait();
+        if (row_ok) {
+            const float* pa = &ep.a[buf][chunk * 32];
+            const float* pb = &ep.b[buf][chunk * 32];
+            const float* pq = &ep.q[buf][chunk * 32];
+            if (n0 + 32 <= P.N) epilogue_chunk<KIND, true>(P, v, pa, pb, pq, orow, colbase, n0);
+            else epilogue_chunk<KIND, false>(P, v, pa, pb, pq, orow, colbase, n0);
+        }
+        __syncwarp();
     }
 }
 
@@ -222,13 +313,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                const __grid_constant__ GemmParams P) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ Bars bars;
+    __shared__ __align__(16) EpiParams epi_params;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+    uint8_t* const smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
     const uint32_t stage_i = P.ia_bytes + P.ib_bytes, stage_p = P.pa_bytes + P.pb_bytes;
-    const uint32_t packed_base = smem_base + (uint32_t)P.ns_i * stage_i;
+    const uint32_t packed_off = (uint32_t)P.ns_i * stage_i;
+    const bool any_packed = !(P.a_direct && P.b_direct), any_direct = P.a_direct || P.b_direct;
     volatile int* abort_ptr = &abort_flag;
 
     if (threadIdx.x == 0) {
@@ -236,13 +330,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int s = 0; s < MAX_STAGES; ++s) {
             ptx::mbar_init(ptx::smem_addr(&bars.p_full[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&bars.p_empty[s]), UNPACK_WARPS);
-            ptx::mbar_init(ptx::smem_addr(&bars.i_full[s]), UNPACK_WARPS);
+            ptx::mbar_init(ptx::smem_addr(&bars.i_full[s]), (any_packed ? UNPACK_WARPS : 0) + (any_direct ? 1 : 0));
             ptx::mbar_init(ptx::smem_addr(&bars.i_empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(ptx::smem_addr(&bars.acc_full[b]), 1);
             ptx::mbar_init(ptx::smem_addr(&bars.acc_empty[b]), EPI_WARPS);
         }
+        ptx::mbar_init(ptx::smem_addr(&bars.epi_sync), EPI_WARPS * 32);
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
     }
@@ -265,29 +360,46 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
             int it = 0;
             bool ok = true;
+            const uint32_t packed_bytes = (P.a_direct ? 0u : P.pa_bytes) + (P.b_direct ? 0u : P.pb_bytes);
+            const uint32_t direct_bytes = (P.a_direct ? P.ia_bytes : 0u) + (P.b_direct ? P.ib_bytes : 0u);
             for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
                 int m_tile, n_tile, inner, outer;
                 tile_coords(P, tile, m_tile, n_tile, inner, outer);
                 for (int kb = 0; kb < P.k_blocks; ++kb, ++it) {
-                    const int s = it % P.ns_p;
-                    const uint32_t ph = (uint32_t)(it / P.ns_p) & 1u;
-                    if (!mbar_wait(ptx::smem_addr(&bars.p_empty[s]), ph ^ 1u, abort_ptr)) { ok = false; break; }
-                    const uint32_t full = ptx::smem_addr(&bars.p_full[s]);
-                    ptx::mbar_arrive_expect_tx(full, stage_p);
-                    const uint32_t dst = packed_base + (uint32_t)s * stage_p;
-                    ptx::tma_load_4d(dst, &map_a, full, kb * 16 * P.ca, m_tile * BM, inner, outer);
-                    if (P.b_mn_major)
-                        ptx::tma_load_4d(dst + P.pa_bytes, &map_b, full, 0, kb * BK, inner, outer);
+                    const int sp = it % P.ns_p, si = it % P.ns_i;
+                    const uint32_t php = (uint32_t)(it / P.ns_p) & 1u, phi = (uint32_t)(it / P.ns_i) & 1u;
+                    const uint32_t p_full = ptx::smem_addr(&bars.p_full[sp]), i_full = ptx::smem_addr(&bars.i_full[si]);
+                    const uint32_t p_dst = smem_base + packed_off + (uint32_t)sp * stage_p;
+                    const uint32_t i_dst = smem_base + (uint32_t)si * stage_i;
+                    if (any_packed) {
+                        if (!mbar_wait(ptx::smem_addr(&bars.p_empty[sp]), php ^ 1u, abort_ptr)) { ok = false; break; }
+                        ptx::mbar_arrive_expect_tx(p_full, packed_bytes);
+                    }
+                    if (any_direct) {
+                        if (!mbar_wait(ptx::smem_addr(&bars.i_empty[si]), phi ^ 1u, abort_ptr)) { ok = false; break; }
+                        ptx::mbar_arrive_expect_tx(i_full, direct_bytes);
+                    }
+                    if (P.a_direct) ptx::tma_load_4d(i_dst, &map_a, i_full, kb * BK, m_tile * BM, inner, outer);
+                    else ptx::tma_load_4d(p_dst, &map_a, p_full, kb * 16 * P.ca, m_tile * BM, inner, outer);
+                    if (P.b_direct)
+                        ptx::tma_load_4d(i_dst + P.ia_bytes, &map_b, i_full, kb * BK, n_tile * P.bn, inner, outer);
+                    else if (P.b_mn_major)
+                        ptx::tma_load_4d(p_dst + P.pa_bytes, &map_b, p_full, 0, kb * BK, inner, outer);
                     else
-                        ptx::tma_load_4d(dst + P.pa_bytes, &map_b, full, kb * 16 * P.cb, n_tile * P.bn, inner, outer);
+                        ptx::tma_load_4d(p_dst + P.pa_bytes, &map_b, p_full, kb * 16 * P.cb, n_tile * P.bn, inner, outer);
                 }
             }
             if (!ok) {
                 // give the copies still in flight a bounded chance to land before the CTA exits
-                for (int j = (it > P.ns_p ? it - P.ns_p : 0); j < it; ++j) {
-                    const uint32_t bar = ptx::smem_addr(&bars.p_full[j % P.ns_p]);
-                    const uint32_t ph = (uint32_t)(j / P.ns_p) & 1u;
-                    for (int spin = 0; spin < (1 << 20) && !ptx::mbar_try_wait(bar, ph); ++spin) {}
+                for (int j = (it > MAX_STAGES ? it - MAX_STAGES : 0); j < it; ++j) {
+                    if (any_packed && j + P.ns_p >= it) {
+                        const uint32_t bar = ptx::smem_addr(&bars.p_full[j % P.ns_p]);
+                        for (int spin = 0; spin < (1 << 20) && !ptx::mbar_try_wait(bar, (uint32_t)(j / P.ns_p) & 1u); ++spin) {}
+                    }
+                    if (any_direct && j + P.ns_i >= it) {
+                        const uint32_t bar = ptx::smem_addr(&bars.i_full[j % P.ns_i]);
+                        for (int spin = 0; spin < (1 << 20) && !ptx::mbar_try_wait(bar, (uint32_t)(j / P.ns_i) & 1u); ++spin) {}
+                    }
                 }
             }
         }
@@ -329,85 +441,93 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if (warp >= WARP_UNPACK0) {
         // --------------------------------- unpack ----------------------------------
-        const int tid_u = threadIdx.x - WARP_UNPACK0 * 32;
-        constexpr int NU = UNPACK_WARPS * 32;
-        const int la = P.ca == 2 ? 1 : (P.ca == 4 ? 2 : 3);        // log2(chunks per packed A row)
-        const int lb = P.cb == 2 ? 1 : (P.cb == 4 ? 2 : 3);
-        const int ea = 8 / P.ca, eb = 8 / P.cb;                    // int8 chunks per packed chunk
-        const int chunks_a = BM << la;
-        const int chunks_b = P.b_mn_major ? (BK << lb) >> 1 : P.bn << lb;
-        int it = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
-            for (int kb = 0; kb < P.k_blocks; ++kb, ++it) {
-                const int sp = it % P.ns_p, si = it % P.ns_i;
-                const uint32_t php = (uint32_t)(it / P.ns_p) & 1u, phi = (uint32_t)(it / P.ns_i) & 1u;
-                bool w = mbar_wait(ptx::smem_addr(&bars.p_full[sp]), php, abort_ptr);
-                w = w && mbar_wait(ptx::smem_addr(&bars.i_empty[si]), phi ^ 1u, abort_ptr);
-                if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
-                ptx::tc_fence_after();
-                const uint32_t pa = packed_base + (uint32_t)sp * stage_p, pb = pa + P.pa_bytes;
-                const uint32_t ia = smem_base + (uint32_t)si * stage_i, ib = ia + P.ia_bytes;
-                for (int q = tid_u; q < chunks_a; q += NU) {
-                    const int r = q >> la, j = q & ((1 << la) - 1);
-                    const uint32_t row = ia + (uint32_t)r * 128u;
-                    const int oc0 = j * ea, sw = r & 7;
-                    expand_chunk(lds128(pa + (uint32_t)q * 16u), P.ca, P.a_signed,
-                                 [&](int e) { return row + (uint32_t)(((oc0 + e) ^ sw) << 4); });
-                }
-                if (!P.b_mn_major) {
-                    for (int q = tid_u; q < chunks_b; q += NU) {
-                        const int r = q >> lb, j = q & ((1 << lb) - 1);
-                        const uint32_t row = ib + (uint32_t)r * 128u;
-                        const int oc0 = j * eb, sw = r & 7;
-                        expand_chunk(lds128(pb + (uint32_t)q * 16u), P.cb, P.b_signed,
-                                     [&](int e) { return row + (uint32_t)(((oc0 + e) ^ sw) << 4); });
+        if (any_packed) {
+            const int tid_u = threadIdx.x - WARP_UNPACK0 * 32;
+            constexpr int NU = UNPACK_WARPS * 32;
+            int it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+                for (int kb = 0; kb < P.k_blocks; ++kb, ++it) {
+                    const int sp = it % P.ns_p, si = it % P.ns_i;
+                    const uint32_t php = (uint32_t)(it / P.ns_p) & 1u, phi = (uint32_t)(it / P.ns_i) & 1u;
+                    bool w = mbar_wait(ptx::smem_addr(&bars.p_full[sp]), php, abort_ptr);
+                    w = w && mbar_wait(ptx::smem_addr(&bars.i_empty[si]), phi ^ 1u, abort_ptr);
+                    if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint8_t* pa = smem_gen + packed_off + (size_t)sp * stage_p;
+                    const uint8_t* pb = pa + P.pa_bytes;
+                    uint8_t* ia = smem_gen + (size_t)si * stage_i;
+                    uint8_t* ib = ia + P.ia_bytes;
+                    if (!P.a_direct) {
+                        if (P.a_signed) unpack_k_major_c<1>(P.ca, pa, ia, BM, tid_u, NU);
+                        else unpack_k_major_c<0>(P.ca, pa, ia, BM, tid_u, NU);
                     }
-                } else {
-                    // B tile = 128 rows of K, 64 codes of N each: rows of 64 int8, 64-byte swizzle
-                    const int lh = lb - 1;                         // log2(packed chunks per row)
-                    for (int q = tid_u; q < chunks_b; q += NU) {
-                        const int r = q >> lh, h = q & ((1 << lh) - 1);
-                        const uint32_t row = ib + (uint32_t)(r >> 3) * 512u + (uint32_t)(r & 7) * 64u;
-                        const int oc0 = h * eb, sw = (r >> 1) & 3;
-                        expand_chunk(lds128(pb + (uint32_t)q * 16u), P.cb, P.b_signed,
-                                     [&](int e) { return row + (uint32_t)(((oc0 + e) ^ sw) << 4); });
+                    if (!P.b_direct) {
+                        if (!P.b_mn_major) {
+                            if (P.b_signed) unpack_k_major_c<1>(P.cb, pb, ib, P.bn, tid_u, NU);
+                            else unpack_k_major_c<0>(P.cb, pb, ib, P.bn, tid_u, NU);
+                        } else {
+                            if (P.b_signed) unpack_mn_major_c<1>(P.cb, pb, ib, tid_u, NU);
+                            else unpack_mn_major_c<0>(P.cb, pb, ib, tid_u, NU);
+                        }
                     }
-                }
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    ptx::mbar_arrive(ptx::smem_addr(&bars.i_full[si]));
-                    ptx::mbar_arrive(ptx::smem_addr(&bars.p_empty[sp]));
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::mbar_arrive(ptx::smem_addr(&bars.i_full[si]));
+                        ptx::mbar_arrive(ptx::smem_addr(&bars.p_empty[sp]));
+                    }
                 }
             }
         }
     } else {
         // -------------------------------- epilogue ---------------------------------
         const int q4 = warp;   // TMEM lane quarter
+        const int tid_e = threadIdx.x;                       // 0..127
+        const float down = __int_as_float((127 - P.shift) << 23);   // 2^-shift
         int tl = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++tl) {
             int m_tile, n_tile, inner, outer;
             tile_coords(P, tile, m_tile, n_tile, inner, outer);
             const int buf = tl & 1;
+            const long long colbase = (long long)inner * P.col_off_inner;
+            // stage this tile's per-column parameters while its MMAs are still running
+            if (P.kind != EK_ACC) {
+                for (int c = tid_e; c < P.bn; c += EPI_WARPS * 32) {
+                    const int n = n_tile * P.bn + c;
+                    float a = 0.0f, b = 0.0f, q = 0.0f;
+                    if (n < P.N) {
+                        const long long cidx = colbase + n;
+                        if (P.kind == EK_REQUANT) {
+                            a = __ldg(P.col_a + cidx);
+                        } else {
+                            a = P.col_a ? __fmul_rn(P.x_step, __ldg(P.col_a + cidx)) : P.x_step;
+                            if (P.kind == EK_REQUANT_GELU) q = __ldg(P.inv_s + cidx);
+                        }
+                        b = P.col_b ? __ldg(P.col_b + cidx) : 0.0f;
+                        a *= down;
+                    }
+                    epi_params.a[buf][c] = a;
+                    epi_params.b[buf][c] = b;
+                    epi_params.q[buf][c] = q;
+                }
+            }
             const uint32_t acc_ph = (uint32_t)(tl >> 1) & 1u;
-            const bool w = mbar_wait(ptx::smem_addr(&bars.acc_full[buf]), acc_ph, abort_ptr);
+            bool w = P.kind == EK_ACC || epi_barrier(ptx::smem_addr(&bars.epi_sync), (uint32_t)tl & 1u, abort_ptr);
+            w = w && mbar_wait(ptx::smem_addr(&bars.acc_full[buf]), acc_ph, abort_ptr);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
             ptx::tc_fence_after();
             const int row_in_problem = m_tile * BM + q4 * 32 + lane;
             const bool row_ok = row_in_problem < P.M;
             const long long orow = (long long)outer * P.row_off_outer + (long long)inner * P.row_off_inner + row_in_problem;
-            const long long colbase = (long long)inner * P.col_off_inner;
             const uint32_t t_row = tmem_base + (uint32_t)buf * acc_stride + ((uint32_t)(q4 * 32) << 16);
-            for (int chunk = 0; chunk * 32 < P.bn; ++chunk) {
-                const int n0 = n_tile * P.bn + chunk * 32;
-                if (n0 >= P.N) break;
-                uint32_t v[32];
-                ptx::tmem_ld32(t_row + (uint32_t)(chunk * 32), v);
-                ptx::tmem_ld_wait();
-                if (row_ok) epilogue_chunk(P, v, orow, colbase, n0);
-                __syncwarp();
+            switch (P.kind) {
+                case EK_ACC: epilogue_tile<EK_ACC>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
+                case EK_DEQUANT: epilogue_tile<EK_DEQUANT>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
+                case EK_DEQUANT_GELU: epilogue_tile<EK_DEQUANT_GELU>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
+                case EK_REQUANT: epilogue_tile<EK_REQUANT>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
+                default: epilogue_tile<EK_REQUANT_GELU>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
             }
             ptx::tc_fence_before();
             __syncwarp();
@@ -447,7 +567,7 @@ EncodeTiledFn encode_fn() {
 
 // 4-D byte tensor (inner bytes, rows, inner problems, outer problems); out-of-range reads give zero.
 int make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t d3, uint64_t s1,
-             uint64_t s2, uint64_t s3, uint32_t box0, uint32_t box1) {
+             uint64_t s2, uint64_t s3, uint32_t box0, uint32_t box1, bool swizzle128) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return VITINT_ERR_CUDA;
     cuuint64_t dims[4] = {d0, d1, d2, d3};
@@ -455,8 +575,8 @@ int make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint6
     cuuint32_t box[4] = {box0, box1, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? VITINT_OK : VITINT_ERR_CUDA;
 }
 
@@ -479,6 +599,8 @@ int sm_count() {
     return n;
 }
 
+constexpr uint32_t SMEM_TILE_BUDGET = 204u * 1024u;   // dynamic shared memory spent on operand rings
+
 }  // namespace
 
 // Batched NT integer GEMM launcher shared by the linear layer, Q K^T and P V.
@@ -487,12 +609,14 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     const int ca = container_bits(A.bits), cb = container_bits(B.bits);
     P.M = M; P.N = N; P.K = K;
     P.ca = ca; P.cb = cb; P.a_signed = A.is_signed; P.b_signed = B.is_signed; P.b_mn_major = b_mn_major;
+    P.a_direct = ca == 8 ? 1 : 0;
+    P.b_direct = (cb == 8 && !b_mn_major) ? 1 : 0;
     P.shift = (A.is_signed ? 8 - ca : 0) + (B.is_signed ? 8 - cb : 0);
     // exact int32 contraction, also after the power-of-two operand scaling
     const long long bound = (long long)K * max_abs_code(A.bits, A.is_signed) * max_abs_code(B.bits, B.is_signed);
     if (bound >= (1ll << 31)) return VITINT_ERR_OVERFLOW_BOUND;
     if ((bound << P.shift) >= (1ll << 31)) return VITINT_ERR_UNSUPPORTED;
-    int bn = N >= 256 ? 256 : ((N + 15) / 16) * 16;
+    int bn = N >= MAX_BN ? MAX_BN : ((N + 15) / 16) * 16;
     if (b_mn_major) { if (N != 64) return VITINT_ERR_UNSUPPORTED; bn = 64; }
     P.bn = bn;
     P.m_tiles = (M + BM - 1) / BM;
@@ -504,37 +628,50 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     P.k_blocks = (K + BK - 1) / BK;
     P.ia_bytes = BM * BK;
     P.ib_bytes = b_mn_major ? BK * 64 : (uint32_t)bn * BK;
-    P.pa_bytes = BM * 16 * ca;
-    P.pb_bytes = b_mn_major ? BK * 8 * cb : (uint32_t)bn * 16 * cb;
-    const uint32_t per_stage = P.ia_bytes + P.ib_bytes + P.pa_bytes + P.pb_bytes;
-    int ns = (int)((220u * 1024u) / per_stage);
-    if (ns > 4) ns = 4;
-    if (ns < 2) return VITINT_ERR_UNSUPPORTED;
-    P.ns_i = P.ns_p = ns;
+    P.pa_bytes = P.a_direct ? 0u : (uint32_t)(BM * 16 * ca);
+    P.pb_bytes = P.b_direct ? 0u : (b_mn_major ? (uint32_t)(BK * 8 * cb) : (uint32_t)bn * 16 * cb);
+    const uint32_t stage_i = P.ia_bytes + P.ib_bytes, stage_p = P.pa_bytes + P.pb_bytes;
+    // The packed ring hides the global-memory latency of the TMA loads; the int8 ring only
+    // decouples unpack from MMA issue, unless TMA writes it directly.
+    int ns_i, ns_p;
+    if (stage_p == 0) {
+        ns_i = (int)(SMEM_TILE_BUDGET / stage_i);
+        ns_p = 1;
+    } else {
+        ns_i = (P.a_direct || P.b_direct) ? 3 : 2;
+        while (ns_i > 2 && (uint32_t)ns_i * stage_i + 2u * stage_p > SMEM_TILE_BUDGET) --ns_i;
+        if ((uint32_t)ns_i * stage_i + 2u * stage_p > SMEM_TILE_BUDGET) return VITINT_ERR_UNSUPPORTED;
+        ns_p = (int)((SMEM_TILE_BUDGET - (uint32_t)ns_i * stage_i) / stage_p);
+    }
+    if (ns_i > MAX_STAGES) ns_i = MAX_STAGES;
+    if (ns_p > MAX_STAGES) ns_p = MAX_STAGES;
+    if (ns_i < 2) return VITINT_ERR_UNSUPPORTED;
+    P.ns_i = ns_i; P.ns_p = ns_p;
     uint32_t cols = 32;
     while (cols < 2u * (uint32_t)((bn + 31) / 32 * 32)) cols <<= 1;
     P.tmem_cols = cols;
 
     CUtensorMap map_a, map_b;
     if (int rc = make_map(&map_a, A.data, A.row_bytes, A.rows, (uint64_t)n_inner, (uint64_t)n_outer, A.pitch,
-                          A.inner_stride, A.outer_stride, 16u * ca, BM))
+                          A.inner_stride, A.outer_stride, P.a_direct ? (uint32_t)BK : 16u * ca, BM, P.a_direct != 0))
         return rc;
     if (b_mn_major) {
         if (int rc = make_map(&map_b, B.data, B.row_bytes, B.rows, (uint64_t)n_inner, (uint64_t)n_outer, B.pitch,
-                              B.inner_stride, B.outer_stride, 8u * cb, BK))
+                              B.inner_stride, B.outer_stride, 8u * cb, BK, false))
             return rc;
     } else {
         if (int rc = make_map(&map_b, B.data, B.row_bytes, B.rows, (uint64_t)n_inner, (uint64_t)n_outer, B.pitch,
-                              B.inner_stride, B.outer_stride, 16u * cb, (uint32_t)bn))
+                              B.inner_stride, B.outer_stride, P.b_direct ? (uint32_t)BK : 16u * cb, (uint32_t)bn,
+                              P.b_direct != 0))
             return rc;
     }
     // at least ~120 KB so that two CTAs never share an SM (and its tensor memory)
-    size_t smem = (size_t)ns * per_stage + 1024;
+    size_t smem = (size_t)ns_i * stage_i + (size_t)ns_p * stage_p + 1024;
     if (smem < 120 * 1024) smem = 120 * 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)SMEM_TILE_BUDGET + 2048) != cudaSuccess)
             return VITINT_ERR_CUDA;
         attr_set = true;
     }
@@ -547,7 +684,7 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
 static int fill_epilogue(GemmParams& P, const vitint_epilogue* epi, float x_step, const float* w_step,
                          const float* bias, void* out, int64_t ld_out, int64_t n_cols_total) {
     if (!epi || !out) return VITINT_ERR_INVALID_ARG;
-    P.mode = epi->mode; P.act = epi->act; P.out = out; P.ld_out = ld_out;
+    P.out = out; P.ld_out = ld_out;
     P.x_step = x_step; P.col_a = nullptr; P.col_b = nullptr; P.inv_s = nullptr; P.residual = nullptr; P.ld_res = 0;
     P.out_c = 4; P.out_qn = 0; P.out_qp = 0;
     if (epi->act != 0 && epi->act != 1) return VITINT_ERR_INVALID_ARG;
@@ -555,12 +692,14 @@ static int fill_epilogue(GemmParams& P, const vitint_epilogue* epi, float x_step
         case VITINT_EPI_ACC_I32:
             if (epi->act) return VITINT_ERR_INVALID_ARG;
             if (ld_out < n_cols_total || (reinterpret_cast<uintptr_t>(out) & 3u)) return VITINT_ERR_INVALID_ARG;
+            P.kind = EK_ACC;
             break;
         case VITINT_EPI_DEQUANT_F32:
             if (ld_out < n_cols_total || (reinterpret_cast<uintptr_t>(out) & 3u)) return VITINT_ERR_INVALID_ARG;
             if (!(x_step > 0.0f && x_step < INFINITY)) return VITINT_ERR_INVALID_ARG;
             P.col_a = w_step; P.col_b = bias; P.residual = epi->residual; P.ld_res = epi->ld_res;
             if (epi->residual && epi->ld_res < n_cols_total) return VITINT_ERR_INVALID_ARG;
+            P.kind = epi->act ? EK_DEQUANT_GELU : EK_DEQUANT;
             break;
         case VITINT_EPI_REQUANT: {
             if (!valid_bits(epi->out_bits)) return VITINT_ERR_INVALID_ARG;
@@ -572,9 +711,11 @@ static int fill_epilogue(GemmParams& P, const vitint_epilogue* epi, float x_step
             if (epi->act == 0) {
                 if (!epi->alpha) return VITINT_ERR_INVALID_ARG;
                 P.col_a = epi->alpha; P.col_b = epi->beta;
+                P.kind = EK_REQUANT;
             } else {
                 if (!epi->inv_out_step || !(x_step > 0.0f && x_step < INFINITY)) return VITINT_ERR_INVALID_ARG;
                 P.col_a = w_step; P.col_b = bias; P.inv_s = epi->inv_out_step;
+                P.kind = EK_REQUANT_GELU;
             }
             break;
         }

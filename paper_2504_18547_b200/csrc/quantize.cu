@@ -121,6 +121,32 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
     }
 }
 
+// One thread expands one 32-bit word of packed codes (32/C codes) into as many bytes.
+template <int C>
+__global__ void __launch_bounds__(256)
+widen_kernel(const uint8_t* __restrict__ in, int64_t in_pitch, uint8_t* __restrict__ out, int64_t out_pitch,
+             int64_t rows, int words_in, int is_signed) {
+    constexpr int E = 32 / C;
+    const int w = blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t row = blockIdx.y; row < rows; row += gridDim.y) {
+        if ((int64_t)w * E >= out_pitch) continue;
+        const uint32_t word = (w < words_in) ? *reinterpret_cast<const uint32_t*>(in + row * in_pitch + (int64_t)w * 4) : 0u;
+        uint32_t o[E / 4];
+#pragma unroll
+        for (int i = 0; i < E / 4; ++i) o[i] = 0;
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+            int v = (int)((word >> (C * i)) & ((1u << C) - 1u));
+            if (is_signed && (v & (1 << (C - 1)))) v -= (1 << C);
+            o[i >> 2] |= ((uint32_t)v & 0xFFu) << (8 * (i & 3));
+        }
+        uint8_t* dst = out + row * out_pitch + (int64_t)w * E;
+#pragma unroll
+        for (int i = 0; i < E / 4; ++i)
+            if ((int64_t)w * E + 4 * i + 4 <= out_pitch) reinterpret_cast<uint32_t*>(dst)[i] = o[i];
+    }
+}
+
 template <int C>
 static int launch_ln(int nv, const float* x, int64_t rows, int cols, int64_t ldx, const float* gamma,
                      const float* beta, float eps, float step, uint8_t* out, int64_t pitch, float* y, int64_t ld_y,
@@ -174,6 +200,28 @@ extern "C" int vitint_quantize(const float* x, int64_t rows, int64_t cols, int64
     else
         quantize_pack_kernel<8><<<grid, block, 0, st>>>(x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
                                                         words, (float)qn, (float)qp, vec_ok);
+    return cuda_status(cudaGetLastError());
+}
+
+extern "C" int vitint_widen(const vitint_codes* in, const vitint_codes* out, void* stream) {
+    if (int rc = check_codes(in)) return rc;
+    if (int rc = check_codes(out)) return rc;
+    if (out->bits != 8 || in->bits == 8 || in->rows != out->rows || in->cols != out->cols ||
+        in->is_signed != out->is_signed)
+        return VITINT_ERR_INVALID_ARG;
+    const int c = container_bits(in->bits);
+    const int e = 32 / c;
+    const int words_in = (int)(in->pitch_bytes / 4);
+    const int words_out = (int)((out->pitch_bytes + e - 1) / e);    // threads needed to cover the output pitch
+    const int threads = words_out > words_in ? words_out : words_in;
+    dim3 block(128), grid((threads + 127) / 128, (unsigned)(in->rows < 32768 ? in->rows : 32768));
+    cudaStream_t st = (cudaStream_t)stream;
+    if (c == 2)
+        widen_kernel<2><<<grid, block, 0, st>>>((const uint8_t*)in->data, in->pitch_bytes, (uint8_t*)out->data,
+                                                out->pitch_bytes, in->rows, words_in, in->is_signed);
+    else
+        widen_kernel<4><<<grid, block, 0, st>>>((const uint8_t*)in->data, in->pitch_bytes, (uint8_t*)out->data,
+                                                out->pitch_bytes, in->rows, words_in, in->is_signed);
     return cuda_status(cudaGetLastError());
 }
 

@@ -22,7 +22,7 @@ def _dev(a, device):
 
 class EncoderLayer:
     def __init__(self, batch: int, tokens: int, heads: int, mlp_dim: int, bits: int, prm: dict, device="cuda",
-                 eps: float = 1e-6):
+                 eps: float = 1e-6, widen_weights: bool = True):
         self.batch, self.tokens, self.heads, self.bits, self.eps = batch, tokens, heads, bits, eps
         self.dim = D = heads * 64
         self.mlp_dim = F = mlp_dim
@@ -37,6 +37,11 @@ class EncoderLayer:
         self.w = {}
         for name in ("qkv", "proj", "fc1", "fc2"):
             self.w[name] = B.vitint_quantize(d(prm[f"w_{name}"]), 0.0, bits, True, row_steps=d(prm[f"s_w_{name}"]))
+        # the low-bit weight codes, re-stored once in 8-bit containers: the GEMM then feeds this
+        # operand to the tensor cores straight from the TMA copy
+        self.w_packed = dict(self.w)
+        if widen_weights and bits != 8:
+            self.w = {n: B.vitint_widen(c) for n, c in self.w.items()}
         self.s_w = {n: d(prm[f"s_w_{n}"]) for n in ("proj", "fc1", "fc2")}
         self.bias = {n: d(prm[f"b_{n}"]) for n in ("proj", "fc1", "fc2")}
         seg = np.concatenate([np.full(D, prm["s_q"]), np.full(D, prm["s_k"]), np.full(D, prm["s_v"])]).astype(np.float32)

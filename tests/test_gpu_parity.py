@@ -56,6 +56,14 @@ def test_quantize_row_steps_strided_input_and_ties():
     assert np.array_equal(from_codes(got), vo.quantize(t, 0.25, 4, True))
 
 
+@pytest.mark.parametrize("bits,signed", [(2, True), (3, True), (4, True), (2, False), (4, False)])
+@pytest.mark.parametrize("rows,cols", [(70, 197), (5, 1), (300, 768)])
+def test_widen_keeps_values(bits, signed, rows, cols):
+    q = rand_codes(50 + bits, (rows, cols), bits, signed)
+    got = vt.vitint_widen(to_codes(q, bits, signed))
+    assert got.bits == 8 and np.array_equal(from_codes(got), q) and padding_is_zero(got)
+
+
 # ---------------------------------------------------------------------------
 # a2 + a3
 # ---------------------------------------------------------------------------
@@ -90,6 +98,17 @@ def test_linear_mixed_widths():
     qw = rand_codes(4, (N, K), 4, True)
     acc = vt.vitint_linear(to_codes(qx, 8, False), 1.0, to_codes(qw, 4, True), None, None,
                            vt.Epilogue(mode=vt.EPI_ACC_I32))
+    assert np.array_equal(acc.cpu().numpy(), vo.matmul_i32(qx, qw))
+
+
+@pytest.mark.parametrize("M,K,N", [(197, 192, 576), (515, 1000, 264), (260, 3072, 768), (1000, 768, 2304)])
+@pytest.mark.parametrize("bits,xs", [(4, True), (2, True), (3, True), (4, False)])
+def test_linear_with_widened_weights(M, K, N, bits, xs):
+    """Weights held in 8-bit containers (TMA-direct operand), activations packed low-bit."""
+    qx = rand_codes(7, (M, K), bits, xs)
+    qw = rand_codes(8, (N, K), bits, True)
+    w8 = vt.vitint_widen(to_codes(qw, bits, True))
+    acc = vt.vitint_linear(to_codes(qx, bits, xs), 1.0, w8, None, None, vt.Epilogue(mode=vt.EPI_ACC_I32))
     assert np.array_equal(acc.cpu().numpy(), vo.matmul_i32(qx, qw))
 
 
