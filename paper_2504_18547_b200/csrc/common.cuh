@@ -41,12 +41,68 @@ __device__ __forceinline__ int round_clamp(float r, float qn, float qp) {
     return (int)n;
 }
 
-// GELU(y) = y * Phi(y).  Positive side: 0.5*y*(1 + erf(y/sqrt2)); negative side through
-// erfc so the small tail keeps its relative accuracy.
+// ---- quantizer arithmetic without the conversion / special-function unit ----------------
+// The streaming kernels run several conversions per element; fp32<->int, fp32<->fp64, rint
+// and the reciprocal of an IEEE division all issue on the quarter-rate XU pipe, which then
+// bounds the kernel long before HBM does.  The helpers below produce the same bits with
+// FMA-pipe and integer instructions only.
+
+// Correctly rounded a / b from r = RN(1/b) by one Newton correction on the quotient
+// (Markstein): q0 = RN(a*r); rem = a - q0*b (exact in an FMA); q = RN(q0 + rem*r) = RN(a/b)
+// whenever b's significand is not all ones and nothing underflows.  A quotient that
+// underflows is below 2^-100 in magnitude and quantizes to code 0 either way.
+struct Divisor {
+    float b, r;
+    int exact;   // 0: significand of b is all ones, use the IEEE division instead
+};
+__device__ __forceinline__ Divisor make_divisor(float b) {
+    Divisor d;
+    d.b = b;
+    d.r = __frcp_rn(b);
+    d.exact = ((__float_as_uint(b) & 0x007FFFFFu) != 0x007FFFFFu) ? 1 : 0;
+    return d;
+}
+__device__ __forceinline__ float div_rn(float a, const Divisor& d) {
+    if (!d.exact) return __fdiv_rn(a, d.b);
+    const float q0 = a * d.r;
+    const float rem = fmaf(-q0, d.b, a);
+    return fmaf(rem, d.r, q0);
+}
+
+// clamp(rint(r)) as an integer code, ties to even, NaN -> qn.  The clamp to the integer
+// bounds commutes with rounding; adding 1.5*2^23 rounds to an integer in the FMA pipe and
+// leaves the two's-complement code in the low mantissa bits.
+__device__ __forceinline__ uint32_t round_clamp_bits(float r, float qn, float qp) {
+    const float c = fminf(fmaxf(r, qn), qp);
+    return __float_as_uint(c + 12582912.0f);   // low bits = code (mod 2^22)
+}
+
+// (float)v for |v| < 2^22 without a conversion instruction.
+__device__ __forceinline__ float small_int_to_float(int v) {
+    return __int_as_float(0x4B400000 + v) - 12582912.0f;
+}
+
+// GELU(y) = y * Phi(y) = 0.5*y*(1 + erf(y/sqrt 2)), with erf from
+//   erf(z) = sign(z) * (1 - 2^(-q(|z|))),   q(z) = -log2(erfc(z)) ~ z*(c0 + c1 z + ... + c6 z^6)
+// on |z| <= 4 (beyond that erf is 1 to 2e-8).  The coefficients are a weighted minimax fit
+// (max |erf error| 7.8e-8 in exact arithmetic); with ex2.approx (2 ulp) and the fp32 Horner
+// steps the absolute error of Phi stays below 2.5e-7, i.e. |GELU error| < 2^-21 * |y|.
 __device__ __forceinline__ float gelu_f32(float y) {
-    const float z = y * 0.70710678118654752440f;
-    if (y >= 0.0f) return 0.5f * y * (1.0f + erff(z));
-    return 0.5f * y * erfcf(-z);
+    const float z = fminf(fabsf(y) * 0.70710678118654752440f, 4.0f);
+    float q = -1.00217749e-04f;
+    q = fmaf(q, z, 4.61550077e-04f);
+    q = fmaf(q, z, 2.30229650e-03f);
+    q = fmaf(q, z, -2.94525847e-02f);
+    q = fmaf(q, z, 1.48963709e-01f);
+    q = fmaf(q, z, 9.18328634e-01f);
+    q = fmaf(q, z, 1.62791373e+00f);
+    q = q * z;
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-q));
+    const float erf_abs = 1.0f - e;
+    const float t = copysignf(erf_abs, y);
+    const float hy = 0.5f * y;
+    return fmaf(hy, t, hy);
 }
 
 }  // namespace vitint

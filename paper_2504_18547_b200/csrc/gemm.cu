@@ -44,6 +44,7 @@ struct GemmParams {
     int bn, m_tiles, n_tiles, n_inner, total_tiles, k_blocks;
     int ca, cb, a_signed, b_signed, shift, b_mn_major;
     int a_direct, b_direct;            // operand already int8: TMA writes the operand ring itself
+    int small_acc;                     // |acc| < 2^22: int -> float without a conversion instruction
     int ns_i, ns_p;
     uint32_t ia_bytes, ib_bytes, pa_bytes, pb_bytes, tmem_cols;
     int kind, out_c;
@@ -192,7 +193,7 @@ __device__ __forceinline__ bool epi_barrier(uint32_t bar, uint32_t parity, volat
 // Epilogue of one row x 32 columns.  v[]: accumulators scaled by 2^shift; pa/pb/pq: the 32
 // columns' parameters in shared memory (multiplier already carries 2^-shift).
 // FULL: all 32 columns exist and 16-byte vector accesses are legal.
-template <int KIND, bool FULL>
+template <int KIND, bool FULL, bool SMALL>
 __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32_t (&v)[32], const float* pa,
                                                const float* pb, const float* pq, long long orow, long long colbase,
                                                int n0) {
@@ -210,23 +211,29 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
         }
         return;
     }
-    float y[32];
     // residual first: independent 16-byte loads in flight while the arithmetic runs
-    float res[32];
-    const bool has_res = (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU) && P.residual != nullptr;
+    const bool deq = (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU);
+    const bool has_res = deq && P.residual != nullptr;
+    float4 res[8];
     if (has_res) {
         const float* r = P.residual + orow * P.ld_res + colbase + n0;
         if (FULL && ((reinterpret_cast<uintptr_t>(r) & 15u) == 0)) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float4 t = __ldg(reinterpret_cast<const float4*>(r) + i);
-                res[4 * i] = t.x; res[4 * i + 1] = t.y; res[4 * i + 2] = t.z; res[4 * i + 3] = t.w;
-            }
+            for (int i = 0; i < 8; ++i) res[i] = __ldg(reinterpret_cast<const float4*>(r) + i);
         } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) res[i] = (i < nvalid) ? __ldg(r + i) : 0.0f;
+            for (int i = 0; i < 8; ++i) {
+                res[i].x = (4 * i + 0 < nvalid) ? __ldg(r + 4 * i + 0) : 0.0f;
+                res[i].y = (4 * i + 1 < nvalid) ? __ldg(r + 4 * i + 1) : 0.0f;
+                res[i].z = (4 * i + 2 < nvalid) ? __ldg(r + 4 * i + 2) : 0.0f;
+                res[i].w = (4 * i + 3 < nvalid) ? __ldg(r + 4 * i + 3) : 0.0f;
+            }
         }
     }
+    float* of = (float*)P.out + orow * P.ld_out + colbase + n0;                   // DEQUANT
+    const bool vec_out = FULL && ((reinterpret_cast<uintptr_t>(of) & 15u) == 0);
+    uint32_t wds[8] = {0, 0, 0, 0, 0, 0, 0, 0};                                   // REQUANT
+    const uint32_t mask = (1u << P.out_c) - 1u;
 #pragma unroll
     for (int i4 = 0; i4 < 8; ++i4) {
         const float4 a4 = *reinterpret_cast<const float4*>(pa + 4 * i4);
@@ -237,39 +244,35 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
             const float4 q4 = *reinterpret_cast<const float4*>(pq + 4 * i4);
             qq[0] = q4.x; qq[1] = q4.y; qq[2] = q4.z; qq[3] = q4.w;
         }
+        const float rr[4] = {res[i4].x, res[i4].y, res[i4].z, res[i4].w};
+        float y[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int i = 4 * i4 + j;
-            float val = fmaf((float)(int)v[i], aa[j], bb[j]);
+            const float f = SMALL ? small_int_to_float((int)v[i] >> P.shift) : (float)(int)v[i];
+            float val = fmaf(f, aa[j], bb[j]);
             if (KIND == EK_DEQUANT_GELU || KIND == EK_REQUANT_GELU) val = gelu_f32(val);
             if (KIND == EK_REQUANT_GELU) val = val * qq[j];
-            if (has_res) val = val + res[i];
-            y[i] = val;
+            if (has_res) val = val + rr[j];
+            y[j] = val;
+            if (!deq) {
+                const uint32_t code = (FULL || i < nvalid) ? (round_clamp_bits(val, P.out_qn, P.out_qp) & mask) : 0u;
+                // static word index for each container width keeps wds[] in registers
+                if (P.out_c == 4) wds[i >> 3] |= code << (4 * (i & 7));
+                else if (P.out_c == 2) wds[i >> 4] |= code << (2 * (i & 15));
+                else wds[i >> 2] |= code << (8 * (i & 3));
+            }
+        }
+        if (deq) {
+            if (vec_out) {
+                reinterpret_cast<float4*>(of)[i4] = make_float4(y[0], y[1], y[2], y[3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (4 * i4 + j < nvalid) of[4 * i4 + j] = y[j];
+            }
         }
     }
-    if (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU) {
-        float* o = (float*)P.out + orow * P.ld_out + colbase + n0;
-        if (FULL && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                reinterpret_cast<float4*>(o)[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) if (i < nvalid) o[i] = y[i];
-        }
-        return;
-    }
-    // REQUANT: 32 codes -> out_c 32-bit words
-    uint32_t wds[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    const uint32_t mask = (1u << P.out_c) - 1u;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        const uint32_t code = (FULL || i < nvalid) ? ((uint32_t)round_clamp(y[i], P.out_qn, P.out_qp) & mask) : 0u;
-        // static word index for each container width keeps wds[] in registers
-        if (P.out_c == 4) wds[i >> 3] |= code << (4 * (i & 7));
-        else if (P.out_c == 2) wds[i >> 4] |= code << (2 * (i & 15));
-        else wds[i >> 2] |= code << (8 * (i & 3));
-    }
+    if (deq) return;
     const int out_words = P.out_c;   // 32 codes = 4*out_c bytes
     const long long byte0 = ((colbase + n0) * P.out_c) >> 3;
     uint8_t* o = (uint8_t*)P.out + orow * P.ld_out + byte0;
@@ -281,14 +284,13 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
             if (k < out_words && byte0 + 4 * k + 4 <= P.ld_out) reinterpret_cast<uint32_t*>(o)[k] = wds[k];
     }
     // row padding behind the last chunk of the last column tile
-    if (!FULL || (P.col_off_inner == 0 && n0 + 32 >= P.N)) {
-        if (P.col_off_inner == 0)
-            for (long long off = byte0 + 4 * out_words; off + 4 <= P.ld_out; off += 4)
-                *reinterpret_cast<uint32_t*>((uint8_t*)P.out + orow * P.ld_out + off) = 0u;
+    if (P.col_off_inner == 0 && (!FULL || n0 + 32 >= P.N)) {
+        for (long long off = byte0 + 4 * out_words; off + 4 <= P.ld_out; off += 4)
+            *reinterpret_cast<uint32_t*>((uint8_t*)P.out + orow * P.ld_out + off) = 0u;
     }
 }
 
-template <int KIND>
+template <int KIND, bool SMALL>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiParams& ep, int buf, uint32_t t_row,
                                               bool row_ok, long long orow, long long colbase, int n_tile) {
     for (int chunk = 0; chunk * 32 < P.bn; ++chunk) {
@@ -301,13 +303,14 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiPara
             const float* pa = &ep.a[buf][chunk * 32];
             const float* pb = &ep.b[buf][chunk * 32];
             const float* pq = &ep.q[buf][chunk * 32];
-            if (n0 + 32 <= P.N) epilogue_chunk<KIND, true>(P, v, pa, pb, pq, orow, colbase, n0);
-            else epilogue_chunk<KIND, false>(P, v, pa, pb, pq, orow, colbase, n0);
+            if (n0 + 32 <= P.N) epilogue_chunk<KIND, true, SMALL>(P, v, pa, pb, pq, orow, colbase, n0);
+            else epilogue_chunk<KIND, false, SMALL>(P, v, pa, pb, pq, orow, colbase, n0);
         }
         __syncwarp();
     }
 }
 
+template <int KIND>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ GemmParams P) {
@@ -484,7 +487,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // -------------------------------- epilogue ---------------------------------
         const int q4 = warp;   // TMEM lane quarter
         const int tid_e = threadIdx.x;                       // 0..127
-        const float down = __int_as_float((127 - P.shift) << 23);   // 2^-shift
+        // small accumulators are shifted back as integers; otherwise 2^-shift rides on the multiplier
+        const float down = P.small_acc ? 1.0f : __int_as_float((127 - P.shift) << 23);
         int tl = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++tl) {
@@ -493,17 +497,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int buf = tl & 1;
             const long long colbase = (long long)inner * P.col_off_inner;
             // stage this tile's per-column parameters while its MMAs are still running
-            if (P.kind != EK_ACC) {
+            if (KIND != EK_ACC) {
                 for (int c = tid_e; c < P.bn; c += EPI_WARPS * 32) {
                     const int n = n_tile * P.bn + c;
                     float a = 0.0f, b = 0.0f, q = 0.0f;
                     if (n < P.N) {
                         const long long cidx = colbase + n;
-                        if (P.kind == EK_REQUANT) {
+                        if (KIND == EK_REQUANT) {
                             a = __ldg(P.col_a + cidx);
                         } else {
                             a = P.col_a ? __fmul_rn(P.x_step, __ldg(P.col_a + cidx)) : P.x_step;
-                            if (P.kind == EK_REQUANT_GELU) q = __ldg(P.inv_s + cidx);
+                            if (KIND == EK_REQUANT_GELU) q = __ldg(P.inv_s + cidx);
                         }
                         b = P.col_b ? __ldg(P.col_b + cidx) : 0.0f;
                         a *= down;
@@ -514,7 +518,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
             }
             const uint32_t acc_ph = (uint32_t)(tl >> 1) & 1u;
-            bool w = P.kind == EK_ACC || epi_barrier(ptx::smem_addr(&bars.epi_sync), (uint32_t)tl & 1u, abort_ptr);
+            bool w = KIND == EK_ACC || epi_barrier(ptx::smem_addr(&bars.epi_sync), (uint32_t)tl & 1u, abort_ptr);
             w = w && mbar_wait(ptx::smem_addr(&bars.acc_full[buf]), acc_ph, abort_ptr);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
             ptx::tc_fence_after();
@@ -522,13 +526,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool row_ok = row_in_problem < P.M;
             const long long orow = (long long)outer * P.row_off_outer + (long long)inner * P.row_off_inner + row_in_problem;
             const uint32_t t_row = tmem_base + (uint32_t)buf * acc_stride + ((uint32_t)(q4 * 32) << 16);
-            switch (P.kind) {
-                case EK_ACC: epilogue_tile<EK_ACC>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
-                case EK_DEQUANT: epilogue_tile<EK_DEQUANT>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
-                case EK_DEQUANT_GELU: epilogue_tile<EK_DEQUANT_GELU>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
-                case EK_REQUANT: epilogue_tile<EK_REQUANT>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
-                default: epilogue_tile<EK_REQUANT_GELU>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile); break;
-            }
+            if (P.small_acc) epilogue_tile<KIND, true>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
+            else epilogue_tile<KIND, false>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&bars.acc_empty[buf]));
@@ -616,6 +615,7 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     const long long bound = (long long)K * max_abs_code(A.bits, A.is_signed) * max_abs_code(B.bits, B.is_signed);
     if (bound >= (1ll << 31)) return VITINT_ERR_OVERFLOW_BOUND;
     if ((bound << P.shift) >= (1ll << 31)) return VITINT_ERR_UNSUPPORTED;
+    P.small_acc = bound < (1ll << 22) ? 1 : 0;
     int bn = N >= MAX_BN ? MAX_BN : ((N + 15) / 16) * 16;
     if (b_mn_major) { if (N != 64) return VITINT_ERR_UNSUPPORTED; bn = 64; }
     P.bn = bn;
@@ -668,16 +668,28 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     // at least ~120 KB so that two CTAs never share an SM (and its tensor memory)
     size_t smem = (size_t)ns_i * stage_i + (size_t)ns_p * stage_p + 1024;
     if (smem < 120 * 1024) smem = 120 * 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)SMEM_TILE_BUDGET + 2048) != cudaSuccess)
-            return VITINT_ERR_CUDA;
-        attr_set = true;
-    }
     int grid = sm_count();
     if (grid > P.total_tiles) grid = P.total_tiles;
-    gemm_i8_kernel<<<grid, NUM_THREADS, smem, st>>>(map_a, map_b, P);
+    static bool attr_set[5] = {false, false, false, false, false};
+#define VITINT_LAUNCH(KIND)                                                                                        \
+    case KIND:                                                                                                     \
+        if (!attr_set[KIND]) {                                                                                     \
+            if (cudaFuncSetAttribute(gemm_i8_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,            \
+                                     (int)SMEM_TILE_BUDGET + 2048) != cudaSuccess)                                 \
+                return VITINT_ERR_CUDA;                                                                            \
+            attr_set[KIND] = true;                                                                                 \
+        }                                                                                                          \
+        gemm_i8_kernel<KIND><<<grid, NUM_THREADS, smem, st>>>(map_a, map_b, P);                                    \
+        break;
+    switch (P.kind) {
+        VITINT_LAUNCH(EK_ACC)
+        VITINT_LAUNCH(EK_DEQUANT)
+        VITINT_LAUNCH(EK_DEQUANT_GELU)
+        VITINT_LAUNCH(EK_REQUANT)
+        VITINT_LAUNCH(EK_REQUANT_GELU)
+        default: return VITINT_ERR_INVALID_ARG;
+    }
+#undef VITINT_LAUNCH
     return cuda_status(cudaGetLastError());
 }
 

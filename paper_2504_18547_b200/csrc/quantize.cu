@@ -18,7 +18,7 @@ quantize_pack_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, in
     const int64_t col0 = (int64_t)w * E;
     for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows;
          row += (int64_t)gridDim.y * blockDim.y) {
-        const float s = row_steps ? row_steps[row] : step;
+        const Divisor dv = make_divisor(row_steps ? row_steps[row] : step);
         const float* xr = x + row * ldx + col0;
         float v[E];
         if (vec_ok && col0 + E <= cols) {
@@ -34,8 +34,7 @@ quantize_pack_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, in
         uint32_t word = 0;
 #pragma unroll
         for (int i = 0; i < E; ++i) {
-            const int q = round_clamp(__fdiv_rn(v[i], s), qn, qp);
-            word |= ((uint32_t)q & ((1u << C) - 1u)) << (C * i);
+            word |= (round_clamp_bits(div_rn(v[i], dv), qn, qp) & ((1u << C) - 1u)) << (C * i);
         }
         *reinterpret_cast<uint32_t*>(out + row * pitch + (int64_t)w * 4) = word;
     }
@@ -43,8 +42,8 @@ quantize_pack_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, in
 
 // One warp per row; the row stays in registers between the statistics and the
 // normalisation.  Lane l owns float4 number v*32 + l of the row, v < NV.
-// Sums run in fp64 so that the result stays inside a few fp32 ulp of the exact
-// normalisation even when |mean| >> sigma.
+// All per-element arithmetic is fp32 on the FMA pipe (no conversions); the corrected
+// two-pass mean keeps the result inside a few ulp of the exact normalisation.
 template <int C, int NV>
 __global__ void __launch_bounds__(256)
 layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, int64_t ldx,
@@ -56,32 +55,44 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
     if (row >= rows) return;
     const float* xr = x + row * ldx;
     float4 f[NV];
-    double sum = 0.0;
+    float sum = 0.0f;
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
         const int col = (v * 32 + lane) * 4;
         f[v] = (col < cols) ? __ldg(reinterpret_cast<const float4*>(xr + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        sum += ((double)f[v].x + (double)f[v].y) + ((double)f[v].z + (double)f[v].w);
+        sum += (f[v].x + f[v].y) + (f[v].z + f[v].w);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    const double mean = sum / (double)cols;
-    double m2 = 0.0;
+    const float inv_n = 1.0f / (float)cols;
+    // corrected two-pass mean: centre on the fp32 estimate, then remove the mean of the
+    // residuals, which carries the estimate's rounding error even when |mean| >> sigma
+    const float mean0 = sum * inv_n;
+    float rsum = 0.0f;
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
         const int col = (v * 32 + lane) * 4;
         if (col < cols) {
-            f[v].x = (float)((double)f[v].x - mean);
-            f[v].y = (float)((double)f[v].y - mean);
-            f[v].z = (float)((double)f[v].z - mean);
-            f[v].w = (float)((double)f[v].w - mean);
-            m2 += ((double)f[v].x * f[v].x + (double)f[v].y * f[v].y) +
-                  ((double)f[v].z * f[v].z + (double)f[v].w * f[v].w);
+            f[v].x -= mean0; f[v].y -= mean0; f[v].z -= mean0; f[v].w -= mean0;
+            rsum += (f[v].x + f[v].y) + (f[v].z + f[v].w);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
+    const float corr = rsum * inv_n;
+    float m2 = 0.0f;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int col = (v * 32 + lane) * 4;
+        if (col < cols) {
+            f[v].x -= corr; f[v].y -= corr; f[v].z -= corr; f[v].w -= corr;
+            m2 += fmaf(f[v].x, f[v].x, f[v].y * f[v].y) + fmaf(f[v].z, f[v].z, f[v].w * f[v].w);
         }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
-    const float rstd = (float)(1.0 / sqrt(m2 / (double)cols + (double)eps));
+    const float rstd = (float)(1.0 / sqrt((double)m2 / (double)cols + (double)eps));   // once per row
+    const Divisor dv = make_divisor(step);
 
     constexpr int LANES_PER_WORD = 8 / C;          // 4 codes per lane per v -> 4*C bits
     const int words_per_row = (int)(pitch >> 2);
@@ -103,10 +114,10 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
             y.w = fmaf(d.w * rstd, g.w, b.w);
             if (y_out) *reinterpret_cast<float4*>(y_out + row * ld_y + col) = y;
             const uint32_t m = (1u << C) - 1u;
-            bits = ((uint32_t)round_clamp(__fdiv_rn(y.x, step), qn, qp) & m) |
-                   (((uint32_t)round_clamp(__fdiv_rn(y.y, step), qn, qp) & m) << C) |
-                   (((uint32_t)round_clamp(__fdiv_rn(y.z, step), qn, qp) & m) << (2 * C)) |
-                   (((uint32_t)round_clamp(__fdiv_rn(y.w, step), qn, qp) & m) << (3 * C));
+            bits = (round_clamp_bits(div_rn(y.x, dv), qn, qp) & m) |
+                   ((round_clamp_bits(div_rn(y.y, dv), qn, qp) & m) << C) |
+                   ((round_clamp_bits(div_rn(y.z, dv), qn, qp) & m) << (2 * C)) |
+                   ((round_clamp_bits(div_rn(y.w, dv), qn, qp) & m) << (3 * C));
         }
         // gather 8/C neighbouring lanes into one 32-bit word
         if (C == 4) {
