@@ -142,7 +142,7 @@ def run_ours(args, cfg):
     import torch.distributed as dist
 
     import paper_2504_18547_b200 as vt
-    from paper_2504_18547_b200.encoder import GEMM_STAGES, STAGES, EncoderLayer
+    from paper_2504_18547_b200.encoder import GEMM_STAGES, EncoderLayer
 
     rank, local_rank, world = dist_env()
     torch.cuda.set_device(local_rank)
@@ -151,7 +151,10 @@ def run_ours(args, cfg):
         dist.init_process_group("nccl", device_id=device)
 
     prm = si.layer_parameters(cfg)
-    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, device)
+    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, device,
+                         fused_attention=not args.unfused_attention)
+    STAGES = layer.stages
+    gemm_stages = [s for s in STAGES if s in GEMM_STAGES]
     M, D = cfg.rows, cfg.dim
     # each rank owns a disjoint range of images (weak scaling, no exchange on the data path)
     first = rank * cfg.batch
@@ -224,8 +227,8 @@ def run_ours(args, cfg):
     e2e_tops = world * ops_step / (ms_e2e / args.steps * 1e-3) / 1e12
 
     sops = layer.stage_ops()
-    gemm_ms = sum(stage_ms[s] for s in GEMM_STAGES)
-    gemm_ops = sum(sops[s] for s in GEMM_STAGES)
+    gemm_ms = sum(stage_ms[s] for s in gemm_stages)
+    gemm_ops = sum(sops[s] for s in gemm_stages)
     int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
     sbytes = layer.stage_bytes()
@@ -260,12 +263,13 @@ def run_ours(args, cfg):
         "images_per_s": world * cfg.batch / (ms_step * 1e-3),
         "config": {"workload": cfg.name, "bits": cfg.bits, "batch_per_gpu": cfg.batch, "tokens": cfg.tokens,
                    "dim": cfg.dim, "heads": cfg.heads, "mlp_dim": cfg.mlp_dim,
+                   "attention": "fused" if layer.fused_attention else "unfused",
                    "l2": f"inputs rotate over {N_INPUT_BUFFERS} buffers of {M * D * 4 / 1e6:.1f} MB (> 126 MB L2)"},
         "clocks": clocks,
         "e2e": {"value": e2e_tops, "unit": "TOPS", "h2d_bytes_per_step": M * D * 4, "d2h_bytes_per_step": M * D * 4,
                 "ms_per_step": ms_e2e / args.steps},
-        "gpu_launches": len(STAGES) * args.steps,
-        "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel (6 launches per step)", "achieved": achieved,
+        "gpu_launches": (len(STAGES) + (1 if layer.fused_attention else 0)) * args.steps,
+        "roofline": {"bound": "tensor", "kernel": f"gemm_i8_kernel ({len(gemm_stages)} launches per step)", "achieved": achieved,
                      "peak": int8_peak, "unit": "TOPS", "frac": achieved / int8_peak, "traffic": None,
                      "peak_source": f"{peaks['source']} sustained bf16 cuBLAS x {INT8_OVER_BF16:g} (nominal int8:bf16)",
                      "frac_of_nominal_4500": achieved / 4500.0},
@@ -287,6 +291,7 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="images per GPU (default: the configuration's 128)")
     ap.add_argument("--ref-images", type=int, default=None, help="images per step of the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--unfused-attention", action="store_true", help="run Q K^T, softmax and P V as separate kernels")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = si.VIT_BASE_LAYER.with_(bits=args.bits)

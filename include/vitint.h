@@ -163,6 +163,24 @@ int vitint_softmax_quantize(const int32_t* s, int64_t rows, int32_t cols, int64_
 int vitint_pv(const vitint_codes* p, const vitint_slabs* v, int32_t batch, int32_t heads, int32_t tokens,
               float p_step, float v_step, const vitint_epilogue* epi, void* out, int64_t ld_out, void* stream);
 
+/* a4 + a5 + a6 fused (Eq. 3 and the W_attn V product of Section IV-B in one kernel): for every
+ *   (image, head)  S = Q K^T,  P = quantize(softmax(c S), p_step, unsigned p_bits),  O = P V,
+ *   o = clamp(rint(fmaf((float)O, alpha_o[h*64+c], beta_o[h*64+c])))  with c = fl32(q_step k_step/8).
+ *   S, the probabilities and P stay on the SM.  Results equal the unfused sequence
+ *   vitint_qk -> vitint_softmax_quantize -> vitint_pv up to the fp32 tolerance of the softmax
+ *   (probabilities within 2 ulp, hence P codes that may differ on near-ties only).
+ *   qkv: signed codes [batch*tokens, 3*heads*64] (Q | K | V column blocks);  o_out: codes
+ *   [batch*tokens, heads*64] whose bits / signedness select the output format;  alpha_o: device
+ *   [heads*64];  beta_o: device [heads*64] or NULL.
+ *   workspace: >= vitint_attention_core_workspace_bytes(bits) bytes of device scratch, 256-byte
+ *   aligned (holds a table of exp(fl32(s*c)) over all integer scores s); contents undefined after.
+ *   Errors: UNSUPPORTED when tokens > 256, the codes are 8-bit, or 64*max|q|*max|k|*c > 80 (use the
+ *   unfused calls then); INVALID_ARG, ALIGNMENT, WORKSPACE, CUDA. */
+size_t vitint_attention_core_workspace_bytes(int32_t bits);
+int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens, float q_step,
+                          float k_step, float p_step, int32_t p_bits, const float* alpha_o, const float* beta_o,
+                          const vitint_codes* o_out, void* workspace, size_t workspace_bytes, void* stream);
+
 /* a7. Integerized self-attention block (Fig. 1(b)):
  *   QKV linear (requantized with per-channel alpha_qkv/beta_qkv, i.e. three per-tensor
  *   steps q_step, k_step, v_step laid out per output channel) -> Q K^T -> scale, softmax,
@@ -176,7 +194,9 @@ int vitint_pv(const vitint_codes* p, const vitint_slabs* v, int32_t batch, int32
  *   that receive copies of the intermediate codes: QKV [M, 3D], P [batch*heads*tokens, tokens],
  *   O [M, D]; NULL to skip.
  *   workspace: device scratch of at least vitint_attention_block_workspace_bytes(...) bytes,
- *   256-byte aligned; contents are undefined afterwards. */
+ *   256-byte aligned; contents are undefined afterwards.
+ *   The middle of the block runs as vitint_attention_core when that call supports the shape and
+ *   dbg_p is NULL, otherwise as vitint_qk -> vitint_softmax_quantize -> vitint_pv. */
 typedef struct {
     int32_t batch, tokens, heads;
     int32_t bits;                 /* activation / weight code width of the block */

@@ -70,6 +70,10 @@ def lib():
                                               c_void_p, c_int64, c_void_p]
         L.vitint_pv.argtypes = [POINTER(_Codes), POINTER(_Slabs), c_int32, c_int32, c_int32, c_float, c_float,
                                 POINTER(_Epilogue), c_void_p, c_int64, c_void_p]
+        L.vitint_attention_core_workspace_bytes.restype = c_size_t
+        L.vitint_attention_core_workspace_bytes.argtypes = [c_int32]
+        L.vitint_attention_core.argtypes = [POINTER(_Codes), c_int32, c_int32, c_int32, c_float, c_float, c_float,
+                                            c_int32, c_void_p, c_void_p, POINTER(_Codes), c_void_p, c_size_t, c_void_p]
         L.vitint_attention_block_workspace_bytes.restype = c_size_t
         L.vitint_attention_block_workspace_bytes.argtypes = [POINTER(_AttentionDesc)]
         L.vitint_attention_block.argtypes = [POINTER(_Codes), POINTER(_AttentionDesc), c_void_p, c_int64,
@@ -266,6 +270,27 @@ def vitint_pv(p: Codes, v: Slabs, batch: int, heads: int, tokens: int, p_step: f
     dp, dv, de = p.desc(), v.desc(), epi.desc()
     _check(lib().vitint_pv(byref(dp), byref(dv), batch, heads, tokens, float(p_step), float(v_step), byref(de), ptr,
                            ld, _stream()), "vitint_pv")
+    return out
+
+
+def vitint_attention_core_workspace_bytes(bits: int) -> int:
+    return int(lib().vitint_attention_core_workspace_bytes(bits))
+
+
+def vitint_attention_core(qkv: Codes, batch: int, heads: int, tokens: int, q_step: float, k_step: float,
+                          p_step: float, p_bits: int, alpha_o: torch.Tensor, beta_o: torch.Tensor | None,
+                          out: Codes | None = None, out_bits: int | None = None,
+                          workspace: torch.Tensor | None = None) -> Codes:
+    """Fused Q K^T -> softmax -> quantize -> P V -> requantize; `out` holds signed codes [batch*tokens, heads*64]."""
+    if out is None:
+        out = Codes.empty(batch * tokens, heads * 64, qkv.bits if out_bits is None else out_bits, True, qkv.data.device)
+    if workspace is None:
+        workspace = torch.empty(vitint_attention_core_workspace_bytes(qkv.bits), dtype=torch.uint8,
+                                device=qkv.data.device)
+    dq, do = qkv.desc(), out.desc()
+    _check(lib().vitint_attention_core(byref(dq), batch, heads, tokens, float(q_step), float(k_step), float(p_step),
+                                       p_bits, _ptr(alpha_o), _ptr(beta_o), byref(do), workspace.data_ptr(),
+                                       workspace.numel(), _stream()), "vitint_attention_core")
     return out
 
 

@@ -12,7 +12,7 @@ namespace {
 struct AttnLayout {
     int64_t M, D, n_rows_p;
     int64_t pitch_qkv, pitch_p, pitch_o, ld_s;
-    size_t off_qkv, off_s, off_p, off_o, total;
+    size_t off_qkv, off_s, off_p, off_o, off_tab, tab_bytes, total;
 };
 
 inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
@@ -32,6 +32,8 @@ int attn_layout(const vitint_attention_desc* d, AttnLayout* L) {
     L->off_s = off;   off = align256(off + (size_t)(L->n_rows_p * L->ld_s) * 4);
     L->off_p = off;   off = align256(off + (size_t)(L->n_rows_p * L->pitch_p));
     L->off_o = off;   off = align256(off + (size_t)(L->M * L->pitch_o));
+    L->tab_bytes = vitint_attention_core_workspace_bytes(d->bits);
+    L->off_tab = off; off = align256(off + L->tab_bytes);
     L->total = off;
     return VITINT_OK;
 }
@@ -84,30 +86,38 @@ extern "C" int vitint_attention_block(const vitint_codes* x, const vitint_attent
     if (int rc = vitint_linear(x, 1.0f, &d->w_qkv, nullptr, nullptr, &e1, qkv.data, qkv.pitch_bytes, stream)) return rc;
     if (int rc = copy_codes(dbg_qkv, qkv.data, L.pitch_qkv, L.M, row_bytes(3 * L.D, d->bits), st)) return rc;
 
-    // 2. S = Q K^T per (image, head)
-    const int64_t head_bytes = 64 * cbits / 8, seg_bytes = L.D * cbits / 8;
-    vitint_slabs q{ws + L.off_qkv, L.pitch_qkv, L.pitch_qkv * d->tokens, head_bytes, d->bits, 1};
-    vitint_slabs k = q, v = q;
-    k.data = ws + L.off_qkv + seg_bytes;
-    v.data = ws + L.off_qkv + 2 * seg_bytes;
-    int32_t* S = (int32_t*)(ws + L.off_s);
-    if (int rc = vitint_qk(&q, &k, d->batch, d->heads, d->tokens, S, L.ld_s, stream)) return rc;
-
-    // 3. P = quantize(softmax(c * S)),  c = s_q s_k / sqrt(64)
-    const float c = (float)((double)d->q_step * (double)d->k_step / 8.0);
-    vitint_codes p{ws + L.off_p, L.n_rows_p, d->tokens, L.pitch_p, d->p_bits, 0};
-    if (int rc = vitint_softmax_quantize(S, L.n_rows_p, d->tokens, L.ld_s, c, d->p_step, &p, nullptr, 0, stream))
-        return rc;
-    if (int rc = copy_codes(dbg_p, p.data, L.pitch_p, L.n_rows_p, row_bytes(d->tokens, d->p_bits), st)) return rc;
-
-    // 4. O = P V, requantized to the projection's input step
     vitint_codes o{ws + L.off_o, L.M, L.D, L.pitch_o, d->bits, 1};
-    vitint_epilogue e4{};
-    e4.mode = VITINT_EPI_REQUANT; e4.alpha = d->alpha_o; e4.beta = d->beta_o;
-    e4.out_bits = d->bits; e4.out_signed = 1;
-    if (int rc = vitint_pv(&p, &v, d->batch, d->heads, d->tokens, d->p_step, d->v_step, &e4, o.data, o.pitch_bytes,
-                           stream))
-        return rc;
+    // 2-4 fused when the shape allows and no copy of P is wanted
+    int fused = VITINT_ERR_UNSUPPORTED;
+    if (!dbg_p && L.tab_bytes)
+        fused = vitint_attention_core(&qkv, d->batch, d->heads, d->tokens, d->q_step, d->k_step, d->p_step, d->p_bits,
+                                      d->alpha_o, d->beta_o, &o, ws + L.off_tab, L.tab_bytes, stream);
+    if (fused != VITINT_OK && fused != VITINT_ERR_UNSUPPORTED) return fused;
+    if (fused == VITINT_ERR_UNSUPPORTED) {
+        // 2. S = Q K^T per (image, head)
+        const int64_t head_bytes = 64 * cbits / 8, seg_bytes = L.D * cbits / 8;
+        vitint_slabs q{ws + L.off_qkv, L.pitch_qkv, L.pitch_qkv * d->tokens, head_bytes, d->bits, 1};
+        vitint_slabs k = q, v = q;
+        k.data = ws + L.off_qkv + seg_bytes;
+        v.data = ws + L.off_qkv + 2 * seg_bytes;
+        int32_t* S = (int32_t*)(ws + L.off_s);
+        if (int rc = vitint_qk(&q, &k, d->batch, d->heads, d->tokens, S, L.ld_s, stream)) return rc;
+
+        // 3. P = quantize(softmax(c * S)),  c = s_q s_k / sqrt(64)
+        const float c = (float)((double)d->q_step * (double)d->k_step / 8.0);
+        vitint_codes p{ws + L.off_p, L.n_rows_p, d->tokens, L.pitch_p, d->p_bits, 0};
+        if (int rc = vitint_softmax_quantize(S, L.n_rows_p, d->tokens, L.ld_s, c, d->p_step, &p, nullptr, 0, stream))
+            return rc;
+        if (int rc = copy_codes(dbg_p, p.data, L.pitch_p, L.n_rows_p, row_bytes(d->tokens, d->p_bits), st)) return rc;
+
+        // 4. O = P V, requantized to the projection's input step
+        vitint_epilogue e4{};
+        e4.mode = VITINT_EPI_REQUANT; e4.alpha = d->alpha_o; e4.beta = d->beta_o;
+        e4.out_bits = d->bits; e4.out_signed = 1;
+        if (int rc = vitint_pv(&p, &v, d->batch, d->heads, d->tokens, d->p_step, d->v_step, &e4, o.data, o.pitch_bytes,
+                               stream))
+            return rc;
+    }
     if (int rc = copy_codes(dbg_o, o.data, L.pitch_o, L.M, row_bytes(L.D, d->bits), st)) return rc;
 
     // 5. output projection

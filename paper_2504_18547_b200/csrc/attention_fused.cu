@@ -1,0 +1,422 @@
+// a4 + a5 + a6 fused: per (image, head, 128-query tile)  S = Q K^T  ->  softmax + quantize  ->
+// O = P V  ->  requantize, with S, the probabilities and P never leaving the SM.
+//
+// A persistent CTA runs TWO independent pipelines ("groups"), each with four compute warps
+// (thread = query row = TMEM lane) and one control warp (TMA + MMA issue); while one group's
+// threads are busy with the softmax the other group's loads and MMAs proceed.
+//
+// Per item and group:
+//   control   TMA: packed Q [128 x 64], K [T x 64], V [T x 64] code slabs -> shared memory
+//   compute   unpack to int8 operand tiles (rows of 64 bytes, 64-byte swizzle)
+//   control   tcgen05.mma  S[128, T] = Q K^T   (K = 64: two MMAs) into TMEM
+//   compute   e_j = EXP[S_j] from a table of exp(fl32(s*c)) over every possible integer score
+//             (|S| <= 64*max|q|*max|k|: 8193 entries for 4-bit codes); row sum in fp64;
+//             p_j = e_j / Z;  code = clamp(rint(p_j / s_P));  codes written as int8 rows (128-byte
+//             swizzle) = the A operand of P V.  e_j is parked in TMEM over S between the passes.
+//   control   tcgen05.mma  O[128, 64] = P V  (V is the N-contiguous B operand) into TMEM
+//   compute   requantize O, pack, store the head's 64 columns of the [M, D] code matrix
+//
+// Softmax accuracy: exp(t_j)/sum_k exp(t_k) equals Eq. 3's softmax exactly (the maximum is only
+// subtracted there for range); every table entry is a correctly rounded fp32, the sum is fp64,
+// and p_j = RN(e_j * (1/Z)) with 1/Z carried as two floats, so p_j stays within 2 ulp.
+// The host only selects this kernel when smax*|c| <= 80 (no overflow without max subtraction).
+#include "common.cuh"
+#include "ptx.cuh"
+#include "tile_ops.cuh"
+
+namespace vitint {
+namespace {
+
+constexpr int AT_GROUPS = 2;
+constexpr int AT_COMPUTE_WARPS = 4;
+constexpr int AT_THREADS = (AT_GROUPS * AT_COMPUTE_WARPS + AT_GROUPS) * 32;   // 320
+
+struct AttnParams {
+    int batch, heads, tokens, q_tiles, total_items;
+    int c;                       // container bits of Q, K, V (2 or 4)
+    int n_k;                     // MMA N of Q K^T: tokens rounded up to 16
+    int kv_rows;                 // tokens rounded up to 32: K extent of P V, rows of the V tile
+    int smax;                    // table covers scores -smax .. smax
+    int part_bytes;              // bytes of one of the Q / K / V column blocks in a QKV row
+    uint32_t off_table, off_group, group_bytes;         // shared-memory layout
+    uint32_t off_pq, off_pk, off_pv, off_q, off_k, off_v, off_p, off_col;   // within a group
+    const float* table;          // global copy of the exp table, 2*smax+1 floats
+    float p_step, p_qp;
+    const float* alpha_o;        // [D]
+    const float* beta_o;         // [D] or null
+    int out_c;
+    float out_qn, out_qp;
+    uint8_t* out;
+    long long out_pitch;
+};
+
+struct AttnBars {
+    uint64_t packed_full, ops_ready, s_full, p_ready, o_full, o_done, grp_sync;
+};
+
+// exp(fl32(s * c)) for every integer score, correctly rounded to fp32 (fp64 exp, one rounding).
+__global__ void exp_table_kernel(float* table, int smax, float c) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i > 2 * smax) return;
+    const float t = __fmul_rn((float)(i - smax), c);
+    table[i] = (float)exp((double)t);
+}
+
+template <int C>
+__global__ void __launch_bounds__(AT_THREADS, 1)
+attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv,
+                       const __grid_constant__ AttnParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ AttnBars bars[AT_GROUPS];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+    uint8_t* const smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
+    volatile int* abort_ptr = &abort_flag;
+    const bool is_control = warp >= AT_GROUPS * AT_COMPUTE_WARPS;
+    const int g = is_control ? warp - AT_GROUPS * AT_COMPUTE_WARPS : warp / AT_COMPUTE_WARPS;
+    AttnBars& B = bars[g];
+    const uint32_t gbase = smem_base + P.off_group + (uint32_t)g * P.group_bytes;
+    uint8_t* const ggen = smem_gen + P.off_group + (size_t)g * P.group_bytes;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int k = 0; k < AT_GROUPS; ++k) {
+            ptx::mbar_init(ptx::smem_addr(&bars[k].packed_full), 1);
+            ptx::mbar_init(ptx::smem_addr(&bars[k].ops_ready), AT_COMPUTE_WARPS);
+            ptx::mbar_init(ptx::smem_addr(&bars[k].s_full), 1);
+            ptx::mbar_init(ptx::smem_addr(&bars[k].p_ready), AT_COMPUTE_WARPS);
+            ptx::mbar_init(ptx::smem_addr(&bars[k].o_full), 1);
+            ptx::mbar_init(ptx::smem_addr(&bars[k].o_done), AT_COMPUTE_WARPS);
+            ptx::mbar_init(ptx::smem_addr(&bars[k].grp_sync), AT_COMPUTE_WARPS * 32);
+        }
+        ptx::fence_mbar_init();
+        ptx::fence_proxy_async_smem();
+    }
+    if (warp == AT_GROUPS * AT_COMPUTE_WARPS) {          // first control warp owns the TMEM allocation
+        ptx::tmem_alloc(ptx::smem_addr(&tmem_base_slot), 512);
+        ptx::tmem_relinquish();
+    }
+    // the exp table: global -> shared, once per CTA
+    {
+        float* tab = reinterpret_cast<float*>(smem_gen + P.off_table);
+        for (int i = threadIdx.x; i <= 2 * P.smax; i += AT_THREADS) tab[i] = __ldg(P.table + i);
+    }
+    if (is_control && lane == 0) { ptx::prefetch_tensormap(&map_q); ptx::prefetch_tensormap(&map_kv); }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_grp = tmem_base_slot + (uint32_t)g * 256u;
+
+    const int T = P.tokens;
+    const int item0 = blockIdx.x * AT_GROUPS + g, item_stride = gridDim.x * AT_GROUPS;
+    const int head_bytes = 8 * C;                      // 64 codes
+    const uint32_t q_bytes = 128u * head_bytes, kv_bytes = (uint32_t)P.kv_rows * head_bytes;   // TMA boxes
+
+    auto item_coords = [&](int item, int& b, int& h, int& qt) {
+        qt = item % P.q_tiles;
+        const int bh = item / P.q_tiles;
+        h = bh % P.heads;
+        b = bh / P.heads;
+    };
+
+    if (is_control) {
+        // --------------------------- control: TMA + MMA issue ----------------------------
+        if (lane == 0) {
+            auto issue_loads = [&](int item) {
+                int b, h, qt;
+                item_coords(item, b, h, qt);
+                const uint32_t bar = ptx::smem_addr(&B.packed_full);
+                ptx::mbar_arrive_expect_tx(bar, q_bytes + 2u * kv_bytes);
+                ptx::tma_load_3d(gbase + P.off_pq, &map_q, bar, h * head_bytes, qt * 128, b);
+                ptx::tma_load_3d(gbase + P.off_pk, &map_kv, bar, P.part_bytes + h * head_bytes, 0, b);
+                ptx::tma_load_3d(gbase + P.off_pv, &map_kv, bar, 2 * P.part_bytes + h * head_bytes, 0, b);
+            };
+            const uint32_t idesc_qk = ptx::idesc_i8(128, P.n_k, 1, 1, 0);
+            const uint32_t idesc_pv = ptx::idesc_i8(128, 64, 0, 1, 1);
+            const uint64_t q_desc = ptx::smem_desc(gbase + P.off_q, 16, 512, ptx::SWIZZLE_64B);
+            const uint64_t k_desc = ptx::smem_desc(gbase + P.off_k, 16, 512, ptx::SWIZZLE_64B);
+            const uint64_t v_desc = ptx::smem_desc(gbase + P.off_v, 16, 512, ptx::SWIZZLE_64B);
+            const int pv_steps = P.kv_rows / 32;
+            bool ok = true;
+            int pending = -1;                       // local index of the item whose loads are in flight
+            if (item0 < P.total_items) { issue_loads(item0); pending = 0; }
+            int n = 0;
+            for (int item = item0; ok && item < P.total_items; item += item_stride, ++n) {
+                const uint32_t ph = (uint32_t)n & 1u;
+                if (!mbar_wait(ptx::smem_addr(&B.ops_ready), ph, abort_ptr)) { ok = false; break; }
+                pending = -1;
+                if (item + item_stride < P.total_items) { issue_loads(item + item_stride); pending = n + 1; }
+                if (n > 0 && !mbar_wait(ptx::smem_addr(&B.o_done), ph ^ 1u, abort_ptr)) { ok = false; break; }
+                ptx::tc_fence_after();
+                for (int k = 0; k < 2; ++k)                        // K = 64 -> two MMAs of 32
+                    ptx::mma_i8(tmem_grp, q_desc + (uint64_t)(k * 2), k_desc + (uint64_t)(k * 2), idesc_qk, k);
+                ptx::mma_commit(ptx::smem_addr(&B.s_full));
+                if (!mbar_wait(ptx::smem_addr(&B.p_ready), ph, abort_ptr)) { ok = false; break; }
+                ptx::tc_fence_after();
+                for (int ks = 0; ks < pv_steps; ++ks) {
+                    const uint64_t p_desc = ptx::smem_desc(gbase + P.off_p + (uint32_t)(ks >> 2) * 16384u, 16, 1024,
+                                                           ptx::SWIZZLE_128B) + (uint64_t)((ks & 3) * 2);
+                    ptx::mma_i8(tmem_grp, p_desc, v_desc + (uint64_t)(ks * 128), idesc_pv, ks);
+                }
+                ptx::mma_commit(ptx::smem_addr(&B.o_full));
+            }
+            if (!ok && pending >= 0) {
+                // give the copies still in flight a bounded chance to land before the CTA exits
+                const uint32_t bar = ptx::smem_addr(&B.packed_full);
+                for (int spin = 0; spin < (1 << 20) && !ptx::mbar_try_wait(bar, (uint32_t)pending & 1u); ++spin) {}
+            }
+        }
+    } else {
+        // ------------------------------ compute warps ------------------------------------
+        const int wq = warp % AT_COMPUTE_WARPS;                     // TMEM lane quarter
+        const int tid_g = wq * 32 + lane;                           // 0..127 within the group
+        const int row = tid_g;                                      // query row of the tile
+        const uint32_t t_row = tmem_grp + ((uint32_t)(wq * 32) << 16);
+        const char* const tab_mid = reinterpret_cast<const char*>(smem_gen + P.off_table) + (size_t)P.smax * 4;
+        float* const colp = reinterpret_cast<float*>(ggen + P.off_col);   // alpha[64], beta[64] of this head
+        const int sh_idx = 2 * (8 - C) - 2;                         // scaled score -> byte offset 4*S
+        const int chunks = P.kv_rows / 32;
+        const int tab_half = 4 * P.smax;
+        const Divisor dv = make_divisor(P.p_step);
+        bool ok = true;
+        int n = 0;
+        for (int item = item0; ok && item < P.total_items; item += item_stride, ++n) {
+            const uint32_t ph = (uint32_t)n & 1u;
+            int b, h, qt;
+            item_coords(item, b, h, qt);
+            // ---- operands: packed -> int8 -------------------------------------------------
+            bool w = mbar_wait(ptx::smem_addr(&B.packed_full), ph, abort_ptr);
+            if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+            unpack_rows64<C, 1>(ggen + P.off_pq, ggen + P.off_q, 128, tid_g, 128);
+            unpack_rows64<C, 1>(ggen + P.off_pk, ggen + P.off_k, P.n_k, tid_g, 128);
+            unpack_rows64<C, 1>(ggen + P.off_pv, ggen + P.off_v, P.kv_rows, tid_g, 128);
+            if (tid_g < 64) colp[tid_g] = __ldg(P.alpha_o + h * 64 + tid_g);
+            else colp[tid_g] = P.beta_o ? __ldg(P.beta_o + h * 64 + (tid_g - 64)) : 0.0f;
+            ptx::fence_proxy_async_smem();
+            // the four warps exchange the staged column parameters through shared memory
+            ptx::mbar_arrive(ptx::smem_addr(&B.grp_sync));
+            w = mbar_wait(ptx::smem_addr(&B.grp_sync), ph, abort_ptr);
+            if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&B.ops_ready));
+            // ---- softmax over the row -------------------------------------------------------
+            w = mbar_wait(ptx::smem_addr(&B.s_full), ph, abort_ptr);
+            if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+            ptx::tc_fence_after();
+            double z = 0.0;
+            for (int ch = 0; ch < chunks; ++ch) {
+                uint32_t v[32];
+                ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    // columns past the last token hold no score: no lookup there
+                    const bool valid = ch * 32 + i < T;
+                    int off = valid ? ((int)v[i] >> sh_idx) : 0;   // 4 * S
+                    off = max(-tab_half, min(tab_half, off));            // never index outside the table
+                    float e = *reinterpret_cast<const float*>(tab_mid + off);
+                    if (!valid) e = 0.0f;
+                    z += (double)e;
+                    v[i] = __float_as_uint(e);
+                }
+                ptx::tmem_st32(t_row + (uint32_t)(ch * 32), v);
+            }
+            ptx::tmem_st_wait();
+            const double rz = 1.0 / z;
+            const float rzh = (float)rz;
+            const float rzl = (float)(rz - (double)rzh);
+            uint8_t* const prow = ggen + P.off_p + row * 128;
+            const int sw = row & 7;
+            for (int ch = 0; ch < chunks; ++ch) {
+                uint32_t v[32];
+                ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
+                ptx::tmem_ld_wait();
+                uint32_t wd[8];
+#pragma unroll
+                for (int i4 = 0; i4 < 8; ++i4) {
+                    uint32_t word = 0;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float e = __uint_as_float(v[4 * i4 + j]);
+                        const float p = fmaf(e, rzh, e * rzl);
+                        word |= (round_clamp_bits(div_rn(p, dv), 0.0f, P.p_qp) & 0xFFu) << (8 * j);
+                    }
+                    wd[i4] = word;
+                }
+                // 32 codes = two 16-byte chunks cc = 2*ch, 2*ch+1 of this row's 256-byte K extent
+                const int cc = 2 * ch;
+                uint8_t* const blk = prow + (cc >> 3) * 16384;
+                *reinterpret_cast<uint4*>(blk + (((cc & 7) ^ sw) << 4)) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                *reinterpret_cast<uint4*>(blk + ((((cc + 1) & 7) ^ sw) << 4)) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
+            }
+            ptx::fence_proxy_async_smem();
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&B.p_ready));
+            // ---- O = P V: requantize and store ------------------------------------------------
+            w = mbar_wait(ptx::smem_addr(&B.o_full), ph, abort_ptr);
+            if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+            ptx::tc_fence_after();
+            const int token = qt * 128 + row;
+            uint32_t ow[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) ow[k] = 0;
+            const uint32_t omask = (1u << P.out_c) - 1u;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t v[32];
+                ptx::tmem_ld32(t_row + (uint32_t)(half * 32), v);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int col = half * 32 + i;
+                    const float f = small_int_to_float((int)v[i] >> (8 - C));
+                    const float y = fmaf(f, colp[col], colp[64 + col]);
+                    const uint32_t code = round_clamp_bits(y, P.out_qn, P.out_qp) & omask;
+                    if (P.out_c == 4) ow[col >> 3] |= code << (4 * (col & 7));
+                    else if (P.out_c == 2) ow[col >> 4] |= code << (2 * (col & 15));
+                    else ow[col >> 2] |= code << (8 * (col & 3));
+                }
+            }
+            if (token < T) {
+                uint8_t* o = P.out + ((long long)b * T + token) * P.out_pitch + (long long)h * (8 * P.out_c);
+                const int nwords = 2 * P.out_c;                     // 64 codes
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (4 * k < nwords)
+                        reinterpret_cast<uint4*>(o)[k] = make_uint4(ow[4 * k], ow[4 * k + 1], ow[4 * k + 2], ow[4 * k + 3]);
+            }
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&B.o_done));
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == AT_GROUPS * AT_COMPUTE_WARPS) {
+        ptx::tc_fence_after();
+        __syncwarp();
+        ptx::tmem_dealloc(tmem_base_slot, 512);
+    }
+}
+
+inline uint32_t up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+}  // namespace vitint
+
+using namespace vitint;
+
+extern "C" size_t vitint_attention_core_workspace_bytes(int32_t bits) {
+    if (bits != 2 && bits != 3 && bits != 4) return 0;
+    const int m = 1 << (container_bits(bits) - 1);   // sized by the container: any bit pattern indexes inside
+    return (size_t)(2 * 64 * m * m + 1) * sizeof(float) + 256;
+}
+
+extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
+                                     float q_step, float k_step, float p_step, int32_t p_bits, const float* alpha_o,
+                                     const float* beta_o, const vitint_codes* o_out, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+    if (int rc = check_codes(qkv)) return rc;
+    if (int rc = check_codes(o_out)) return rc;
+    if (batch <= 0 || heads <= 0 || tokens <= 0 || !alpha_o) return VITINT_ERR_INVALID_ARG;
+    const int64_t M = (int64_t)batch * tokens, D = (int64_t)heads * 64;
+    if (qkv->rows != M || qkv->cols != 3 * D || !qkv->is_signed || o_out->rows != M || o_out->cols != D)
+        return VITINT_ERR_INVALID_ARG;
+    const float steps[3] = {q_step, k_step, p_step};
+    for (float s : steps) if (!(s > 0.0f && s < INFINITY)) return VITINT_ERR_INVALID_ARG;
+    if (!valid_bits(p_bits)) return VITINT_ERR_INVALID_ARG;
+    if (qkv->bits == 8 || tokens > 256 || batch > 65535) return VITINT_ERR_UNSUPPORTED;
+    const int c = container_bits(qkv->bits);
+    const int m = 1 << (c - 1);
+    const int smax = 64 * m * m;
+    const float cs = (float)((double)q_step * (double)k_step / 8.0);
+    // exp without max subtraction must not overflow for any score the declared code range can produce
+    // (the table itself is sized by the container so that any bit pattern indexes inside it)
+    const int mq = 1 << (qkv->bits - 1);
+    if (64.0 * mq * mq * (double)cs > 80.0) return VITINT_ERR_UNSUPPORTED;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < vitint_attention_core_workspace_bytes(qkv->bits))
+        return VITINT_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    AttnParams P{};
+    P.batch = batch; P.heads = heads; P.tokens = tokens;
+    P.q_tiles = (tokens + 127) / 128;
+    P.total_items = batch * heads * P.q_tiles;
+    P.c = c;
+    P.n_k = (tokens + 15) / 16 * 16;
+    P.kv_rows = (tokens + 31) / 32 * 32;
+    P.smax = smax;
+    P.part_bytes = (int)(D * c / 8);
+    P.table = (const float*)workspace;
+    P.p_step = p_step;
+    int qn, qp;
+    code_range(p_bits, 0, &qn, &qp);
+    P.p_qp = (float)qp;
+    P.alpha_o = alpha_o; P.beta_o = beta_o;
+    P.out_c = container_bits(o_out->bits);
+    code_range(o_out->bits, o_out->is_signed, &qn, &qp);
+    P.out_qn = (float)qn; P.out_qp = (float)qp;
+    P.out = (uint8_t*)o_out->data; P.out_pitch = o_out->pitch_bytes;
+    // shared-memory layout
+    const uint32_t hb = 8u * c;
+    P.off_table = 0;
+    P.off_group = up((uint32_t)(2 * smax + 1) * 4u, 1024);
+    uint32_t o = 0;
+    P.off_q = o; o += 128 * 64;
+    P.off_k = o; o += up((uint32_t)P.n_k * 64, 1024);
+    P.off_v = o; o += up((uint32_t)P.kv_rows * 64, 1024);
+    P.off_p = o; o += (uint32_t)((P.kv_rows + 127) / 128) * 16384u;
+    P.off_pq = o; o += up(128 * hb, 128);
+    P.off_pk = o; o += up((uint32_t)P.kv_rows * hb, 128);
+    P.off_pv = o; o += up((uint32_t)P.kv_rows * hb, 128);
+    P.off_col = o; o += 512;
+    P.group_bytes = up(o, 1024);
+    const size_t smem = (size_t)P.off_group + (size_t)AT_GROUPS * P.group_bytes + 1024;
+    if (smem > 225 * 1024) return VITINT_ERR_UNSUPPORTED;
+
+    CUtensorMap map_q, map_kv;
+    {
+        // 3-D byte view of the QKV code matrix: (row bytes, token, image); rows past an image's
+        // last token read as zero.  Q tiles are 128 rows high, K and V tiles kv_rows.
+        EncodeTiledFn fn = encode_fn();
+        if (!fn) return VITINT_ERR_CUDA;
+        cuuint64_t dims[3] = {(cuuint64_t)row_bytes(3 * D, qkv->bits), (cuuint64_t)tokens, (cuuint64_t)batch};
+        cuuint64_t strides[2] = {(cuuint64_t)qkv->pitch_bytes, (cuuint64_t)qkv->pitch_bytes * tokens};
+        cuuint32_t estr[3] = {1, 1, 1};
+        cuuint32_t box_q[3] = {hb, 128, 1}, box_kv[3] = {hb, (cuuint32_t)P.kv_rows, 1};
+        if (fn(&map_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, qkv->data, dims, strides, box_q, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+            fn(&map_kv, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, qkv->data, dims, strides, box_kv, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return VITINT_ERR_CUDA;
+    }
+    exp_table_kernel<<<(2 * smax + 1 + 255) / 256, 256, 0, st>>>((float*)workspace, smax, cs);
+    if (cudaGetLastError() != cudaSuccess) return VITINT_ERR_CUDA;
+    int grid = sm_count();
+    const int want = (P.total_items + AT_GROUPS - 1) / AT_GROUPS;
+    if (grid > want) grid = want;
+    static bool attr2 = false, attr4 = false;
+    if (c == 4) {
+        if (!attr4) {
+            if (cudaFuncSetAttribute(attention_fused_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess)
+                return VITINT_ERR_CUDA;
+            attr4 = true;
+        }
+        attention_fused_kernel<4><<<grid, AT_THREADS, smem, st>>>(map_q, map_kv, P);
+    } else {
+        if (!attr2) {
+            if (cudaFuncSetAttribute(attention_fused_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess)
+                return VITINT_ERR_CUDA;
+            attr2 = true;
+        }
+        attention_fused_kernel<2><<<grid, AT_THREADS, smem, st>>>(map_q, map_kv, P);
+    }
+    return cuda_status(cudaGetLastError());
+}

@@ -3,4 +3,5 @@
 #include "quantize.cu"
 #include "softmax.cu"
 #include "gemm.cu"
+#include "attention_fused.cu"
 #include "attention.cu"

@@ -11,8 +11,10 @@ import torch
 
 from . import binding as B
 
-STAGES = ("ln1_quant", "qkv_linear", "qk", "softmax_quant", "pv", "proj_linear", "ln2_quant", "fc1_linear",
-          "fc2_linear")
+STAGES_UNFUSED = ("ln1_quant", "qkv_linear", "qk", "softmax_quant", "pv", "proj_linear", "ln2_quant", "fc1_linear",
+                  "fc2_linear")
+STAGES_FUSED = ("ln1_quant", "qkv_linear", "attention_core", "proj_linear", "ln2_quant", "fc1_linear", "fc2_linear")
+# stages that run in the integer GEMM kernel
 GEMM_STAGES = ("qkv_linear", "qk", "pv", "proj_linear", "fc1_linear", "fc2_linear")
 
 
@@ -22,12 +24,14 @@ def _dev(a, device):
 
 class EncoderLayer:
     def __init__(self, batch: int, tokens: int, heads: int, mlp_dim: int, bits: int, prm: dict, device="cuda",
-                 eps: float = 1e-6, widen_weights: bool = True):
+                 eps: float = 1e-6, widen_weights: bool = True, fused_attention: bool = True):
         self.batch, self.tokens, self.heads, self.bits, self.eps = batch, tokens, heads, bits, eps
         self.dim = D = heads * 64
         self.mlp_dim = F = mlp_dim
         self.rows = M = batch * tokens
         self.device = device
+        self.fused_attention = fused_attention and bits != 8 and tokens <= 256
+        self.stages = STAGES_FUSED if self.fused_attention else STAGES_UNFUSED
         d = lambda a: _dev(a, device)
         f = lambda k: float(prm[k])
         self.s_ln, self.s_q, self.s_k, self.s_v = f("s_ln"), f("s_q"), f("s_k"), f("s_v")
@@ -55,8 +59,11 @@ class EncoderLayer:
         self.x1 = B.Codes.empty(M, D, bits, True, device)
         self.qkv = B.Codes.empty(M, 3 * D, bits, True, device)
         self.ld_s = (tokens + 3) // 4 * 4
-        self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
-        self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
+        if self.fused_attention:
+            self.attn_ws = torch.empty(B.vitint_attention_core_workspace_bytes(bits), dtype=torch.uint8, device=device)
+        else:
+            self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
+            self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
         self.O = B.Codes.empty(M, D, bits, True, device)
         self.h = torch.empty((M, D), dtype=torch.float32, device=device)
         self.x2 = B.Codes.empty(M, D, bits, True, device)
@@ -69,7 +76,7 @@ class EncoderLayer:
 
     def forward(self, x: torch.Tensor, out: torch.Tensor, events: list | None = None) -> torch.Tensor:
         """x, out: fp32 [batch*tokens, dim] on the device.  `events`, when given, receives
-        len(STAGES)+1 recorded CUDA events bracketing the stages."""
+        len(self.stages)+1 recorded CUDA events bracketing the stages."""
         def mark():
             if events is not None:
                 e = torch.cuda.Event(enable_timing=True)
@@ -81,11 +88,15 @@ class EncoderLayer:
         mark()
         B.vitint_linear(self.x1, self.s_ln, self.w["qkv"], None, None, self.epi_qkv, out=self.qkv)
         mark()
-        B.vitint_qk(self.slabs[0], self.slabs[1], b, h, t, out=self.S, ld_s=self.ld_s)
-        mark()
-        B.vitint_softmax_quantize(self.S, t, self.c, self.s_p, self.bits, out=self.P)
-        mark()
-        B.vitint_pv(self.P, self.slabs[2], b, h, t, self.s_p, self.s_v, self.epi_o, out=self.O)
+        if self.fused_attention:
+            B.vitint_attention_core(self.qkv, b, h, t, self.s_q, self.s_k, self.s_p, self.bits, self.alpha_o, None,
+                                    out=self.O, workspace=self.attn_ws)
+        else:
+            B.vitint_qk(self.slabs[0], self.slabs[1], b, h, t, out=self.S, ld_s=self.ld_s)
+            mark()
+            B.vitint_softmax_quantize(self.S, t, self.c, self.s_p, self.bits, out=self.P)
+            mark()
+            B.vitint_pv(self.P, self.slabs[2], b, h, t, self.s_p, self.s_v, self.epi_o, out=self.O)
         mark()
         B.vitint_linear(self.O, self.s_o, self.w["proj"], self.s_w["proj"], self.bias["proj"],
                         B.Epilogue(mode=B.EPI_DEQUANT_F32, residual=x), out=self.h)
@@ -104,7 +115,8 @@ class EncoderLayer:
         M, D, F, T = self.rows, self.dim, self.mlp_dim, self.tokens
         n = self.batch * self.heads
         return {"qkv_linear": 2 * M * D * 3 * D, "qk": 2 * n * T * T * 64, "pv": 2 * n * T * T * 64,
-                "proj_linear": 2 * M * D * D, "fc1_linear": 2 * M * D * F, "fc2_linear": 2 * M * F * D}
+                "attention_core": 4 * n * T * T * 64, "proj_linear": 2 * M * D * D, "fc1_linear": 2 * M * D * F,
+                "fc2_linear": 2 * M * F * D}
 
     def stage_bytes(self) -> dict:
         """Algorithmic HBM bytes of the streaming stages (4 + c/8 per element)."""

@@ -18,15 +18,17 @@ vt = pytest.importorskip("paper_2504_18547_b200")
 from gpu_util import dev, from_codes  # noqa: E402
 
 
+@pytest.mark.parametrize("fused", [True, False], ids=["fused_attention", "unfused_attention"])
 @pytest.mark.parametrize("bits", [4, 3, 2])
-def test_encoder_layer_staged(bits):
+def test_encoder_layer_staged(bits, fused):
     from paper_2504_18547_b200.encoder import EncoderLayer
     cfg = si.VIT_BASE_LAYER.with_(batch=3, bits=bits)
     prm = si.layer_parameters(cfg)
     x = si.activations(cfg)
     st = vp.encoder_layer(x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits)
     att = st["attn"]
-    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm)
+    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, fused_attention=fused)
+    assert layer.fused_attention == fused
     out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
     layer.forward(dev(x), out)
     assert vt.vitint_device_status() == 0
@@ -44,10 +46,14 @@ def test_encoder_layer_staged(bits):
     qkv = from_codes(layer.qkv)
     assert np.array_equal(qkv[rows_img], att["qkv_codes"][rows_img])
 
-    P = from_codes(layer.P).reshape(B * H, T, T)
     prob_ok = np.repeat(img_ok, H)
-    assert np.all(P[prob_ok] >= att["p_lo"][prob_ok]) and np.all(P[prob_ok] <= att["p_hi"][prob_ok])
-    p_row_ok = (P == att["p_codes"]).all(axis=2) & prob_ok[:, None]           # [B*H, T]
+    if fused:
+        # P never leaves the SM: rows whose every code is unique under the 2-ulp band must agree downstream
+        p_row_ok = (att["p_lo"] == att["p_hi"]).all(axis=2) & prob_ok[:, None]
+    else:
+        P = from_codes(layer.P).reshape(B * H, T, T)
+        assert np.all(P[prob_ok] >= att["p_lo"][prob_ok]) and np.all(P[prob_ok] <= att["p_hi"][prob_ok])
+        p_row_ok = (P == att["p_codes"]).all(axis=2) & prob_ok[:, None]           # [B*H, T]
     assert p_row_ok[prob_ok].mean() > 0.97
 
     O = from_codes(layer.O)

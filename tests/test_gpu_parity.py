@@ -256,6 +256,43 @@ def test_softmax_error_statistics_on_attention_like_rows():
     assert np.all(g >= lo) and np.all(g <= hi)
 
 
+@pytest.mark.parametrize("bits", [4, 2, 3])
+@pytest.mark.parametrize("batch,tokens,heads,scale", [(1, 197, 3, 1.0), (3, 197, 2, 3.0), (2, 50, 1, 3.0), (1, 256, 2, 2.0),
+                                                      (5, 128, 1, 0.3), (2, 129, 2, 2.5)])
+def test_attention_core_fused(batch, tokens, heads, bits, scale):
+    """Fused Q K^T -> softmax -> P V against the oracle stages; rows whose P codes are unique must be bit-exact."""
+    D = heads * 64
+    qkv = _qkv_codes(batch, tokens, heads, bits, 61 + tokens)
+    qmax = si.code_range(bits, True)[1] + 1
+    # random codes give scores with spread ~ 8*qmax^2/3; choose the steps so the logits' spread is `scale`
+    s_q = s_k = np.float32(math.sqrt(8.0 * scale * 3.0 / (8.0 * qmax * qmax)))
+    s_p = np.float32(2.0 / (tokens * math.sqrt(si.code_range(bits, False)[1])))
+    q = vp.split_heads(qkv, batch, tokens, heads, 64, 0)
+    k = vp.split_heads(qkv, batch, tokens, heads, 64, D)
+    v = vp.split_heads(qkv, batch, tokens, heads, 64, 2 * D)
+    S = vo.qk(q, k)
+    c = vp.softmax_scale(s_q, s_k, 64)
+    n = batch * heads
+    _, pc, plo, phi = vo.softmax_quantize(S.reshape(n * tokens, tokens), c, s_p, bits)
+    acc = vo.pv(pc.reshape(n, tokens, tokens), v)
+    alpha, beta = vp.fold(s_p, np.full(D, 0.17, np.float32), None, np.float32(0.17 * 0.6 * qmax / math.sqrt(8 * scale + 1)))
+    beta = si.normal(5, (D,), 0.0, 0.3)
+    want = vo.epilogue_requant(vp.merge_heads(acc, batch, tokens, heads, 64), alpha, beta, bits, True)
+    got = from_codes(vt.vitint_attention_core(to_codes(qkv, bits, True), batch, heads, tokens, s_q, s_k, s_p, bits,
+                                              dev(alpha), dev(beta)))
+    unique_row = (plo == phi).all(axis=1).reshape(n, tokens)             # [B*H, T]
+    ok = np.ones((batch * tokens, D), bool)
+    for b in range(batch):
+        for h in range(heads):
+            ok[b * tokens:(b + 1) * tokens, h * 64:(h + 1) * 64] = unique_row[b * heads + h][:, None]
+    assert ok.mean() > 0.8
+    assert np.array_equal(got[ok], want[ok])
+    assert np.all(np.abs(got.astype(int) - want) <= 1)
+    assert len(np.unique(want)) >= 3
+    if scale >= 1.0:
+        assert len(np.unique(pc)) >= 3
+
+
 # ---------------------------------------------------------------------------
 # glue
 # ---------------------------------------------------------------------------

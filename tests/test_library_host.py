@@ -96,8 +96,12 @@ def test_attention_workspace_query_and_errors(L):
     d.batch, d.tokens, d.heads, d.bits, d.p_bits = 2, 197, 3, 4, 4
     n = lib.vitint_attention_block_workspace_bytes(ctypes.byref(d))
     M, D = 2 * 197, 192
-    expect_min = M * 288 + 2 * 3 * 197 * 200 * 4 + 2 * 3 * 197 * 112 + M * 96
-    assert expect_min <= n <= expect_min + 4 * 256
+    expect_min = M * 288 + 2 * 3 * 197 * 200 * 4 + 2 * 3 * 197 * 112 + M * 96 + (2 * 4096 + 1) * 4 + 256
+    assert expect_min <= n <= expect_min + 5 * 256
+    assert lib.vitint_attention_core_workspace_bytes(4) == (2 * 4096 + 1) * 4 + 256
+    assert lib.vitint_attention_core_workspace_bytes(3) == (2 * 4096 + 1) * 4 + 256
+    assert lib.vitint_attention_core_workspace_bytes(2) == (2 * 256 + 1) * 4 + 256
+    assert lib.vitint_attention_core_workspace_bytes(8) == 0
     d.batch = 0
     assert lib.vitint_attention_block_workspace_bytes(ctypes.byref(d)) == 0
     d.batch = 2
