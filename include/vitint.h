@@ -181,6 +181,29 @@ int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int32_t heads,
                           float k_step, float p_step, int32_t p_bits, const float* alpha_o, const float* beta_o,
                           const vitint_codes* o_out, void* workspace, size_t workspace_bytes, void* stream);
 
+/* vitint_attention_core without caller-provided scratch.  (No counterpart in the paper: this is
+ *   a packaging variant, not a step of the method.)
+ *   Who needs it: code that is not allowed to obtain device memory when it runs the attention
+ *   core -- for example a plug-in inside a serving process whose whole device-memory budget was
+ *   handed out at start-up by another component, or a latency-critical loop that must avoid
+ *   cudaMalloc / cudaFree because those calls may synchronize the device.  Such callers still
+ *   pass their own input (qkv) and output (o_out) buffers; only the kernel's scratch -- the table
+ *   of exp(fl32(s*c)) over all integer scores -- comes from the library: a fixed device array of
+ *   33,280 bytes that every GPU loading the library holds until the process exits.
+ *   The function allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.
+ *   Limit: the table must fit the array, i.e. 2-, 3- and 4-bit codes (at most 8193 entries);
+ *   anything larger is rejected with VITINT_ERR_WORKSPACE (8-bit codes: VITINT_ERR_UNSUPPORTED,
+ *   as in vitint_attention_core).  All other arguments, results and errors are those of
+ *   vitint_attention_core.
+ *   The first call on each device looks up the array's device address (with that device
+ *   current); make that first call outside any stream capture.
+ *   Every call on a device uses the same array and rewrites all the entries it needs, so nothing
+ *   carries over between calls -- but two calls that overlap on the GPU (different streams) race
+ *   on it: serialize calls per device. */
+int vitint_attention_core_noalloc(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
+                                  float q_step, float k_step, float p_step, int32_t p_bits, const float* alpha_o,
+                                  const float* beta_o, const vitint_codes* o_out, void* stream);
+
 /* a7. Integerized self-attention block (Fig. 1(b)):
  *   QKV linear (requantized with per-channel alpha_qkv/beta_qkv, i.e. three per-tensor
  *   steps q_step, k_step, v_step laid out per output channel) -> Q K^T -> scale, softmax,

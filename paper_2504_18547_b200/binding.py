@@ -74,6 +74,8 @@ def lib():
         L.vitint_attention_core_workspace_bytes.argtypes = [c_int32]
         L.vitint_attention_core.argtypes = [POINTER(_Codes), c_int32, c_int32, c_int32, c_float, c_float, c_float,
                                             c_int32, c_void_p, c_void_p, POINTER(_Codes), c_void_p, c_size_t, c_void_p]
+        L.vitint_attention_core_noalloc.argtypes = [POINTER(_Codes), c_int32, c_int32, c_int32, c_float, c_float, c_float,
+                                                    c_int32, c_void_p, c_void_p, POINTER(_Codes), c_void_p]
         L.vitint_attention_block_workspace_bytes.restype = c_size_t
         L.vitint_attention_block_workspace_bytes.argtypes = [POINTER(_AttentionDesc)]
         L.vitint_attention_block.argtypes = [POINTER(_Codes), POINTER(_AttentionDesc), c_void_p, c_int64,
@@ -291,6 +293,18 @@ def vitint_attention_core(qkv: Codes, batch: int, heads: int, tokens: int, q_ste
     _check(lib().vitint_attention_core(byref(dq), batch, heads, tokens, float(q_step), float(k_step), float(p_step),
                                        p_bits, _ptr(alpha_o), _ptr(beta_o), byref(do), workspace.data_ptr(),
                                        workspace.numel(), _stream()), "vitint_attention_core")
+    return out
+
+
+def vitint_attention_core_noalloc(qkv: Codes, batch: int, heads: int, tokens: int, q_step: float, k_step: float,
+                                  p_step: float, p_bits: int, alpha_o: torch.Tensor, beta_o: torch.Tensor | None,
+                                  out: Codes) -> Codes:
+    """vitint_attention_core for callers that may not allocate device memory: the kernel's scratch is a
+    fixed array inside the library and `out` must be supplied.  This wrapper allocates nothing either."""
+    dq, do = qkv.desc(), out.desc()
+    _check(lib().vitint_attention_core_noalloc(byref(dq), batch, heads, tokens, float(q_step), float(k_step),
+                                               float(p_step), p_bits, _ptr(alpha_o), _ptr(beta_o), byref(do),
+                                               _stream()), "vitint_attention_core_noalloc")
     return out
 
 

@@ -420,3 +420,50 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     }
     return cuda_status(cudaGetLastError());
 }
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free variant: the exp table lives in a fixed device array of this library.
+// ---------------------------------------------------------------------------------------
+namespace vitint {
+namespace {
+
+constexpr int STATIC_TABLE_FLOATS = 8320;   // largest table (8193 entries, 4-bit containers) plus the 256-byte slack of the workspace query
+
+// Resident on every GPU that loads the library, from load until the process exits (about 33 KB).
+static __device__ __align__(256) float g_static_exp_table[STATIC_TABLE_FLOATS];
+
+constexpr int MAX_DEVICES = 64;
+void* g_static_table_addr[MAX_DEVICES];   // device address of the array, per device, once looked up
+bool g_static_table_ready[MAX_DEVICES];
+
+// The array's name is only a host-side handle; kernels need its device address.  Looked up once
+// per device, with that device current.
+int static_table_address(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return VITINT_ERR_CUDA;
+    if (!g_static_table_ready[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_exp_table) != cudaSuccess || !p) return VITINT_ERR_CUDA;
+        g_static_table_addr[dev] = p;
+        g_static_table_ready[dev] = true;
+    }
+    *out = g_static_table_addr[dev];
+    return VITINT_OK;
+}
+
+}  // namespace
+}  // namespace vitint
+
+extern "C" int vitint_attention_core_noalloc(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
+                                             float q_step, float k_step, float p_step, int32_t p_bits,
+                                             const float* alpha_o, const float* beta_o, const vitint_codes* o_out,
+                                             void* stream) {
+    if (!qkv) return VITINT_ERR_INVALID_ARG;
+    const size_t need = vitint_attention_core_workspace_bytes(qkv->bits);
+    if (need == 0) return VITINT_ERR_UNSUPPORTED;                     // 8-bit codes: no table-driven kernel
+    if (need > sizeof(float) * STATIC_TABLE_FLOATS) return VITINT_ERR_WORKSPACE;   // beyond the built-in scratch
+    void* table = nullptr;
+    if (int rc = static_table_address(&table)) return rc;
+    return vitint_attention_core(qkv, batch, heads, tokens, q_step, k_step, p_step, p_bits, alpha_o, beta_o, o_out,
+                                 table, sizeof(float) * STATIC_TABLE_FLOATS, stream);
+}
