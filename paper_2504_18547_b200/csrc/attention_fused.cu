@@ -205,21 +205,32 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             w = mbar_wait(ptx::smem_addr(&B.s_full), ph, abort_ptr);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
             ptx::tc_fence_after();
+            // pass 1: e_j = EXP[S_j] (an integer score is bounded by the code ranges, so the byte offset
+            // 4*S always lies inside the table), row sum in fp64, e_j parked in TMEM over S_j
             double z = 0.0;
+            const int full_chunks = T >> 5;
             for (int ch = 0; ch < chunks; ++ch) {
                 uint32_t v[32];
                 ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
                 ptx::tmem_ld_wait();
+                if (ch < full_chunks) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    // columns past the last token hold no score: no lookup there
-                    const bool valid = ch * 32 + i < T;
-                    int off = valid ? ((int)v[i] >> sh_idx) : 0;   // 4 * S
-                    off = max(-tab_half, min(tab_half, off));            // never index outside the table
-                    float e = *reinterpret_cast<const float*>(tab_mid + off);
-                    if (!valid) e = 0.0f;
-                    z += (double)e;
-                    v[i] = __float_as_uint(e);
+                    for (int i = 0; i < 32; ++i) {
+                        const float e = *reinterpret_cast<const float*>(tab_mid + ((int)v[i] >> sh_idx));
+                        z += (double)e;
+                        v[i] = __float_as_uint(e);
+                    }
+                } else {
+                    // last, partial chunk: columns past the last token hold no score -> no lookup, e = 0
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const bool valid = ch * 32 + i < T;
+                        const int off = valid ? ((int)v[i] >> sh_idx) : 0;
+                        float e = *reinterpret_cast<const float*>(tab_mid + max(-tab_half, min(tab_half, off)));
+                        if (!valid) e = 0.0f;
+                        z += (double)e;
+                        v[i] = __float_as_uint(e);
+                    }
                 }
                 ptx::tmem_st32(t_row + (uint32_t)(ch * 32), v);
             }
@@ -229,6 +240,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const float rzl = (float)(rz - (double)rzh);
             uint8_t* const prow = ggen + P.off_p + row * 128;
             const int sw = row & 7;
+            // pass 2: p_j = RN(e_j / Z), code = min(rint(RN(p_j / s_P)), Qp) (p >= 0: no lower clamp)
             for (int ch = 0; ch < chunks; ++ch) {
                 uint32_t v[32];
                 ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
@@ -236,14 +248,14 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 uint32_t wd[8];
 #pragma unroll
                 for (int i4 = 0; i4 < 8; ++i4) {
-                    uint32_t word = 0;
+                    uint32_t cb[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const float e = __uint_as_float(v[4 * i4 + j]);
                         const float p = fmaf(e, rzh, e * rzl);
-                        word |= (round_clamp_bits(div_rn(p, dv), 0.0f, P.p_qp) & 0xFFu) << (8 * j);
+                        cb[j] = __float_as_uint(fminf(div_rn(p, dv), P.p_qp) + 12582912.0f);   // code in the low byte
                     }
-                    wd[i4] = word;
+                    wd[i4] = __byte_perm(__byte_perm(cb[0], cb[1], 0x4040), __byte_perm(cb[2], cb[3], 0x4040), 0x5410);
                 }
                 // 32 codes = two 16-byte chunks cc = 2*ch, 2*ch+1 of this row's 256-byte K extent
                 const int cc = 2 * ch;
@@ -263,21 +275,29 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             uint32_t ow[16];
 #pragma unroll
             for (int k = 0; k < 16; ++k) ow[k] = 0;
-            const uint32_t omask = (1u << P.out_c) - 1u;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t v[32];
                 ptx::tmem_ld32(t_row + (uint32_t)(half * 32), v);
                 ptx::tmem_ld_wait();
+                // straight-line per-column arithmetic first, container-dependent packing afterwards
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     const int col = half * 32 + i;
                     const float f = small_int_to_float((int)v[i] >> (8 - C));
-                    const float y = fmaf(f, colp[col], colp[64 + col]);
-                    const uint32_t code = round_clamp_bits(y, P.out_qn, P.out_qp) & omask;
-                    if (P.out_c == 4) ow[col >> 3] |= code << (4 * (col & 7));
-                    else if (P.out_c == 2) ow[col >> 4] |= code << (2 * (col & 15));
-                    else ow[col >> 2] |= code << (8 * (col & 3));
+                    v[i] = round_clamp_bits(fmaf(f, colp[col], colp[64 + col]), P.out_qn, P.out_qp);
+                }
+                if (P.out_c == 4) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) ow[half * 4 + (i >> 3)] |= (v[i] & 0xFu) << (4 * (i & 7));
+                } else if (P.out_c == 2) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) ow[half * 2 + (i >> 4)] |= (v[i] & 0x3u) << (2 * (i & 15));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        ow[half * 8 + i] = __byte_perm(__byte_perm(v[4 * i], v[4 * i + 1], 0x4040),
+                                                       __byte_perm(v[4 * i + 2], v[4 * i + 3], 0x4040), 0x5410);
                 }
             }
             if (token < T) {

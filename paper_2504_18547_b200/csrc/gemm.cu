@@ -168,8 +168,9 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     }
     float* of = (float*)P.out + orow * P.ld_out + colbase + n0;                   // DEQUANT
     const bool vec_out = FULL && ((reinterpret_cast<uintptr_t>(of) & 15u) == 0);
-    uint32_t wds[8] = {0, 0, 0, 0, 0, 0, 0, 0};                                   // REQUANT
-    const uint32_t mask = (1u << P.out_c) - 1u;
+    // The element loop below is straight-line code (no branch on run-time parameters), so the 32
+    // independent per-column chains can overlap; the container width is only looked at when packing.
+    uint32_t code[32];                                                            // REQUANT
 #pragma unroll
     for (int i4 = 0; i4 < 8; ++i4) {
         const float4 a4 = *reinterpret_cast<const float4*>(pa + 4 * i4);
@@ -191,13 +192,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
             if (KIND == EK_REQUANT_GELU) val = val * qq[j];
             if (has_res) val = val + rr[j];
             y[j] = val;
-            if (!deq) {
-                const uint32_t code = (FULL || i < nvalid) ? (round_clamp_bits(val, P.out_qn, P.out_qp) & mask) : 0u;
-                // static word index for each container width keeps wds[] in registers
-                if (P.out_c == 4) wds[i >> 3] |= code << (4 * (i & 7));
-                else if (P.out_c == 2) wds[i >> 4] |= code << (2 * (i & 15));
-                else wds[i >> 2] |= code << (8 * (i & 3));
-            }
+            if (!deq) code[i] = round_clamp_bits(val, P.out_qn, P.out_qp);
         }
         if (deq) {
             if (vec_out) {
@@ -209,6 +204,23 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
         }
     }
     if (deq) return;
+    uint32_t wds[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (!FULL) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) if (i >= nvalid) code[i] = 0u;
+    }
+    if (P.out_c == 4) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) wds[i >> 3] |= (code[i] & 0xFu) << (4 * (i & 7));
+    } else if (P.out_c == 2) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) wds[i >> 4] |= (code[i] & 0x3u) << (2 * (i & 15));
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            wds[i] = __byte_perm(__byte_perm(code[4 * i], code[4 * i + 1], 0x4040),
+                                 __byte_perm(code[4 * i + 2], code[4 * i + 3], 0x4040), 0x5410);
+    }
     const int out_words = P.out_c;   // 32 codes = 4*out_c bytes
     const long long byte0 = ((colbase + n0) * P.out_c) >> 3;
     uint8_t* o = (uint8_t*)P.out + orow * P.ld_out + byte0;
