@@ -129,7 +129,7 @@ __device__ __forceinline__ bool epi_barrier(uint32_t bar, uint32_t parity, volat
 // Epilogue of one row x 32 columns.  v[]: accumulators scaled by 2^shift; pa/pb/pq: the 32
 // columns' parameters in shared memory (multiplier already carries 2^-shift).
 // FULL: all 32 columns exist and 16-byte vector accesses are legal.
-template <int KIND, bool FULL, bool SMALL>
+template <int KIND, bool FULL, bool SMALL, bool HAS_RES>
 __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32_t (&v)[32], const float* pa,
                                                const float* pb, const float* pq, long long orow, long long colbase,
                                                int n0) {
@@ -149,7 +149,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     }
     // residual first: independent 16-byte loads in flight while the arithmetic runs
     const bool deq = (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU);
-    const bool has_res = deq && P.residual != nullptr;
+    constexpr bool has_res = HAS_RES;
     float4 res[8];
     if (has_res) {
         const float* r = P.residual + orow * P.ld_res + colbase + n0;
@@ -251,8 +251,14 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiPara
             const float* pa = &ep.a[buf][chunk * 32];
             const float* pb = &ep.b[buf][chunk * 32];
             const float* pq = &ep.q[buf][chunk * 32];
-            if (n0 + 32 <= P.N) epilogue_chunk<KIND, true, SMALL>(P, v, pa, pb, pq, orow, colbase, n0);
-            else epilogue_chunk<KIND, false, SMALL>(P, v, pa, pb, pq, orow, colbase, n0);
+            constexpr bool can_res = (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU);
+            if (can_res && P.residual != nullptr) {
+                if (n0 + 32 <= P.N) epilogue_chunk<KIND, true, SMALL, can_res>(P, v, pa, pb, pq, orow, colbase, n0);
+                else epilogue_chunk<KIND, false, SMALL, can_res>(P, v, pa, pb, pq, orow, colbase, n0);
+            } else {
+                if (n0 + 32 <= P.N) epilogue_chunk<KIND, true, SMALL, false>(P, v, pa, pb, pq, orow, colbase, n0);
+                else epilogue_chunk<KIND, false, SMALL, false>(P, v, pa, pb, pq, orow, colbase, n0);
+            }
         }
         __syncwarp();
     }
