@@ -56,8 +56,11 @@ typedef struct {
     void* data;          /* device, 16-byte aligned */
     int64_t rows, cols;  /* logical code counts */
     int64_t pitch_bytes; /* multiple of 16, >= ceil(cols*c/8) */
-    int32_t bits;        /* 2, 3, 4 or 8 */
+    int32_t bits;        /* 2, 3, 4 or 8: the value range of the codes */
     int32_t is_signed;   /* 0 / 1 */
+    int32_t container_bits; /* 0: the default container of `bits` (2, 4, 4, 8); 8: b-bit codes stored one per
+                               byte (what vitint_widen produces).  Other values are invalid. */
+    int32_t reserved_;   /* set to 0 */
 } vitint_codes;
 
 typedef enum {
@@ -87,6 +90,8 @@ typedef struct {
     const float* inv_out_step;  /* REQUANT, act 1 */
     int32_t out_bits;           /* REQUANT: 2, 3, 4, 8 */
     int32_t out_signed;
+    int32_t out_container_bits; /* REQUANT: 0 = default container of out_bits, 8 = one code per byte */
+    int32_t reserved_;          /* set to 0 */
 } vitint_epilogue;
 
 const char* vitint_status_string(int status);
@@ -111,8 +116,8 @@ int64_t vitint_packed_pitch(int64_t cols, int32_t bits);
 int vitint_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, float step, const float* row_steps,
                     const vitint_codes* out, void* stream);
 
-/* Re-stores b-bit codes in 8-bit containers (same values, same signedness): out->bits must be 8,
- *   rows/cols equal to the input's.  Weights widened once this way let vitint_linear feed the
+/* Re-stores b-bit codes in 8-bit containers (same values, same signedness): out->bits equals
+ *   in->bits, out->container_bits is 8, rows/cols equal the input's.  Weights widened once this way let vitint_linear feed the
  *   tensor cores straight from the TMA copy, with no in-kernel unpacking of that operand; the
  *   value range of the codes is unchanged, so Eq. 1's integer contraction is the same.
  *   Errors: INVALID_ARG, ALIGNMENT. */

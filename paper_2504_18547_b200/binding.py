@@ -22,13 +22,14 @@ class VitintError(RuntimeError):
 
 class _Codes(Structure):
     _fields_ = [("data", c_void_p), ("rows", c_int64), ("cols", c_int64), ("pitch_bytes", c_int64),
-                ("bits", c_int32), ("is_signed", c_int32)]
+                ("bits", c_int32), ("is_signed", c_int32), ("container_bits", c_int32), ("reserved_", c_int32)]
 
 
 class _Epilogue(Structure):
     _fields_ = [("mode", c_int32), ("act", c_int32), ("residual", c_void_p), ("ld_res", c_int64),
                 ("alpha", c_void_p), ("beta", c_void_p), ("inv_out_step", c_void_p),
-                ("out_bits", c_int32), ("out_signed", c_int32)]
+                ("out_bits", c_int32), ("out_signed", c_int32), ("out_container_bits", c_int32),
+                ("reserved_", c_int32)]
 
 
 class _Slabs(Structure):
@@ -129,11 +130,18 @@ class Codes:
     cols: int
     bits: int
     signed: bool
+    container: int = 0        # 0: default container of `bits`; 8: one code per byte
 
     @staticmethod
-    def empty(rows: int, cols: int, bits: int, signed: bool, device="cuda", pitch: int | None = None) -> "Codes":
-        pitch = packed_pitch(cols, bits) if pitch is None else pitch
-        return Codes(torch.empty((rows, pitch), dtype=torch.uint8, device=device), rows, cols, bits, signed)
+    def empty(rows: int, cols: int, bits: int, signed: bool, device="cuda", pitch: int | None = None,
+              container: int = 0) -> "Codes":
+        pitch = packed_pitch(cols, container or bits) if pitch is None else pitch
+        return Codes(torch.empty((rows, pitch), dtype=torch.uint8, device=device), rows, cols, bits, signed, container)
+
+    @property
+    def stored_bits(self) -> int:
+        """Bits per stored code."""
+        return self.container or (4 if self.bits == 3 else self.bits)
 
     @staticmethod
     def from_packed(packed: np.ndarray, cols: int, bits: int, signed: bool, device="cuda") -> "Codes":
@@ -145,7 +153,8 @@ class Codes:
         return int(self.data.stride(0))
 
     def desc(self) -> _Codes:
-        return _Codes(self.data.data_ptr(), self.rows, self.cols, self.pitch, self.bits, int(self.signed))
+        return _Codes(self.data.data_ptr(), self.rows, self.cols, self.pitch, self.bits, int(self.signed),
+                      self.container, 0)
 
 
 @dataclass
@@ -158,11 +167,12 @@ class Epilogue:
     inv_out_step: torch.Tensor | None = None
     out_bits: int = 4
     out_signed: bool = True
+    out_container: int = 0
 
     def desc(self) -> _Epilogue:
         ld_res = _ld(self.residual) if self.residual is not None else 0
         return _Epilogue(self.mode, self.act, _ptr(self.residual), ld_res, _ptr(self.alpha), _ptr(self.beta),
-                         _ptr(self.inv_out_step), self.out_bits, int(self.out_signed))
+                         _ptr(self.inv_out_step), self.out_bits, int(self.out_signed), self.out_container, 0)
 
 
 @dataclass
@@ -213,7 +223,7 @@ def vitint_quantize(x: torch.Tensor, step: float, bits: int, signed: bool, row_s
 
 def vitint_widen(x: Codes, out: Codes | None = None) -> Codes:
     """The same codes in 8-bit containers (used once for weights)."""
-    out = Codes.empty(x.rows, x.cols, 8, x.signed, x.data.device) if out is None else out
+    out = Codes.empty(x.rows, x.cols, x.bits, x.signed, x.data.device, container=8) if out is None else out
     di, do = x.desc(), out.desc()
     _check(lib().vitint_widen(byref(di), byref(do), _stream()), "vitint_widen")
     return out
@@ -224,7 +234,7 @@ def _alloc_out(epi: Epilogue, rows: int, cols: int, device):
         return torch.empty((rows, cols), dtype=torch.int32, device=device)
     if epi.mode == EPI_DEQUANT_F32:
         return torch.empty((rows, cols), dtype=torch.float32, device=device)
-    return Codes.empty(rows, cols, epi.out_bits, epi.out_signed, device)
+    return Codes.empty(rows, cols, epi.out_bits, epi.out_signed, device, container=epi.out_container)
 
 
 def _out_ptr_ld(out):

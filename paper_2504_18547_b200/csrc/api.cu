@@ -10,7 +10,9 @@ int check_codes(const vitint_codes* c) {
     if (!valid_bits(c->bits) || (c->is_signed != 0 && c->is_signed != 1)) return VITINT_ERR_INVALID_ARG;
     if (c->rows <= 0 || c->cols <= 0) return VITINT_ERR_INVALID_ARG;
     if (!aligned16(c->data) || c->pitch_bytes % 16 != 0) return VITINT_ERR_ALIGNMENT;
-    if (c->pitch_bytes < row_bytes(c->cols, c->bits)) return VITINT_ERR_INVALID_ARG;
+    if (c->container_bits != 0 && c->container_bits != 8 && c->container_bits != container_bits(c->bits))
+        return VITINT_ERR_INVALID_ARG;
+    if (c->pitch_bytes < codes_row_bytes(c, c->cols)) return VITINT_ERR_INVALID_ARG;
     return VITINT_OK;
 }
 

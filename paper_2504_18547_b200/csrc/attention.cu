@@ -79,14 +79,14 @@ extern "C" int vitint_attention_block(const vitint_codes* x, const vitint_attent
     const int cbits = container_bits(d->bits);
 
     // 1. QKV linear, requantized per output channel (three per-tensor steps)
-    vitint_codes qkv{ws + L.off_qkv, L.M, 3 * L.D, L.pitch_qkv, d->bits, 1};
+    vitint_codes qkv{ws + L.off_qkv, L.M, 3 * L.D, L.pitch_qkv, d->bits, 1, 0, 0};
     vitint_epilogue e1{};
     e1.mode = VITINT_EPI_REQUANT; e1.alpha = d->alpha_qkv; e1.beta = d->beta_qkv;
     e1.out_bits = d->bits; e1.out_signed = 1;
     if (int rc = vitint_linear(x, 1.0f, &d->w_qkv, nullptr, nullptr, &e1, qkv.data, qkv.pitch_bytes, stream)) return rc;
     if (int rc = copy_codes(dbg_qkv, qkv.data, L.pitch_qkv, L.M, row_bytes(3 * L.D, d->bits), st)) return rc;
 
-    vitint_codes o{ws + L.off_o, L.M, L.D, L.pitch_o, d->bits, 1};
+    vitint_codes o{ws + L.off_o, L.M, L.D, L.pitch_o, d->bits, 1, 0, 0};
     // 2-4 fused when the shape allows and no copy of P is wanted
     int fused = VITINT_ERR_UNSUPPORTED;
     if (!dbg_p && L.tab_bytes)
@@ -105,7 +105,7 @@ extern "C" int vitint_attention_block(const vitint_codes* x, const vitint_attent
 
         // 3. P = quantize(softmax(c * S)),  c = s_q s_k / sqrt(64)
         const float c = (float)((double)d->q_step * (double)d->k_step / 8.0);
-        vitint_codes p{ws + L.off_p, L.n_rows_p, d->tokens, L.pitch_p, d->p_bits, 0};
+        vitint_codes p{ws + L.off_p, L.n_rows_p, d->tokens, L.pitch_p, d->p_bits, 0, 0, 0};
         if (int rc = vitint_softmax_quantize(S, L.n_rows_p, d->tokens, L.ld_s, c, d->p_step, &p, nullptr, 0, stream))
             return rc;
         if (int rc = copy_codes(dbg_p, p.data, L.pitch_p, L.n_rows_p, row_bytes(d->tokens, d->p_bits), st)) return rc;

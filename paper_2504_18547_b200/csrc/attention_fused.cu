@@ -209,7 +209,10 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // 4*S always lies inside the table), row sum in fp64, e_j parked in TMEM over S_j
             double z = 0.0;
             const int full_chunks = T >> 5;
-            for (int ch = 0; ch < chunks; ++ch) {
+            // a warp whose 32 query rows all lie past the last token has nothing to compute: its P rows
+            // only feed accumulator rows that are never stored (whatever int8 they hold)
+            const bool warp_live = qt * 128 + wq * 32 < T;
+            for (int ch = 0; warp_live && ch < chunks; ++ch) {
                 uint32_t v[32];
                 ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
                 ptx::tmem_ld_wait();
@@ -235,13 +238,13 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 ptx::tmem_st32(t_row + (uint32_t)(ch * 32), v);
             }
             ptx::tmem_st_wait();
-            const double rz = 1.0 / z;
+            const double rz = warp_live ? 1.0 / z : 0.0;
             const float rzh = (float)rz;
             const float rzl = (float)(rz - (double)rzh);
             uint8_t* const prow = ggen + P.off_p + row * 128;
             const int sw = row & 7;
             // pass 2: p_j = RN(e_j / Z), code = min(rint(RN(p_j / s_P)), Qp) (p >= 0: no lower clamp)
-            for (int ch = 0; ch < chunks; ++ch) {
+            for (int ch = 0; warp_live && ch < chunks; ++ch) {
                 uint32_t v[32];
                 ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
                 ptx::tmem_ld_wait();
@@ -349,7 +352,7 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     const float steps[3] = {q_step, k_step, p_step};
     for (float s : steps) if (!(s > 0.0f && s < INFINITY)) return VITINT_ERR_INVALID_ARG;
     if (!valid_bits(p_bits)) return VITINT_ERR_INVALID_ARG;
-    if (qkv->bits == 8 || tokens > 256 || batch > 65535) return VITINT_ERR_UNSUPPORTED;
+    if (qkv->bits == 8 || qkv->container_bits == 8 || tokens > 256 || batch > 65535) return VITINT_ERR_UNSUPPORTED;
     const int c = container_bits(qkv->bits);
     const int m = 1 << (c - 1);
     const int smax = 64 * m * m;
@@ -378,7 +381,7 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     code_range(p_bits, 0, &qn, &qp);
     P.p_qp = (float)qp;
     P.alpha_o = alpha_o; P.beta_o = beta_o;
-    P.out_c = container_bits(o_out->bits);
+    P.out_c = codes_container(o_out);
     code_range(o_out->bits, o_out->is_signed, &qn, &qp);
     P.out_qn = (float)qn; P.out_qp = (float)qp;
     P.out = (uint8_t*)o_out->data; P.out_pitch = o_out->pitch_bytes;

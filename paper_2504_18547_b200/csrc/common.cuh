@@ -17,6 +17,9 @@ inline int container_bits(int bits) { return bits == 3 ? 4 : bits; }
 inline bool valid_bits(int bits) { return bits == 2 || bits == 3 || bits == 4 || bits == 8; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t row_bytes(int64_t cols, int bits) { return (cols * container_bits(bits) + 7) / 8; }
+// Container actually used by a code matrix (a descriptor may ask for one code per byte).
+inline int codes_container(const vitint_codes* c) { return c->container_bits ? c->container_bits : container_bits(c->bits); }
+inline int64_t codes_row_bytes(const vitint_codes* c, int64_t cols) { return (cols * codes_container(c) + 7) / 8; }
 inline int max_abs_code(int bits, int is_signed) { return is_signed ? (1 << (bits - 1)) : (1 << bits) - 1; }
 inline void code_range(int bits, int is_signed, int* qn, int* qp) {
     if (is_signed) { *qn = -(1 << (bits - 1)); *qp = (1 << (bits - 1)) - 1; }
@@ -87,7 +90,8 @@ __device__ __forceinline__ float small_int_to_float(int v) {
 // on |z| <= 4 (beyond that erf is 1 to 2e-8).  The coefficients are a weighted minimax fit
 // (max |erf error| 7.8e-8 in exact arithmetic); with ex2.approx (2 ulp) and the fp32 Horner
 // steps the absolute error of Phi stays below 2.5e-7, i.e. |GELU error| < 2^-21 * |y|.
-__device__ __forceinline__ float gelu_f32(float y) {
+// gelu_scaled(y, h) = 2*h*GELU(y); h = 0.5 gives GELU itself, h = 0.5/s_out folds the output step.
+__device__ __forceinline__ float gelu_scaled(float y, float h) {
     const float z = fminf(fabsf(y) * 0.70710678118654752440f, 4.0f);
     float q = -1.00217749e-04f;
     q = fmaf(q, z, 4.61550077e-04f);
@@ -101,8 +105,9 @@ __device__ __forceinline__ float gelu_f32(float y) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-q));
     const float erf_abs = 1.0f - e;
     const float t = copysignf(erf_abs, y);
-    const float hy = 0.5f * y;
+    const float hy = h * y;
     return fmaf(hy, t, hy);
 }
+__device__ __forceinline__ float gelu_f32(float y) { return gelu_scaled(y, 0.5f); }
 
 }  // namespace vitint

@@ -129,7 +129,7 @@ __device__ __forceinline__ bool epi_barrier(uint32_t bar, uint32_t parity, volat
 // Epilogue of one row x 32 columns.  v[]: accumulators scaled by 2^shift; pa/pb/pq: the 32
 // columns' parameters in shared memory (multiplier already carries 2^-shift).
 // FULL: all 32 columns exist and 16-byte vector accesses are legal.
-template <int KIND, bool FULL, bool SMALL, bool HAS_RES>
+template <int KIND, bool FULL, int SMALL, bool HAS_RES>
 __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32_t (&v)[32], const float* pa,
                                                const float* pb, const float* pq, long long orow, long long colbase,
                                                int n0) {
@@ -170,7 +170,13 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     const bool vec_out = FULL && ((reinterpret_cast<uintptr_t>(of) & 15u) == 0);
     // The element loop below is straight-line code (no branch on run-time parameters), so the 32
     // independent per-column chains can overlap; the container width is only looked at when packing.
-    uint32_t code[32];                                                            // REQUANT
+    // REQUANT: clamp, then add 1.5*2^23 + 2^(c-1) for signed codes (c = container bits): the sum's low
+    // mantissa bits hold the code in offset binary (q + 2^(c-1) >= 0).  Offset codes pack with one
+    // shift-add each and no masking; the constant high bits are subtracted per word and one XOR of
+    // every container's top bit turns offset binary into two's complement.
+    const bool sgn = P.out_qn < 0.0f;
+    const float magic = 12582912.0f + (sgn ? (float)(1 << (P.out_c - 1)) : 0.0f);
+    uint32_t code[32];
 #pragma unroll
     for (int i4 = 0; i4 < 8; ++i4) {
         const float4 a4 = *reinterpret_cast<const float4*>(pa + 4 * i4);
@@ -186,13 +192,16 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int i = 4 * i4 + j;
-            const float f = SMALL ? small_int_to_float((int)v[i] >> P.shift) : (float)(int)v[i];
+            // SMALL 2: scaled accumulator below 2^22, no shift (2^-shift rides on the multiplier);
+            // SMALL 1: shift back first; SMALL 0: conversion instruction
+            const float f = SMALL == 2 ? small_int_to_float((int)v[i])
+                          : SMALL == 1 ? small_int_to_float((int)v[i] >> P.shift) : (float)(int)v[i];
             float val = fmaf(f, aa[j], bb[j]);
-            if (KIND == EK_DEQUANT_GELU || KIND == EK_REQUANT_GELU) val = gelu_f32(val);
-            if (KIND == EK_REQUANT_GELU) val = val * qq[j];
+            if (KIND == EK_DEQUANT_GELU) val = gelu_f32(val);
+            if (KIND == EK_REQUANT_GELU) val = gelu_scaled(val, qq[j]);      // qq = 0.5 / s_out
             if (has_res) val = val + rr[j];
             y[j] = val;
-            if (!deq) code[i] = round_clamp_bits(val, P.out_qn, P.out_qp);
+            if (!deq) code[i] = __float_as_uint(fminf(fmaxf(val, P.out_qn), P.out_qp) + magic);
         }
         if (deq) {
             if (vec_out) {
@@ -206,20 +215,31 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     if (deq) return;
     uint32_t wds[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (!FULL) {
+        const uint32_t zero_code = __float_as_uint(magic);            // q = 0
 #pragma unroll
-        for (int i = 0; i < 32; ++i) if (i >= nvalid) code[i] = 0u;
+        for (int i = 0; i < 32; ++i) if (i >= nvalid) code[i] = zero_code;
     }
     if (P.out_c == 4) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) wds[i >> 3] |= (code[i] & 0xFu) << (4 * (i & 7));
+        for (int w = 0; w < 4; ++w) {
+            uint32_t acc = code[8 * w];
+#pragma unroll
+            for (int j = 1; j < 8; ++j) acc += code[8 * w + j] << (4 * j);
+            wds[w] = (acc - 0x4B400000u * 0x11111111u) ^ (sgn ? 0x88888888u : 0u);
+        }
     } else if (P.out_c == 2) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) wds[i >> 4] |= (code[i] & 0x3u) << (2 * (i & 15));
+        for (int w = 0; w < 2; ++w) {
+            uint32_t acc = code[16 * w];
+#pragma unroll
+            for (int j = 1; j < 16; ++j) acc += code[16 * w + j] << (2 * j);
+            wds[w] = (acc - 0x4B400000u * 0x55555555u) ^ (sgn ? 0xAAAAAAAAu : 0u);
+        }
     } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i)
             wds[i] = __byte_perm(__byte_perm(code[4 * i], code[4 * i + 1], 0x4040),
-                                 __byte_perm(code[4 * i + 2], code[4 * i + 3], 0x4040), 0x5410);
+                                 __byte_perm(code[4 * i + 2], code[4 * i + 3], 0x4040), 0x5410) ^ (sgn ? 0x80808080u : 0u);
     }
     const int out_words = P.out_c;   // 32 codes = 4*out_c bytes
     const long long byte0 = ((colbase + n0) * P.out_c) >> 3;
@@ -238,7 +258,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     }
 }
 
-template <int KIND, bool SMALL>
+template <int KIND, int SMALL>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiParams& ep, int buf, uint32_t t_row,
                                               bool row_ok, long long orow, long long colbase, int n_tile) {
     for (int chunk = 0; chunk * 32 < P.bn; ++chunk) {
@@ -442,7 +462,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int q4 = warp;   // TMEM lane quarter
         const int tid_e = threadIdx.x;                       // 0..127
         // small accumulators are shifted back as integers; otherwise 2^-shift rides on the multiplier
-        const float down = P.small_acc ? 1.0f : __int_as_float((127 - P.shift) << 23);
+        const float down = P.small_acc == 1 ? 1.0f : __int_as_float((127 - P.shift) << 23);
         int tl = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++tl) {
@@ -461,7 +481,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             a = __ldg(P.col_a + cidx);
                         } else {
                             a = P.col_a ? __fmul_rn(P.x_step, __ldg(P.col_a + cidx)) : P.x_step;
-                            if (KIND == EK_REQUANT_GELU) q = __ldg(P.inv_s + cidx);
+                            if (KIND == EK_REQUANT_GELU) q = 0.5f * __ldg(P.inv_s + cidx);   // folds GELU's 1/2
                         }
                         b = P.col_b ? __ldg(P.col_b + cidx) : 0.0f;
                         a *= down;
@@ -480,8 +500,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool row_ok = row_in_problem < P.M;
             const long long orow = (long long)outer * P.row_off_outer + (long long)inner * P.row_off_inner + row_in_problem;
             const uint32_t t_row = tmem_base + (uint32_t)buf * acc_stride + ((uint32_t)(q4 * 32) << 16);
-            if (P.small_acc) epilogue_tile<KIND, true>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
-            else epilogue_tile<KIND, false>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
+            if (P.small_acc == 2) epilogue_tile<KIND, 2>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
+            else if (P.small_acc == 1) epilogue_tile<KIND, 1>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
+            else epilogue_tile<KIND, 0>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&bars.acc_empty[buf]));
@@ -535,7 +556,8 @@ int make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint6
 
 struct Operand {
     const void* data;
-    int bits, is_signed;
+    int bits, is_signed;   // value range of the codes
+    int container;         // bits per stored code
     uint64_t row_bytes;   // valid bytes of one row (inner extent of the tensor map)
     uint64_t rows;        // rows per problem
     uint64_t pitch, inner_stride, outer_stride;
@@ -559,7 +581,7 @@ constexpr uint32_t SMEM_TILE_BUDGET = 204u * 1024u;   // dynamic shared memory s
 // Batched NT integer GEMM launcher shared by the linear layer, Q K^T and P V.
 int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_inner, int n_outer, int b_mn_major,
                 GemmParams P, cudaStream_t st) {
-    const int ca = container_bits(A.bits), cb = container_bits(B.bits);
+    const int ca = A.container, cb = B.container;
     P.M = M; P.N = N; P.K = K;
     P.ca = ca; P.cb = cb; P.a_signed = A.is_signed; P.b_signed = B.is_signed; P.b_mn_major = b_mn_major;
     P.a_direct = ca == 8 ? 1 : 0;
@@ -569,7 +591,7 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     const long long bound = (long long)K * max_abs_code(A.bits, A.is_signed) * max_abs_code(B.bits, B.is_signed);
     if (bound >= (1ll << 31)) return VITINT_ERR_OVERFLOW_BOUND;
     if ((bound << P.shift) >= (1ll << 31)) return VITINT_ERR_UNSUPPORTED;
-    P.small_acc = bound < (1ll << 22) ? 1 : 0;
+    P.small_acc = (bound << P.shift) < (1ll << 22) ? 2 : (bound < (1ll << 22) ? 1 : 0);
     int bn = N >= MAX_BN ? MAX_BN : ((N + 15) / 16) * 16;
     if (b_mn_major) { if (N != 64) return VITINT_ERR_UNSUPPORTED; bn = 64; }
     P.bn = bn;
@@ -673,7 +695,12 @@ static int fill_epilogue(GemmParams& P, const vitint_epilogue* epi, float x_step
             if (ld_out < row_bytes(n_cols_total, epi->out_bits)) return VITINT_ERR_INVALID_ARG;
             int qn, qp;
             code_range(epi->out_bits, epi->out_signed, &qn, &qp);
-            P.out_c = container_bits(epi->out_bits); P.out_qn = (float)qn; P.out_qp = (float)qp;
+            if (epi->out_container_bits != 0 && epi->out_container_bits != 8 &&
+                epi->out_container_bits != container_bits(epi->out_bits))
+                return VITINT_ERR_INVALID_ARG;
+            P.out_c = epi->out_container_bits ? epi->out_container_bits : container_bits(epi->out_bits);
+            if (ld_out < (n_cols_total * P.out_c + 7) / 8) return VITINT_ERR_INVALID_ARG;
+            P.out_qn = (float)qn; P.out_qp = (float)qp;
             if (epi->act == 0) {
                 if (!epi->alpha) return VITINT_ERR_INVALID_ARG;
                 P.col_a = epi->alpha; P.col_b = epi->beta;
@@ -716,10 +743,10 @@ extern "C" int vitint_linear(const vitint_codes* x, float x_step, const vitint_c
     if ((epi->mode == VITINT_EPI_DEQUANT_F32 || (epi->mode == VITINT_EPI_REQUANT && epi->act == 1)) && !w_step)
         return VITINT_ERR_INVALID_ARG;
     P.row_off_outer = 0; P.row_off_inner = 0; P.col_off_inner = 0;
-    Operand A{x->data, x->bits, x->is_signed, (uint64_t)row_bytes(x->cols, x->bits), (uint64_t)x->rows,
+    Operand A{x->data, x->bits, x->is_signed, codes_container(x), (uint64_t)codes_row_bytes(x, x->cols), (uint64_t)x->rows,
               (uint64_t)x->pitch_bytes, (uint64_t)x->pitch_bytes * (uint64_t)x->rows,
               (uint64_t)x->pitch_bytes * (uint64_t)x->rows};
-    Operand B{w->data, w->bits, w->is_signed, (uint64_t)row_bytes(w->cols, w->bits), (uint64_t)w->rows,
+    Operand B{w->data, w->bits, w->is_signed, codes_container(w), (uint64_t)codes_row_bytes(w, w->cols), (uint64_t)w->rows,
               (uint64_t)w->pitch_bytes, (uint64_t)w->pitch_bytes * (uint64_t)w->rows,
               (uint64_t)w->pitch_bytes * (uint64_t)w->rows};
     return launch_gemm(A, B, (int)x->rows, (int)w->rows, (int)x->cols, 1, 1, 0, P, (cudaStream_t)stream);
@@ -736,9 +763,9 @@ extern "C" int vitint_qk(const vitint_slabs* q, const vitint_slabs* k, int32_t b
     epi.mode = VITINT_EPI_ACC_I32;
     if (int rc = fill_epilogue(P, &epi, 1.0f, nullptr, nullptr, s_out, ld_s, tokens)) return rc;
     P.row_off_outer = (long long)heads * tokens; P.row_off_inner = tokens; P.col_off_inner = 0;
-    Operand A{q->data, q->bits, q->is_signed, (uint64_t)row_bytes(64, q->bits), (uint64_t)tokens,
+    Operand A{q->data, q->bits, q->is_signed, container_bits(q->bits), (uint64_t)row_bytes(64, q->bits), (uint64_t)tokens,
               (uint64_t)q->pitch_bytes, (uint64_t)q->head_stride_bytes, (uint64_t)q->image_stride_bytes};
-    Operand B{k->data, k->bits, k->is_signed, (uint64_t)row_bytes(64, k->bits), (uint64_t)tokens,
+    Operand B{k->data, k->bits, k->is_signed, container_bits(k->bits), (uint64_t)row_bytes(64, k->bits), (uint64_t)tokens,
               (uint64_t)k->pitch_bytes, (uint64_t)k->head_stride_bytes, (uint64_t)k->image_stride_bytes};
     return launch_gemm(A, B, tokens, tokens, 64, heads, batch, 0, P, (cudaStream_t)stream);
 }
@@ -758,9 +785,9 @@ extern "C" int vitint_pv(const vitint_codes* p, const vitint_slabs* v, int32_t b
         return rc;
     if (epi->mode == VITINT_EPI_REQUANT && epi->act == 1) return VITINT_ERR_UNSUPPORTED;
     P.row_off_outer = tokens; P.row_off_inner = 0; P.col_off_inner = 64;
-    Operand A{p->data, p->bits, p->is_signed, (uint64_t)row_bytes(tokens, p->bits), (uint64_t)tokens,
+    Operand A{p->data, p->bits, p->is_signed, codes_container(p), (uint64_t)codes_row_bytes(p, tokens), (uint64_t)tokens,
               (uint64_t)p->pitch_bytes, (uint64_t)p->pitch_bytes * tokens, (uint64_t)p->pitch_bytes * tokens * heads};
-    Operand B{v->data, v->bits, v->is_signed, (uint64_t)row_bytes(64, v->bits), (uint64_t)tokens,
+    Operand B{v->data, v->bits, v->is_signed, container_bits(v->bits), (uint64_t)row_bytes(64, v->bits), (uint64_t)tokens,
               (uint64_t)v->pitch_bytes, (uint64_t)v->head_stride_bytes, (uint64_t)v->image_stride_bytes};
     return launch_gemm(A, B, tokens, 64, tokens, heads, batch, 1, P, (cudaStream_t)stream);
 }

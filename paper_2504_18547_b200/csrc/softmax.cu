@@ -155,7 +155,7 @@ extern "C" int vitint_softmax_quantize(const int32_t* s, int64_t rows, int32_t c
     if (p_f32 && ld_p < cols) return VITINT_ERR_INVALID_ARG;
     if (cols > 1024) return VITINT_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(s) & 3u) != 0) return VITINT_ERR_ALIGNMENT;
-    const int cb = container_bits(p_out->bits);
+    const int cb = codes_container(p_out);
     int qn, qp;
     code_range(p_out->bits, 0, &qn, &qp);
     const int nch = (cols + 255) / 256;

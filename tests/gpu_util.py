@@ -15,13 +15,13 @@ def to_codes(q: np.ndarray, bits: int, signed: bool, pitch: int | None = None) -
 
 def from_codes(c: vt.Codes) -> np.ndarray:
     """Packed device codes -> int16 [rows, cols], unpacked by the oracle's unpacker."""
-    return vo.unpack(c.data.cpu().numpy(), c.cols, c.bits, c.signed)
+    return vo.unpack(c.data.cpu().numpy(), c.cols, c.stored_bits, c.signed)
 
 
 def padding_is_zero(c: vt.Codes) -> bool:
     """Bytes between the last code of each row and the pitch must be zero."""
     raw = c.data.cpu().numpy()
-    cb = 4 if c.bits == 3 else c.bits
+    cb = c.stored_bits
     nbits = c.cols * cb
     full = nbits // 8
     ok = not raw[:, (nbits + 7) // 8:].any()

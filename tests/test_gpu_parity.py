@@ -61,7 +61,8 @@ def test_quantize_row_steps_strided_input_and_ties():
 def test_widen_keeps_values(bits, signed, rows, cols):
     q = rand_codes(50 + bits, (rows, cols), bits, signed)
     got = vt.vitint_widen(to_codes(q, bits, signed))
-    assert got.bits == 8 and np.array_equal(from_codes(got), q) and padding_is_zero(got)
+    assert got.bits == bits and got.container == 8 and got.pitch >= cols
+    assert np.array_equal(from_codes(got), q) and padding_is_zero(got)
 
 
 # ---------------------------------------------------------------------------
@@ -110,6 +111,29 @@ def test_linear_with_widened_weights(M, K, N, bits, xs):
     w8 = vt.vitint_widen(to_codes(qw, bits, True))
     acc = vt.vitint_linear(to_codes(qx, bits, xs), 1.0, w8, None, None, vt.Epilogue(mode=vt.EPI_ACC_I32))
     assert np.array_equal(acc.cpu().numpy(), vo.matmul_i32(qx, qw))
+
+
+def test_byte_containers_for_low_bit_codes():
+    """4-bit-range codes stored one per byte: produced by the quantizer and by a requantizing epilogue,
+    consumed by the linear layer (both operands then go from the TMA copy straight to the tensor cores)."""
+    M, K, N = 300, 320, 200
+    x = si.normal(71, (M, K))
+    step = si.lsq_step(x, 4, True)
+    out = vt.Codes.empty(M, K, 4, True, container=8)
+    got = vt.vitint_quantize(dev(x), float(step), 4, True, out=out)
+    qx = vo.quantize(x, step, 4, True)
+    assert np.array_equal(from_codes(got), qx) and padding_is_zero(got)
+    qw = rand_codes(72, (N, K), 4, True)
+    w8 = vt.vitint_widen(to_codes(qw, 4, True))
+    acc = vo.matmul_i32(qx, qw)
+    got_acc = vt.vitint_linear(got, 1.0, w8, None, None, vt.Epilogue(mode=vt.EPI_ACC_I32))
+    assert np.array_equal(got_acc.cpu().numpy(), acc)
+    alpha = np.full(N, 0.02, np.float32)
+    beta = si.normal(73, (N,), 0.0, 0.5)
+    epi = vt.Epilogue(mode=vt.EPI_REQUANT, alpha=dev(alpha), beta=dev(beta), out_bits=4, out_signed=True, out_container=8)
+    q8 = vt.vitint_linear(got, 1.0, w8, None, None, epi)
+    assert q8.container == 8 and q8.pitch >= N
+    assert np.array_equal(from_codes(q8), vo.epilogue_requant(acc, alpha, beta, 4, True)) and padding_is_zero(q8)
 
 
 @pytest.mark.parametrize("M,K,N", [(197, 192, 576), (300, 320, 100)])
