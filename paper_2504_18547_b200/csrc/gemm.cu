@@ -3,13 +3,13 @@
 // post-contraction epilogue of Eq. 2.
 //
 // One persistent CTA per SM walks 128 x BN output tiles.  Warp roles:
-//   warps 0-3  epilogue: stage the tile's per-column scale / bias in shared memory,
+//   warps 0-7  epilogue: stage the tile's per-column scale / bias in shared memory,
 //              tcgen05.ld of their 32 TMEM lanes, rescale / bias / GELU / requantize /
-//              pack, global stores (warp w owns TMEM lanes 32w..32w+31);
-//   warp  4    TMA producer: packed low-bit tiles -> shared-memory ring; operands that are
+//              pack, global stores (warp w owns TMEM lanes 32(w%4).. and half of the columns);
+//   warp  8    TMA producer: packed low-bit tiles -> shared-memory ring; operands that are
 //              already 8-bit go straight into the swizzled int8 operand ring;
-//   warp  5    MMA issuer (one thread) and owner of the TMEM allocation;
-//   warps 6-9  unpack: packed codes -> int8 operand tiles in the shared-memory layout
+//   warp  9    MMA issuer (one thread) and owner of the TMEM allocation;
+//   warps 10-13 unpack: packed codes -> int8 operand tiles in the shared-memory layout
 //              the tensor core expects (128-byte swizzle, K contiguous; or 64-byte
 //              swizzle, N contiguous, for the V operand of P*V).
 // The accumulator is double buffered in TMEM so the epilogue of tile i overlaps the
@@ -30,9 +30,9 @@ namespace {
 
 constexpr int BM = 128;   // rows per tile (= TMEM lanes)
 constexpr int BK = 128;   // int8 elements per K block (= one 128-byte swizzle row)
-constexpr int EPI_WARPS = 4;
+constexpr int EPI_WARPS = 8;   // two warps per TMEM lane quarter, each taking half of the tile's columns
 constexpr int UNPACK_WARPS = 4;
-constexpr int WARP_TMA = 4, WARP_MMA = 5, WARP_UNPACK0 = 6;
+constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_UNPACK0 = 10;
 constexpr int NUM_THREADS = (WARP_UNPACK0 + UNPACK_WARPS) * 32;
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_BN = 256;
@@ -45,6 +45,7 @@ struct GemmParams {
     int ca, cb, a_signed, b_signed, shift, b_mn_major;
     int a_direct, b_direct;            // operand already int8: TMA writes the operand ring itself
     int small_acc;                     // |acc| < 2^22: int -> float without a conversion instruction
+    uint32_t stage_off;                // fp32 epilogue: byte offset of the per-warp transposition buffers (0 = none)
     int ns_i, ns_p;
     uint32_t ia_bytes, ib_bytes, pa_bytes, pb_bytes, tmem_cols;
     int kind, out_c;
@@ -119,7 +120,7 @@ __device__ __forceinline__ void tile_coords(const GemmParams& P, int tile, int& 
     inner = prob - outer * P.n_inner;
 }
 
-// Barrier among the 128 epilogue threads, bounded like every other wait (an mbarrier with one
+// Barrier among the epilogue threads, bounded like every other wait (an mbarrier with one
 // phase per tile instead of bar.sync, which could not give up).
 __device__ __forceinline__ bool epi_barrier(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     ptx::mbar_arrive(bar);
@@ -258,16 +259,92 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     }
 }
 
+constexpr int STAGE_LD = 36;                                  // floats per staged row: 144 bytes keeps 16-byte accesses conflict-free
+constexpr int STAGE_BYTES = 32 * STAGE_LD * 4;                // one 32 x 32 fp32 block per epilogue warp
+
+// fp32 epilogue of a 32 x 32 block through a shared-memory transposition, so that every global
+// access of the warp covers whole 128-byte lines: the TMEM layout gives each thread one ROW of the
+// block, while coalesced loads / stores want each instruction to cover four rows of 128 bytes.
+//   residual: coalesced float4 loads -> stage -> each thread reads its own row;
+//   result  : each thread writes its own row -> stage -> coalesced float4 stores.
+// Whole-warp call (rows past M take part and are masked at the global accesses).
+template <int KIND, int SMALL, bool HAS_RES>
+__device__ __forceinline__ void epilogue_chunk_staged(const GemmParams& P, const uint32_t (&v)[32], const float* pa,
+                                                     const float* pb, float* stage, int lane, long long orow0,
+                                                     int rows_valid, long long colbase, int n0) {
+    const int cr = lane >> 3, cc = (lane & 7) * 4;              // cooperative phase: row cr + 4*i, columns cc..cc+3
+    float* const my_row = stage + lane * STAGE_LD;
+    if (HAS_RES) {
+        const float* r0 = P.residual + orow0 * P.ld_res + colbase + n0 + cc;
+        float4 t[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = cr + 4 * i;
+            t[i] = (r < rows_valid) ? __ldg(reinterpret_cast<const float4*>(r0 + (long long)r * P.ld_res))
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(stage + (cr + 4 * i) * STAGE_LD + cc) = t[i];
+        __syncwarp();
+    }
+    float4 y[8];
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4) {
+        const float4 a4 = *reinterpret_cast<const float4*>(pa + 4 * i4);
+        const float4 b4 = *reinterpret_cast<const float4*>(pb + 4 * i4);
+        float4 r4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (HAS_RES) r4 = *reinterpret_cast<const float4*>(my_row + 4 * i4);
+        const float aa[4] = {a4.x, a4.y, a4.z, a4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w}, rr[4] = {r4.x, r4.y, r4.z, r4.w};
+        float o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = 4 * i4 + j;
+            const float f = SMALL == 2 ? small_int_to_float((int)v[i])
+                          : SMALL == 1 ? small_int_to_float((int)v[i] >> P.shift) : (float)(int)v[i];
+            float val = fmaf(f, aa[j], bb[j]);
+            if (KIND == EK_DEQUANT_GELU) val = gelu_f32(val);
+            if (HAS_RES) val = val + rr[j];
+            o[j] = val;
+        }
+        y[i4] = make_float4(o[0], o[1], o[2], o[3]);
+    }
+    if (HAS_RES) __syncwarp();                                  // every row has been read before it is overwritten
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4) *reinterpret_cast<float4*>(my_row + 4 * i4) = y[i4];
+    __syncwarp();
+    float* o0 = (float*)P.out + orow0 * P.ld_out + colbase + n0 + cc;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = cr + 4 * i;
+        const float4 t = *reinterpret_cast<const float4*>(stage + r * STAGE_LD + cc);
+        if (r < rows_valid) *reinterpret_cast<float4*>(o0 + (long long)r * P.ld_out) = t;
+    }
+    __syncwarp();                                               // the buffer is free for the next chunk
+}
+
 template <int KIND, int SMALL>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiParams& ep, int buf, uint32_t t_row,
-                                              bool row_ok, long long orow, long long colbase, int n_tile) {
-    for (int chunk = 0; chunk * 32 < P.bn; ++chunk) {
+                                              bool row_ok, long long orow, long long colbase, int n_tile, int half,
+                                              float* stage, int lane, int rows_valid) {
+    // the two warps of a lane quarter split the tile's 32-column chunks: first half / second half
+    const int n_chunks = (P.bn + 31) / 32, split = (n_chunks + 1) / 2;
+    const int c_begin = half ? split : 0, c_end = half ? n_chunks : split;
+    for (int chunk = c_begin; chunk < c_end; ++chunk) {
         const int n0 = n_tile * P.bn + chunk * 32;
         if (n0 >= P.N) break;
         uint32_t v[32];
         ptx::tmem_ld32(t_row + (uint32_t)(chunk * 32), v);
         ptx::tmem_ld_wait();
-        if (row_ok) {
+        constexpr bool is_deq = (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU);
+        if (is_deq && stage != nullptr && n0 + 32 <= P.N) {
+            // full 32-column chunk of an fp32 output: coalesced path (stage is only set when the host has
+            // checked 16-byte alignment of the output, the residual and their leading dimensions)
+            const float* pa = &ep.a[buf][chunk * 32];
+            const float* pb = &ep.b[buf][chunk * 32];
+            const long long orow0 = orow - lane;
+            if (P.residual != nullptr) epilogue_chunk_staged<is_deq ? KIND : EK_DEQUANT, SMALL, true>(P, v, pa, pb, stage, lane, orow0, rows_valid, colbase, n0);
+            else epilogue_chunk_staged<is_deq ? KIND : EK_DEQUANT, SMALL, false>(P, v, pa, pb, stage, lane, orow0, rows_valid, colbase, n0);
+        } else if (row_ok) {
             const float* pa = &ep.a[buf][chunk * 32];
             const float* pb = &ep.b[buf][chunk * 32];
             const float* pq = &ep.q[buf][chunk * 32];
@@ -459,8 +536,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // -------------------------------- epilogue ---------------------------------
-        const int q4 = warp;   // TMEM lane quarter
-        const int tid_e = threadIdx.x;                       // 0..127
+        const int q4 = warp & 3;   // TMEM lane quarter
+        const int half = warp >> 2;   // which half of the tile's columns
+        const int tid_e = threadIdx.x;                       // 0..255
         // small accumulators are shifted back as integers; otherwise 2^-shift rides on the multiplier
         const float down = P.small_acc == 1 ? 1.0f : __int_as_float((127 - P.shift) << 23);
         int tl = 0;
@@ -500,9 +578,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool row_ok = row_in_problem < P.M;
             const long long orow = (long long)outer * P.row_off_outer + (long long)inner * P.row_off_inner + row_in_problem;
             const uint32_t t_row = tmem_base + (uint32_t)buf * acc_stride + ((uint32_t)(q4 * 32) << 16);
-            if (P.small_acc == 2) epilogue_tile<KIND, 2>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
-            else if (P.small_acc == 1) epilogue_tile<KIND, 1>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
-            else epilogue_tile<KIND, 0>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile);
+            int rows_valid = P.M - (m_tile * BM + q4 * 32);
+            rows_valid = rows_valid < 0 ? 0 : (rows_valid > 32 ? 32 : rows_valid);
+            float* const stage = P.stage_off ? reinterpret_cast<float*>(smem_gen + P.stage_off + (size_t)warp * STAGE_BYTES) : nullptr;
+            if (P.small_acc == 2) epilogue_tile<KIND, 2>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, half, stage, lane, rows_valid);
+            else if (P.small_acc == 1) epilogue_tile<KIND, 1>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, half, stage, lane, rows_valid);
+            else epilogue_tile<KIND, 0>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, half, stage, lane, rows_valid);
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&bars.acc_empty[buf]));
@@ -607,17 +688,23 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     P.pa_bytes = P.a_direct ? 0u : (uint32_t)(BM * 16 * ca);
     P.pb_bytes = P.b_direct ? 0u : (b_mn_major ? (uint32_t)(BK * 8 * cb) : (uint32_t)bn * 16 * cb);
     const uint32_t stage_i = P.ia_bytes + P.ib_bytes, stage_p = P.pa_bytes + P.pb_bytes;
+    // fp32 epilogues go through a per-warp transposition buffer when every access can be a 16-byte one
+    bool staged = (P.kind == EK_DEQUANT || P.kind == EK_DEQUANT_GELU) && n_inner == 1 && n_outer == 1 &&
+                  aligned16(P.out) && P.ld_out % 4 == 0 &&
+                  (!P.residual || (aligned16(P.residual) && P.ld_res % 4 == 0));
+    const uint32_t stage_total = staged ? (uint32_t)(EPI_WARPS * STAGE_BYTES) : 0u;
+    const uint32_t ring_budget = SMEM_TILE_BUDGET + 12u * 1024u - stage_total;   // staging comes out of the ring space
     // The packed ring hides the global-memory latency of the TMA loads; the int8 ring only
     // decouples unpack from MMA issue, unless TMA writes it directly.
     int ns_i, ns_p;
     if (stage_p == 0) {
-        ns_i = (int)(SMEM_TILE_BUDGET / stage_i);
+        ns_i = (int)(ring_budget / stage_i);
         ns_p = 1;
     } else {
         ns_i = (P.a_direct || P.b_direct) ? 3 : 2;
-        while (ns_i > 2 && (uint32_t)ns_i * stage_i + 2u * stage_p > SMEM_TILE_BUDGET) --ns_i;
-        if ((uint32_t)ns_i * stage_i + 2u * stage_p > SMEM_TILE_BUDGET) return VITINT_ERR_UNSUPPORTED;
-        ns_p = (int)((SMEM_TILE_BUDGET - (uint32_t)ns_i * stage_i) / stage_p);
+        while (ns_i > 2 && (uint32_t)ns_i * stage_i + 2u * stage_p > ring_budget) --ns_i;
+        if ((uint32_t)ns_i * stage_i + 2u * stage_p > ring_budget) return VITINT_ERR_UNSUPPORTED;
+        ns_p = (int)((ring_budget - (uint32_t)ns_i * stage_i) / stage_p);
     }
     if (ns_i > MAX_STAGES) ns_i = MAX_STAGES;
     if (ns_p > MAX_STAGES) ns_p = MAX_STAGES;
@@ -642,7 +729,9 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
             return rc;
     }
     // at least ~120 KB so that two CTAs never share an SM (and its tensor memory)
-    size_t smem = (size_t)ns_i * stage_i + (size_t)ns_p * stage_p + 1024;
+    const size_t rings = (size_t)ns_i * stage_i + (size_t)ns_p * stage_p;
+    P.stage_off = staged ? (uint32_t)rings : 0u;
+    size_t smem = rings + stage_total + 1024;
     if (smem < 120 * 1024) smem = 120 * 1024;
     int grid = sm_count();
     if (grid > P.total_tiles) grid = P.total_tiles;
@@ -651,7 +740,7 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     case KIND:                                                                                                     \
         if (!attr_set[KIND]) {                                                                                     \
             if (cudaFuncSetAttribute(gemm_i8_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,            \
-                                     (int)SMEM_TILE_BUDGET + 2048) != cudaSuccess)                                 \
+                                     (int)SMEM_TILE_BUDGET + 14 * 1024) != cudaSuccess)                                 \
                 return VITINT_ERR_CUDA;                                                                            \
             attr_set[KIND] = true;                                                                                 \
         }                                                                                                          \
