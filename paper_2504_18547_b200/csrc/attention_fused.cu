@@ -28,8 +28,8 @@ namespace vitint {
 namespace {
 
 constexpr int AT_GROUPS = 2;
-constexpr int AT_COMPUTE_WARPS = 4;
-constexpr int AT_THREADS = (AT_GROUPS * AT_COMPUTE_WARPS + AT_GROUPS) * 32;   // 320
+constexpr int AT_COMPUTE_WARPS = 8;   // two warps per TMEM lane quarter: a query row is shared by two threads
+constexpr int AT_THREADS = (AT_GROUPS * AT_COMPUTE_WARPS + AT_GROUPS) * 32;   // 576
 
 struct AttnParams {
     int batch, heads, tokens, q_tiles, total_items;
@@ -39,7 +39,7 @@ struct AttnParams {
     int smax;                    // table covers scores -smax .. smax
     int part_bytes;              // bytes of one of the Q / K / V column blocks in a QKV row
     uint32_t off_table, off_group, group_bytes;         // shared-memory layout
-    uint32_t off_pq, off_pk, off_pv, off_q, off_k, off_v, off_p, off_col;   // within a group
+    uint32_t off_pq, off_pk, off_pv, off_q, off_k, off_v, off_p, off_col, off_z;   // within a group
     const float* table;          // global copy of the exp table, 2*smax+1 floats
     float p_step, p_qp;
     const float* alpha_o;        // [D]
@@ -51,7 +51,7 @@ struct AttnParams {
 };
 
 struct AttnBars {
-    uint64_t packed_full, ops_ready, s_full, p_ready, o_full, o_done, grp_sync;
+    uint64_t packed_full, ops_ready, s_full, p_ready, o_full, o_done, grp_sync, z_sync;
 };
 
 // exp(fl32(s * c)) for every integer score, correctly rounded to fp32 (fp64 exp, one rounding).
@@ -91,6 +91,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             ptx::mbar_init(ptx::smem_addr(&bars[k].o_full), 1);
             ptx::mbar_init(ptx::smem_addr(&bars[k].o_done), AT_COMPUTE_WARPS);
             ptx::mbar_init(ptx::smem_addr(&bars[k].grp_sync), AT_COMPUTE_WARPS * 32);
+            ptx::mbar_init(ptx::smem_addr(&bars[k].z_sync), AT_COMPUTE_WARPS * 32);
         }
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
@@ -171,9 +172,11 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         }
     } else {
         // ------------------------------ compute warps ------------------------------------
-        const int wq = warp % AT_COMPUTE_WARPS;                     // TMEM lane quarter
-        const int tid_g = wq * 32 + lane;                           // 0..127 within the group
-        const int row = tid_g;                                      // query row of the tile
+        const int wq = warp & 3;                                    // TMEM lane quarter
+        const int hf = (warp % AT_COMPUTE_WARPS) >> 2;              // which of the row's two threads: even / odd 32-column chunks
+        const int tid_g = (warp % AT_COMPUTE_WARPS) * 32 + lane;    // 0..255 within the group
+        const int row = wq * 32 + lane;                             // query row of the tile
+        double* const zx = reinterpret_cast<double*>(ggen + P.off_z);   // partial row sums, [2][128]
         const uint32_t t_row = tmem_grp + ((uint32_t)(wq * 32) << 16);
         const char* const tab_mid = reinterpret_cast<const char*>(smem_gen + P.off_table) + (size_t)P.smax * 4;
         float* const colp = reinterpret_cast<float*>(ggen + P.off_col);   // alpha[64], beta[64] of this head
@@ -190,13 +193,13 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // ---- operands: packed -> int8 -------------------------------------------------
             bool w = mbar_wait(ptx::smem_addr(&B.packed_full), ph, abort_ptr);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
-            unpack_rows64<C, 1>(ggen + P.off_pq, ggen + P.off_q, 128, tid_g, 128);
-            unpack_rows64<C, 1>(ggen + P.off_pk, ggen + P.off_k, P.n_k, tid_g, 128);
-            unpack_rows64<C, 1>(ggen + P.off_pv, ggen + P.off_v, P.kv_rows, tid_g, 128);
+            unpack_rows64<C, 1>(ggen + P.off_pq, ggen + P.off_q, 128, tid_g, AT_COMPUTE_WARPS * 32);
+            unpack_rows64<C, 1>(ggen + P.off_pk, ggen + P.off_k, P.n_k, tid_g, AT_COMPUTE_WARPS * 32);
+            unpack_rows64<C, 1>(ggen + P.off_pv, ggen + P.off_v, P.kv_rows, tid_g, AT_COMPUTE_WARPS * 32);
             if (tid_g < 64) colp[tid_g] = __ldg(P.alpha_o + h * 64 + tid_g);
-            else colp[tid_g] = P.beta_o ? __ldg(P.beta_o + h * 64 + (tid_g - 64)) : 0.0f;
+            else if (tid_g < 128) colp[tid_g] = P.beta_o ? __ldg(P.beta_o + h * 64 + (tid_g - 64)) : 0.0f;
             ptx::fence_proxy_async_smem();
-            // the four warps exchange the staged column parameters through shared memory
+            // the group's warps exchange the staged column parameters through shared memory
             ptx::mbar_arrive(ptx::smem_addr(&B.grp_sync));
             w = mbar_wait(ptx::smem_addr(&B.grp_sync), ph, abort_ptr);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
@@ -212,7 +215,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             // a warp whose 32 query rows all lie past the last token has nothing to compute: its P rows
             // only feed accumulator rows that are never stored (whatever int8 they hold)
             const bool warp_live = qt * 128 + wq * 32 < T;
-            for (int ch = 0; warp_live && ch < chunks; ++ch) {
+            for (int ch = hf; warp_live && ch < chunks; ch += 2) {
                 uint32_t v[32];
                 ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
                 ptx::tmem_ld_wait();
@@ -238,13 +241,19 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 ptx::tmem_st32(t_row + (uint32_t)(ch * 32), v);
             }
             ptx::tmem_st_wait();
+            // the row's two threads add their partial sums (every thread takes part in the barrier)
+            zx[hf * 128 + row] = z;
+            ptx::mbar_arrive(ptx::smem_addr(&B.z_sync));
+            w = mbar_wait(ptx::smem_addr(&B.z_sync), ph, abort_ptr);
+            if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+            z = zx[row] + zx[128 + row];
             const double rz = warp_live ? 1.0 / z : 0.0;
             const float rzh = (float)rz;
             const float rzl = (float)(rz - (double)rzh);
             uint8_t* const prow = ggen + P.off_p + row * 128;
             const int sw = row & 7;
             // pass 2: p_j = RN(e_j / Z), code = min(rint(RN(p_j / s_P)), Qp) (p >= 0: no lower clamp)
-            for (int ch = 0; warp_live && ch < chunks; ++ch) {
+            for (int ch = hf; warp_live && ch < chunks; ch += 2) {
                 uint32_t v[32];
                 ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
                 ptx::tmem_ld_wait();
@@ -275,41 +284,45 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
             ptx::tc_fence_after();
             const int token = qt * 128 + row;
-            uint32_t ow[16];
+            // each of the row's two threads requantizes and stores 32 of the head's 64 columns
+            uint32_t ow[8];
 #pragma unroll
-            for (int k = 0; k < 16; ++k) ow[k] = 0;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
+            for (int k = 0; k < 8; ++k) ow[k] = 0;
+            {
                 uint32_t v[32];
-                ptx::tmem_ld32(t_row + (uint32_t)(half * 32), v);
+                ptx::tmem_ld32(t_row + (uint32_t)(hf * 32), v);
                 ptx::tmem_ld_wait();
                 // straight-line per-column arithmetic first, container-dependent packing afterwards
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                    const int col = half * 32 + i;
+                    const int col = hf * 32 + i;
                     const float f = small_int_to_float((int)v[i] >> (8 - C));
                     v[i] = round_clamp_bits(fmaf(f, colp[col], colp[64 + col]), P.out_qn, P.out_qp);
                 }
                 if (P.out_c == 4) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) ow[half * 4 + (i >> 3)] |= (v[i] & 0xFu) << (4 * (i & 7));
+                    for (int i = 0; i < 32; ++i) ow[i >> 3] |= (v[i] & 0xFu) << (4 * (i & 7));
                 } else if (P.out_c == 2) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) ow[half * 2 + (i >> 4)] |= (v[i] & 0x3u) << (2 * (i & 15));
+                    for (int i = 0; i < 32; ++i) ow[i >> 4] |= (v[i] & 0x3u) << (2 * (i & 15));
                 } else {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        ow[half * 8 + i] = __byte_perm(__byte_perm(v[4 * i], v[4 * i + 1], 0x4040),
-                                                       __byte_perm(v[4 * i + 2], v[4 * i + 3], 0x4040), 0x5410);
+                        ow[i] = __byte_perm(__byte_perm(v[4 * i], v[4 * i + 1], 0x4040),
+                                            __byte_perm(v[4 * i + 2], v[4 * i + 3], 0x4040), 0x5410);
                 }
             }
             if (token < T) {
-                uint8_t* o = P.out + ((long long)b * T + token) * P.out_pitch + (long long)h * (8 * P.out_c);
-                const int nwords = 2 * P.out_c;                     // 64 codes
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    if (4 * k < nwords)
-                        reinterpret_cast<uint4*>(o)[k] = make_uint4(ow[4 * k], ow[4 * k + 1], ow[4 * k + 2], ow[4 * k + 3]);
+                // 32 codes = 4*out_c bytes at column block h*64 + hf*32
+                uint8_t* o = P.out + ((long long)b * T + token) * P.out_pitch + (long long)h * (8 * P.out_c) + hf * (4 * P.out_c);
+                if (P.out_c == 4) {
+                    *reinterpret_cast<uint4*>(o) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                } else if (P.out_c == 2) {
+                    *reinterpret_cast<uint2*>(o) = make_uint2(ow[0], ow[1]);
+                } else {
+                    reinterpret_cast<uint4*>(o)[0] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                    reinterpret_cast<uint4*>(o)[1] = make_uint4(ow[4], ow[5], ow[6], ow[7]);
+                }
             }
             ptx::tc_fence_before();
             __syncwarp();
@@ -398,6 +411,7 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     P.off_pk = o; o += up((uint32_t)P.kv_rows * hb, 128);
     P.off_pv = o; o += up((uint32_t)P.kv_rows * hb, 128);
     P.off_col = o; o += 512;
+    P.off_z = o; o += 2 * 128 * 8;
     P.group_bytes = up(o, 1024);
     const size_t smem = (size_t)P.off_group + (size_t)AT_GROUPS * P.group_bytes + 1024;
     if (smem > 225 * 1024) return VITINT_ERR_UNSUPPORTED;
