@@ -20,6 +20,8 @@
 // subtracted there for range); every table entry is a correctly rounded fp32, the sum is fp64,
 // and p_j = RN(e_j * (1/Z)) with 1/Z carried as two floats, so p_j stays within 2 ulp.
 // The host only selects this kernel when smax*|c| <= 80 (no overflow without max subtraction).
+#include <cstring>
+
 #include "common.cuh"
 #include "ptx.cuh"
 #include "tile_ops.cuh"
@@ -265,7 +267,8 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     for (int j = 0; j < 4; ++j) {
                         const float e = __uint_as_float(v[4 * i4 + j]);
                         const float p = fmaf(e, rzh, e * rzl);
-                        cb[j] = __float_as_uint(fminf(div_rn(p, dv), P.p_qp) + 12582912.0f);   // code in the low byte
+                        // straight-line quotient (host selects this kernel only for such a step, see below)
+                        cb[j] = __float_as_uint(fminf(div_rn_exact(p, dv), P.p_qp) + 12582912.0f);   // code in the low byte
                     }
                     wd[i4] = __byte_perm(__byte_perm(cb[0], cb[1], 0x4040), __byte_perm(cb[2], cb[3], 0x4040), 0x5410);
                 }
@@ -366,6 +369,11 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     for (float s : steps) if (!(s > 0.0f && s < INFINITY)) return VITINT_ERR_INVALID_ARG;
     if (!valid_bits(p_bits)) return VITINT_ERR_INVALID_ARG;
     if (qkv->bits == 8 || qkv->container_bits == 8 || tokens > 256 || batch > 65535) return VITINT_ERR_UNSUPPORTED;
+    {   // the kernel divides by p_step with the two-FMA correction, exact unless the significand is all ones
+        uint32_t bits;
+        memcpy(&bits, &p_step, sizeof(bits));
+        if ((bits & 0x007FFFFFu) == 0x007FFFFFu) return VITINT_ERR_UNSUPPORTED;
+    }
     const int c = container_bits(qkv->bits);
     const int m = 1 << (c - 1);
     const int smax = 64 * m * m;

@@ -65,11 +65,15 @@ __device__ __forceinline__ Divisor make_divisor(float b) {
     d.exact = ((__float_as_uint(b) & 0x007FFFFFu) != 0x007FFFFFu) ? 1 : 0;
     return d;
 }
-__device__ __forceinline__ float div_rn(float a, const Divisor& d) {
-    if (!d.exact) return __fdiv_rn(a, d.b);
+// Straight-line form for inner loops; valid only when d.exact (callers test that once, outside
+// the loop, because a branch per element would serialise the otherwise independent elements).
+__device__ __forceinline__ float div_rn_exact(float a, const Divisor& d) {
     const float q0 = a * d.r;
     const float rem = fmaf(-q0, d.b, a);
     return fmaf(rem, d.r, q0);
+}
+__device__ __forceinline__ float div_rn(float a, const Divisor& d) {
+    return d.exact ? div_rn_exact(a, d) : __fdiv_rn(a, d.b);
 }
 
 // clamp(rint(r)) as an integer code, ties to even, NaN -> qn.  The clamp to the integer

@@ -32,9 +32,14 @@ quantize_pack_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, in
             for (int i = 0; i < E; ++i) v[i] = (col0 + i < cols) ? __ldg(xr + i) : 0.0f;
         }
         uint32_t word = 0;
+        if (dv.exact) {
 #pragma unroll
-        for (int i = 0; i < E; ++i) {
-            word |= (round_clamp_bits(div_rn(v[i], dv), qn, qp) & ((1u << C) - 1u)) << (C * i);
+            for (int i = 0; i < E; ++i)
+                word |= (round_clamp_bits(div_rn_exact(v[i], dv), qn, qp) & ((1u << C) - 1u)) << (C * i);
+        } else {
+#pragma unroll
+            for (int i = 0; i < E; ++i)
+                word |= (round_clamp_bits(__fdiv_rn(v[i], dv.b), qn, qp) & ((1u << C) - 1u)) << (C * i);
         }
         *reinterpret_cast<uint32_t*>(out + row * pitch + (int64_t)w * 4) = word;
     }
