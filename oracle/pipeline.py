@@ -125,3 +125,14 @@ def encoder_layer(x, prm: dict, batch: int, tokens: int, heads: int, bits: int, 
     st["acc_fc2"] = vo.matmul_i32(st["g_codes"], w_fc2)
     st["out"] = vo.epilogue_dequant(st["acc_fc2"], prm["s_g"], prm["s_w_fc2"], prm["b_fc2"], h)
     return st
+
+
+def encoder_stack(x, layer_params: list, batch: int, tokens: int, heads: int, bits: int) -> list:
+    """Encoder layers in sequence; returns the list of per-layer stage dicts (the last one's "out" is the result)."""
+    stages = []
+    cur = x
+    for prm in layer_params:
+        st = encoder_layer(cur, prm, batch, tokens, heads, bits)
+        stages.append(st)
+        cur = st["out"]
+    return stages

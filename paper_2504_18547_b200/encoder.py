@@ -125,3 +125,26 @@ class EncoderLayer:
         n = self.batch * self.heads * T
         return {"ln1_quant": M * D * 4 + M * D * c // 8, "ln2_quant": M * D * 4 + M * D * c // 8,
                 "softmax_quant": n * T * 4 + n * ((T * c + 7) // 8)}
+
+
+class EncoderStack:
+    """`layers` integerized encoder layers applied in sequence (each with its own weights and steps);
+    the fp32 residual stream ping-pongs between two device buffers."""
+
+    def __init__(self, layer_params: list, batch: int, tokens: int, heads: int, mlp_dim: int, bits: int,
+                 device="cuda", **kw):
+        self.layers = [EncoderLayer(batch, tokens, heads, mlp_dim, bits, prm, device, **kw) for prm in layer_params]
+        rows, dim = batch * tokens, heads * 64
+        self.buf = [torch.empty((rows, dim), dtype=torch.float32, device=device) for _ in range(2)]
+
+    def forward(self, x: torch.Tensor, out: torch.Tensor) -> torch.Tensor:
+        cur = x
+        n = len(self.layers)
+        for i, layer in enumerate(self.layers):
+            dst = out if i == n - 1 else self.buf[i & 1]
+            layer.forward(cur, dst)
+            cur = dst
+        return out
+
+    def ops(self) -> int:
+        return sum(sum(v for k, v in l.stage_ops().items() if k in l.stages) for l in self.layers)

@@ -161,3 +161,39 @@ def test_attention_block_full_size_sampled_images():
             tok_ok[blk] &= sel
     assert tok_ok.mean() > 0.5
     assert np.array_equal(_rows(from_codes(outc), images, T)[tok_ok], st["out_codes"][tok_ok])
+
+
+def test_twelve_layer_encoder_sampled_images():
+    """12 integerized ViT-Base layers (the 12-layer configuration at a reduced batch; the oracle follows two of
+    the images through all layers).  Near-tie code flips accumulate with depth, so the end-to-end check is a
+    closeness bound, while the first layer is checked stage by stage and bit-exactly where codes agree."""
+    from paper_2504_18547_b200.encoder import EncoderStack
+    cfg = si.VIT_BASE_ENCODER.with_(batch=8)
+    T, H = cfg.tokens, cfg.heads
+    prms = [si.layer_parameters(cfg, layer=l) for l in range(cfg.layers)]
+    x = si.activations(cfg)
+    stack = EncoderStack(prms, cfg.batch, T, H, cfg.mlp_dim, cfg.bits)
+    out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
+    stack.forward(dev(x), out)
+    assert vt.vitint_device_status() == 0
+    images = [0, 7]
+    sts = vp.encoder_stack(_rows(x, images, T), prms, len(images), T, H, cfg.bits)
+    # Every layer, fed with the ORACLE's previous-layer output for the sampled images (tiled to the batch), is
+    # checked stage by stage: this exercises each layer's own weights and steps without any cascade.
+    for l in (0, 5, 11):
+        xin = _rows(x, images, T) if l == 0 else sts[l - 1]["out"]
+        xin_b = np.concatenate([xin] * (cfg.batch // len(images)))
+        out_l = torch.empty_like(out)
+        stack.layers[l].forward(dev(xin_b), out_l)
+        g = gpu_stages(stack.layers[l], out_l, range(len(images)), T, H)
+        compare_stages(g, sts[l], len(images), T, H, cfg.dim, True, min_images_ok=1)
+    # End to end, near-tie code flips (legitimate one-code differences) spread through attention and are
+    # re-quantized twelve times, so the two results are compared statistically.
+    o = _rows(out.cpu().numpy(), images, T)
+    ref = sts[-1]["out"]
+    err = (o - ref).astype(np.float64)
+    rel_rms = np.sqrt((err ** 2).mean()) / ref.std()
+    corr = np.corrcoef(o.ravel(), ref.ravel())[0, 1]
+    assert vt.vitint_device_status() == 0
+    assert rel_rms < 0.25 and corr > 0.97 and ref.std() > 0.5, (rel_rms, corr)
+    print(f"12 layers: relative rms difference {rel_rms:.4f}, correlation {corr:.5f}")
