@@ -846,7 +846,6 @@ extern "C" int vitint_qk(const vitint_slabs* q, const vitint_slabs* k, int32_t b
     if (int rc = check_slabs(q)) return rc;
     if (int rc = check_slabs(k)) return rc;
     if (batch <= 0 || heads <= 0 || tokens <= 0 || !s_out || ld_s < tokens) return VITINT_ERR_INVALID_ARG;
-    if (tokens > 256) return VITINT_ERR_UNSUPPORTED;   // one column tile per problem in this kernel
     GemmParams P{};
     vitint_epilogue epi{};
     epi.mode = VITINT_EPI_ACC_I32;

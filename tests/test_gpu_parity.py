@@ -200,7 +200,7 @@ def _qkv_codes(batch, tokens, heads, bits, seed):
 
 
 @pytest.mark.parametrize("bits", [4, 2, 8])
-@pytest.mark.parametrize("batch,tokens,heads", [(1, 197, 3), (3, 197, 2), (2, 50, 1), (1, 256, 2)])
+@pytest.mark.parametrize("batch,tokens,heads", [(1, 197, 3), (3, 197, 2), (2, 50, 1), (1, 256, 2), (2, 577, 1), (1, 785, 2)])
 def test_qk_bit_exact(batch, tokens, heads, bits):
     D = heads * 64
     qkv = _qkv_codes(batch, tokens, heads, bits, 21)
@@ -211,7 +211,7 @@ def test_qk_bit_exact(batch, tokens, heads, bits):
 
 
 @pytest.mark.parametrize("bits", [4, 2, 8])
-@pytest.mark.parametrize("batch,tokens,heads", [(1, 197, 3), (3, 197, 2), (2, 50, 1), (1, 256, 2)])
+@pytest.mark.parametrize("batch,tokens,heads", [(1, 197, 3), (3, 197, 2), (2, 50, 1), (1, 256, 2), (2, 577, 1), (1, 785, 2)])
 def test_pv_bit_exact(batch, tokens, heads, bits):
     D = heads * 64
     qkv = _qkv_codes(batch, tokens, heads, bits, 22)
@@ -406,3 +406,68 @@ def test_attention_block_requant_output():
     assert rows_ok.mean() > 0.9
     assert np.array_equal(from_codes(out)[rows_ok], st["out_codes"][rows_ok])
     assert len(np.unique(st["out_codes"])) >= 8
+
+
+# ---------------------------------------------------------------------------
+# sweep over the linear shapes of the scaling study
+# ---------------------------------------------------------------------------
+
+SWEEP_KN = [192, 384, 768, 1024, 3072, 4096]
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+@pytest.mark.parametrize("tokens,batch", [(197, 1), (577, 1), (785, 2)])
+def test_linear_sweep_shapes(tokens, batch, bits):
+    """K, N over {192 ... 4096}, M = batch*tokens, Gaussian inputs with 1 % outlier channels, every bit width;
+    quantize -> integer linear (requantizing epilogue) against the oracle, bit for bit."""
+    M = tokens * batch
+    for idx, K in enumerate(SWEEP_KN):
+        N = SWEEP_KN[(idx * 5 + 2 + bits) % len(SWEEP_KN)]
+        x = si.normal(300 + K + bits, (M, K))
+        ch = si.choice_without_replacement(9 + K, K, max(1, K // 100))
+        x[:, ch] *= np.float32(10.0)
+        w = si.normal(400 + N + bits, (N, K), 0.0, 0.02)
+        s_x = si.lsq_step(x, bits, True)
+        s_w = si.lsq_step_rows(w, bits)
+        qx = vo.quantize(x, s_x, bits, True)
+        qw = vo.quantize(w, 0.0, bits, True, row_steps=s_w)
+        bias = si.normal(500 + N, (N,), 0.0, 0.01)
+        s_out = si.gaussian_lsq_step(float(s_x) * float(np.mean(s_w)) * math.sqrt(K) * (2 ** (bits - 1)) / 2, bits)
+        alpha, beta = vp.fold(s_x, s_w, bias, s_out)
+        gx = vt.vitint_quantize(dev(x), float(s_x), bits, True)
+        gw = vt.vitint_quantize(dev(w), 0.0, bits, True, row_steps=dev(s_w))
+        assert np.array_equal(from_codes(gx), qx) and np.array_equal(from_codes(gw), qw)
+        if bits != 8:
+            gw = vt.vitint_widen(gw)
+        epi = vt.Epilogue(mode=vt.EPI_REQUANT, alpha=dev(alpha), beta=dev(beta), out_bits=bits, out_signed=True)
+        got = vt.vitint_linear(gx, float(s_x), gw, None, None, epi)
+        want = vo.epilogue_requant(vo.matmul_i32(qx, qw), alpha, beta, bits, True)
+        assert np.array_equal(from_codes(got), want), (K, N)
+        assert len(np.unique(want)) >= min(4, 2 ** bits - 1)
+
+
+@pytest.mark.parametrize("tokens", [577, 785])
+def test_unfused_attention_long_sequences(tokens):
+    """Token counts beyond one 256-column tile: Q K^T -> softmax+quantize -> P V through the unfused calls."""
+    batch, heads, bits = 1, 2, 4
+    D = heads * 64
+    qkv = _qkv_codes(batch, tokens, heads, bits, 81 + tokens)
+    c8 = to_codes(qkv, bits, True)
+    S = vt.vitint_qk(vt.Slabs.of_qkv(c8, tokens, D, 0), vt.Slabs.of_qkv(c8, tokens, D, 1), batch, heads, tokens)
+    q = vp.split_heads(qkv, batch, tokens, heads, 64, 0)
+    k = vp.split_heads(qkv, batch, tokens, heads, 64, D)
+    v = vp.split_heads(qkv, batch, tokens, heads, 64, 2 * D)
+    S_ref = vo.qk(q, k)
+    assert np.array_equal(S.cpu().numpy()[:, :, :tokens], S_ref)
+    c = np.float32(0.004)
+    s_p = np.float32(2.0 / (tokens * math.sqrt(15.0)))
+    n = batch * heads
+    P = vt.vitint_softmax_quantize(S.reshape(n * tokens, -1), tokens, c, s_p, bits)
+    _, pc, plo, phi = vo.softmax_quantize(S_ref.reshape(n * tokens, tokens), c, s_p, bits)
+    gp = from_codes(P)
+    assert np.all(gp >= plo) and np.all(gp <= phi) and len(np.unique(pc)) >= 8
+    # P V from the oracle's own codes, so the comparison is exact
+    O = vt.vitint_pv(to_codes(pc, bits, False), vt.Slabs.of_qkv(c8, tokens, D, 2), batch, heads, tokens, 1.0, 1.0,
+                     vt.Epilogue(mode=vt.EPI_ACC_I32))
+    want = vp.merge_heads(vo.pv(pc.reshape(n, tokens, tokens), v), batch, tokens, heads, 64)
+    assert np.array_equal(O.cpu().numpy(), want)

@@ -82,9 +82,8 @@ def test_argument_errors_are_caught_on_the_host(L):
     assert lib.vitint_softmax_quantize(ctypes.c_void_p(fake), 4, 2000, 2000, 1.0, 1.0, br(pc), None, 0, None) == -2
     ps = _codes(L, fake, 4, 100, 64, 4, 1)
     assert lib.vitint_softmax_quantize(ctypes.c_void_p(fake), 4, 100, 100, 1.0, 1.0, br(ps), None, 0, None) == -1
-    # qk: more tokens than one column tile
     sl = L._Slabs(fake, 384, 384 * 300, 32, 4, 1)
-    assert lib.vitint_qk(br(sl), br(sl), 1, 1, 300, out, 300, None) == -2
+    assert lib.vitint_qk(br(sl), br(sl), 1, 1, 300, out, 299, None) == -1      # ld_s < tokens
     sl_bad = L._Slabs(fake, 380, 384 * 100, 32, 4, 1)
     assert lib.vitint_qk(br(sl_bad), br(sl), 1, 1, 100, out, 100, None) == -3
 
