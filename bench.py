@@ -8,8 +8,9 @@ LayerNorm+quantize -> fc1 (GELU, requantize) -> fc2.  Prints ONE JSON line (rank
 
 value      effective TOPS (2 x true multiply-accumulates of the six integer contractions per
            second), inputs resident in HBM, whole job over all ranks (ranks hold disjoint images).
-e2e        same metric through the same calls with the step's fp32 input copied from pinned host
-           memory and the fp32 output copied back inside the timed region.
+e2e        same metric through the same calls with every step's fp32 input copied from pinned host
+           memory and its fp32 output copied back inside the timed region (copies of neighbouring
+           steps overlap the kernels on separate streams).
 roofline   the integer GEMM kernel: achieved TOPS over its launches inside the timed region
            (CUDA events around each call) against the int8 tensor peak.
 cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the same workload.
@@ -201,14 +202,38 @@ def run_ours(args, cfg):
     stage_ms = {s: v / args.steps for s, v in stage_ms.items()}
 
     # ---- end to end: host -> device, step, device -> host, every step -----------------
+    # Three streams, double-buffered device input and output: the copy of step i+1's input and the read-back
+    # of step i-1's result overlap step i's kernels (every step still moves its own input and output).
     barrier()
+    main = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    x_dev = [torch.empty_like(xs[0]) for _ in range(2)]
+    out_dev = [torch.empty_like(out) for _ in range(2)]
+    ev_in = [torch.cuda.Event() for _ in range(2)]       # input i landed
+    ev_done = [torch.cuda.Event() for _ in range(2)]     # step i finished (its input buffer is free, its output ready)
+    ev_read = [torch.cuda.Event() for _ in range(2)]     # output i read back (its output buffer is free)
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    x_dev = torch.empty_like(xs[0])
     t0.record()
+    s_in.wait_stream(main)
+    s_out.wait_stream(main)
     for i in range(args.steps):
-        x_dev.copy_(host_x[i % N_INPUT_BUFFERS], non_blocking=True)
-        layer.forward(x_dev, out)
-        host_out.copy_(out, non_blocking=True)
+        b = i & 1
+        with torch.cuda.stream(s_in):
+            if i >= 2:
+                s_in.wait_event(ev_done[b])              # step i-2 no longer reads this input buffer
+            x_dev[b].copy_(host_x[i % N_INPUT_BUFFERS], non_blocking=True)
+            ev_in[b].record(s_in)
+        main.wait_event(ev_in[b])
+        if i >= 2:
+            main.wait_event(ev_read[b])                  # step i-2's result has left this output buffer
+        layer.forward(x_dev[b], out_dev[b])
+        ev_done[b].record(main)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_done[b])
+            host_out.copy_(out_dev[b], non_blocking=True)
+            ev_read[b].record(s_out)
+    main.wait_stream(s_in)
+    main.wait_stream(s_out)
     t1.record()
     barrier()
     ms_e2e = max_over_ranks(t0.elapsed_time(t1), world, device)
@@ -250,11 +275,16 @@ def run_ours(args, cfg):
         from oracle import pipeline as vp
         sample = args.ref_images
         xs_cpu = si.activations(cfg, batch=sample)
-        t0c = time.perf_counter()
-        vp.encoder_layer(xs_cpu, prm, sample, cfg.tokens, cfg.heads, cfg.bits)
-        dtc = time.perf_counter() - t0c
-        cpu = {"value": layer_ops(cfg, sample) / dtc / 1e12, "unit": "TOPS", "cores": vo.get_threads(),
-               "kind": "oracle", "sample": f"{sample} of {cfg.batch} images, whole encoder layer, {dtc:.1f} s"}
+        reps, t0c = 0, time.perf_counter()
+        while True:                                  # about ten seconds of CPU work, whole passes only
+            vp.encoder_layer(xs_cpu, prm, sample, cfg.tokens, cfg.heads, cfg.bits)
+            reps += 1
+            dtc = time.perf_counter() - t0c
+            if dtc >= 10.0 or reps >= 20:
+                break
+        cpu = {"value": reps * layer_ops(cfg, sample) / dtc / 1e12, "unit": "TOPS", "cores": vo.get_threads(),
+               "kind": "oracle",
+               "sample": f"{sample} of {cfg.batch} images, whole encoder layer, {reps} passes in {dtc:.1f} s"}
 
     line = {
         "metric": "integerized ViT-B block effective TOPS", "value": tops, "unit": "TOPS", "n_gpus": world,

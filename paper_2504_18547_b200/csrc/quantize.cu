@@ -96,13 +96,19 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
-    const float rstd = (float)(1.0 / sqrt((double)m2 / (double)cols + (double)eps));   // once per row
+    // 1/sqrt(var + eps): hardware estimate plus one Newton step (about 1 ulp), all in fp32
+    const float var = fmaf(m2, inv_n, eps);
+    float rstd = rsqrtf(var);
+    rstd = rstd * fmaf(-0.5f * var, rstd * rstd, 1.5f);
     // y / step as y * RN(1/step): at most 1.5 ulp from the exact quotient, far inside the tolerance
     // that the fp32 normalisation itself is granted, and one instruction instead of three
     const float rstep = __frcp_rn(step);
+    const bool sgn = qn < 0.0f;
+    const float magic = 12582912.0f + (sgn ? (float)(1 << (C - 1)) : 0.0f);
+    const uint32_t top = 1u << (C - 1);
+    const uint32_t flip = sgn ? (top | (top << C) | (top << (2 * C)) | (top << (3 * C))) : 0u;   // offset binary -> two's complement
 
     constexpr int LANES_PER_WORD = 8 / C;          // 4 codes per lane per v -> 4*C bits
-    constexpr uint32_t MASK = (1u << C) - 1u;
     const int words_per_row = (int)(pitch >> 2);
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
@@ -117,10 +123,13 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
             y.z = fmaf(f[v].z * rstd, g.z, b.z);
             y.w = fmaf(f[v].w * rstd, g.w, b.w);
             if (y_out) *reinterpret_cast<float4*>(y_out + row * ld_y + col) = y;
-            bits = (round_clamp_bits(y.x * rstep, qn, qp) & MASK) |
-                   ((round_clamp_bits(y.y * rstep, qn, qp) & MASK) << C) |
-                   ((round_clamp_bits(y.z * rstep, qn, qp) & MASK) << (2 * C)) |
-                   ((round_clamp_bits(y.w * rstep, qn, qp) & MASK) << (3 * C));
+            // clamp, then add 1.5*2^23 (+ 2^(C-1) for signed codes): the low mantissa bits hold the code in
+            // offset binary, so the four codes combine by shift-add without masking
+            const float cx = fminf(fmaxf(y.x * rstep, qn), qp) + magic, cy = fminf(fmaxf(y.y * rstep, qn), qp) + magic;
+            const float cz = fminf(fmaxf(y.z * rstep, qn), qp) + magic, cw = fminf(fmaxf(y.w * rstep, qn), qp) + magic;
+            bits = (__float_as_uint(cx) + (__float_as_uint(cy) << C) + (__float_as_uint(cz) << (2 * C)) +
+                    (__float_as_uint(cw) << (3 * C)) - 0x4B400000u * (1u + (1u << C) + (1u << (2 * C)) + (1u << (3 * C))));
+            bits = (bits ^ flip) & (C == 8 ? 0xFFFFFFFFu : ((1u << ((4 * C) & 31)) - 1u));
         }
         // gather 8/C neighbouring lanes into one 32-bit word
         if (C == 4) {
