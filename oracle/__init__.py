@@ -203,6 +203,18 @@ def softmax_quantize(S, c, p_step, bits: int, ulp_band: int = SOFTMAX_ULP_BAND):
     return p, q, lo, hi
 
 
+def softmax_shift_quantize(S, c2, p_step, bits: int, want_p: bool = False):
+    """Eq. 4 softmax (2^r ~ 1+r, integer shifts) with the division-free comparator quantizer.
+    S [rows, cols] int32 -> codes (and, optionally, the approximate probabilities E_j/Sigma in fp64)."""
+    S = np.ascontiguousarray(S, dtype=np.int32)
+    rows, cols = S.shape
+    q = np.empty((rows, cols), dtype=np.int16)
+    p = np.empty((rows, cols), dtype=np.float64) if want_p else None
+    lib().vo_softmax_shift_quantize(_p(S), I64(rows), I64(cols), I64(cols), F32(float(c2)), F32(float(p_step)),
+                                    I32(bits), _p(q), I64(cols), _p(p), I64(cols))
+    return (q, p) if want_p else q
+
+
 # ---- glue ---------------------------------------------------------------------
 
 def layernorm(x, gamma, beta, eps: float = 1e-6):

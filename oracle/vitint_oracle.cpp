@@ -18,7 +18,8 @@
 // Pins (tests/test_oracle_*.py): Eq. 1 reordering identity against an fp64
 // dequantize-then-matmul, brute force on tiny operands, closed-form sums, the
 // int32 overflow bound, the 3-bit threshold ladder, pack/unpack round trips,
-// exact-rational epilogue cases, softmax closed forms and invariants, LayerNorm
+// exact-rational epilogue cases, softmax closed forms and invariants, the shift softmax
+// against big-integer / rational arithmetic and its 2^r ~ 1+r error bound, LayerNorm
 // against the Welford recurrence of Eq. 5.  Parity unpinned: none of the
 // functions below; the paper's accuracy and power tables are out of scope.
 
@@ -284,6 +285,55 @@ void vo_softmax_quantize(const int32_t* S, int64_t rows, int64_t cols, int64_t l
                 if (q_lo) q_lo[r * ldq + j] = round_clamp(lo / p_step, qn, qp);
                 if (q_hi) q_hi[r * ldq + j] = round_clamp(hi / p_step, qn, qp);
             }
+        }
+    });
+}
+
+// ---- shift-based softmax with the division-free quantizer (Eq. 4, Section IV-B) ---------------
+// Follows the paper's steps with integers wherever it says "shift":
+//   z_j = fl32(float(S_j) * c2),  c2 = s*log2(e) supplied by the caller      (exponent of 2, Eq. 4 line 1)
+//   f_j = floor(z_j),  r_j = z_j - f_j (exact)                                (integer part and residual)
+//   M_j = (1 + r_j) * 2^23   as an integer: 2^r ~ 1 + r                       (Eq. 4 last line)
+//   E_j = M_j << (30 + f_j - m),  m = max_j f_j; negative counts shift right  ("<< floor(...)")
+//         (a common factor 2^(30-m) changes neither side of the comparison below; it only keeps the
+//          integers inside 64 bits; bits shifted out on the right are dropped, as a shifter drops them)
+//   Sigma = sum_j E_j   (exact integer sum: the systolic row adder)
+//   code_j = number of k in 1..Qp with  float(E_j) > fl32(b_k * float(Sigma)),  b_k = fl32((k - 1/2) * step)
+//         (comparator references scaled by the row sum instead of dividing by it; strict '>' as drawn)
+// Every operation is an integer one or a single IEEE fp32 operation, so the codes are unique.
+// p_approx (optional) = float(E_j) / float(Sigma) in fp64, for error studies only.
+void vo_softmax_shift_quantize(const int32_t* S, int64_t rows, int64_t cols, int64_t lds, float c2, float p_step,
+                               int bits, int16_t* q, int64_t ldq, double* p_approx, int64_t ldp) {
+    int qn, qp;
+    code_range(bits, 0, &qn, &qp);
+    parallel_for(rows, [&](int64_t r) {
+        std::vector<int64_t> f((size_t)cols);
+        std::vector<uint64_t> M((size_t)cols), E((size_t)cols);
+        int64_t m = INT64_MIN;
+        for (int64_t j = 0; j < cols; ++j) {
+            const float z = (float)S[r * lds + j] * c2;
+            const float fl = floorf(z);
+            const float res = z - fl;
+            f[j] = (int64_t)fl;
+            M[j] = (uint64_t)((1.0f + res) * 8388608.0f);
+            m = std::max(m, f[j]);
+        }
+        uint64_t sigma = 0;
+        for (int64_t j = 0; j < cols; ++j) {
+            const int64_t sh = 30 + f[j] - m;
+            E[j] = sh >= 0 ? (M[j] << sh) : (sh > -64 ? (M[j] >> (-sh)) : 0);
+            sigma += E[j];
+        }
+        const float sig_f = (float)sigma;
+        for (int64_t j = 0; j < cols; ++j) {
+            const float e_f = (float)E[j];
+            int code = 0;
+            for (int k = 1; k <= qp; ++k) {
+                const float b_k = ((float)k - 0.5f) * p_step;
+                if (e_f > b_k * sig_f) ++code;
+            }
+            q[r * ldq + j] = (int16_t)code;
+            if (p_approx) p_approx[r * ldp + j] = (double)E[j] / (double)sigma;
         }
     });
 }

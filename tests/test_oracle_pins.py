@@ -470,3 +470,79 @@ def test_attention_block_matches_dequantize_first_datapath(w_std):
     ref = o_all @ wp.T + prm["b_proj"].astype(np.float64)
     mag = np.abs(o_all) @ np.abs(wp).T + np.abs(prm["b_proj"].astype(np.float64))
     assert np.all(np.abs(st["out"] - ref) <= 2.0 ** -22 * mag)
+
+
+# ---------------------------------------------------------------------------
+# shift-based softmax with the division-free quantizer (Eq. 4)
+# ---------------------------------------------------------------------------
+
+def _shift_softmax_by_hand(S_row, c2, step, bits):
+    """Independent evaluation with Python integers and exact rational rounding."""
+    qp = (1 << bits) - 1
+    z = (S_row.astype(np.float32) * np.float32(c2)).astype(np.float32)
+    f = np.floor(z)
+    r = (z - f).astype(np.float32)
+    one_plus_r = (np.float32(1.0) + r).astype(np.float32)
+    M = [int(Fraction(float(v)) * (1 << 23)) for v in one_plus_r]
+    m = int(f.max())
+    E = []
+    for Mj, fj in zip(M, f):
+        sh = 30 + int(fj) - m
+        E.append(Mj << sh if sh >= 0 else (Mj >> -sh if sh > -64 else 0))
+    sigma = sum(E)
+    sig_f = Fraction(float(f32_from_fraction(Fraction(sigma))))
+    codes = []
+    for Ej in E:
+        e_f = Fraction(float(f32_from_fraction(Fraction(Ej))))
+        c = 0
+        for k in range(1, qp + 1):
+            b_k = f32_from_fraction(Fraction(k) * 1 - Fraction(1, 2)) * np.float32(step)   # (k - 1/2) is exact in fp32
+            t_k = f32_from_fraction(Fraction(float(np.float32(b_k))) * sig_f)
+            if e_f > Fraction(float(t_k)):
+                c += 1
+        codes.append(c)
+    return codes, [Fraction(e, sigma) for e in E]
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_shift_softmax_against_integer_and_rational_arithmetic(bits):
+    S = (si.splitmix64(91 + bits, 6 * 23) % np.uint64(801)).astype(np.int64).reshape(6, 23) - 400
+    S[1] = 7                                    # all equal
+    S[2, :] = -400
+    S[2, 5] = 400                               # one dominant score: the others are shifted far to the right
+    c2, step = np.float32(0.0211 * 1.4426950408889634), np.float32(2.0 / (23 * math.sqrt(2 ** bits - 1)))
+    q, p = vo.softmax_shift_quantize(S, c2, step, bits, want_p=True)
+    for r in range(6):
+        codes, probs = _shift_softmax_by_hand(S[r], c2, step, bits)
+        assert q[r].tolist() == codes
+        assert np.allclose(p[r], [float(x) for x in probs], rtol=1e-15, atol=0)
+    assert q.max() == 2 ** bits - 1 and q.min() == 0
+
+
+def test_shift_softmax_error_bound_of_the_linear_residual():
+    """2^r ~ 1 + r overestimates by at most 6.15 % (r = 0.5288), so every probability stays within that
+    factor of the exact base-2 softmax; integer-valued exponents make it exact."""
+    T = 197
+    S = (si.splitmix64(95, 16 * T) % np.uint64(1201)).astype(np.int64).reshape(16, T) - 600
+    c2 = np.float32(0.01 * 1.4426950408889634)
+    _, p = vo.softmax_shift_quantize(S, c2, np.float32(0.0026), 4, want_p=True)
+    z = (S.astype(np.float32) * c2).astype(np.float64)
+    e = np.exp2(z - z.max(1, keepdims=True))
+    ref = e / e.sum(1, keepdims=True)
+    ratio = p[ref > 1e-9] / ref[ref > 1e-9]
+    assert ratio.max() <= 1.0616 and ratio.min() >= 1.0 / 1.0616 and ratio.std() > 0.005
+    assert np.all(np.abs(p.sum(1) - 1.0) < 1e-12)
+    # integer exponents: no residual, the shifts are the exact powers of two
+    Si = np.array([[0, 1, 2, 5, -3]], np.int32)
+    _, pi = vo.softmax_shift_quantize(Si, np.float32(1.0), np.float32(0.05), 4, want_p=True)
+    w = np.array([1, 2, 4, 32, 0.125])
+    assert np.allclose(pi[0], w / w.sum(), rtol=1e-15)
+
+
+def test_shift_softmax_comparator_is_strict_and_scaled_by_the_row_sum():
+    # two equal scores: p = 1/2 each; thresholds b_k * Sigma with step 0.25: (k - 1/2)/4 < 1/2  <=>  k < 2.5
+    q = vo.softmax_shift_quantize(np.array([[3, 3]], np.int32), np.float32(1.0), np.float32(0.25), 4)
+    assert q.tolist() == [[2, 2]]
+    # exact tie: p = 1/2 against the reference (k - 1/2) * step = 1/2 at k = 1, step = 1: not exceeded (strict '>')
+    q = vo.softmax_shift_quantize(np.array([[3, 3]], np.int32), np.float32(1.0), np.float32(1.0), 4)
+    assert q.tolist() == [[0, 0]]
