@@ -244,8 +244,9 @@ def run_ours(args, cfg):
         if world > 1:
             dist.destroy_process_group()
         return
+    peaks_early = measured_peaks()
 
-    peaks = measured_peaks()
+    peaks = peaks_early
     ops_step = layer_ops(cfg, cfg.batch)
     ms_step = ms_total / args.steps
     tops = world * ops_step / (ms_step * 1e-3) / 1e12
@@ -267,6 +268,36 @@ def run_ours(args, cfg):
             k["gbs"] = round(sbytes[s] / (stage_ms[s] * 1e-3) / 1e9, 1)
             k["frac_hbm_peak"] = round(k["gbs"] / peaks["hbm_gbs"], 4)
         kernels[s] = k
+
+    # ---- streaming kernels that the fused step does not launch, timed alone (HBM roofline) -------------
+    standalone = {}
+    if world == 1:
+        def timed(fn, reps=10):
+            for _ in range(3):
+                fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+        cb = 4 if cfg.bits == 3 else cfg.bits
+        n_rows, T = cfg.batch * cfg.heads * cfg.tokens, cfg.tokens
+        S = torch.randint(-300, 300, (n_rows, (T + 3) // 4 * 4), dtype=torch.int32, device=device)   # 242 MB > L2
+        Pq = vt.Codes.empty(n_rows, T, cfg.bits, False, device)
+        xq = vt.Codes.empty(M, D, cfg.bits, True, device)
+        sm_bytes = n_rows * T * 4 + n_rows * ((T * cb + 7) // 8)
+        q_bytes = M * D * 4 + M * D * cb // 8
+        for name, fn, nbytes in (
+                ("quantize", lambda: vt.vitint_quantize(xs[1], layer.s_ln, cfg.bits, True, out=xq), q_bytes),
+                ("softmax_quant", lambda: vt.vitint_softmax_quantize(S, T, layer.c, layer.s_p, cfg.bits, out=Pq), sm_bytes),
+                ("softmax_shift_quant", lambda: vt.vitint_softmax_shift_quantize(S, T, layer.c * 1.4426950408889634,
+                                                                                 layer.s_p, cfg.bits, out=Pq), sm_bytes)):
+            ms = timed(fn)
+            standalone[name] = {"ms": round(ms, 4), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                                "frac_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks_early["hbm_gbs"], 4)}
+        del S, Pq, xq
 
     # ---- CPU oracle on a bounded sample (rank 0, single-GPU runs only) -----------------
     cpu = None
@@ -304,6 +335,7 @@ def run_ours(args, cfg):
                      "peak_source": f"{peaks['source']} sustained bf16 cuBLAS x {INT8_OVER_BF16:g} (nominal int8:bf16)",
                      "frac_of_nominal_4500": achieved / 4500.0},
         "kernels": kernels,
+        "kernels_standalone": standalone,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))

@@ -159,6 +159,18 @@ int vitint_qk(const vitint_slabs* q, const vitint_slabs* k, int32_t batch, int32
 int vitint_softmax_quantize(const int32_t* s, int64_t rows, int32_t cols, int64_t ld_s, float c, float p_step,
                             const vitint_codes* p_out, float* p_f32, int64_t ld_p, void* stream);
 
+/* a5, shift form (Eq. 4 with the division-free comparator quantizer of Section IV-B).  Integer and
+ *   single-rounding fp32 operations only, so the codes are unique (bit-exact against the definition):
+ *     z_j = fl32((float)S_j * c2)   (c2 = s*log2(e): the exponent of 2);  f_j = floor(z_j), r_j = z_j - f_j;
+ *     E_j = ((1 + r_j) * 2^23 as an integer) << (30 + f_j - max_k f_k)   (2^r ~ 1 + r; negative counts shift
+ *           right and drop bits; the common factor 2^(30 - max f) only keeps the integers inside 64 bits);
+ *     Sigma = sum_j E_j (exact);  q_j = #{ k in 1..2^bits-1 : (float)E_j > fl32(fl32((k - 1/2)*p_step) * (float)Sigma) }
+ *   i.e. the comparator references are scaled by the row sum instead of dividing by it; the comparison is
+ *   strict, as drawn in the paper (it differs from round-to-nearest-even only on exact ties).
+ *   s, rows, cols, ld_s, p_out as in vitint_softmax_quantize.  cols <= 1024. */
+int vitint_softmax_shift_quantize(const int32_t* s, int64_t rows, int32_t cols, int64_t ld_s, float c2, float p_step,
+                                  const vitint_codes* p_out, void* stream);
+
 /* a6. O[p][i][c] = sum_j P_p[i][j] * V_p[j][c] (Section IV-B, W_attn V), then the epilogue
  *   with s_x*s_w[n] replaced by p_step*v_step (bias NULL; alpha/beta/inv_out_step, when
  *   used, are indexed by the output column h*64 + c).

@@ -69,6 +69,8 @@ def lib():
         L.vitint_qk.argtypes = [POINTER(_Slabs), POINTER(_Slabs), c_int32, c_int32, c_int32, c_void_p, c_int64, c_void_p]
         L.vitint_softmax_quantize.argtypes = [c_void_p, c_int64, c_int32, c_int64, c_float, c_float, POINTER(_Codes),
                                               c_void_p, c_int64, c_void_p]
+        L.vitint_softmax_shift_quantize.argtypes = [c_void_p, c_int64, c_int32, c_int64, c_float, c_float,
+                                                    POINTER(_Codes), c_void_p]
         L.vitint_pv.argtypes = [POINTER(_Codes), POINTER(_Slabs), c_int32, c_int32, c_int32, c_float, c_float,
                                 POINTER(_Epilogue), c_void_p, c_int64, c_void_p]
         L.vitint_attention_core_workspace_bytes.restype = c_size_t
@@ -273,6 +275,17 @@ def vitint_softmax_quantize(s: torch.Tensor, cols: int, c: float, p_step: float,
     _check(lib().vitint_softmax_quantize(s.data_ptr(), rows, cols, ld_s, float(c), float(p_step), byref(d), _ptr(p),
                                          cols if want_p else 0, _stream()), "vitint_softmax_quantize")
     return (out, p) if want_p else out
+
+
+def vitint_softmax_shift_quantize(s: torch.Tensor, cols: int, c2: float, p_step: float, bits: int,
+                                  out: Codes | None = None) -> Codes:
+    """Eq. 4 softmax (2^r ~ 1 + r, integer shifts) with the division-free comparator quantizer."""
+    rows, ld_s = s.shape[0], _ld(s)
+    out = Codes.empty(rows, cols, bits, False, s.device) if out is None else out
+    d = out.desc()
+    _check(lib().vitint_softmax_shift_quantize(s.data_ptr(), rows, cols, ld_s, float(c2), float(p_step), byref(d),
+                                               _stream()), "vitint_softmax_shift_quantize")
+    return out
 
 
 def vitint_pv(p: Codes, v: Slabs, batch: int, heads: int, tokens: int, p_step: float, v_step: float, epi: Epilogue,

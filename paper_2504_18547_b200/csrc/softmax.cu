@@ -10,6 +10,8 @@
 //   * exp(d) = 2^k * exp(r), k = rint(d*log2 e), r = d - k*ln2 reduced in fp64, then a
 //     degree-7 Taylor polynomial in fp32 on |r| <= ln2/2 (truncation < 0.1 ulp);
 //   * the normaliser is accumulated in fp64 and applied as one fp64 multiply.
+#include <climits>
+
 #include "common.cuh"
 
 namespace vitint {
@@ -79,6 +81,8 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
     const double rz = 1.0 / z;
+    const float rzh = (float)rz, rzl = (float)(rz - (double)(float)rz);   // 1/Z as two floats
+    const Divisor dv = make_divisor(p_step);
 
     constexpr uint32_t MASK = (1u << C) - 1u;
     const int chunk_bytes = 32 * C;                                   // 256 codes
@@ -91,7 +95,7 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
             for (int u = 0; u < NCH; ++u)
                 if (u == k) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) p[i] = (float)((double)t[u][i] * rz);
+                    for (int i = 0; i < 8; ++i) p[i] = fmaf(t[u][i], rzh, t[u][i] * rzl);
                 }
             const int col = k * 256 + lane * 8;
             if (p_out && col < cols) {
@@ -106,7 +110,7 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const uint32_t q = (col + i < cols) ? (uint32_t)round_clamp(__fdiv_rn(p[i], p_step), 0.0f, qp) : 0u;
+                const uint32_t q = (col + i < cols) ? (round_clamp_bits(div_rn(p[i], dv), 0.0f, qp) & 0xFFu) : 0u;
                 if (C == 8) { if (i < 4) w0 |= q << (8 * i); else w1 |= q << (8 * (i - 4)); }
                 else w0 |= (q & MASK) << (C * i);
             }
@@ -140,6 +144,124 @@ static int launch_softmax(int nch, const int32_t* s, int64_t rows, int cols, int
     return cuda_status(cudaGetLastError());
 }
 
+// Shift-based softmax with the division-free quantizer (Eq. 4 and the comparator of Section IV-B),
+// one warp per row.  Integer and single-rounding fp32 operations only, so the codes are unique:
+//   z = fl32(float(S) * c2);  f = floor(z);  r = z - f;  M = (1 + r) * 2^23 as an integer  (2^r ~ 1 + r)
+//   E = M << (30 + f - max_j f)   (right shift, dropping bits, when the count is negative)
+//   Sigma = sum_j E (exact, 64-bit);  code = #{ k in 1..Qp : float(E) > fl32(fl32((k - 1/2) * step) * float(Sigma)) }
+// The thresholds grow with k, so the count is found by a bit-by-bit search (one comparison per code bit).
+// Explicit _rn intrinsics keep the compiler from contracting a multiply and a subtract into one FMA.
+template <int C, int NCH>
+__global__ void __launch_bounds__(256)
+softmax_shift_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, int64_t ld_s, float c2,
+                              float p_step, uint8_t* __restrict__ out, int64_t pitch, int code_bits, int vec_in) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int32_t* sr = s + row * ld_s;
+    int fi[NCH][8];
+    uint32_t mant[NCH][8];
+    int m = INT_MIN;
+#pragma unroll
+    for (int k = 0; k < NCH; ++k) {
+        const int col = k * 256 + lane * 8;
+        int sv[8];
+        if (vec_in && col + 8 <= cols) {
+            const int4 a = __ldg(reinterpret_cast<const int4*>(sr + col));
+            const int4 b = __ldg(reinterpret_cast<const int4*>(sr + col) + 1);
+            sv[0] = a.x; sv[1] = a.y; sv[2] = a.z; sv[3] = a.w; sv[4] = b.x; sv[5] = b.y; sv[6] = b.z; sv[7] = b.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sv[i] = (col + i < cols) ? __ldg(sr + col + i) : 0;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float z = __fmul_rn((float)sv[i], c2);
+            const float fl = floorf(z);
+            const float res = __fsub_rn(z, fl);
+            mant[k][i] = (uint32_t)__fmul_rn(__fadd_rn(1.0f, res), 8388608.0f);
+            fi[k][i] = (int)fl;
+            if (col + i < cols) m = max(m, fi[k][i]);
+            else mant[k][i] = 0u;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+
+    unsigned long long sigma = 0ull;
+#pragma unroll
+    for (int k = 0; k < NCH; ++k) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            // shift count 30 + f - m <= 30; far negative counts shift everything out
+            int sh = 30 + fi[k][i] - m;
+            sh = mant[k][i] ? max(sh, -63) : 0;
+            const unsigned long long mj = (unsigned long long)mant[k][i];
+            const unsigned long long e = sh >= 0 ? (mj << sh) : (mj >> (-sh));
+            sigma += e;
+            // keep E as (high, low) in the two register arrays that are free now
+            fi[k][i] = (int)(uint32_t)(e >> 32);
+            mant[k][i] = (uint32_t)e;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sigma += __shfl_xor_sync(0xffffffffu, sigma, o);
+    const float sig_f = __ull2float_rn(sigma);
+
+    constexpr uint32_t MASK = (1u << C) - 1u;
+    const int chunk_bytes = 32 * C;
+    const int n_out_chunks = (int)((pitch + chunk_bytes - 1) / chunk_bytes);
+    for (int k = 0; k < n_out_chunks; ++k) {
+        uint32_t w0 = 0, w1 = 0;
+        if (k < NCH) {
+#pragma unroll
+            for (int u = 0; u < NCH; ++u)
+                if (u == k) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const unsigned long long e = ((unsigned long long)(uint32_t)fi[u][i] << 32) | mant[u][i];
+                        const float e_f = __ull2float_rn(e);
+                        uint32_t code = 0;
+                        for (int b = code_bits - 1; b >= 0; --b) {
+                            const uint32_t t = code | (1u << b);
+                            const float thr = __fmul_rn(__fmul_rn(__fsub_rn((float)t, 0.5f), p_step), sig_f);
+                            code = (e_f > thr) ? t : code;
+                        }
+                        const int col = k * 256 + lane * 8 + i;
+                        if (col >= cols) code = 0;
+                        if (C == 8) { if (i < 4) w0 |= code << (8 * i); else w1 |= code << (8 * (i - 4)); }
+                        else w0 |= (code & MASK) << (C * i);
+                    }
+                }
+        }
+        uint8_t* orow = out + row * pitch;
+        const int64_t off = (int64_t)k * chunk_bytes + lane * C;
+        if (C == 8) {
+            if (off + 8 <= pitch) *reinterpret_cast<uint2*>(orow + off) = make_uint2(w0, w1);
+        } else if (C == 4) {
+            if (off + 4 <= pitch) *reinterpret_cast<uint32_t*>(orow + off) = w0;
+        } else {
+            w0 |= __shfl_xor_sync(0xffffffffu, w0, 1) << 16;
+            if ((lane & 1) == 0 && off + 4 <= pitch) *reinterpret_cast<uint32_t*>(orow + off) = w0;
+        }
+    }
+}
+
+template <int C>
+static int launch_softmax_shift(int nch, const int32_t* s, int64_t rows, int cols, int64_t ld_s, float c2, float p_step,
+                                uint8_t* out, int64_t pitch, int code_bits, int vec_in, cudaStream_t st) {
+    const int warps = 8;
+    dim3 grid((unsigned)((rows + warps - 1) / warps)), block(32 * warps);
+    switch (nch) {
+        case 1: softmax_shift_quantize_kernel<C, 1><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
+        case 2: softmax_shift_quantize_kernel<C, 2><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
+        case 3: softmax_shift_quantize_kernel<C, 3><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
+        case 4: softmax_shift_quantize_kernel<C, 4><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
+        default: return VITINT_ERR_UNSUPPORTED;
+    }
+    return cuda_status(cudaGetLastError());
+}
+
 }  // namespace vitint
 
 using namespace vitint;
@@ -166,4 +288,23 @@ extern "C" int vitint_softmax_quantize(const int32_t* s, int64_t rows, int32_t c
     if (cb == 2) return launch_softmax<2>(nch, s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
     if (cb == 4) return launch_softmax<4>(nch, s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
     return launch_softmax<8>(nch, s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
+}
+
+extern "C" int vitint_softmax_shift_quantize(const int32_t* s, int64_t rows, int32_t cols, int64_t ld_s, float c2,
+                                             float p_step, const vitint_codes* p_out, void* stream) {
+    if (!s || !p_out) return VITINT_ERR_INVALID_ARG;
+    if (int rc = check_codes(p_out)) return rc;
+    if (rows <= 0 || cols <= 0 || ld_s < cols || p_out->rows != rows || p_out->cols != cols || p_out->is_signed)
+        return VITINT_ERR_INVALID_ARG;
+    if (!(p_step > 0.0f && p_step < INFINITY) || !(c2 == c2) || fabsf(c2) == INFINITY) return VITINT_ERR_INVALID_ARG;
+    if (cols > 1024) return VITINT_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(s) & 3u) != 0) return VITINT_ERR_ALIGNMENT;
+    const int cb = codes_container(p_out);
+    const int nch = (cols + 255) / 256;
+    const int vec_in = (aligned16(s) && ld_s % 4 == 0) ? 1 : 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* o = (uint8_t*)p_out->data;
+    if (cb == 2) return launch_softmax_shift<2>(nch, s, rows, cols, ld_s, c2, p_step, o, p_out->pitch_bytes, p_out->bits, vec_in, st);
+    if (cb == 4) return launch_softmax_shift<4>(nch, s, rows, cols, ld_s, c2, p_step, o, p_out->pitch_bytes, p_out->bits, vec_in, st);
+    return launch_softmax_shift<8>(nch, s, rows, cols, ld_s, c2, p_step, o, p_out->pitch_bytes, p_out->bits, vec_in, st);
 }

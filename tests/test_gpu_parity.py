@@ -268,6 +268,26 @@ def test_softmax_quantize_within_two_ulp_and_band(rows, cols, ld, bits):
     assert padding_is_zero(got)
 
 
+@pytest.mark.parametrize("bits", [4, 2, 3, 8])
+@pytest.mark.parametrize("rows,cols,ld", [(591, 197, 200), (64, 197, 197), (33, 50, 52), (40, 577, 580), (24, 785, 785), (9, 1, 4)])
+def test_softmax_shift_quantize_bit_exact(rows, cols, ld, bits):
+    """Eq. 4 softmax with the division-free comparator quantizer: integer / single-rounding arithmetic, unique codes."""
+    S = np.zeros((rows, ld), np.int32)
+    S[:, :cols] = (si.splitmix64(131 + cols, rows * cols) % np.uint64(1401)).astype(np.int64).reshape(rows, cols) - 700
+    S[0, :cols] = 5
+    if cols > 3:
+        S[1, :cols] = -700
+        S[1, 2] = 700
+    c2 = np.float32(0.0211 * 1.4426950408889634)
+    s_p = np.float32(2.0 / (cols * math.sqrt(si.code_range(bits, False)[1])))
+    got = vt.vitint_softmax_shift_quantize(dev(S), cols, c2, s_p, bits)
+    want = vo.softmax_shift_quantize(S[:, :cols], c2, s_p, bits)
+    assert np.array_equal(from_codes(got), want)
+    assert padding_is_zero(got)
+    if cols > 3:
+        assert want.max() == si.code_range(bits, False)[1]
+
+
 def test_softmax_error_statistics_on_attention_like_rows():
     rows, cols = 4096, 197
     S = (si.splitmix64(77, rows * cols) % np.uint64(257)).astype(np.int64).reshape(rows, cols) - 128
