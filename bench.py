@@ -153,7 +153,8 @@ def run_ours(args, cfg):
 
     prm = si.layer_parameters(cfg)
     layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, device,
-                         fused_attention=not args.unfused_attention)
+                         fused_attention=not args.unfused_attention,
+                         wide_activations=not args.packed_activations)
     STAGES = layer.stages
     gemm_stages = [s for s in STAGES if s in GEMM_STAGES]
     M, D = cfg.rows, cfg.dim
@@ -325,6 +326,7 @@ def run_ours(args, cfg):
         "config": {"workload": cfg.name, "bits": cfg.bits, "batch_per_gpu": cfg.batch, "tokens": cfg.tokens,
                    "dim": cfg.dim, "heads": cfg.heads, "mlp_dim": cfg.mlp_dim,
                    "attention": "fused" if layer.fused_attention else "unfused",
+                   "activation_codes": "packed" if args.packed_activations else "one per byte between linear layers",
                    "l2": f"inputs rotate over {N_INPUT_BUFFERS} buffers of {M * D * 4 / 1e6:.1f} MB (> 126 MB L2)"},
         "clocks": clocks,
         "e2e": {"value": e2e_tops, "unit": "TOPS", "h2d_bytes_per_step": M * D * 4, "d2h_bytes_per_step": M * D * 4,
@@ -353,6 +355,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="images per GPU (default: the configuration's 128)")
     ap.add_argument("--ref-images", type=int, default=None, help="images per step of the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--packed-activations", action="store_true",
+                    help="keep every activation code matrix bit-packed (default: one code per byte where only a linear layer reads it)")
     ap.add_argument("--unfused-attention", action="store_true", help="run Q K^T, softmax and P V as separate kernels")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

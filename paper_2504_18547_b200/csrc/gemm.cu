@@ -247,6 +247,9 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     uint8_t* o = (uint8_t*)P.out + orow * P.ld_out + byte0;
     if (P.out_c == 4 && byte0 + 16 <= P.ld_out) {
         *reinterpret_cast<uint4*>(o) = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+    } else if (P.out_c == 8 && byte0 + 32 <= P.ld_out) {
+        reinterpret_cast<uint4*>(o)[0] = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+        reinterpret_cast<uint4*>(o)[1] = make_uint4(wds[4], wds[5], wds[6], wds[7]);
     } else {
 #pragma unroll
         for (int k = 0; k < 8; ++k)

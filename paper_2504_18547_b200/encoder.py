@@ -24,7 +24,8 @@ def _dev(a, device):
 
 class EncoderLayer:
     def __init__(self, batch: int, tokens: int, heads: int, mlp_dim: int, bits: int, prm: dict, device="cuda",
-                 eps: float = 1e-6, widen_weights: bool = True, fused_attention: bool = True):
+                 eps: float = 1e-6, widen_weights: bool = True, fused_attention: bool = True,
+                 wide_activations: bool = True):
         self.batch, self.tokens, self.heads, self.bits, self.eps = batch, tokens, heads, bits, eps
         self.dim = D = heads * 64
         self.mlp_dim = F = mlp_dim
@@ -55,8 +56,11 @@ class EncoderLayer:
         self.alpha_o = d(a)
         self.inv_s_g = d((1.0 / np.full(F, prm["s_g"], np.float64)).astype(np.float32))
         self.c = float(np.float32(float(prm["s_q"]) * float(prm["s_k"]) / 8.0))
-        # activations
-        self.x1 = B.Codes.empty(M, D, bits, True, device)
+        # activations.  The codes that only feed a linear layer (x1, O, x2, g) are stored one per
+        # byte, so that layer's TMA copy is already the tensor-core operand; q, k, v stay packed
+        # (the attention kernels unpack them per head).
+        ca = 8 if wide_activations and bits != 8 else 0
+        self.x1 = B.Codes.empty(M, D, bits, True, device, container=ca)
         self.qkv = B.Codes.empty(M, 3 * D, bits, True, device)
         self.ld_s = (tokens + 3) // 4 * 4
         if self.fused_attention:
@@ -64,15 +68,16 @@ class EncoderLayer:
         else:
             self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
             self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
-        self.O = B.Codes.empty(M, D, bits, True, device)
+        self.O = B.Codes.empty(M, D, bits, True, device, container=ca)
         self.h = torch.empty((M, D), dtype=torch.float32, device=device)
-        self.x2 = B.Codes.empty(M, D, bits, True, device)
-        self.g = B.Codes.empty(M, F, bits, False, device)
+        self.x2 = B.Codes.empty(M, D, bits, True, device, container=ca)
+        self.g = B.Codes.empty(M, F, bits, False, device, container=ca)
         self.slabs = [B.Slabs.of_qkv(self.qkv, tokens, D, i) for i in range(3)]
         self.epi_qkv = B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_qkv, beta=self.beta_qkv, out_bits=bits,
                                   out_signed=True)
-        self.epi_o = B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_o, out_bits=bits, out_signed=True)
-        self.epi_fc1 = B.Epilogue(mode=B.EPI_REQUANT, act=1, inv_out_step=self.inv_s_g, out_bits=bits, out_signed=False)
+        self.epi_o = B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_o, out_bits=bits, out_signed=True, out_container=ca)
+        self.epi_fc1 = B.Epilogue(mode=B.EPI_REQUANT, act=1, inv_out_step=self.inv_s_g, out_bits=bits, out_signed=False,
+                                  out_container=ca)
 
     def forward(self, x: torch.Tensor, out: torch.Tensor, events: list | None = None) -> torch.Tensor:
         """x, out: fp32 [batch*tokens, dim] on the device.  `events`, when given, receives
@@ -121,9 +126,10 @@ class EncoderLayer:
     def stage_bytes(self) -> dict:
         """Algorithmic HBM bytes of the streaming stages (4 + c/8 per element)."""
         c = 4 if self.bits == 3 else self.bits
+        cx = self.x1.stored_bits
         M, D, T = self.rows, self.dim, self.tokens
         n = self.batch * self.heads * T
-        return {"ln1_quant": M * D * 4 + M * D * c // 8, "ln2_quant": M * D * 4 + M * D * c // 8,
+        return {"ln1_quant": M * D * 4 + M * D * cx // 8, "ln2_quant": M * D * 4 + M * D * cx // 8,
                 "softmax_quant": n * T * 4 + n * ((T * c + 7) // 8)}
 
 

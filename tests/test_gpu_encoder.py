@@ -80,15 +80,17 @@ def compare_stages(g, st, B, T, H, D, fused, min_images_ok):
     return tok_ok3.mean()
 
 
+@pytest.mark.parametrize("wide", [True, False], ids=["byte_codes", "packed_codes"])
 @pytest.mark.parametrize("fused", [True, False], ids=["fused_attention", "unfused_attention"])
 @pytest.mark.parametrize("bits", [4, 3, 2])
-def test_encoder_layer_staged(bits, fused):
+def test_encoder_layer_staged(bits, fused, wide):
     from paper_2504_18547_b200.encoder import EncoderLayer
     cfg = si.VIT_BASE_LAYER.with_(batch=3, bits=bits)
     prm = si.layer_parameters(cfg)
     x = si.activations(cfg)
     st = vp.encoder_layer(x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits)
-    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, fused_attention=fused)
+    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, fused_attention=fused,
+                         wide_activations=wide)
     assert layer.fused_attention == fused
     out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
     layer.forward(dev(x), out)
