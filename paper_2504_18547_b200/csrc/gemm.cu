@@ -5,13 +5,15 @@
 // One persistent CTA per SM walks 128 x BN output tiles.  Warp roles:
 //   warps 0-7  epilogue: stage the tile's per-column scale / bias in shared memory,
 //              tcgen05.ld of their 32 TMEM lanes, rescale / bias / GELU / requantize /
-//              pack, global stores (warp w owns TMEM lanes 32(w%4).. and half of the columns);
+//              pack, global stores (warp w owns TMEM lanes 32(w%4).. and a share of the columns);
 //   warp  8    TMA producer: packed low-bit tiles -> shared-memory ring; operands that are
 //              already 8-bit go straight into the swizzled int8 operand ring;
 //   warp  9    MMA issuer (one thread) and owner of the TMEM allocation;
 //   warps 10-13 unpack: packed codes -> int8 operand tiles in the shared-memory layout
 //              the tensor core expects (128-byte swizzle, K contiguous; or 64-byte
-//              swizzle, N contiguous, for the V operand of P*V).
+//              swizzle, N contiguous, for the V operand of P*V).  When both operands are
+//              stored one code per byte there is nothing to unpack and these four warps
+//              serve as a third epilogue warp per lane quarter.
 // The accumulator is double buffered in TMEM so the epilogue of tile i overlaps the
 // MMAs of tile i+1.
 //
@@ -30,8 +32,9 @@ namespace {
 
 constexpr int BM = 128;   // rows per tile (= TMEM lanes)
 constexpr int BK = 128;   // int8 elements per K block (= one 128-byte swizzle row)
-constexpr int EPI_WARPS = 8;   // two warps per TMEM lane quarter, each taking half of the tile's columns
-constexpr int UNPACK_WARPS = 4;
+constexpr int EPI_WARPS = 8;   // two warps per TMEM lane quarter, each taking a share of the tile's columns
+constexpr int UNPACK_WARPS = 4;   // with nothing to unpack these become a third epilogue warp per lane quarter
+constexpr int MAX_EPI_WARPS = EPI_WARPS + UNPACK_WARPS;
 constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_UNPACK0 = 10;
 constexpr int NUM_THREADS = (WARP_UNPACK0 + UNPACK_WARPS) * 32;
 constexpr int MAX_STAGES = 8;
@@ -45,6 +48,7 @@ struct GemmParams {
     int ca, cb, a_signed, b_signed, shift, b_mn_major;
     int a_direct, b_direct;            // operand already int8: TMA writes the operand ring itself
     int small_acc;                     // |acc| < 2^22: int -> float without a conversion instruction
+    int epi_warps;                     // EPI_WARPS, or MAX_EPI_WARPS when both operands come straight from TMA
     uint32_t stage_off;                // fp32 epilogue: byte offset of the per-warp transposition buffers (0 = none)
     int ns_i, ns_p;
     uint32_t ia_bytes, ib_bytes, pa_bytes, pb_bytes, tmem_cols;
@@ -262,6 +266,76 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     }
 }
 
+// Requantizing epilogue of whole 16-column blocks as a ROLLED loop.  The fully unrolled 32-column
+// form above is ~900 instructions of straight-line code that every warp walks once per chunk, so it
+// streams through the instruction cache; this body (16 independent element chains) is a quarter of
+// that and is re-used by every block of the warp's share.  Columns [col_begin, col_end) of the tile,
+// all of them real columns; col_begin and col_end are multiples of 16.  Whole-warp call: the TMEM
+// load is a warp-wide instruction, so lanes whose row lies past M run the arithmetic too and only
+// their stores are masked.
+template <int KIND, int SMALL>
+__device__ __forceinline__ void epilogue_requant_blocks(const GemmParams& P, const EpiParams& ep, int buf,
+                                                       uint32_t t_row, bool row_ok, long long orow, long long col0,
+                                                       int col_begin, int col_end) {
+    const bool sgn = P.out_qn < 0.0f;
+    const float magic = 12582912.0f + (sgn ? (float)(1 << (P.out_c - 1)) : 0.0f);
+    uint8_t* const o_row = (uint8_t*)P.out + orow * P.ld_out;
+#pragma unroll 1
+    for (int col = col_begin; col < col_end; col += 16) {
+        uint32_t v[16];
+        ptx::tmem_ld16(t_row + (uint32_t)col, v);
+        ptx::tmem_ld_wait();
+        const float4* pa = reinterpret_cast<const float4*>(&ep.a[buf][col]);
+        const float4* pb = reinterpret_cast<const float4*>(&ep.b[buf][col]);
+        const float4* pq = reinterpret_cast<const float4*>(&ep.q[buf][col]);
+        uint32_t code[16];
+#pragma unroll
+        for (int i4 = 0; i4 < 4; ++i4) {
+            const float4 a4 = pa[i4], b4 = pb[i4];
+            const float aa[4] = {a4.x, a4.y, a4.z, a4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w};
+            float qq[4] = {0.f, 0.f, 0.f, 0.f};
+            if (KIND == EK_REQUANT_GELU) {
+                const float4 q4 = pq[i4];
+                qq[0] = q4.x; qq[1] = q4.y; qq[2] = q4.z; qq[3] = q4.w;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int i = 4 * i4 + j;
+                const float f = SMALL == 2 ? small_int_to_float((int)v[i])
+                              : SMALL == 1 ? small_int_to_float((int)v[i] >> P.shift) : (float)(int)v[i];
+                float val = fmaf(f, aa[j], bb[j]);
+                if (KIND == EK_REQUANT_GELU) val = gelu_scaled(val, qq[j]);
+                code[i] = __float_as_uint(fminf(fmaxf(val, P.out_qn), P.out_qp) + magic);
+            }
+        }
+        // offset-binary packing as in epilogue_chunk: 16 codes = 2 * out_c bytes
+        const long long c = col0 + col;
+        if (P.out_c == 8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                w[i] = __byte_perm(__byte_perm(code[4 * i], code[4 * i + 1], 0x4040),
+                                   __byte_perm(code[4 * i + 2], code[4 * i + 3], 0x4040), 0x5410) ^ (sgn ? 0x80808080u : 0u);
+            if (row_ok) *reinterpret_cast<uint4*>(o_row + c) = make_uint4(w[0], w[1], w[2], w[3]);
+        } else if (P.out_c == 4) {
+            uint32_t w[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t acc = code[8 * h];
+#pragma unroll
+                for (int j = 1; j < 8; ++j) acc += code[8 * h + j] << (4 * j);
+                w[h] = (acc - 0x4B400000u * 0x11111111u) ^ (sgn ? 0x88888888u : 0u);
+            }
+            if (row_ok) *reinterpret_cast<uint2*>(o_row + (c >> 1)) = make_uint2(w[0], w[1]);
+        } else {
+            uint32_t acc = code[0];
+#pragma unroll
+            for (int j = 1; j < 16; ++j) acc += code[j] << (2 * j);
+            if (row_ok) *reinterpret_cast<uint32_t*>(o_row + (c >> 2)) = (acc - 0x4B400000u * 0x55555555u) ^ (sgn ? 0xAAAAAAAAu : 0u);
+        }
+    }
+}
+
 constexpr int STAGE_LD = 36;                                  // floats per staged row: 144 bytes keeps 16-byte accesses conflict-free
 constexpr int STAGE_BYTES = 32 * STAGE_LD * 4;                // one 32 x 32 fp32 block per epilogue warp
 
@@ -327,11 +401,25 @@ __device__ __forceinline__ void epilogue_chunk_staged(const GemmParams& P, const
 
 template <int KIND, int SMALL>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiParams& ep, int buf, uint32_t t_row,
-                                              bool row_ok, long long orow, long long colbase, int n_tile, int half,
+                                              bool row_ok, long long orow, long long colbase, int n_tile, int slice,
                                               float* stage, int lane, int rows_valid) {
-    // the two warps of a lane quarter split the tile's 32-column chunks: first half / second half
-    const int n_chunks = (P.bn + 31) / 32, split = (n_chunks + 1) / 2;
-    const int c_begin = half ? split : 0, c_end = half ? n_chunks : split;
+    // the warps of a lane quarter split the tile's 32-column chunks into contiguous shares
+    const int n_slices = P.epi_warps >> 2;
+    const int n_chunks = (P.bn + 31) / 32, base = n_chunks / n_slices, rem = n_chunks % n_slices;
+    const int c_begin = slice * base + (slice < rem ? slice : rem), c_end = c_begin + base + (slice < rem ? 1 : 0);
+    constexpr bool is_req = (KIND == EK_REQUANT || KIND == EK_REQUANT_GELU);
+    if (is_req && (n_tile + 1) * P.bn <= P.N && (P.bn & 31) == 0 && (colbase & 15) == 0) {
+        // every column of the tile is real: rolled 16-column blocks
+        epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL>(P, ep, buf, t_row, row_ok, orow,
+                                                                  colbase + (long long)n_tile * P.bn, c_begin * 32, c_end * 32);
+        // row padding behind the last column of the matrix
+        if (row_ok && P.col_off_inner == 0 && n_tile * P.bn + c_end * 32 >= P.N && c_end > c_begin) {
+            for (long long off = ((long long)P.N * P.out_c) >> 3; off + 4 <= P.ld_out; off += 4)
+                *reinterpret_cast<uint32_t*>((uint8_t*)P.out + orow * P.ld_out + off) = 0u;
+        }
+        __syncwarp();
+        return;
+    }
     for (int chunk = c_begin; chunk < c_end; ++chunk) {
         const int n0 = n_tile * P.bn + chunk * 32;
         if (n0 >= P.N) break;
@@ -392,9 +480,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(ptx::smem_addr(&bars.acc_full[b]), 1);
-            ptx::mbar_init(ptx::smem_addr(&bars.acc_empty[b]), EPI_WARPS);
+            ptx::mbar_init(ptx::smem_addr(&bars.acc_empty[b]), P.epi_warps);
         }
-        ptx::mbar_init(ptx::smem_addr(&bars.epi_sync), EPI_WARPS * 32);
+        ptx::mbar_init(ptx::smem_addr(&bars.epi_sync), P.epi_warps * 32);
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
     }
@@ -496,7 +584,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (ok) ptx::mma_commit(ptx::smem_addr(&bars.acc_full[buf]));
             }
         }
-    } else if (warp >= WARP_UNPACK0) {
+    } else if (warp >= WARP_UNPACK0 && P.epi_warps == EPI_WARPS) {
         // --------------------------------- unpack ----------------------------------
         if (any_packed) {
             const int tid_u = threadIdx.x - WARP_UNPACK0 * 32;
@@ -539,9 +627,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // -------------------------------- epilogue ---------------------------------
-        const int q4 = warp & 3;   // TMEM lane quarter
-        const int half = warp >> 2;   // which half of the tile's columns
-        const int tid_e = threadIdx.x;                       // 0..255
+        const int q4 = warp & 3;   // TMEM lane quarter (fixed by the warp's index in the CTA)
+        const int slice = warp < EPI_WARPS ? warp >> 2 : 2;   // which share of the tile's columns
+        const int ewarp = warp < EPI_WARPS ? warp : warp - (WARP_UNPACK0 - EPI_WARPS);   // 0 .. epi_warps-1
+        const int tid_e = ewarp * 32 + lane;
         // small accumulators are shifted back as integers; otherwise 2^-shift rides on the multiplier
         const float down = P.small_acc == 1 ? 1.0f : __int_as_float((127 - P.shift) << 23);
         int tl = 0;
@@ -553,7 +642,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const long long colbase = (long long)inner * P.col_off_inner;
             // stage this tile's per-column parameters while its MMAs are still running
             if (KIND != EK_ACC) {
-                for (int c = tid_e; c < P.bn; c += EPI_WARPS * 32) {
+                for (int c = tid_e; c < P.bn; c += P.epi_warps * 32) {
                     const int n = n_tile * P.bn + c;
                     float a = 0.0f, b = 0.0f, q = 0.0f;
                     if (n < P.N) {
@@ -583,10 +672,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t t_row = tmem_base + (uint32_t)buf * acc_stride + ((uint32_t)(q4 * 32) << 16);
             int rows_valid = P.M - (m_tile * BM + q4 * 32);
             rows_valid = rows_valid < 0 ? 0 : (rows_valid > 32 ? 32 : rows_valid);
-            float* const stage = P.stage_off ? reinterpret_cast<float*>(smem_gen + P.stage_off + (size_t)warp * STAGE_BYTES) : nullptr;
-            if (P.small_acc == 2) epilogue_tile<KIND, 2>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, half, stage, lane, rows_valid);
-            else if (P.small_acc == 1) epilogue_tile<KIND, 1>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, half, stage, lane, rows_valid);
-            else epilogue_tile<KIND, 0>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, half, stage, lane, rows_valid);
+            float* const stage = P.stage_off ? reinterpret_cast<float*>(smem_gen + P.stage_off + (size_t)ewarp * STAGE_BYTES) : nullptr;
+            if (P.small_acc == 2) epilogue_tile<KIND, 2>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid);
+            else if (P.small_acc == 1) epilogue_tile<KIND, 1>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid);
+            else epilogue_tile<KIND, 0>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid);
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&bars.acc_empty[buf]));
@@ -695,7 +784,8 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     bool staged = (P.kind == EK_DEQUANT || P.kind == EK_DEQUANT_GELU) && n_inner == 1 && n_outer == 1 &&
                   aligned16(P.out) && P.ld_out % 4 == 0 &&
                   (!P.residual || (aligned16(P.residual) && P.ld_res % 4 == 0));
-    const uint32_t stage_total = staged ? (uint32_t)(EPI_WARPS * STAGE_BYTES) : 0u;
+    P.epi_warps = (P.a_direct && P.b_direct) ? MAX_EPI_WARPS : EPI_WARPS;
+    const uint32_t stage_total = staged ? (uint32_t)(P.epi_warps * STAGE_BYTES) : 0u;
     const uint32_t ring_budget = SMEM_TILE_BUDGET + 12u * 1024u - stage_total;   // staging comes out of the ring space
     // The packed ring hides the global-memory latency of the TMA loads; the int8 ring only
     // decouples unpack from MMA issue, unless TMA writes it directly.
