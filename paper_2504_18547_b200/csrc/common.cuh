@@ -89,28 +89,87 @@ __device__ __forceinline__ float small_int_to_float(int v) {
     return __int_as_float(0x4B400000 + v) - 12582912.0f;
 }
 
+// ---- packed fp32 pairs ---------------------------------------------------------------------
+// sm_100 issues add / mul / fma on two fp32 values held in a 64-bit register pair as ONE
+// instruction (f32x2); each half is the IEEE round-to-nearest result of the scalar operation, so
+// pairing elements changes no bit of the outcome and halves the issue slots of an
+// instruction-bound element-wise stage.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 f2_pack(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ f32x2 f2_dup(float v) { return f2_pack(v, v); }
+__device__ __forceinline__ void f2_unpack(f32x2 r, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ f32x2 f2_fma(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 f2_mul(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 f2_add(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 // GELU(y) = y * Phi(y) = 0.5*y*(1 + erf(y/sqrt 2)), with erf from
 //   erf(z) = sign(z) * (1 - 2^(-q(|z|))),   q(z) = -log2(erfc(z)) ~ z*(c0 + c1 z + ... + c6 z^6)
 // on |z| <= 4 (beyond that erf is 1 to 2e-8).  The coefficients are a weighted minimax fit
 // (max |erf error| 7.8e-8 in exact arithmetic); with ex2.approx (2 ulp) and the fp32 Horner
 // steps the absolute error of Phi stays below 2.5e-7, i.e. |GELU error| < 2^-21 * |y|.
-// gelu_scaled(y, h) = 2*h*GELU(y); h = 0.5 gives GELU itself, h = 0.5/s_out folds the output step.
-__device__ __forceinline__ float gelu_scaled(float y, float h) {
-    const float z = fminf(fabsf(y) * 0.70710678118654752440f, 4.0f);
-    float q = -1.00217749e-04f;
-    q = fmaf(q, z, 4.61550077e-04f);
-    q = fmaf(q, z, 2.30229650e-03f);
-    q = fmaf(q, z, -2.94525847e-02f);
-    q = fmaf(q, z, 1.48963709e-01f);
-    q = fmaf(q, z, 9.18328634e-01f);
-    q = fmaf(q, z, 1.62791373e+00f);
-    q = q * z;
+// The polynomial runs in t = z/4 (coefficients scaled by exact powers of four), so the clamp
+// of z to [0, 4] is the saturate modifier of the multiply that forms t.
+__device__ __forceinline__ float gelu_erfc_term(float y) {               // 2^(-q(|y|/sqrt 2)) = erfc(|y|/sqrt 2)
+    const float t = __saturatef(fabsf(y) * 0.17677669529663688110f);     // min(|y|/sqrt 2, 4) / 4
+    float q = -1.00217749e-04f * 16384.0f;
+    q = fmaf(q, t, 4.61550077e-04f * 4096.0f);
+    q = fmaf(q, t, 2.30229650e-03f * 1024.0f);
+    q = fmaf(q, t, -2.94525847e-02f * 256.0f);
+    q = fmaf(q, t, 1.48963709e-01f * 64.0f);
+    q = fmaf(q, t, 9.18328634e-01f * 16.0f);
+    q = fmaf(q, t, 1.62791373e+00f * 4.0f);
+    q = q * t;
     float e;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-q));
-    const float erf_abs = 1.0f - e;
-    const float t = copysignf(erf_abs, y);
-    const float hy = h * y;
-    return fmaf(hy, t, hy);
+    return e;
+}
+// The same term for two elements: the Horner steps run as packed pairs.
+__device__ __forceinline__ void gelu_erfc_term2(float y0, float y1, float& e0, float& e1) {
+    const f32x2 t = f2_pack(__saturatef(fabsf(y0) * 0.17677669529663688110f),
+                            __saturatef(fabsf(y1) * 0.17677669529663688110f));
+    f32x2 q = f2_dup(-1.00217749e-04f * 16384.0f);
+    q = f2_fma(q, t, f2_dup(4.61550077e-04f * 4096.0f));
+    q = f2_fma(q, t, f2_dup(2.30229650e-03f * 1024.0f));
+    q = f2_fma(q, t, f2_dup(-2.94525847e-02f * 256.0f));
+    q = f2_fma(q, t, f2_dup(1.48963709e-01f * 64.0f));
+    q = f2_fma(q, t, f2_dup(9.18328634e-01f * 16.0f));
+    q = f2_fma(q, t, f2_dup(1.62791373e+00f * 4.0f));
+    q = f2_mul(q, t);
+    float q0, q1;
+    f2_unpack(q, q0, q1);
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(-q0));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(-q1));
+}
+// gelu_scaled(y, h) = 2*h*GELU(y); h = 0.5 gives GELU itself, h = 0.5/s_out folds the output step.
+// With w = h*y:  w*(1 + erf) = (w + |w|) - |w|*erfc, one rounding after an exact first term.
+__device__ __forceinline__ float gelu_scaled(float y, float h) {
+    const float e = gelu_erfc_term(y);
+    const float w = h * y;
+    return fmaf(-fabsf(w), e, w + fabsf(w));
+}
+// The same value clamped to [0, 1] by the saturate modifier of the last FMA (NaN -> 0).
+__device__ __forceinline__ float gelu_scaled_unit(float y, float h) {
+    const float e = gelu_erfc_term(y);
+    const float w = h * y;
+    return __saturatef(fmaf(-fabsf(w), e, w + fabsf(w)));
 }
 __device__ __forceinline__ float gelu_f32(float y) { return gelu_scaled(y, 0.5f); }
 

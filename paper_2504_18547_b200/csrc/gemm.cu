@@ -48,6 +48,7 @@ struct GemmParams {
     int ca, cb, a_signed, b_signed, shift, b_mn_major;
     int a_direct, b_direct;            // operand already int8: TMA writes the operand ring itself
     int small_acc;                     // |acc| < 2^22: int -> float without a conversion instruction
+    int unit_out;                      // GELU + unsigned requantization: the GELU multiplier carries 1/Qp and values clamp to [0, 1]
     int epi_warps;                     // EPI_WARPS, or MAX_EPI_WARPS when both operands come straight from TMA
     uint32_t stage_off;                // fp32 epilogue: byte offset of the per-warp transposition buffers (0 = none)
     int ns_i, ns_p;
@@ -181,6 +182,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     // every container's top bit turns offset binary into two's complement.
     const bool sgn = P.out_qn < 0.0f;
     const float magic = 12582912.0f + (sgn ? (float)(1 << (P.out_c - 1)) : 0.0f);
+    const float c_lo = P.unit_out ? 0.0f : P.out_qn, c_hi = P.unit_out ? 1.0f : P.out_qp, c_mul = P.unit_out ? P.out_qp : 1.0f;
     uint32_t code[32];
 #pragma unroll
     for (int i4 = 0; i4 < 8; ++i4) {
@@ -203,10 +205,10 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
                           : SMALL == 1 ? small_int_to_float((int)v[i] >> P.shift) : (float)(int)v[i];
             float val = fmaf(f, aa[j], bb[j]);
             if (KIND == EK_DEQUANT_GELU) val = gelu_f32(val);
-            if (KIND == EK_REQUANT_GELU) val = gelu_scaled(val, qq[j]);      // qq = 0.5 / s_out
+            if (KIND == EK_REQUANT_GELU) val = gelu_scaled(val, qq[j]);      // qq = 0.5 / s_out (/ Qp when unit_out)
             if (has_res) val = val + rr[j];
             y[j] = val;
-            if (!deq) code[i] = __float_as_uint(fminf(fmaxf(val, P.out_qn), P.out_qp) + magic);
+            if (!deq) code[i] = __float_as_uint(fmaf(fminf(fmaxf(val, c_lo), c_hi), c_mul, magic));
         }
         if (deq) {
             if (vec_out) {
@@ -273,7 +275,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
 // all of them real columns; col_begin and col_end are multiples of 16.  Whole-warp call: the TMEM
 // load is a warp-wide instruction, so lanes whose row lies past M run the arithmetic too and only
 // their stores are masked.
-template <int KIND, int SMALL>
+template <int KIND, int SMALL, bool UNIT>
 __device__ __forceinline__ void epilogue_requant_blocks(const GemmParams& P, const EpiParams& ep, int buf,
                                                        uint32_t t_row, bool row_ok, long long orow, long long col0,
                                                        int col_begin, int col_end) {
@@ -285,27 +287,51 @@ __device__ __forceinline__ void epilogue_requant_blocks(const GemmParams& P, con
         uint32_t v[16];
         ptx::tmem_ld16(t_row + (uint32_t)col, v);
         ptx::tmem_ld_wait();
-        const float4* pa = reinterpret_cast<const float4*>(&ep.a[buf][col]);
-        const float4* pb = reinterpret_cast<const float4*>(&ep.b[buf][col]);
-        const float4* pq = reinterpret_cast<const float4*>(&ep.q[buf][col]);
+        const float* pa = &ep.a[buf][col];
+        const float* pb = &ep.b[buf][col];
+        const float* pq = &ep.q[buf][col];
         uint32_t code[16];
 #pragma unroll
-        for (int i4 = 0; i4 < 4; ++i4) {
-            const float4 a4 = pa[i4], b4 = pb[i4];
-            const float aa[4] = {a4.x, a4.y, a4.z, a4.w}, bb[4] = {b4.x, b4.y, b4.z, b4.w};
-            float qq[4] = {0.f, 0.f, 0.f, 0.f};
-            if (KIND == EK_REQUANT_GELU) {
-                const float4 q4 = pq[i4];
-                qq[0] = q4.x; qq[1] = q4.y; qq[2] = q4.z; qq[3] = q4.w;
+        for (int i2 = 0; i2 < 8; ++i2) {
+            // two columns per step: the fp32 arithmetic runs as packed pairs (bit-identical per element)
+            const float2 a2 = reinterpret_cast<const float2*>(pa)[i2], b2 = reinterpret_cast<const float2*>(pb)[i2];
+            float f0, f1;
+            if (SMALL == 0) {
+                f0 = (float)(int)v[2 * i2];
+                f1 = (float)(int)v[2 * i2 + 1];
+            } else {
+                // 1.5*2^23 + acc as float bits, then the packed subtraction of 1.5*2^23
+                const int s = SMALL == 1 ? P.shift : 0;
+                const f32x2 m = f2_pack(__int_as_float(0x4B400000 + ((int)v[2 * i2] >> s)),
+                                        __int_as_float(0x4B400000 + ((int)v[2 * i2 + 1] >> s)));
+                f2_unpack(f2_add(m, f2_dup(-12582912.0f)), f0, f1);
             }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int i = 4 * i4 + j;
-                const float f = SMALL == 2 ? small_int_to_float((int)v[i])
-                              : SMALL == 1 ? small_int_to_float((int)v[i] >> P.shift) : (float)(int)v[i];
-                float val = fmaf(f, aa[j], bb[j]);
-                if (KIND == EK_REQUANT_GELU) val = gelu_scaled(val, qq[j]);
-                code[i] = __float_as_uint(fminf(fmaxf(val, P.out_qn), P.out_qp) + magic);
+            const f32x2 y = f2_fma(f2_pack(f0, f1), f2_pack(a2.x, a2.y), f2_pack(b2.x, b2.y));
+            float y0, y1;
+            f2_unpack(y, y0, y1);
+            if (UNIT) {
+                // unsigned codes after GELU: the value arrives clamped to [0, 1] in units of Qp
+                const float2 q2 = reinterpret_cast<const float2*>(pq)[i2];
+                float e0, e1, w0, w1;
+                gelu_erfc_term2(y0, y1, e0, e1);
+                f2_unpack(f2_mul(y, f2_pack(q2.x, q2.y)), w0, w1);
+                const float u0 = __saturatef(fmaf(-fabsf(w0), e0, w0 + fabsf(w0)));
+                const float u1 = __saturatef(fmaf(-fabsf(w1), e1, w1 + fabsf(w1)));
+                float c0, c1;
+                f2_unpack(f2_fma(f2_pack(u0, u1), f2_dup(P.out_qp), f2_dup(magic)), c0, c1);
+                code[2 * i2] = __float_as_uint(c0);
+                code[2 * i2 + 1] = __float_as_uint(c1);
+            } else {
+                if (KIND == EK_REQUANT_GELU) {
+                    const float2 q2 = reinterpret_cast<const float2*>(pq)[i2];
+                    y0 = gelu_scaled(y0, q2.x);
+                    y1 = gelu_scaled(y1, q2.y);
+                }
+                float c0, c1;
+                f2_unpack(f2_add(f2_pack(fminf(fmaxf(y0, P.out_qn), P.out_qp), fminf(fmaxf(y1, P.out_qn), P.out_qp)),
+                                 f2_dup(magic)), c0, c1);
+                code[2 * i2] = __float_as_uint(c0);
+                code[2 * i2 + 1] = __float_as_uint(c1);
             }
         }
         // offset-binary packing as in epilogue_chunk: 16 codes = 2 * out_c bytes
@@ -410,8 +436,11 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiPara
     constexpr bool is_req = (KIND == EK_REQUANT || KIND == EK_REQUANT_GELU);
     if (is_req && (n_tile + 1) * P.bn <= P.N && (P.bn & 31) == 0 && (colbase & 15) == 0) {
         // every column of the tile is real: rolled 16-column blocks
-        epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL>(P, ep, buf, t_row, row_ok, orow,
-                                                                  colbase + (long long)n_tile * P.bn, c_begin * 32, c_end * 32);
+        const long long col0 = colbase + (long long)n_tile * P.bn;
+        if (KIND == EK_REQUANT_GELU && P.unit_out)
+            epilogue_requant_blocks<EK_REQUANT_GELU, SMALL, true>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+        else
+            epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL, false>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
         // row padding behind the last column of the matrix
         if (row_ok && P.col_off_inner == 0 && n_tile * P.bn + c_end * 32 >= P.N && c_end > c_begin) {
             for (long long off = ((long long)P.N * P.out_c) >> 3; off + 4 <= P.ld_out; off += 4)
@@ -584,7 +613,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (ok) ptx::mma_commit(ptx::smem_addr(&bars.acc_full[buf]));
             }
         }
-    } else if (warp >= WARP_UNPACK0 && P.epi_warps == EPI_WARPS) {
+    } else if (warp >= WARP_UNPACK0 + (P.epi_warps - EPI_WARPS)) {
         // --------------------------------- unpack ----------------------------------
         if (any_packed) {
             const int tid_u = threadIdx.x - WARP_UNPACK0 * 32;
@@ -628,11 +657,42 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         // -------------------------------- epilogue ---------------------------------
         const int q4 = warp & 3;   // TMEM lane quarter (fixed by the warp's index in the CTA)
-        const int slice = warp < EPI_WARPS ? warp >> 2 : 2;   // which share of the tile's columns
+        const int slice = warp < EPI_WARPS ? warp >> 2 : 2 + ((warp - WARP_UNPACK0) >> 2);   // which share of the tile's columns
         const int ewarp = warp < EPI_WARPS ? warp : warp - (WARP_UNPACK0 - EPI_WARPS);   // 0 .. epi_warps-1
         const int tid_e = ewarp * 32 + lane;
         // small accumulators are shifted back as integers; otherwise 2^-shift rides on the multiplier
         const float down = P.small_acc == 1 ? 1.0f : __int_as_float((127 - P.shift) << 23);
+        // Per-column parameters of a tile (multiplier, bias, GELU output factor), column c of the tile.
+        auto fetch_params = [&](int tile, int c, float& a, float& b, float& q) {
+            int m_tile, n_tile, inner, outer;
+            tile_coords(P, tile, m_tile, n_tile, inner, outer);
+            const int n = n_tile * P.bn + c;
+            a = 0.0f; b = 0.0f; q = 0.0f;
+            if (n < P.N) {
+                const long long cidx = (long long)inner * P.col_off_inner + n;
+                if (KIND == EK_REQUANT) {
+                    a = __ldg(P.col_a + cidx);
+                } else {
+                    a = P.col_a ? __fmul_rn(P.x_step, __ldg(P.col_a + cidx)) : P.x_step;
+                    if (KIND == EK_REQUANT_GELU) {                                  // folds GELU's 1/2 (and 1/Qp)
+                        q = 0.5f * __ldg(P.inv_s + cidx);
+                        if (P.unit_out) q = __fdiv_rn(q, P.out_qp);
+                    }
+                }
+                b = P.col_b ? __ldg(P.col_b + cidx) : 0.0f;
+                a *= down;
+            }
+        };
+        // The parameters of tile i+1 are fetched while the warps wait for tile i's accumulators and are
+        // stored to the other half of epi_params before tile i is processed, so no tile waits for them.
+        const bool my_col = KIND != EK_ACC && tid_e < P.bn;          // bn <= 256 <= epilogue threads
+        if (my_col && (int)blockIdx.x < P.total_tiles) {
+            float a, b, q;
+            fetch_params(blockIdx.x, tid_e, a, b, q);
+            epi_params.a[0][tid_e] = a;
+            epi_params.b[0][tid_e] = b;
+            epi_params.q[0][tid_e] = q;
+        }
         int tl = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++tl) {
@@ -640,32 +700,21 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tile_coords(P, tile, m_tile, n_tile, inner, outer);
             const int buf = tl & 1;
             const long long colbase = (long long)inner * P.col_off_inner;
-            // stage this tile's per-column parameters while its MMAs are still running
-            if (KIND != EK_ACC) {
-                for (int c = tid_e; c < P.bn; c += P.epi_warps * 32) {
-                    const int n = n_tile * P.bn + c;
-                    float a = 0.0f, b = 0.0f, q = 0.0f;
-                    if (n < P.N) {
-                        const long long cidx = colbase + n;
-                        if (KIND == EK_REQUANT) {
-                            a = __ldg(P.col_a + cidx);
-                        } else {
-                            a = P.col_a ? __fmul_rn(P.x_step, __ldg(P.col_a + cidx)) : P.x_step;
-                            if (KIND == EK_REQUANT_GELU) q = 0.5f * __ldg(P.inv_s + cidx);   // folds GELU's 1/2
-                        }
-                        b = P.col_b ? __ldg(P.col_b + cidx) : 0.0f;
-                        a *= down;
-                    }
-                    epi_params.a[buf][c] = a;
-                    epi_params.b[buf][c] = b;
-                    epi_params.q[buf][c] = q;
-                }
-            }
+            const int next_tile = tile + (int)gridDim.x;
+            const bool fetch_next = my_col && next_tile < P.total_tiles;
+            float na = 0.0f, nb = 0.0f, nq = 0.0f;
+            if (fetch_next) fetch_params(next_tile, tid_e, na, nb, nq);
             const uint32_t acc_ph = (uint32_t)(tl >> 1) & 1u;
             bool w = KIND == EK_ACC || epi_barrier(ptx::smem_addr(&bars.epi_sync), (uint32_t)tl & 1u, abort_ptr);
             w = w && mbar_wait(ptx::smem_addr(&bars.acc_full[buf]), acc_ph, abort_ptr);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
             ptx::tc_fence_after();
+            if (fetch_next) {
+                // every epilogue warp has arrived at this tile's barrier, so none still reads the other half
+                epi_params.a[buf ^ 1][tid_e] = na;
+                epi_params.b[buf ^ 1][tid_e] = nb;
+                epi_params.q[buf ^ 1][tid_e] = nq;
+            }
             const int row_in_problem = m_tile * BM + q4 * 32 + lane;
             const bool row_ok = row_in_problem < P.M;
             const long long orow = (long long)outer * P.row_off_outer + (long long)inner * P.row_off_inner + row_in_problem;
@@ -891,6 +940,7 @@ static int fill_epilogue(GemmParams& P, const vitint_epilogue* epi, float x_step
                 if (!epi->inv_out_step || !(x_step > 0.0f && x_step < INFINITY)) return VITINT_ERR_INVALID_ARG;
                 P.col_a = w_step; P.col_b = bias; P.inv_s = epi->inv_out_step;
                 P.kind = EK_REQUANT_GELU;
+                P.unit_out = qn == 0 ? 1 : 0;
             }
             break;
         }

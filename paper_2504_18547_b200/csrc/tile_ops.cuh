@@ -14,15 +14,15 @@ constexpr long long WAIT_LIMIT_CYCLES = 2000000000ll;   // about one second
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    for (uint32_t spin = 1;; ++spin) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((spin & 127u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-                *abort_flag = 1;
-                atomicExch(&g_device_status, (int)VITINT_ERR_TIMEOUT);
-                return false;
-            }
+    for (;;) {
+        // sleeps in hardware until the phase completes or ~50 us pass, so a waiting warp leaves the
+        // issue slots to the warps that have work
+        if (ptx::mbar_try_wait_hint(bar, parity, 50000u)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort_flag = 1;
+            atomicExch(&g_device_status, (int)VITINT_ERR_TIMEOUT);
+            return false;
         }
     }
 }
