@@ -185,7 +185,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         const int sh_idx = 2 * (8 - C) - 2;                         // scaled score -> byte offset 4*S
         const int chunks = P.kv_rows / 32;
         const int tab_half = 4 * P.smax;
-        const Divisor dv = make_divisor(P.p_step);
+        const double inv_p_step = 1.0 / (double)P.p_step;
         bool ok = true;
         int n = 0;
         for (int item = item0; ok && item < P.total_items; item += item_stride, ++n) {
@@ -224,9 +224,12 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 if (ch < full_chunks) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        const float e = *reinterpret_cast<const float*>(tab_mid + ((int)v[i] >> sh_idx));
-                        z += (double)e;
-                        v[i] = __float_as_uint(e);
+                        // every table entry is a positive normal float (exp of a bounded argument), so its
+                        // double is formed from the bits with two integer operations instead of a conversion
+                        // (the conversion unit runs at a quarter of the fp64 adder's rate)
+                        const uint32_t eb = *reinterpret_cast<const uint32_t*>(tab_mid + ((int)v[i] >> sh_idx));
+                        z += __hiloint2double((int)((eb >> 3) + 0x38000000u), (int)(eb << 29));
+                        v[i] = eb;
                     }
                 } else {
                     // last, partial chunk: columns past the last token hold no score -> no lookup, e = 0
@@ -234,10 +237,10 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     for (int i = 0; i < 32; ++i) {
                         const bool valid = ch * 32 + i < T;
                         const int off = valid ? ((int)v[i] >> sh_idx) : 0;
-                        float e = *reinterpret_cast<const float*>(tab_mid + max(-tab_half, min(tab_half, off)));
-                        if (!valid) e = 0.0f;
-                        z += (double)e;
-                        v[i] = __float_as_uint(e);
+                        uint32_t eb = *reinterpret_cast<const uint32_t*>(tab_mid + max(-tab_half, min(tab_half, off)));
+                        if (!valid) eb = 0u;
+                        z += __hiloint2double(valid ? (int)((eb >> 3) + 0x38000000u) : 0, (int)(eb << 29));
+                        v[i] = eb;
                     }
                 }
                 ptx::tmem_st32(t_row + (uint32_t)(ch * 32), v);
@@ -249,12 +252,15 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             w = mbar_wait(ptx::smem_addr(&B.z_sync), ph, abort_ptr);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
             z = zx[row] + zx[128 + row];
-            const double rz = warp_live ? 1.0 / z : 0.0;
+            // r = 1 / (Z * s_P) as a two-float number: e * r then carries the quantizer argument p / s_P to
+            // about half an ulp, i.e. it is the exact-division result for a probability that differs from
+            // RN(e / Z) by less than one ulp
+            const double rz = warp_live ? inv_p_step / z : 0.0;
             const float rzh = (float)rz;
             const float rzl = (float)(rz - (double)rzh);
             uint8_t* const prow = ggen + P.off_p + row * 128;
             const int sw = row & 7;
-            // pass 2: p_j = RN(e_j / Z), code = min(rint(RN(p_j / s_P)), Qp) (p >= 0: no lower clamp)
+            // pass 2: code = min(rint(e_j / (Z s_P)), Qp) (p >= 0: no lower clamp)
             for (int ch = hf; warp_live && ch < chunks; ch += 2) {
                 uint32_t v[32];
                 ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
@@ -266,9 +272,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const float e = __uint_as_float(v[4 * i4 + j]);
-                        const float p = fmaf(e, rzh, e * rzl);
-                        // straight-line quotient (host selects this kernel only for such a step, see below)
-                        cb[j] = __float_as_uint(fminf(div_rn_exact(p, dv), P.p_qp) + 12582912.0f);   // code in the low byte
+                        cb[j] = __float_as_uint(fminf(fmaf(e, rzh, e * rzl), P.p_qp) + 12582912.0f);   // code in the low byte
                     }
                     wd[i4] = __byte_perm(__byte_perm(cb[0], cb[1], 0x4040), __byte_perm(cb[2], cb[3], 0x4040), 0x5410);
                 }
@@ -369,11 +373,6 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     for (float s : steps) if (!(s > 0.0f && s < INFINITY)) return VITINT_ERR_INVALID_ARG;
     if (!valid_bits(p_bits)) return VITINT_ERR_INVALID_ARG;
     if (qkv->bits == 8 || qkv->container_bits == 8 || tokens > 256 || batch > 65535) return VITINT_ERR_UNSUPPORTED;
-    {   // the kernel divides by p_step with the two-FMA correction, exact unless the significand is all ones
-        uint32_t bits;
-        memcpy(&bits, &p_step, sizeof(bits));
-        if ((bits & 0x007FFFFFu) == 0x007FFFFFu) return VITINT_ERR_UNSUPPORTED;
-    }
     const int c = container_bits(qkv->bits);
     const int m = 1 << (c - 1);
     const int smax = 64 * m * m;
