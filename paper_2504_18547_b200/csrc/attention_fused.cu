@@ -212,7 +212,8 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             ptx::tc_fence_after();
             // pass 1: e_j = EXP[S_j] (an integer score is bounded by the code ranges, so the byte offset
             // 4*S always lies inside the table), row sum in fp64, e_j parked in TMEM over S_j
-            double z = 0.0;
+            // four interleaved partial sums: a single fp64 accumulator would chain 32 dependent additions per chunk
+            double zp[4] = {0.0, 0.0, 0.0, 0.0};
             const int full_chunks = T >> 5;
             // a warp whose 32 query rows all lie past the last token has nothing to compute: its P rows
             // only feed accumulator rows that are never stored (whatever int8 they hold)
@@ -228,7 +229,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         // double is formed from the bits with two integer operations instead of a conversion
                         // (the conversion unit runs at a quarter of the fp64 adder's rate)
                         const uint32_t eb = *reinterpret_cast<const uint32_t*>(tab_mid + ((int)v[i] >> sh_idx));
-                        z += __hiloint2double((int)((eb >> 3) + 0x38000000u), (int)(eb << 29));
+                        zp[i & 3] += __hiloint2double((int)((eb >> 3) + 0x38000000u), (int)(eb << 29));
                         v[i] = eb;
                     }
                 } else {
@@ -239,7 +240,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         const int off = valid ? ((int)v[i] >> sh_idx) : 0;
                         uint32_t eb = *reinterpret_cast<const uint32_t*>(tab_mid + max(-tab_half, min(tab_half, off)));
                         if (!valid) eb = 0u;
-                        z += __hiloint2double(valid ? (int)((eb >> 3) + 0x38000000u) : 0, (int)(eb << 29));
+                        zp[i & 3] += __hiloint2double(valid ? (int)((eb >> 3) + 0x38000000u) : 0, (int)(eb << 29));
                         v[i] = eb;
                     }
                 }
@@ -247,6 +248,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             }
             ptx::tmem_st_wait();
             // the row's two threads add their partial sums (every thread takes part in the barrier)
+            double z = (zp[0] + zp[1]) + (zp[2] + zp[3]);
             zx[hf * 128 + row] = z;
             ptx::mbar_arrive(ptx::smem_addr(&B.z_sync));
             w = mbar_wait(ptx::smem_addr(&B.z_sync), ph, abort_ptr);
