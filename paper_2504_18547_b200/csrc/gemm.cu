@@ -363,12 +363,29 @@ __device__ __forceinline__ void epilogue_requant_blocks(const GemmParams& P, con
 }
 
 constexpr int STAGE_LD = 36;                                  // floats per staged row: 144 bytes keeps 16-byte accesses conflict-free
-constexpr int STAGE_BYTES = 32 * STAGE_LD * 4;                // one 32 x 32 fp32 block per epilogue warp
+constexpr int STAGE_FLOATS = 32 * STAGE_LD;                   // one 32 x 32 fp32 block
+constexpr int STAGE_BYTES = 2 * STAGE_FLOATS * 4;             // two blocks per epilogue warp: the residual of the next
+                                                              // chunk lands in one while the other is worked on
+
+// Starts the asynchronous copy of one 32 x 32 block of the residual into a staging block (coalesced:
+// each instruction covers four rows of 128 bytes) and closes it as one copy group of the calling thread.
+__device__ __forceinline__ void residual_prefetch(const GemmParams& P, float* block, int lane, long long orow0,
+                                                  int rows_valid, long long col) {
+    const int cr = lane >> 3, cc = (lane & 7) * 4;
+    const float* r0 = P.residual + orow0 * P.ld_res + col + cc;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = cr + 4 * i;
+        if (r < rows_valid) ptx::cp_async16(ptx::smem_addr(block + r * STAGE_LD + cc), r0 + (long long)r * P.ld_res);
+    }
+    ptx::cp_async_commit();
+}
 
 // fp32 epilogue of a 32 x 32 block through a shared-memory transposition, so that every global
 // access of the warp covers whole 128-byte lines: the TMEM layout gives each thread one ROW of the
 // block, while coalesced loads / stores want each instruction to cover four rows of 128 bytes.
-//   residual: coalesced float4 loads -> stage -> each thread reads its own row;
+//   residual: already copied into `stage` by residual_prefetch (the caller has waited for the copy
+//             group and synchronised the warp) -> each thread reads its own row;
 //   result  : each thread writes its own row -> stage -> coalesced float4 stores.
 // Whole-warp call (rows past M take part and are masked at the global accesses).
 template <int KIND, int SMALL, bool HAS_RES>
@@ -377,19 +394,6 @@ __device__ __forceinline__ void epilogue_chunk_staged(const GemmParams& P, const
                                                      int rows_valid, long long colbase, int n0) {
     const int cr = lane >> 3, cc = (lane & 7) * 4;              // cooperative phase: row cr + 4*i, columns cc..cc+3
     float* const my_row = stage + lane * STAGE_LD;
-    if (HAS_RES) {
-        const float* r0 = P.residual + orow0 * P.ld_res + colbase + n0 + cc;
-        float4 t[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int r = cr + 4 * i;
-            t[i] = (r < rows_valid) ? __ldg(reinterpret_cast<const float4*>(r0 + (long long)r * P.ld_res))
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) *reinterpret_cast<float4*>(stage + (cr + 4 * i) * STAGE_LD + cc) = t[i];
-        __syncwarp();
-    }
     float4 y[8];
 #pragma unroll
     for (int i4 = 0; i4 < 8; ++i4) {
@@ -425,14 +429,35 @@ __device__ __forceinline__ void epilogue_chunk_staged(const GemmParams& P, const
     __syncwarp();                                               // the buffer is free for the next chunk
 }
 
+// The warps of a lane quarter split the tile's 32-column chunks into contiguous shares.
+__device__ __forceinline__ void chunk_share(const GemmParams& P, int slice, int& c_begin, int& c_end) {
+    const int n_slices = P.epi_warps >> 2;
+    const int n_chunks = (P.bn + 31) / 32, base = n_chunks / n_slices, rem = n_chunks % n_slices;
+    c_begin = slice * base + (slice < rem ? slice : rem);
+    c_end = c_begin + base + (slice < rem ? 1 : 0);
+}
+
+// Residual of the warp's first chunk of a tile, requested before the warp waits for the tile's
+// accumulators.  Returns whether a copy group was opened (the chunk takes the staged path).
+template <int KIND>
+__device__ __forceinline__ bool epilogue_prefetch_first(const GemmParams& P, long long colbase, int n_tile, int slice,
+                                                        float* stage, int lane, long long orow0, int rows_valid) {
+    constexpr bool is_deq = (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU);
+    if (!is_deq || stage == nullptr || P.residual == nullptr) return false;
+    int c_begin, c_end;
+    chunk_share(P, slice, c_begin, c_end);
+    const int n0 = n_tile * P.bn + c_begin * 32;
+    if (c_begin >= c_end || n0 + 32 > P.N) return false;
+    residual_prefetch(P, stage, lane, orow0, rows_valid, colbase + n0);
+    return true;
+}
+
 template <int KIND, int SMALL>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiParams& ep, int buf, uint32_t t_row,
                                               bool row_ok, long long orow, long long colbase, int n_tile, int slice,
-                                              float* stage, int lane, int rows_valid) {
-    // the warps of a lane quarter split the tile's 32-column chunks into contiguous shares
-    const int n_slices = P.epi_warps >> 2;
-    const int n_chunks = (P.bn + 31) / 32, base = n_chunks / n_slices, rem = n_chunks % n_slices;
-    const int c_begin = slice * base + (slice < rem ? slice : rem), c_end = c_begin + base + (slice < rem ? 1 : 0);
+                                              float* stage, int lane, int rows_valid, bool first_prefetched) {
+    int c_begin, c_end;
+    chunk_share(P, slice, c_begin, c_end);
     constexpr bool is_req = (KIND == EK_REQUANT || KIND == EK_REQUANT_GELU);
     if (is_req && (n_tile + 1) * P.bn <= P.N && (P.bn & 31) == 0 && (colbase & 15) == 0) {
         // every column of the tile is real: rolled 16-column blocks
@@ -449,21 +474,37 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiPara
         __syncwarp();
         return;
     }
+    bool have_res = first_prefetched;                           // the current chunk's residual copy is already open
     for (int chunk = c_begin; chunk < c_end; ++chunk) {
         const int n0 = n_tile * P.bn + chunk * 32;
         if (n0 >= P.N) break;
         uint32_t v[32];
         ptx::tmem_ld32(t_row + (uint32_t)(chunk * 32), v);
-        ptx::tmem_ld_wait();
         constexpr bool is_deq = (KIND == EK_DEQUANT || KIND == EK_DEQUANT_GELU);
-        if (is_deq && stage != nullptr && n0 + 32 <= P.N) {
+        const bool staged_here = is_deq && stage != nullptr && n0 + 32 <= P.N;
+        float* const block = stage + ((chunk - c_begin) & 1) * STAGE_FLOATS;
+        const long long orow0 = orow - lane;
+        if (staged_here && P.residual != nullptr) {
+            // this chunk's residual block is on its way (or is requested now); the next chunk's is requested
+            // into the other block before this one is awaited, so its latency hides behind the arithmetic
+            if (!have_res) residual_prefetch(P, block, lane, orow0, rows_valid, colbase + n0);
+            have_res = chunk + 1 < c_end && n0 + 64 <= P.N;
+            if (have_res) {
+                residual_prefetch(P, stage + ((chunk + 1 - c_begin) & 1) * STAGE_FLOATS, lane, orow0, rows_valid, colbase + n0 + 32);
+                ptx::cp_async_wait<1>();
+            } else {
+                ptx::cp_async_wait<0>();
+            }
+            __syncwarp();                                       // every lane's copies have landed
+        }
+        ptx::tmem_ld_wait();
+        if (staged_here) {
             // full 32-column chunk of an fp32 output: coalesced path (stage is only set when the host has
             // checked 16-byte alignment of the output, the residual and their leading dimensions)
             const float* pa = &ep.a[buf][chunk * 32];
             const float* pb = &ep.b[buf][chunk * 32];
-            const long long orow0 = orow - lane;
-            if (P.residual != nullptr) epilogue_chunk_staged<is_deq ? KIND : EK_DEQUANT, SMALL, true>(P, v, pa, pb, stage, lane, orow0, rows_valid, colbase, n0);
-            else epilogue_chunk_staged<is_deq ? KIND : EK_DEQUANT, SMALL, false>(P, v, pa, pb, stage, lane, orow0, rows_valid, colbase, n0);
+            if (P.residual != nullptr) epilogue_chunk_staged<is_deq ? KIND : EK_DEQUANT, SMALL, true>(P, v, pa, pb, block, lane, orow0, rows_valid, colbase, n0);
+            else epilogue_chunk_staged<is_deq ? KIND : EK_DEQUANT, SMALL, false>(P, v, pa, pb, block, lane, orow0, rows_valid, colbase, n0);
         } else if (row_ok) {
             const float* pa = &ep.a[buf][chunk * 32];
             const float* pb = &ep.b[buf][chunk * 32];
@@ -704,6 +745,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool fetch_next = my_col && next_tile < P.total_tiles;
             float na = 0.0f, nb = 0.0f, nq = 0.0f;
             if (fetch_next) fetch_params(next_tile, tid_e, na, nb, nq);
+            const int row0_in_problem = m_tile * BM + q4 * 32;
+            int rows_valid = P.M - row0_in_problem;
+            rows_valid = rows_valid < 0 ? 0 : (rows_valid > 32 ? 32 : rows_valid);
+            const long long orow0 = (long long)outer * P.row_off_outer + (long long)inner * P.row_off_inner + row0_in_problem;
+            float* const stage = P.stage_off ? reinterpret_cast<float*>(smem_gen + P.stage_off + (size_t)ewarp * STAGE_BYTES) : nullptr;
+            const bool first_prefetched = epilogue_prefetch_first<KIND>(P, colbase, n_tile, slice, stage, lane, orow0, rows_valid);
             const uint32_t acc_ph = (uint32_t)(tl >> 1) & 1u;
             bool w = KIND == EK_ACC || epi_barrier(ptx::smem_addr(&bars.epi_sync), (uint32_t)tl & 1u, abort_ptr);
             w = w && mbar_wait(ptx::smem_addr(&bars.acc_full[buf]), acc_ph, abort_ptr);
@@ -715,20 +762,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 epi_params.b[buf ^ 1][tid_e] = nb;
                 epi_params.q[buf ^ 1][tid_e] = nq;
             }
-            const int row_in_problem = m_tile * BM + q4 * 32 + lane;
-            const bool row_ok = row_in_problem < P.M;
-            const long long orow = (long long)outer * P.row_off_outer + (long long)inner * P.row_off_inner + row_in_problem;
+            const bool row_ok = row0_in_problem + lane < P.M;
+            const long long orow = orow0 + lane;
             const uint32_t t_row = tmem_base + (uint32_t)buf * acc_stride + ((uint32_t)(q4 * 32) << 16);
-            int rows_valid = P.M - (m_tile * BM + q4 * 32);
-            rows_valid = rows_valid < 0 ? 0 : (rows_valid > 32 ? 32 : rows_valid);
-            float* const stage = P.stage_off ? reinterpret_cast<float*>(smem_gen + P.stage_off + (size_t)ewarp * STAGE_BYTES) : nullptr;
-            if (P.small_acc == 2) epilogue_tile<KIND, 2>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid);
-            else if (P.small_acc == 1) epilogue_tile<KIND, 1>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid);
-            else epilogue_tile<KIND, 0>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid);
+            if (P.small_acc == 2) epilogue_tile<KIND, 2>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid, first_prefetched);
+            else if (P.small_acc == 1) epilogue_tile<KIND, 1>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid, first_prefetched);
+            else epilogue_tile<KIND, 0>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid, first_prefetched);
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&bars.acc_empty[buf]));
         }
+        ptx::cp_async_wait<0>();   // a residual copy requested before a wait that gave up has landed before the CTA exits
     }
 
     // ---------------------------------- teardown -----------------------------------
@@ -833,7 +877,8 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     bool staged = (P.kind == EK_DEQUANT || P.kind == EK_DEQUANT_GELU) && n_inner == 1 && n_outer == 1 &&
                   aligned16(P.out) && P.ld_out % 4 == 0 &&
                   (!P.residual || (aligned16(P.residual) && P.ld_res % 4 == 0));
-    P.epi_warps = (P.a_direct && P.b_direct) ? MAX_EPI_WARPS : EPI_WARPS;
+    // the fp32 kinds keep 8 epilogue warps: their two staging blocks per warp come out of the ring space
+    P.epi_warps = (P.a_direct && P.b_direct && !staged) ? MAX_EPI_WARPS : EPI_WARPS;
     const uint32_t stage_total = staged ? (uint32_t)(P.epi_warps * STAGE_BYTES) : 0u;
     const uint32_t ring_budget = SMEM_TILE_BUDGET + 12u * 1024u - stage_total;   // staging comes out of the ring space
     // The packed ring hides the global-memory latency of the TMA loads; the int8 ring only
