@@ -58,6 +58,8 @@ struct AttnBars {
 
 // exp(fl32(s * c)) for every integer score, correctly rounded to fp32 (fp64 exp, one rounding).
 __global__ void exp_table_kernel(float* table, int smax, float c) {
+    grid_dependency_wait();        // an earlier kernel may still read the table
+    grid_dependency_launch();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i > 2 * smax) return;
     const float t = __fmul_rn((float)(i - smax), c);
@@ -102,6 +104,8 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         ptx::tmem_alloc(ptx::smem_addr(&tmem_base_slot), 512);
         ptx::tmem_relinquish();
     }
+    grid_dependency_wait();        // the table and the codes come from earlier kernels of the stream
+    grid_dependency_launch();
     // the exp table: global -> shared, once per CTA
     {
         float* tab = reinterpret_cast<float*>(smem_gen + P.off_table);
@@ -443,7 +447,7 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return VITINT_ERR_CUDA;
     }
-    exp_table_kernel<<<(2 * smax + 1 + 255) / 256, 256, 0, st>>>((float*)workspace, smax, cs);
+    launch_kernel(exp_table_kernel, dim3((2 * smax + 1 + 255) / 256), dim3(256), 0, st, (float*)workspace, smax, cs);
     if (cudaGetLastError() != cudaSuccess) return VITINT_ERR_CUDA;
     int grid = sm_count();
     const int want = (P.total_items + AT_GROUPS - 1) / AT_GROUPS;
@@ -455,14 +459,14 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
                 return VITINT_ERR_CUDA;
             attr4 = true;
         }
-        attention_fused_kernel<4><<<grid, AT_THREADS, smem, st>>>(map_q, map_kv, P);
+        launch_kernel(attention_fused_kernel<4>, dim3(grid), dim3(AT_THREADS), smem, st, map_q, map_kv, P);
     } else {
         if (!attr2) {
             if (cudaFuncSetAttribute(attention_fused_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess)
                 return VITINT_ERR_CUDA;
             attr2 = true;
         }
-        attention_fused_kernel<2><<<grid, AT_THREADS, smem, st>>>(map_q, map_kv, P);
+        launch_kernel(attention_fused_kernel<2>, dim3(grid), dim3(AT_THREADS), smem, st, map_q, map_kv, P);
     }
     return cuda_status(cudaGetLastError());
 }

@@ -31,6 +31,31 @@ int check_codes(const vitint_codes* c);
 
 int cuda_status(cudaError_t e);
 
+// ---- programmatic dependent launch ---------------------------------------------------------
+// Every kernel of the library is launched with programmatic stream serialization: its CTAs may
+// be scheduled while the previous kernel of the stream is still draining, run their set-up
+// (barriers, tensor memory, descriptor prefetch) and then block in grid_dependency_wait() until
+// the previous kernel has completed and its writes are visible.  Nothing that another kernel
+// may have produced is read, and nothing is written, before that wait.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------------------
 // device helpers shared by the element-wise kernels
 // ---------------------------------------------------------------------------

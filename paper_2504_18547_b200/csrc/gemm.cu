@@ -569,6 +569,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t acc_stride = P.tmem_cols >> 1;
+    grid_dependency_wait();        // operands, parameters and the residual may come from the previous kernel
+    grid_dependency_launch();
 
     if (warp == WARP_TMA) {
         // ------------------------------ TMA producer -------------------------------
@@ -931,7 +933,7 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
                 return VITINT_ERR_CUDA;                                                                            \
             attr_set[KIND] = true;                                                                                 \
         }                                                                                                          \
-        gemm_i8_kernel<KIND><<<grid, NUM_THREADS, smem, st>>>(map_a, map_b, P);                                    \
+        launch_kernel(gemm_i8_kernel<KIND>, dim3(grid), dim3(NUM_THREADS), smem, st, map_a, map_b, P);            \
         break;
     switch (P.kind) {
         VITINT_LAUNCH(EK_ACC)

@@ -12,6 +12,8 @@ __global__ void __launch_bounds__(256)
 quantize_pack_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, int64_t ldx, float step,
                      const float* __restrict__ row_steps, uint8_t* __restrict__ out, int64_t pitch,
                      int words_per_row, float qn, float qp, int vec_ok) {
+    grid_dependency_wait();        // inputs may come from the previous kernel of the stream
+    grid_dependency_launch();
     constexpr int E = 32 / C;  // codes per word
     const int w = blockIdx.x * blockDim.x + threadIdx.x;
     if (w >= words_per_row) return;
@@ -55,6 +57,8 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
                           const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float step,
                           uint8_t* __restrict__ out, int64_t pitch, float* __restrict__ y_out, int64_t ld_y,
                           float qn, float qp) {
+    grid_dependency_wait();        // inputs may come from the previous kernel of the stream
+    grid_dependency_launch();
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -152,6 +156,8 @@ template <int C>
 __global__ void __launch_bounds__(256)
 widen_kernel(const uint8_t* __restrict__ in, int64_t in_pitch, uint8_t* __restrict__ out, int64_t out_pitch,
              int64_t rows, int words_in, int is_signed) {
+    grid_dependency_wait();        // inputs may come from the previous kernel of the stream
+    grid_dependency_launch();
     constexpr int E = 32 / C;
     const int w = blockIdx.x * blockDim.x + threadIdx.x;
     for (int64_t row = blockIdx.y; row < rows; row += gridDim.y) {
@@ -181,7 +187,7 @@ static int launch_ln(int nv, const float* x, int64_t rows, int cols, int64_t ldx
     dim3 grid((unsigned)((rows + warps - 1) / warps)), block(32 * warps);
 #define VITINT_LN_CASE(NVV)                                                                                     \
     case NVV:                                                                                                   \
-        layernorm_quantize_kernel<C, NVV><<<grid, block, 0, st>>>(x, rows, cols, ldx, gamma, beta, eps, step,   \
+        launch_kernel(layernorm_quantize_kernel<C, NVV>, dim3(grid), dim3(block), 0, st, x, rows, cols, ldx, gamma, beta, eps, step,   \
                                                                   out, pitch, y, ld_y, qn, qp);                 \
         break;
     switch (nv) {
@@ -218,13 +224,13 @@ extern "C" int vitint_quantize(const float* x, int64_t rows, int64_t cols, int64
     cudaStream_t st = (cudaStream_t)stream;
     uint8_t* o = (uint8_t*)out->data;
     if (c == 2)
-        quantize_pack_kernel<2><<<grid, block, 0, st>>>(x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
+        launch_kernel(quantize_pack_kernel<2>, dim3(grid), dim3(block), 0, st, x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
                                                         words, (float)qn, (float)qp, vec_ok);
     else if (c == 4)
-        quantize_pack_kernel<4><<<grid, block, 0, st>>>(x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
+        launch_kernel(quantize_pack_kernel<4>, dim3(grid), dim3(block), 0, st, x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
                                                         words, (float)qn, (float)qp, vec_ok);
     else
-        quantize_pack_kernel<8><<<grid, block, 0, st>>>(x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
+        launch_kernel(quantize_pack_kernel<8>, dim3(grid), dim3(block), 0, st, x, rows, cols, ldx, step, row_steps, o, out->pitch_bytes,
                                                         words, (float)qn, (float)qp, vec_ok);
     return cuda_status(cudaGetLastError());
 }
@@ -243,10 +249,10 @@ extern "C" int vitint_widen(const vitint_codes* in, const vitint_codes* out, voi
     dim3 block(128), grid((threads + 127) / 128, (unsigned)(in->rows < 32768 ? in->rows : 32768));
     cudaStream_t st = (cudaStream_t)stream;
     if (c == 2)
-        widen_kernel<2><<<grid, block, 0, st>>>((const uint8_t*)in->data, in->pitch_bytes, (uint8_t*)out->data,
+        launch_kernel(widen_kernel<2>, dim3(grid), dim3(block), 0, st, (const uint8_t*)in->data, in->pitch_bytes, (uint8_t*)out->data,
                                                 out->pitch_bytes, in->rows, words_in, in->is_signed);
     else
-        widen_kernel<4><<<grid, block, 0, st>>>((const uint8_t*)in->data, in->pitch_bytes, (uint8_t*)out->data,
+        launch_kernel(widen_kernel<4>, dim3(grid), dim3(block), 0, st, (const uint8_t*)in->data, in->pitch_bytes, (uint8_t*)out->data,
                                                 out->pitch_bytes, in->rows, words_in, in->is_signed);
     return cuda_status(cudaGetLastError());
 }

@@ -41,6 +41,8 @@ __global__ void __launch_bounds__(256)
 softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, int64_t ld_s, float c, float p_step,
                         uint8_t* __restrict__ out, int64_t pitch, float* __restrict__ p_out, int64_t ld_p, float qp,
                         int vec_in, int vec_p) {
+    grid_dependency_wait();        // inputs may come from the previous kernel of the stream
+    grid_dependency_launch();
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -135,10 +137,10 @@ static int launch_softmax(int nch, const int32_t* s, int64_t rows, int cols, int
     const int warps = 8;
     dim3 grid((unsigned)((rows + warps - 1) / warps)), block(32 * warps);
     switch (nch) {
-        case 1: softmax_quantize_kernel<C, 1><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
-        case 2: softmax_quantize_kernel<C, 2><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
-        case 3: softmax_quantize_kernel<C, 3><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
-        case 4: softmax_quantize_kernel<C, 4><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
+        case 1: launch_kernel(softmax_quantize_kernel<C, 1>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
+        case 2: launch_kernel(softmax_quantize_kernel<C, 2>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
+        case 3: launch_kernel(softmax_quantize_kernel<C, 3>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
+        case 4: launch_kernel(softmax_quantize_kernel<C, 4>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
         default: return VITINT_ERR_UNSUPPORTED;
     }
     return cuda_status(cudaGetLastError());
@@ -155,6 +157,8 @@ template <int C, int NCH>
 __global__ void __launch_bounds__(256)
 softmax_shift_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, int64_t ld_s, float c2,
                               float p_step, uint8_t* __restrict__ out, int64_t pitch, int code_bits, int vec_in) {
+    grid_dependency_wait();        // inputs may come from the previous kernel of the stream
+    grid_dependency_launch();
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -253,10 +257,10 @@ static int launch_softmax_shift(int nch, const int32_t* s, int64_t rows, int col
     const int warps = 8;
     dim3 grid((unsigned)((rows + warps - 1) / warps)), block(32 * warps);
     switch (nch) {
-        case 1: softmax_shift_quantize_kernel<C, 1><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
-        case 2: softmax_shift_quantize_kernel<C, 2><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
-        case 3: softmax_shift_quantize_kernel<C, 3><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
-        case 4: softmax_shift_quantize_kernel<C, 4><<<grid, block, 0, st>>>(s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
+        case 1: launch_kernel(softmax_shift_quantize_kernel<C, 1>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
+        case 2: launch_kernel(softmax_shift_quantize_kernel<C, 2>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
+        case 3: launch_kernel(softmax_shift_quantize_kernel<C, 3>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
+        case 4: launch_kernel(softmax_shift_quantize_kernel<C, 4>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c2, p_step, out, pitch, code_bits, vec_in); break;
         default: return VITINT_ERR_UNSUPPORTED;
     }
     return cuda_status(cudaGetLastError());
