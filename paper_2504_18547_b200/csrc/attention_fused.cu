@@ -35,7 +35,8 @@ constexpr int AT_THREADS = (AT_GROUPS * AT_COMPUTE_WARPS + AT_GROUPS) * 32;   //
 
 struct AttnParams {
     int batch, heads, tokens, q_tiles, total_items;
-    int c;                       // container bits of Q, K, V (2 or 4)
+    int c;                       // container bits of Q, K, V (2 or 4: packed, unpacked in the kernel; 8: one code per byte,
+                                 // the TMA copy is the tensor-core operand)
     int n_k;                     // MMA N of Q K^T: tokens rounded up to 16
     int kv_rows;                 // tokens rounded up to 32: K extent of P V, rows of the V tile
     int smax;                    // table covers scores -smax .. smax
@@ -53,7 +54,7 @@ struct AttnParams {
 };
 
 struct AttnBars {
-    uint64_t packed_full, ops_ready, s_full, p_ready, o_full, o_done, grp_sync, z_sync;
+    uint64_t packed_full, v_full, ops_ready, s_full, p_ready, o_full, o_done, grp_sync, z_sync;
 };
 
 // exp(fl32(s * c)) for every integer score, correctly rounded to fp32 (fp64 exp, one rounding).
@@ -89,6 +90,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         abort_flag = 0;
         for (int k = 0; k < AT_GROUPS; ++k) {
             ptx::mbar_init(ptx::smem_addr(&bars[k].packed_full), 1);
+            ptx::mbar_init(ptx::smem_addr(&bars[k].v_full), 1);
             ptx::mbar_init(ptx::smem_addr(&bars[k].ops_ready), AT_COMPUTE_WARPS);
             ptx::mbar_init(ptx::smem_addr(&bars[k].s_full), 1);
             ptx::mbar_init(ptx::smem_addr(&bars[k].p_ready), AT_COMPUTE_WARPS);
@@ -119,6 +121,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 
     const int T = P.tokens;
     const int item0 = blockIdx.x * AT_GROUPS + g, item_stride = gridDim.x * AT_GROUPS;
+    constexpr bool DIRECT = (C == 8);                  // byte codes: no packed staging, no unpack
     const int head_bytes = 8 * C;                      // 64 codes
     const uint32_t q_bytes = 128u * head_bytes, kv_bytes = (uint32_t)P.kv_rows * head_bytes;   // TMA boxes
 
@@ -132,14 +135,24 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     if (is_control) {
         // --------------------------- control: TMA + MMA issue ----------------------------
         if (lane == 0) {
+            // packed codes: one barrier for the three slabs, which the compute warps unpack.
+            // byte codes: Q and K land in their operand tiles under packed_full, V under v_full, so that each
+            // buffer is refilled as soon as the MMA that read it has completed.
             auto issue_loads = [&](int item) {
                 int b, h, qt;
                 item_coords(item, b, h, qt);
                 const uint32_t bar = ptx::smem_addr(&B.packed_full);
-                ptx::mbar_arrive_expect_tx(bar, q_bytes + 2u * kv_bytes);
-                ptx::tma_load_3d(gbase + P.off_pq, &map_q, bar, h * head_bytes, qt * 128, b);
-                ptx::tma_load_3d(gbase + P.off_pk, &map_kv, bar, P.part_bytes + h * head_bytes, 0, b);
-                ptx::tma_load_3d(gbase + P.off_pv, &map_kv, bar, 2 * P.part_bytes + h * head_bytes, 0, b);
+                ptx::mbar_arrive_expect_tx(bar, q_bytes + (DIRECT ? 1u : 2u) * kv_bytes);
+                ptx::tma_load_3d(gbase + (DIRECT ? P.off_q : P.off_pq), &map_q, bar, h * head_bytes, qt * 128, b);
+                ptx::tma_load_3d(gbase + (DIRECT ? P.off_k : P.off_pk), &map_kv, bar, P.part_bytes + h * head_bytes, 0, b);
+                if (!DIRECT) ptx::tma_load_3d(gbase + P.off_pv, &map_kv, bar, 2 * P.part_bytes + h * head_bytes, 0, b);
+            };
+            auto issue_v = [&](int item) {
+                int b, h, qt;
+                item_coords(item, b, h, qt);
+                const uint32_t bar = ptx::smem_addr(&B.v_full);
+                ptx::mbar_arrive_expect_tx(bar, kv_bytes);
+                ptx::tma_load_3d(gbase + P.off_v, &map_kv, bar, 2 * P.part_bytes + h * head_bytes, 0, b);
             };
             const uint32_t idesc_qk = ptx::idesc_i8(128, P.n_k, 1, 1, 0);
             const uint32_t idesc_pv = ptx::idesc_i8(128, 64, 0, 1, 1);
@@ -148,20 +161,38 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const uint64_t v_desc = ptx::smem_desc(gbase + P.off_v, 16, 512, ptx::SWIZZLE_64B);
             const int pv_steps = P.kv_rows / 32;
             bool ok = true;
-            int pending = -1;                       // local index of the item whose loads are in flight
-            if (item0 < P.total_items) { issue_loads(item0); pending = 0; }
+            int pending = -1, pending_v = -1;       // local index of the item whose loads are in flight
+            if (item0 < P.total_items) {
+                issue_loads(item0); pending = 0;
+                if (DIRECT) { issue_v(item0); pending_v = 0; }
+            }
             int n = 0;
             for (int item = item0; ok && item < P.total_items; item += item_stride, ++n) {
                 const uint32_t ph = (uint32_t)n & 1u;
-                if (!mbar_wait(ptx::smem_addr(&B.ops_ready), ph, abort_ptr)) { ok = false; break; }
-                pending = -1;
-                if (item + item_stride < P.total_items) { issue_loads(item + item_stride); pending = n + 1; }
+                const bool has_next = item + item_stride < P.total_items;
+                if (DIRECT) {
+                    if (!mbar_wait(ptx::smem_addr(&B.packed_full), ph, abort_ptr)) { ok = false; break; }
+                    pending = -1;
+                } else {
+                    if (!mbar_wait(ptx::smem_addr(&B.ops_ready), ph, abort_ptr)) { ok = false; break; }
+                    pending = -1;
+                    if (has_next) { issue_loads(item + item_stride); pending = n + 1; }
+                }
                 if (n > 0 && !mbar_wait(ptx::smem_addr(&B.o_done), ph ^ 1u, abort_ptr)) { ok = false; break; }
                 ptx::tc_fence_after();
                 for (int k = 0; k < 2; ++k)                        // K = 64 -> two MMAs of 32
                     ptx::mma_i8(tmem_grp, q_desc + (uint64_t)(k * 2), k_desc + (uint64_t)(k * 2), idesc_qk, k);
                 ptx::mma_commit(ptx::smem_addr(&B.s_full));
+                if (DIRECT) {
+                    // Q K^T has been read out of the Q and K tiles once s_full completes
+                    if (!mbar_wait(ptx::smem_addr(&B.s_full), ph, abort_ptr)) { ok = false; break; }
+                    if (has_next) { issue_loads(item + item_stride); pending = n + 1; }
+                }
                 if (!mbar_wait(ptx::smem_addr(&B.p_ready), ph, abort_ptr)) { ok = false; break; }
+                if (DIRECT) {
+                    if (!mbar_wait(ptx::smem_addr(&B.v_full), ph, abort_ptr)) { ok = false; break; }
+                    pending_v = -1;
+                }
                 ptx::tc_fence_after();
                 for (int ks = 0; ks < pv_steps; ++ks) {
                     const uint64_t p_desc = ptx::smem_desc(gbase + P.off_p + (uint32_t)(ks >> 2) * 16384u, 16, 1024,
@@ -169,11 +200,22 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     ptx::mma_i8(tmem_grp, p_desc, v_desc + (uint64_t)(ks * 128), idesc_pv, ks);
                 }
                 ptx::mma_commit(ptx::smem_addr(&B.o_full));
+                if (DIRECT && has_next) {
+                    // P V has been read out of the V tile once o_full completes
+                    if (!mbar_wait(ptx::smem_addr(&B.o_full), ph, abort_ptr)) { ok = false; break; }
+                    issue_v(item + item_stride); pending_v = n + 1;
+                }
             }
-            if (!ok && pending >= 0) {
+            if (!ok) {
                 // give the copies still in flight a bounded chance to land before the CTA exits
-                const uint32_t bar = ptx::smem_addr(&B.packed_full);
-                for (int spin = 0; spin < (1 << 20) && !ptx::mbar_try_wait(bar, (uint32_t)pending & 1u); ++spin) {}
+                if (pending >= 0) {
+                    const uint32_t bar = ptx::smem_addr(&B.packed_full);
+                    for (int spin = 0; spin < (1 << 20) && !ptx::mbar_try_wait(bar, (uint32_t)pending & 1u); ++spin) {}
+                }
+                if (pending_v >= 0) {
+                    const uint32_t bar = ptx::smem_addr(&B.v_full);
+                    for (int spin = 0; spin < (1 << 20) && !ptx::mbar_try_wait(bar, (uint32_t)pending_v & 1u); ++spin) {}
+                }
             }
         }
     } else {
@@ -185,8 +227,8 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         double* const zx = reinterpret_cast<double*>(ggen + P.off_z);   // partial row sums, [2][128]
         const uint32_t t_row = tmem_grp + ((uint32_t)(wq * 32) << 16);
         const char* const tab_mid = reinterpret_cast<const char*>(smem_gen + P.off_table) + (size_t)P.smax * 4;
-        float* const colp = reinterpret_cast<float*>(ggen + P.off_col);   // alpha[64], beta[64] of this head
-        const int sh_idx = 2 * (8 - C) - 2;                         // scaled score -> byte offset 4*S
+        float* const colp2 = reinterpret_cast<float*>(ggen + P.off_col);  // alpha[64], beta[64] of the head, one copy per item parity
+        const int sh_idx = DIRECT ? 0 : 2 * (8 - C) - 2;            // scaled score -> byte offset 4*S
         const int chunks = P.kv_rows / 32;
         const int tab_half = 4 * P.smax;
         const double inv_p_step = 1.0 / (double)P.p_step;
@@ -196,20 +238,25 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const uint32_t ph = (uint32_t)n & 1u;
             int b, h, qt;
             item_coords(item, b, h, qt);
-            // ---- operands: packed -> int8 -------------------------------------------------
-            bool w = mbar_wait(ptx::smem_addr(&B.packed_full), ph, abort_ptr);
-            if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
-            unpack_rows64<C, 1>(ggen + P.off_pq, ggen + P.off_q, 128, tid_g, AT_COMPUTE_WARPS * 32);
-            unpack_rows64<C, 1>(ggen + P.off_pk, ggen + P.off_k, P.n_k, tid_g, AT_COMPUTE_WARPS * 32);
-            unpack_rows64<C, 1>(ggen + P.off_pv, ggen + P.off_v, P.kv_rows, tid_g, AT_COMPUTE_WARPS * 32);
+            // the head's output parameters; the copy of the other parity may still be read by a warp that is
+            // finishing the previous item, and every reader of this one passes z_sync first
+            float* const colp = colp2 + (n & 1) * 128;
             if (tid_g < 64) colp[tid_g] = __ldg(P.alpha_o + h * 64 + tid_g);
             else if (tid_g < 128) colp[tid_g] = P.beta_o ? __ldg(P.beta_o + h * 64 + (tid_g - 64)) : 0.0f;
-            ptx::fence_proxy_async_smem();
-            // the group's warps exchange the staged column parameters through shared memory
-            ptx::mbar_arrive(ptx::smem_addr(&B.grp_sync));
-            w = mbar_wait(ptx::smem_addr(&B.grp_sync), ph, abort_ptr);
-            if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&B.ops_ready));
+            bool w = true;
+            if constexpr (!DIRECT) {
+                // ---- operands: packed -> int8 ---------------------------------------------
+                w = mbar_wait(ptx::smem_addr(&B.packed_full), ph, abort_ptr);
+                if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+                unpack_rows64<C, 1>(ggen + P.off_pq, ggen + P.off_q, 128, tid_g, AT_COMPUTE_WARPS * 32);
+                unpack_rows64<C, 1>(ggen + P.off_pk, ggen + P.off_k, P.n_k, tid_g, AT_COMPUTE_WARPS * 32);
+                unpack_rows64<C, 1>(ggen + P.off_pv, ggen + P.off_v, P.kv_rows, tid_g, AT_COMPUTE_WARPS * 32);
+                ptx::fence_proxy_async_smem();
+                ptx::mbar_arrive(ptx::smem_addr(&B.grp_sync));
+                w = mbar_wait(ptx::smem_addr(&B.grp_sync), ph, abort_ptr);
+                if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&B.ops_ready));
+            }
             // ---- softmax over the row -------------------------------------------------------
             w = mbar_wait(ptx::smem_addr(&B.s_full), ph, abort_ptr);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
@@ -232,7 +279,9 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         // every table entry is a positive normal float (exp of a bounded argument), so its
                         // double is formed from the bits with two integer operations instead of a conversion
                         // (the conversion unit runs at a quarter of the fp64 adder's rate)
-                        const uint32_t eb = *reinterpret_cast<const uint32_t*>(tab_mid + ((int)v[i] >> sh_idx));
+                        int off = DIRECT ? ((int)v[i] << 2) : ((int)v[i] >> sh_idx);
+                        if (DIRECT) off = max(-tab_half, min(tab_half, off));   // raw bytes: keep any value inside the table
+                        const uint32_t eb = *reinterpret_cast<const uint32_t*>(tab_mid + off);
                         zp[i & 3] += __hiloint2double((int)((eb >> 3) + 0x38000000u), (int)(eb << 29));
                         v[i] = eb;
                     }
@@ -241,7 +290,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const bool valid = ch * 32 + i < T;
-                        const int off = valid ? ((int)v[i] >> sh_idx) : 0;
+                        const int off = valid ? (DIRECT ? ((int)v[i] << 2) : ((int)v[i] >> sh_idx)) : 0;
                         uint32_t eb = *reinterpret_cast<const uint32_t*>(tab_mid + max(-tab_half, min(tab_half, off)));
                         if (!valid) eb = 0u;
                         zp[i & 3] += __hiloint2double(valid ? (int)((eb >> 3) + 0x38000000u) : 0, (int)(eb << 29));
@@ -309,7 +358,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     const int col = hf * 32 + i;
-                    const float f = small_int_to_float((int)v[i] >> (8 - C));
+                    const float f = small_int_to_float((int)v[i] >> (8 - C));     // V codes sit in the high bits of their bytes
                     v[i] = round_clamp_bits(fmaf(f, colp[col], colp[64 + col]), P.out_qn, P.out_qp);
                 }
                 if (P.out_c == 4) {
@@ -378,9 +427,9 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     const float steps[3] = {q_step, k_step, p_step};
     for (float s : steps) if (!(s > 0.0f && s < INFINITY)) return VITINT_ERR_INVALID_ARG;
     if (!valid_bits(p_bits)) return VITINT_ERR_INVALID_ARG;
-    if (qkv->bits == 8 || qkv->container_bits == 8 || tokens > 256 || batch > 65535) return VITINT_ERR_UNSUPPORTED;
-    const int c = container_bits(qkv->bits);
-    const int m = 1 << (c - 1);
+    if (qkv->bits == 8 || tokens > 256 || batch > 65535) return VITINT_ERR_UNSUPPORTED;
+    const int c = codes_container(qkv);                  // 2 / 4: packed; 8: one code per byte
+    const int m = 1 << (container_bits(qkv->bits) - 1);
     const int smax = 64 * m * m;
     const float cs = (float)((double)q_step * (double)k_step / 8.0);
     // exp without max subtraction must not overflow for any score the declared code range can produce
@@ -417,13 +466,15 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     P.off_group = up((uint32_t)(2 * smax + 1) * 4u, 1024);
     uint32_t o = 0;
     P.off_q = o; o += 128 * 64;
-    P.off_k = o; o += up((uint32_t)P.n_k * 64, 1024);
+    P.off_k = o; o += up((uint32_t)(c == 8 ? P.kv_rows : P.n_k) * 64, 1024);   // byte codes: the K box is kv_rows high
     P.off_v = o; o += up((uint32_t)P.kv_rows * 64, 1024);
     P.off_p = o; o += (uint32_t)((P.kv_rows + 127) / 128) * 16384u;
-    P.off_pq = o; o += up(128 * hb, 128);
-    P.off_pk = o; o += up((uint32_t)P.kv_rows * hb, 128);
-    P.off_pv = o; o += up((uint32_t)P.kv_rows * hb, 128);
-    P.off_col = o; o += 512;
+    if (c != 8) {
+        P.off_pq = o; o += up(128 * hb, 128);
+        P.off_pk = o; o += up((uint32_t)P.kv_rows * hb, 128);
+        P.off_pv = o; o += up((uint32_t)P.kv_rows * hb, 128);
+    }
+    P.off_col = o; o += 1024;
     P.off_z = o; o += 2 * 128 * 8;
     P.group_bytes = up(o, 1024);
     const size_t smem = (size_t)P.off_group + (size_t)AT_GROUPS * P.group_bytes + 1024;
@@ -435,15 +486,17 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
         // last token read as zero.  Q tiles are 128 rows high, K and V tiles kv_rows.
         EncodeTiledFn fn = encode_fn();
         if (!fn) return VITINT_ERR_CUDA;
-        cuuint64_t dims[3] = {(cuuint64_t)row_bytes(3 * D, qkv->bits), (cuuint64_t)tokens, (cuuint64_t)batch};
+        cuuint64_t dims[3] = {(cuuint64_t)codes_row_bytes(qkv, 3 * D), (cuuint64_t)tokens, (cuuint64_t)batch};
+        // byte codes land directly in the 64-byte-swizzled operand tiles
+        const CUtensorMapSwizzle swz = c == 8 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE;
         cuuint64_t strides[2] = {(cuuint64_t)qkv->pitch_bytes, (cuuint64_t)qkv->pitch_bytes * tokens};
         cuuint32_t estr[3] = {1, 1, 1};
         cuuint32_t box_q[3] = {hb, 128, 1}, box_kv[3] = {hb, (cuuint32_t)P.kv_rows, 1};
         if (fn(&map_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, qkv->data, dims, strides, box_q, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
             fn(&map_kv, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, qkv->data, dims, strides, box_kv, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return VITINT_ERR_CUDA;
     }
@@ -452,22 +505,21 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     int grid = sm_count();
     const int want = (P.total_items + AT_GROUPS - 1) / AT_GROUPS;
     if (grid > want) grid = want;
-    static bool attr2 = false, attr4 = false;
-    if (c == 4) {
-        if (!attr4) {
-            if (cudaFuncSetAttribute(attention_fused_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess)
-                return VITINT_ERR_CUDA;
-            attr4 = true;
-        }
-        launch_kernel(attention_fused_kernel<4>, dim3(grid), dim3(AT_THREADS), smem, st, map_q, map_kv, P);
-    } else {
-        if (!attr2) {
-            if (cudaFuncSetAttribute(attention_fused_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) != cudaSuccess)
-                return VITINT_ERR_CUDA;
-            attr2 = true;
-        }
-        launch_kernel(attention_fused_kernel<2>, dim3(grid), dim3(AT_THREADS), smem, st, map_q, map_kv, P);
+    static bool attr_set[3] = {false, false, false};
+#define VITINT_ATTN_LAUNCH(CC, SLOT)                                                                               \
+    {                                                                                                              \
+        if (!attr_set[SLOT]) {                                                                                     \
+            if (cudaFuncSetAttribute(attention_fused_kernel<CC>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                                     225 * 1024) != cudaSuccess)                                                   \
+                return VITINT_ERR_CUDA;                                                                            \
+            attr_set[SLOT] = true;                                                                                 \
+        }                                                                                                          \
+        launch_kernel(attention_fused_kernel<CC>, dim3(grid), dim3(AT_THREADS), smem, st, map_q, map_kv, P);       \
     }
+    if (c == 8) VITINT_ATTN_LAUNCH(8, 2)
+    else if (c == 4) VITINT_ATTN_LAUNCH(4, 1)
+    else VITINT_ATTN_LAUNCH(2, 0)
+#undef VITINT_ATTN_LAUNCH
     return cuda_status(cudaGetLastError());
 }
 

@@ -56,12 +56,12 @@ class EncoderLayer:
         self.alpha_o = d(a)
         self.inv_s_g = d((1.0 / np.full(F, prm["s_g"], np.float64)).astype(np.float32))
         self.c = float(np.float32(float(prm["s_q"]) * float(prm["s_k"]) / 8.0))
-        # activations.  The codes that only feed a linear layer (x1, O, x2, g) are stored one per
-        # byte, so that layer's TMA copy is already the tensor-core operand; q, k, v stay packed
-        # (the attention kernels unpack them per head).
+        # activations, stored one code per byte: the consumer's TMA copy is then already the
+        # tensor-core operand (the unfused attention kernels read packed q, k, v slabs instead)
         ca = 8 if wide_activations and bits != 8 else 0
+        cq = ca if self.fused_attention else 0
         self.x1 = B.Codes.empty(M, D, bits, True, device, container=ca)
-        self.qkv = B.Codes.empty(M, 3 * D, bits, True, device)
+        self.qkv = B.Codes.empty(M, 3 * D, bits, True, device, container=cq)
         self.ld_s = (tokens + 3) // 4 * 4
         if self.fused_attention:
             self.attn_ws = torch.empty(B.vitint_attention_core_workspace_bytes(bits), dtype=torch.uint8, device=device)
@@ -72,9 +72,9 @@ class EncoderLayer:
         self.h = torch.empty((M, D), dtype=torch.float32, device=device)
         self.x2 = B.Codes.empty(M, D, bits, True, device, container=ca)
         self.g = B.Codes.empty(M, F, bits, False, device, container=ca)
-        self.slabs = [B.Slabs.of_qkv(self.qkv, tokens, D, i) for i in range(3)]
+        self.slabs = None if self.fused_attention else [B.Slabs.of_qkv(self.qkv, tokens, D, i) for i in range(3)]
         self.epi_qkv = B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_qkv, beta=self.beta_qkv, out_bits=bits,
-                                  out_signed=True)
+                                  out_signed=True, out_container=cq)
         self.epi_o = B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_o, out_bits=bits, out_signed=True, out_container=ca)
         self.epi_fc1 = B.Epilogue(mode=B.EPI_REQUANT, act=1, inv_out_step=self.inv_s_g, out_bits=bits, out_signed=False,
                                   out_container=ca)

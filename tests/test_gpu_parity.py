@@ -300,11 +300,13 @@ def test_softmax_error_statistics_on_attention_like_rows():
     assert np.all(g >= lo) and np.all(g <= hi)
 
 
+@pytest.mark.parametrize("byte_codes", [False, True], ids=["packed_qkv", "byte_qkv"])
 @pytest.mark.parametrize("bits", [4, 2, 3])
 @pytest.mark.parametrize("batch,tokens,heads,scale", [(1, 197, 3, 1.0), (3, 197, 2, 3.0), (2, 50, 1, 3.0), (1, 256, 2, 2.0),
                                                       (5, 128, 1, 0.3), (2, 129, 2, 2.5)])
-def test_attention_core_fused(batch, tokens, heads, bits, scale):
-    """Fused Q K^T -> softmax -> P V against the oracle stages; rows whose P codes are unique must be bit-exact."""
+def test_attention_core_fused(batch, tokens, heads, bits, scale, byte_codes):
+    """Fused Q K^T -> softmax -> P V against the oracle stages; rows whose P codes are unique must be bit-exact.
+    The Q, K, V codes arrive bit-packed (unpacked inside the kernel) or one per byte (the TMA copy is the operand)."""
     D = heads * 64
     qkv = _qkv_codes(batch, tokens, heads, bits, 61 + tokens)
     qmax = si.code_range(bits, True)[1] + 1
@@ -322,8 +324,10 @@ def test_attention_core_fused(batch, tokens, heads, bits, scale):
     alpha, beta = vp.fold(s_p, np.full(D, 0.17, np.float32), None, np.float32(0.17 * 0.6 * qmax / math.sqrt(8 * scale + 1)))
     beta = si.normal(5, (D,), 0.0, 0.3)
     want = vo.epilogue_requant(vp.merge_heads(acc, batch, tokens, heads, 64), alpha, beta, bits, True)
-    got = from_codes(vt.vitint_attention_core(to_codes(qkv, bits, True), batch, heads, tokens, s_q, s_k, s_p, bits,
-                                              dev(alpha), dev(beta)))
+    qkv_dev = to_codes(qkv, bits, True)
+    if byte_codes:
+        qkv_dev = vt.vitint_widen(qkv_dev)
+    got = from_codes(vt.vitint_attention_core(qkv_dev, batch, heads, tokens, s_q, s_k, s_p, bits, dev(alpha), dev(beta)))
     unique_row = (plo == phi).all(axis=1).reshape(n, tokens)             # [B*H, T]
     ok = np.ones((batch * tokens, D), bool)
     for b in range(batch):
