@@ -49,11 +49,13 @@ def merge_heads(slabs, batch: int, tokens: int, heads: int, head_dim: int):
 
 
 def attention_block(x_codes, s_x, prm: dict, batch: int, tokens: int, heads: int, bits: int, head_dim: int = 64,
-                    proj: str = "dequant", residual=None, wq: dict | None = None) -> dict:
+                    proj: str = "dequant", residual=None, wq: dict | None = None, softmax: str = "exp") -> dict:
     """Integerized self-attention: QKV linear -> Q K^T -> softmax -> quantize -> P V -> proj.
 
     proj: "dequant" (fp32 output, optional residual) or "requant" (codes at step prm["s_out"]).
     wq: optional pre-quantized weight codes {"w_qkv", "w_proj"}.
+    softmax: "exp" (Eq. 3, fp32 island: codes come with a band) or "shift" (Eq. 4 with the division-free
+    comparator quantizer: integer and single-rounding operations only, so the codes are unique).
     """
     D = heads * head_dim
     st: dict = {}
@@ -80,9 +82,16 @@ def attention_block(x_codes, s_x, prm: dict, batch: int, tokens: int, heads: int
     c = softmax_scale(prm["s_q"], prm["s_k"], head_dim)
     st["c"] = c
     n = batch * heads
-    p, pc, plo, phi = vo.softmax_quantize(st["S"].reshape(n * tokens, tokens), c, prm["s_p"], bits)
-    st["p"], st["p_codes"] = p.reshape(n, tokens, tokens), pc.reshape(n, tokens, tokens)
-    st["p_lo"], st["p_hi"] = plo.reshape(n, tokens, tokens), phi.reshape(n, tokens, tokens)
+    if softmax == "shift":
+        c2 = np.float32(np.float64(c) * np.log2(np.e))               # exponent of two: z = S * c * log2(e)
+        st["c2"] = c2
+        pc = vo.softmax_shift_quantize(st["S"].reshape(n * tokens, tokens), c2, prm["s_p"], bits)
+        st["p_codes"] = pc.reshape(n, tokens, tokens)
+        st["p_lo"] = st["p_hi"] = st["p_codes"]
+    else:
+        p, pc, plo, phi = vo.softmax_quantize(st["S"].reshape(n * tokens, tokens), c, prm["s_p"], bits)
+        st["p"], st["p_codes"] = p.reshape(n, tokens, tokens), pc.reshape(n, tokens, tokens)
+        st["p_lo"], st["p_hi"] = plo.reshape(n, tokens, tokens), phi.reshape(n, tokens, tokens)
 
     st["acc_o"] = vo.pv(st["p_codes"], v)
     a_o, b_o = fold(prm["s_p"], np.full(head_dim, prm["s_v"], np.float32), None, prm["s_o"])
@@ -101,13 +110,14 @@ def attention_block(x_codes, s_x, prm: dict, batch: int, tokens: int, heads: int
 
 
 def encoder_layer(x, prm: dict, batch: int, tokens: int, heads: int, bits: int, head_dim: int = 64,
-                  eps: float = 1e-6) -> dict:
+                  eps: float = 1e-6, softmax: str = "exp") -> dict:
     """LN1 -> quantize -> attention (+residual) -> LN2 -> quantize -> fc1 -> GELU -> quantize -> fc2 (+residual)."""
     st: dict = {}
     y1, tol1 = vo.layernorm(x, prm["ln1_g"], prm["ln1_b"], eps)
     st["ln1"], st["ln1_tol"] = y1, tol1
     st["x1_codes"], st["x1_lo"], st["x1_hi"] = vo.quantize_band(y1, tol1, prm["s_ln"], bits, True)
-    att = attention_block(st["x1_codes"], prm["s_ln"], prm, batch, tokens, heads, bits, head_dim, "dequant", x)
+    att = attention_block(st["x1_codes"], prm["s_ln"], prm, batch, tokens, heads, bits, head_dim, "dequant", x,
+                          softmax=softmax)
     st["attn"] = att
     h = att["out"]
     st["h"] = h

@@ -25,13 +25,17 @@ def _dev(a, device):
 class EncoderLayer:
     def __init__(self, batch: int, tokens: int, heads: int, mlp_dim: int, bits: int, prm: dict, device="cuda",
                  eps: float = 1e-6, widen_weights: bool = True, fused_attention: bool = True,
-                 wide_activations: bool = True):
+                 wide_activations: bool = True, softmax: str = "exp"):
         self.batch, self.tokens, self.heads, self.bits, self.eps = batch, tokens, heads, bits, eps
         self.dim = D = heads * 64
         self.mlp_dim = F = mlp_dim
         self.rows = M = batch * tokens
         self.device = device
-        self.fused_attention = fused_attention and bits != 8 and tokens <= 256
+        if softmax not in ("exp", "shift"):
+            raise ValueError("softmax must be 'exp' (Eq. 3) or 'shift' (Eq. 4 with the comparator quantizer)")
+        self.softmax = softmax
+        # the shift-based softmax is a separate kernel: it runs in the unfused attention pipeline
+        self.fused_attention = fused_attention and bits != 8 and tokens <= 256 and softmax == "exp"
         self.stages = STAGES_FUSED if self.fused_attention else STAGES_UNFUSED
         d = lambda a: _dev(a, device)
         f = lambda k: float(prm[k])
@@ -56,6 +60,7 @@ class EncoderLayer:
         self.alpha_o = d(a)
         self.inv_s_g = d((1.0 / np.full(F, prm["s_g"], np.float64)).astype(np.float32))
         self.c = float(np.float32(float(prm["s_q"]) * float(prm["s_k"]) / 8.0))
+        self.c2 = float(np.float32(np.float64(np.float32(self.c)) * np.log2(np.e)))   # exponent of two for Eq. 4
         # activations, stored one code per byte: the consumer's TMA copy is then already the
         # tensor-core operand (the unfused attention kernels read packed q, k, v slabs instead)
         ca = 8 if wide_activations and bits != 8 else 0
@@ -99,7 +104,10 @@ class EncoderLayer:
         else:
             B.vitint_qk(self.slabs[0], self.slabs[1], b, h, t, out=self.S, ld_s=self.ld_s)
             mark()
-            B.vitint_softmax_quantize(self.S, t, self.c, self.s_p, self.bits, out=self.P)
+            if self.softmax == "shift":
+                B.vitint_softmax_shift_quantize(self.S, t, self.c2, self.s_p, self.bits, out=self.P)
+            else:
+                B.vitint_softmax_quantize(self.S, t, self.c, self.s_p, self.bits, out=self.P)
             mark()
             B.vitint_pv(self.P, self.slabs[2], b, h, t, self.s_p, self.s_v, self.epi_o, out=self.O)
         mark()

@@ -102,6 +102,34 @@ def test_encoder_layer_staged(bits, fused, wide):
     compare_stages(g, st, cfg.batch, cfg.tokens, cfg.heads, cfg.dim, fused, min_images_ok=2)
 
 
+@pytest.mark.parametrize("bits", [4, 3])
+def test_encoder_layer_shift_softmax_attention_bit_exact(bits):
+    """Encoder layer with the Eq. 4 softmax and the comparator quantizer: the attention stage has no fp32 island,
+    so in every image whose LayerNorm codes agree, P and O must equal the oracle's bit for bit."""
+    from paper_2504_18547_b200.encoder import EncoderLayer
+    cfg = si.VIT_BASE_LAYER.with_(batch=3, bits=bits)
+    prm = si.layer_parameters(cfg)
+    x = si.activations(cfg)
+    st = vp.encoder_layer(x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits, softmax="shift")
+    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, softmax="shift")
+    assert not layer.fused_attention
+    out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
+    layer.forward(dev(x), out)
+    assert vt.vitint_device_status() == 0
+    T, H = cfg.tokens, cfg.heads
+    g = gpu_stages(layer, out, range(cfg.batch), T, H)
+    att = st["attn"]
+    img_ok = np.array([(g["x1"][b * T:(b + 1) * T] == st["x1_codes"][b * T:(b + 1) * T]).all() for b in range(cfg.batch)])
+    assert img_ok.sum() >= 2
+    heads_ok = np.repeat(img_ok, H)
+    rows_ok = np.repeat(img_ok, T)
+    assert np.array_equal(g["P"][heads_ok], att["p_codes"][heads_ok])
+    assert np.array_equal(g["O"][rows_ok], att["o_codes"][rows_ok])
+    assert len(np.unique(att["p_codes"])) >= 4
+    # the rest of the layer as in the exp mode
+    compare_stages(g, st, cfg.batch, T, H, cfg.dim, False, min_images_ok=2)
+
+
 @pytest.mark.parametrize("bits", [4, 2])
 def test_encoder_layer_full_size_sampled_images(bits):
     """The benchmark's own launch configuration (ViT-Base layer, batch 128): the GPU runs the full batch, the
