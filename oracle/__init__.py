@@ -228,6 +228,39 @@ def layernorm(x, gamma, beta, eps: float = 1e-6):
     return y, tol
 
 
+def layernorm_references(gamma, beta, step, bits: int, signed: bool, cols: int):
+    """References of the division- and square-root-free LayerNorm comparator (Fig. 5(b)), fp64 then one
+    rounding: for column j and threshold k = Qn+1..Qp, c = ((k - 1/2) step - beta_j) / gamma_j, taken with
+    the sign flipped where gamma_j < 0.  Returns (ref = c^2 / cols as fp32 [cols, n_thr], neg = c < 0 as
+    uint8 [cols, n_thr], flip = gamma < 0 as uint8 [cols])."""
+    qn, qp = code_range(bits, signed)
+    g = np.asarray(gamma, dtype=np.float64)[:, None]
+    b = np.asarray(beta, dtype=np.float64)[:, None]
+    k = np.arange(qn + 1, qp + 1, dtype=np.float64)[None, :]
+    c = ((k - 0.5) * float(step) - b) / g
+    flip = (g[:, 0] < 0)
+    c = np.where(flip[:, None], -c, c)
+    ref = (c * c / float(cols)).astype(np.float32)
+    return np.ascontiguousarray(ref), np.ascontiguousarray((c < 0).astype(np.uint8)), flip.astype(np.uint8)
+
+
+def layernorm_compare_quantize(x, ref, neg, flip, eps: float, bits: int, signed: bool, want_stats: bool = False):
+    """Eq. 5 running statistics in fp32 + the comparator quantizer of Fig. 5(b).  x fp32 [rows, cols] -> codes
+    (and, optionally, the row means and V = S_n + n*eps)."""
+    x = _f32(x)
+    rows, cols = x.shape
+    ref = _f32(ref)
+    neg = np.ascontiguousarray(neg, dtype=np.uint8)
+    flip = np.ascontiguousarray(flip, dtype=np.uint8)
+    q = np.empty((rows, cols), dtype=np.int16)
+    mu = np.empty(rows, dtype=np.float32)
+    v = np.empty(rows, dtype=np.float32)
+    n_eps = np.float32(np.float64(cols) * np.float64(np.float32(eps)))
+    lib().vo_layernorm_compare_quantize(_p(x), I64(rows), I64(cols), I64(cols), _p(ref), _p(neg), _p(flip),
+                                        F32(float(n_eps)), I32(bits), I32(int(signed)), _p(q), I64(cols), _p(mu), _p(v))
+    return (q, mu, v) if want_stats else q
+
+
 def running_stats(x):
     x = _f32(x).ravel()
     mu = ctypes.c_double()

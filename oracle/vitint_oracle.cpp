@@ -20,7 +20,8 @@
 // int32 overflow bound, the 3-bit threshold ladder, pack/unpack round trips,
 // exact-rational epilogue cases, softmax closed forms and invariants, the shift softmax
 // against big-integer / rational arithmetic and its 2^r ~ 1+r error bound, LayerNorm
-// against the Welford recurrence of Eq. 5.  Parity unpinned: none of the
+// against the Welford recurrence of Eq. 5, the comparator LayerNorm quantizer against exact rational
+// arithmetic, the direct formula of Fig. 5(a), hand-worked rows and its invariances.  Parity unpinned: none of the
 // functions below; the paper's accuracy and power tables are out of scope.
 
 #include <algorithm>
@@ -381,6 +382,60 @@ void vo_running_stats(const float* x, int64_t n, double* mu_out, double* m2_out)
     }
     *mu_out = mu;
     *m2_out = m2;
+}
+
+// ---- quantizing LayerNorm (Section IV-C: Eq. 5 running statistics + the division- and
+//      square-root-free comparator of Fig. 5(b)) ---------------------------------------------
+// Row statistics by the recurrence of Eq. 5 in the order the paper gives, every operation a
+// single fp32 one (the paper fixes no precision; fp32 is the reading taken):
+//   delta = x_i - mu_{i-1};  mu_i = mu_{i-1} + delta / i;  S_i = S_{i-1} + delta * (x_i - mu_i)
+// with mu_0 = S_0 = 0.  S_n is the unnormalised sum of squared deviations (n * variance); the 1/n
+// and LayerNorm's epsilon are absorbed as the paper absorbs scales: V = S_n + n*eps multiplies
+// references that already carry 1/n.
+// Quantizer: code = Qn + number of thresholds s_k = (k - 1/2) * step, k = Qn+1 .. Qp, with
+//   (x - mu)/sigma * gamma + beta > s_k.
+// For gamma > 0 this is  d > sigma * c_k  with d = x - mu, c_k = (s_k - beta)/gamma, decided without
+// sigma and without a division from squares plus sign logic (Fig. 5(b)):
+//   c_k <  0 :  true when d >= 0, otherwise  d*d < V * (c_k^2 / n)
+//   c_k >= 0 :  false when d <= 0, otherwise  d*d > V * (c_k^2 / n)
+// For gamma < 0 the direction flips (d < sigma * c_k): the same logic applied to -d and -c_k.
+// The caller supplies ref[j][t] = c^2 / n >= 0 and neg[j][t] = 1 when the (gamma-sign-adjusted) c is
+// negative, for column j and threshold t = 0 .. 2^bits-2 (ascending k), and flip[j] = 1 for gamma_j < 0.
+void vo_layernorm_compare_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, const float* ref,
+                                   const uint8_t* neg, const uint8_t* flip, float n_eps, int bits, int is_signed,
+                                   int16_t* q, int64_t ldq, float* mu_out, float* v_out) {
+    int qn, qp;
+    code_range(bits, is_signed, &qn, &qp);
+    const int n_thr = qp - qn;
+    parallel_for(rows, [&](int64_t m) {
+        const float* xr = x + m * ldx;
+        float mu = 0.0f, S = 0.0f;
+        for (int64_t i = 1; i <= cols; ++i) {
+            const float xi = xr[i - 1];
+            const float delta = xi - mu;
+            const float step_mu = delta / (float)i;
+            mu = mu + step_mu;
+            const float prod = delta * (xi - mu);
+            S = S + prod;
+        }
+        const float V = S + n_eps;
+        if (mu_out) mu_out[m] = mu;
+        if (v_out) v_out[m] = V;
+        for (int64_t j = 0; j < cols; ++j) {
+            float d = xr[j] - mu;
+            if (flip && flip[j]) d = -d;
+            const float d2 = d * d;
+            int code = qn;
+            for (int t = 0; t < n_thr; ++t) {
+                const float rhs = V * ref[j * n_thr + t];
+                bool above;
+                if (neg[j * n_thr + t]) above = (d >= 0.0f) ? true : (d2 < rhs);
+                else                    above = (d <= 0.0f) ? false : (d2 > rhs);
+                if (above) ++code;
+            }
+            q[m * ldq + j] = (int16_t)code;
+        }
+    });
 }
 
 // Quantize y with absolute tolerance tol: the code of y and the codes reachable

@@ -546,3 +546,145 @@ def test_shift_softmax_comparator_is_strict_and_scaled_by_the_row_sum():
     # exact tie: p = 1/2 against the reference (k - 1/2) * step = 1/2 at k = 1, step = 1: not exceeded (strict '>')
     q = vo.softmax_shift_quantize(np.array([[3, 3]], np.int32), np.float32(1.0), np.float32(1.0), 4)
     assert q.tolist() == [[0, 0]]
+
+
+# ---------------------------------------------------------------------------
+# quantizing LayerNorm: Eq. 5 statistics + the comparator of Fig. 5(b)
+# ---------------------------------------------------------------------------
+
+def _direct_layernorm_codes(x_row, gamma, beta, step, bits, signed, eps):
+    """Fig. 5(a) in exact rational arithmetic: code = Qn + #{k : (x-mu)/sigma*gamma+beta > (k-1/2) step}, the
+    square root avoided by comparing signed squares of exact rationals.  Also returns the smallest relative
+    distance of any comparison from a tie."""
+    qn, qp = vo.code_range(bits, signed)
+    xs = [Fraction(float(v)) for v in x_row]
+    n = len(xs)
+    mu = sum(xs) / n
+    var = sum((v - mu) ** 2 for v in xs) / n + Fraction(float(np.float32(eps)))
+    codes, margin = [], 1.0
+    for j, v in enumerate(xs):
+        g, b = Fraction(float(gamma[j])), Fraction(float(beta[j]))
+        code = qn
+        for k in range(qn + 1, qp + 1):
+            s = (Fraction(k) - Fraction(1, 2)) * Fraction(float(step))
+            lhs = (v - mu) * g                 # (x - mu) * gamma  >  (s - beta) * sigma  ?
+            rhs_over_sigma = s - b
+            sq = lambda t: t * abs(t)          # strictly increasing: compares like t itself
+            a, c = sq(lhs), sq(rhs_over_sigma) * var
+            if a > c:
+                code += 1
+            scale = max(abs(a), abs(c), Fraction(1, 10 ** 30))
+            margin = min(margin, float(abs(a - c) / scale))
+        codes.append(code)
+    return codes, margin
+
+
+def test_layernorm_comparator_hand_worked_row():
+    # x = 1, 2, 3, 4: Eq. 5 gives mu = 1, 1.5, 2, 2.5 and S = 0, 0.5, 2, 5, all exact in binary fp.
+    # variance 5/4, z = (x - 2.5)/sqrt(1.25) = -1.342, -0.447, 0.447, 1.342; step 1/2, 3 bits:
+    # z/step = -2.68, -0.89, 0.89, 2.68 -> levels -3, -1, 1, 3.
+    x = np.array([[1, 2, 3, 4]], np.float32)
+    ref, neg, flip = vo.layernorm_references(np.ones(4), np.zeros(4), 0.5, 3, True, 4)
+    q, mu, v = vo.layernorm_compare_quantize(x, ref, neg, flip, 0.0, 3, True, want_stats=True)
+    assert mu[0] == np.float32(2.5) and v[0] == np.float32(5.0)
+    assert q.tolist() == [[-3, -1, 1, 3]]
+    # the references themselves: c_k = (k - 1/2)/2 for k = -3..3, ref = c^2/4
+    want = [((k - 0.5) * 0.5) ** 2 / 4 for k in range(-3, 4)]
+    assert np.allclose(ref[0], np.array(want, np.float32), rtol=0, atol=0)
+    assert neg[0].tolist() == [1, 1, 1, 1, 0, 0, 0]
+
+
+def test_layernorm_comparator_is_strict_on_exact_ties():
+    # x = 0, 2: Eq. 5 gives mu = 0, 1 and S = 0, 2 exactly; variance 1 (eps = 0), so z = -1, 1 exactly.
+    # With step 2 the boundaries (k - 1/2)*2 = ..., -3, -1, 1, 3 hit z: the comparator is '>' as drawn, so
+    # z = 1 stays at level 0 (not above the boundary 1) and z = -1 at level -1 (not above -1, above -3).
+    x = np.array([[0, 2]], np.float32)
+    ref, neg, flip = vo.layernorm_references(np.ones(2), np.zeros(2), 2.0, 3, True, 2)
+    q = vo.layernorm_compare_quantize(x, ref, neg, flip, 0.0, 3, True)
+    assert q.tolist() == [[-1, 0]]
+    # a gain a hair above one moves z = 1 over its boundary (z = -1 moves away from -1, downwards: no change);
+    # a gain a hair below one moves z = -1 over its boundary instead
+    g = np.full(2, np.nextafter(np.float32(1), np.float32(2)), np.float32)
+    ref2, neg2, flip2 = vo.layernorm_references(g, np.zeros(2), 2.0, 3, True, 2)
+    assert vo.layernorm_compare_quantize(x, ref2, neg2, flip2, 0.0, 3, True).tolist() == [[-1, 1]]
+    g = np.full(2, np.nextafter(np.float32(1), np.float32(0)), np.float32)
+    ref3, neg3, flip3 = vo.layernorm_references(g, np.zeros(2), 2.0, 3, True, 2)
+    assert vo.layernorm_compare_quantize(x, ref3, neg3, flip3, 0.0, 3, True).tolist() == [[0, 0]]
+
+
+@pytest.mark.parametrize("bits,signed", [(2, True), (3, True), (4, True), (4, False)])
+def test_layernorm_comparator_against_exact_rational_direct_formula(bits, signed):
+    rng = np.random.default_rng(2504 + bits)
+    rows, cols = 6, 24
+    x = rng.normal(0.3, 1.7, (rows, cols)).astype(np.float32)
+    gamma = rng.normal(1.0, 0.3, cols).astype(np.float32)
+    gamma[3] = -gamma[3]                     # a negative gain flips the comparison
+    gamma[11] = -0.7
+    beta = rng.normal(0.0, 0.4, cols).astype(np.float32)
+    step = np.float32(0.37)
+    eps = 1e-5
+    ref, neg, flip = vo.layernorm_references(gamma, beta, step, bits, signed, cols)
+    assert flip[3] == 1 and flip[11] == 1 and flip.sum() == 2
+    q = vo.layernorm_compare_quantize(x, ref, neg, flip, eps, bits, signed)
+    checked = 0
+    for r in range(rows):
+        want, margin = _direct_layernorm_codes(x[r], gamma, beta, step, bits, signed, eps)
+        if margin > 1e-4:                    # fp32 statistics move a comparison only this close to a tie
+            assert q[r].tolist() == want, r
+            checked += 1
+    assert checked >= rows - 1
+
+
+def test_layernorm_comparator_equals_layernorm_then_round_off_ties():
+    cfg = si.VIT_BASE_LAYER.with_(batch=1)
+    prm = si.layer_parameters(cfg)
+    x = si.activations(cfg)[:24]
+    y, tol = vo.layernorm(x, prm["ln1_g"], prm["ln1_b"], 1e-6)
+    s = np.float32(prm["s_ln"])
+    ref, neg, flip = vo.layernorm_references(prm["ln1_g"], prm["ln1_b"], s, cfg.bits, True, x.shape[1])
+    q = vo.layernorm_compare_quantize(x, ref, neg, flip, 1e-6, cfg.bits, True)
+    # the plain path: fp64 LayerNorm, round to nearest, clamp (numpy, not the oracle's quantizer)
+    qn, qp = vo.code_range(cfg.bits, True)
+    u = y.astype(np.float64) / float(s)
+    plain = np.clip(np.rint(u), qn, qp).astype(np.int16)
+    frac = np.abs(u - np.floor(u) - 0.5)
+    clear = frac > 1e-3                      # away from a rounding boundary both rules give the same level
+    assert clear.mean() > 0.99
+    assert np.array_equal(q[clear], plain[clear])
+    assert np.abs(q.astype(int) - plain.astype(int)).max() <= 1
+
+
+def test_layernorm_comparator_invariances_on_exact_data():
+    # integers: every step of Eq. 5 that matters stays exact enough that a shift of all inputs by a constant
+    # or a scaling by a power of two (eps = 0) leaves the statistics' ratios, hence every level, unchanged
+    rng = np.random.default_rng(77)
+    x = rng.integers(-8, 9, (5, 16)).astype(np.float32)
+    gamma = np.ones(16, np.float32)
+    beta = np.zeros(16, np.float32)
+    ref, neg, flip = vo.layernorm_references(gamma, beta, 0.3, 4, True, 16)
+    q0 = vo.layernorm_compare_quantize(x, ref, neg, flip, 0.0, 4, True)
+    q1 = vo.layernorm_compare_quantize(x * 4.0, ref, neg, flip, 0.0, 4, True)
+    assert np.array_equal(q0, q1)
+    for r in range(5):
+        want, margin = _direct_layernorm_codes(x[r] + 64.0, gamma, beta, np.float32(0.3), 4, True, 0.0)
+        got = vo.layernorm_compare_quantize((x[r:r + 1] + 64.0), ref, neg, flip, 0.0, 4, True)
+        if margin > 1e-4:
+            assert got[0].tolist() == want
+
+
+def test_layernorm_comparator_brute_force_tiny_rows():
+    # every row of three values from {-2..2}: exact rational decision vs the oracle (2-bit levels)
+    vals = [-2.0, -1.0, 0.0, 1.0, 2.0]
+    gamma = np.array([1.0, 0.5, -1.5], np.float32)
+    beta = np.array([0.25, -0.5, 0.0], np.float32)
+    step = np.float32(0.75)
+    ref, neg, flip = vo.layernorm_references(gamma, beta, step, 2, True, 3)
+    rows = np.array(list(itertools.product(vals, repeat=3)), np.float32)
+    q = vo.layernorm_compare_quantize(rows, ref, neg, flip, 1e-3, 2, True)
+    n_checked = 0
+    for r in range(rows.shape[0]):
+        want, margin = _direct_layernorm_codes(rows[r], gamma, beta, step, 2, True, 1e-3)
+        if margin > 1e-5:
+            assert q[r].tolist() == want, rows[r]
+            n_checked += 1
+    assert n_checked > 100
