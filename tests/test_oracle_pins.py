@@ -592,6 +592,14 @@ def test_layernorm_comparator_hand_worked_row():
     want = [((k - 0.5) * 0.5) ** 2 / 4 for k in range(-3, 4)]
     assert np.allclose(ref[0], np.array(want, np.float32), rtol=0, atol=0)
     assert neg[0].tolist() == [1, 1, 1, 1, 0, 0, 0]
+    # epsilon enters as n*eps added to S: x = 0, 2 has S = 2 (variance 1); eps = 3 makes the variance 4,
+    # z = -1/2, 1/2, and with step 0.3 (boundaries +-0.15, +-0.45, +-0.75, -1.05) the levels are -2, 2;
+    # without eps z = -1, 1 gives -3, 3
+    x = np.array([[0, 2]], np.float32)
+    ref, neg, flip = vo.layernorm_references(np.ones(2), np.zeros(2), 0.3, 3, True, 2)
+    q, mu, v = vo.layernorm_compare_quantize(x, ref, neg, flip, 3.0, 3, True, want_stats=True)
+    assert v[0] == np.float32(8.0) and q.tolist() == [[-2, 2]]
+    assert vo.layernorm_compare_quantize(x, ref, neg, flip, 0.0, 3, True).tolist() == [[-3, 3]]
 
 
 def test_layernorm_comparator_is_strict_on_exact_ties():
