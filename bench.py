@@ -298,8 +298,15 @@ def run_ours(args, cfg):
         xq = vt.Codes.empty(M, D, cfg.bits, True, device)
         sm_bytes = n_rows * T * 4 + n_rows * ((T * cb + 7) // 8)
         q_bytes = M * D * 4 + M * D * cb // 8
+        # the paper's own LayerNorm quantizer (Eq. 5 statistics + comparator), which the default step does not use
+        lrefs, lflip = vt.fold_layernorm_references(prm["ln1_g"], prm["ln1_b"], prm["s_ln"], cfg.bits, True, D)
+        lrefs, lflip = torch.from_numpy(lrefs).to(device), torch.from_numpy(lflip).to(device)
+        lstats = torch.empty((M, 2), dtype=torch.float32, device=device)
+        n_eps = float(np.float32(D * 1e-6))
         for name, fn, nbytes in (
                 ("quantize", lambda: vt.vitint_quantize(xs[1], layer.s_ln, cfg.bits, True, out=xq), q_bytes),
+                ("layernorm_compare_quant", lambda: vt.vitint_layernorm_compare_quantize(
+                    xs[2], lrefs, lflip, n_eps, cfg.bits, True, out=xq, stats=lstats), q_bytes),
                 ("softmax_quant", lambda: vt.vitint_softmax_quantize(S, T, layer.c, layer.s_p, cfg.bits, out=Pq), sm_bytes),
                 ("softmax_shift_quant", lambda: vt.vitint_softmax_shift_quantize(S, T, layer.c * 1.4426950408889634,
                                                                                  layer.s_p, cfg.bits, out=Pq), sm_bytes)):

@@ -267,6 +267,26 @@ int vitint_layernorm_quantize(const float* x, int64_t rows, int64_t cols, int64_
                               const float* beta, float eps, float step, const vitint_codes* out, float* y_f32,
                               int64_t ld_y, void* stream);
 
+/* Quantizing LayerNorm of Section IV-C: running statistics of Eq. 5 and the division- and square-root-free
+ * comparator of Fig. 5(b).
+ *   statistics, per row, in the order of Eq. 5, every operation one round-to-nearest fp32 operation:
+ *     delta = x_i - mu;  mu = mu + delta / i;  S = S + delta * (x_i - mu)      (mu_0 = S_0 = 0)
+ *     V = S + n_eps   (S is the unnormalised sum of squared deviations; n_eps = cols * eps)
+ *   quantizer: level = Qn + number of references t with  copysign(d*d, d) > V * refs[col][t],
+ *     d = x - mu (negated where flip[col] != 0).  This decides (x-mu)/sigma*gamma+beta > (k - 1/2)*step
+ *     for k = Qn+1 .. Qp when the caller supplies refs[col][t] = sgn(c) c^2 / cols with
+ *     c = ((k - 1/2) step - beta_col) / gamma_col (negated where gamma_col < 0, and then flip[col] = 1).
+ * x: device fp32 [rows, ldx], 16-byte aligned, ldx a multiple of 4, finite values.  refs: device fp32
+ * [cols][2^bits - 1], ascending along t (the bisection in the kernel relies on it).  flip: device bytes
+ * [cols] or NULL (no negative gain).  n_eps > 0.  out: codes [rows, cols] of 2, 3 or 4 bits in any
+ * container, cols a multiple of 4; padding bytes up to the pitch are written as zero.  stats: device fp32
+ * [rows][2], receives (mu, V) of every row (it also carries them from the first kernel to the second).
+ * Returns VITINT_ERR_UNSUPPORTED for 8-bit codes, VITINT_ERR_ALIGNMENT / VITINT_ERR_INVALID_ARG otherwise.
+ * Asynchronous on `stream`; nothing is allocated. */
+int vitint_layernorm_compare_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, const float* refs,
+                                      const uint8_t* flip, float n_eps, const vitint_codes* out, float* stats,
+                                      void* stream);
+
 #ifdef __cplusplus
 }
 #endif

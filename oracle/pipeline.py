@@ -110,20 +110,28 @@ def attention_block(x_codes, s_x, prm: dict, batch: int, tokens: int, heads: int
 
 
 def encoder_layer(x, prm: dict, batch: int, tokens: int, heads: int, bits: int, head_dim: int = 64,
-                  eps: float = 1e-6, softmax: str = "exp") -> dict:
-    """LN1 -> quantize -> attention (+residual) -> LN2 -> quantize -> fc1 -> GELU -> quantize -> fc2 (+residual)."""
+                  eps: float = 1e-6, softmax: str = "exp", layernorm: str = "fp32") -> dict:
+    """LN1 -> quantize -> attention (+residual) -> LN2 -> quantize -> fc1 -> GELU -> quantize -> fc2 (+residual).
+    layernorm="compare": both LayerNorm + quantize stages run as Eq. 5 statistics with the comparator quantizer of
+    Fig. 5(b); their levels are then unique (the band collapses to the code itself)."""
     st: dict = {}
-    y1, tol1 = vo.layernorm(x, prm["ln1_g"], prm["ln1_b"], eps)
-    st["ln1"], st["ln1_tol"] = y1, tol1
-    st["x1_codes"], st["x1_lo"], st["x1_hi"] = vo.quantize_band(y1, tol1, prm["s_ln"], bits, True)
+
+    def ln_quant(v, g, b, tag):
+        if layernorm == "compare":
+            ref, neg, flip = vo.layernorm_references(prm[g], prm[b], prm["s_ln"], bits, True, v.shape[1])
+            q = vo.layernorm_compare_quantize(v, ref, neg, flip, eps, bits, True)
+            return q, q, q
+        y, tol = vo.layernorm(v, prm[g], prm[b], eps)
+        st[tag], st[tag + "_tol"] = y, tol
+        return vo.quantize_band(y, tol, prm["s_ln"], bits, True)
+
+    st["x1_codes"], st["x1_lo"], st["x1_hi"] = ln_quant(x, "ln1_g", "ln1_b", "ln1")
     att = attention_block(st["x1_codes"], prm["s_ln"], prm, batch, tokens, heads, bits, head_dim, "dequant", x,
                           softmax=softmax)
     st["attn"] = att
     h = att["out"]
     st["h"] = h
-    y2, tol2 = vo.layernorm(h, prm["ln2_g"], prm["ln2_b"], eps)
-    st["ln2"], st["ln2_tol"] = y2, tol2
-    st["x2_codes"], st["x2_lo"], st["x2_hi"] = vo.quantize_band(y2, tol2, prm["s_ln"], bits, True)
+    st["x2_codes"], st["x2_lo"], st["x2_hi"] = ln_quant(h, "ln2_g", "ln2_b", "ln2")
     w_fc1 = vo.quantize(prm["w_fc1"], 0.0, bits, True, row_steps=prm["s_w_fc1"])
     w_fc2 = vo.quantize(prm["w_fc2"], 0.0, bits, True, row_steps=prm["s_w_fc2"])
     st["w_fc1_codes"], st["w_fc2_codes"] = w_fc1, w_fc2

@@ -84,6 +84,8 @@ def lib():
         L.vitint_attention_block.argtypes = [POINTER(_Codes), POINTER(_AttentionDesc), c_void_p, c_int64,
                                              POINTER(_Codes), POINTER(_Codes), POINTER(_Codes), c_void_p, c_size_t,
                                              c_void_p]
+        L.vitint_layernorm_compare_quantize.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_float,
+                                                        POINTER(_Codes), c_void_p, c_void_p]
         L.vitint_layernorm_quantize.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_float,
                                                 c_float, POINTER(_Codes), c_void_p, c_int64, c_void_p]
         _lib = L
@@ -207,6 +209,23 @@ def fold_requant(s_x, s_w, bias, s_out):
     alpha = (float(s_x) * s_w64 / s_out64).astype(np.float32)
     beta = np.zeros_like(alpha) if bias is None else (np.asarray(bias, np.float64) / s_out64).astype(np.float32)
     return alpha, beta
+
+
+def fold_layernorm_references(gamma, beta, step, bits: int, signed: bool, cols: int):
+    """Host-side parameter preparation for vitint_layernorm_compare_quantize (Fig. 5(b)): the signed
+    references sgn(c) c^2 / cols, c = ((k - 1/2) step - beta) / gamma for k = Qn+1 .. Qp (fp64, one rounding),
+    with c negated for columns of negative gain, and the per-column flip flags.  Returns (refs fp32
+    [cols, 2^bits - 1], flip uint8 [cols])."""
+    qn = -(1 << (bits - 1)) if signed else 0
+    qp = (1 << (bits - 1)) - 1 if signed else (1 << bits) - 1
+    g = np.asarray(gamma, dtype=np.float64).reshape(-1, 1)
+    b = np.asarray(beta, dtype=np.float64).reshape(-1, 1)
+    k = np.arange(qn + 1, qp + 1, dtype=np.float64).reshape(1, -1)
+    c = ((k - 0.5) * float(step) - b) / g
+    flip = g[:, 0] < 0
+    c[flip] = -c[flip]
+    refs = (np.sign(c) * c * c / float(cols)).astype(np.float32)
+    return np.ascontiguousarray(refs), np.ascontiguousarray(flip.astype(np.uint8))
 
 
 # ---------------------------------------------------------------------------
@@ -391,3 +410,17 @@ def vitint_layernorm_quantize(x: torch.Tensor, gamma: torch.Tensor, beta: torch.
                                            float(eps), float(step), byref(d), _ptr(y), cols if want_y else 0,
                                            _stream()), "vitint_layernorm_quantize")
     return (out, y) if want_y else out
+
+
+def vitint_layernorm_compare_quantize(x: torch.Tensor, refs: torch.Tensor, flip: torch.Tensor | None, n_eps: float,
+                                      bits: int, signed: bool = True, out: Codes | None = None,
+                                      stats: torch.Tensor | None = None):
+    """Eq. 5 running statistics + the comparator quantizer of Fig. 5(b).  Returns (codes, stats [rows, 2])."""
+    rows, cols = x.shape
+    out = Codes.empty(rows, cols, bits, signed, x.device) if out is None else out
+    stats = torch.empty((rows, 2), dtype=torch.float32, device=x.device) if stats is None else stats
+    d = out.desc()
+    _check(lib().vitint_layernorm_compare_quantize(x.data_ptr(), rows, cols, _ld(x), refs.data_ptr(), _ptr(flip),
+                                                   float(n_eps), byref(d), stats.data_ptr(), _stream()),
+           "vitint_layernorm_compare_quantize")
+    return out, stats

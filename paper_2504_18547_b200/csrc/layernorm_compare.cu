@@ -1,0 +1,178 @@
+// Quantizing LayerNorm of Section IV-C: the running statistics of Eq. 5 and the division- and
+// square-root-free comparator of Fig. 5(b), as two kernels.
+//
+//   ln_running_stats_kernel    one thread per row walks the row in order:
+//                                delta = x_i - mu;  mu += delta / i;  S += delta * (x_i - mu)
+//                              every operation a single round-to-nearest fp32 one (no contraction), the
+//                              division by i exact-rounded through a reciprocal and one correction step.
+//                              Writes (mu, V = S + n*eps) per row.
+//   ln_compare_quantize_kernel level = Qn + number of references exceeded.  With d = x - mu (negated where
+//                              gamma < 0) the sign logic of the figure collapses into one comparison of
+//                              signed squares,  copysign(d*d, d) > V * r,  r = sgn(c) c^2 / n the caller's
+//                              signed reference.  The references of a column ascend, fp32 multiplication
+//                              by V > 0 keeps their order, so the comparisons are true up to some index
+//                              and false after it: the count is found by bisection (b comparisons for
+//                              2^b - 1 references) with the candidate references kept in registers.
+#include "common.cuh"
+
+namespace vitint {
+namespace {
+
+constexpr int LNC_ROWS_PER_THREAD = 16;
+
+__global__ void __launch_bounds__(32)
+ln_running_stats_kernel(const float* __restrict__ x, int64_t rows, int cols, int64_t ldx, float n_eps,
+                        float* __restrict__ stats) {
+    grid_dependency_wait();        // x may come from the previous kernel of the stream
+    grid_dependency_launch();
+    const int64_t row = (int64_t)blockIdx.x * 32 + threadIdx.x;
+    if (row >= rows) return;
+    const float4* xr = reinterpret_cast<const float4*>(x + row * ldx);
+    const int nv = cols >> 2;
+    float mu = 0.0f, S = 0.0f;
+    // one 128-byte line of the row (eight 16-byte loads) is requested while the previous one is walked
+    float4 cur[8], nxt[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) cur[k] = k < nv ? __ldg(xr + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int v0 = 0; v0 < nv; v0 += 8) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) nxt[k] = v0 + 8 + k < nv ? __ldg(xr + v0 + 8 + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (v0 + k < nv) {
+                const float e[4] = {cur[k].x, cur[k].y, cur[k].z, cur[k].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float fi = (float)(4 * (v0 + k) + j + 1);
+                    const float r = __frcp_rn(fi);                    // off the dependent chain
+                    const float delta = __fadd_rn(e[j], -mu);
+                    // RN(delta / i): q0 = RN(delta*r), remainder exact in one FMA, one correction
+                    const float q0 = __fmul_rn(delta, r);
+                    const float rem = __fmaf_rn(-q0, fi, delta);
+                    const float q = __fmaf_rn(rem, r, q0);
+                    mu = __fadd_rn(mu, q);
+                    S = __fadd_rn(S, __fmul_rn(delta, __fadd_rn(e[j], -mu)));
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) cur[k] = nxt[k];
+    }
+    stats[2 * row] = mu;
+    stats[2 * row + 1] = __fadd_rn(S, n_eps);
+}
+
+// Block (32, 4): lane = four adjacent columns, threadIdx.y = a group of LNC_ROWS_PER_THREAD rows.
+template <int BITS, int C>
+__global__ void __launch_bounds__(128)
+ln_compare_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, int64_t ldx,
+                           const float* __restrict__ refs, const uint8_t* __restrict__ flip,
+                           const float* __restrict__ stats, uint8_t* __restrict__ out, int64_t pitch, int qn) {
+    grid_dependency_wait();
+    grid_dependency_launch();
+    constexpr int NT = (1 << BITS) - 1;
+    constexpr int LANES_PER_WORD = 8 / C;                       // lanes whose 4 codes share one 32-bit word
+    const int lane = threadIdx.x;
+    const int col = (blockIdx.x * 32 + lane) * 4;
+    const bool col_ok = col < cols;                             // cols is a multiple of 4
+    float r[4][NT];
+    float sgn[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        sgn[j] = (col_ok && flip && flip[col + j]) ? -1.0f : 1.0f;
+#pragma unroll
+        for (int t = 0; t < NT; ++t) r[j][t] = col_ok ? __ldg(refs + (int64_t)(col + j) * NT + t) : 0.0f;
+    }
+    const int words_per_row = (int)(pitch / 4);
+    const int word = (blockIdx.x * 32 + lane) / LANES_PER_WORD;
+    const int64_t row0 = ((int64_t)blockIdx.y * 4 + threadIdx.y) * LNC_ROWS_PER_THREAD;
+    for (int rr = 0; rr < LNC_ROWS_PER_THREAD; ++rr) {
+        const int64_t row = row0 + rr;
+        if (row >= rows) break;                                  // uniform across the warp
+        const float mu = __ldg(stats + 2 * row), V = __ldg(stats + 2 * row + 1);
+        const float4 xv = col_ok ? __ldg(reinterpret_cast<const float4*>(x + row * ldx + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float e[4] = {xv.x, xv.y, xv.z, xv.w};
+        uint32_t bits = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float d = __fmul_rn(__fadd_rn(e[j], -mu), sgn[j]);        // exact sign change
+            const float ds = copysignf(__fmul_rn(d, d), d);
+            float cand[NT > 1 ? NT / 2 : 1];
+            int cnt = 0;
+            {
+                constexpr int half = (NT + 1) / 2;
+                const bool p = ds > __fmul_rn(V, r[j][half - 1]);
+                cnt = p ? half : 0;
+#pragma unroll
+                for (int i = 0; i < half - 1; ++i) cand[i] = p ? r[j][i + half] : r[j][i];
+            }
+#pragma unroll
+            for (int half = (NT + 1) / 4; half >= 1; half >>= 1) {
+                const bool p = ds > __fmul_rn(V, cand[half - 1]);
+                cnt += p ? half : 0;
+#pragma unroll
+                for (int i = 0; i < half - 1; ++i) cand[i] = p ? cand[i + half] : cand[i];
+            }
+            bits |= ((uint32_t)(qn + cnt) & ((1u << C) - 1u)) << (C * j);
+        }
+        if (!col_ok) bits = 0;
+        // gather 8/C neighbouring lanes into one 32-bit word
+        if (C == 4) {
+            bits |= __shfl_xor_sync(0xffffffffu, bits, 1) << 16;
+        } else if (C == 2) {
+            bits |= __shfl_xor_sync(0xffffffffu, bits, 1) << 8;
+            bits |= __shfl_xor_sync(0xffffffffu, bits, 2) << 16;
+        }
+        if ((lane % LANES_PER_WORD) == 0 && word < words_per_row)
+            *reinterpret_cast<uint32_t*>(out + row * pitch + (int64_t)word * 4) = bits;
+    }
+}
+
+template <int BITS>
+int launch_ln_compare(int c, dim3 grid, cudaStream_t st, const float* x, int64_t rows, int cols, int64_t ldx,
+                      const float* refs, const uint8_t* flip, const float* stats, uint8_t* out, int64_t pitch, int qn) {
+    const dim3 block(32, 4);
+    if (c == 2)
+        launch_kernel(ln_compare_quantize_kernel<BITS, 2>, grid, block, 0, st, x, rows, cols, ldx, refs, flip, stats, out, pitch, qn);
+    else if (c == 4)
+        launch_kernel(ln_compare_quantize_kernel<BITS, 4>, grid, block, 0, st, x, rows, cols, ldx, refs, flip, stats, out, pitch, qn);
+    else
+        launch_kernel(ln_compare_quantize_kernel<BITS, 8>, grid, block, 0, st, x, rows, cols, ldx, refs, flip, stats, out, pitch, qn);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+}  // namespace vitint
+
+using namespace vitint;
+
+extern "C" int vitint_layernorm_compare_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx,
+                                                 const float* refs, const uint8_t* flip, float n_eps,
+                                                 const vitint_codes* out, float* stats, void* stream) {
+    if (!x || !refs || !out || !stats) return VITINT_ERR_INVALID_ARG;
+    if (int rc = check_codes(out)) return rc;
+    if (rows <= 0 || cols <= 0 || ldx < cols || out->rows != rows || out->cols != cols) return VITINT_ERR_INVALID_ARG;
+    if (!(n_eps > 0.0f && n_eps < INFINITY)) return VITINT_ERR_INVALID_ARG;
+    if (out->bits == 8 || cols % 4 != 0 || cols > (1 << 22)) return VITINT_ERR_UNSUPPORTED;
+    if (!aligned16(x) || ldx % 4 != 0 || (reinterpret_cast<uintptr_t>(stats) & 7u) != 0) return VITINT_ERR_ALIGNMENT;
+    const int c = codes_container(out);
+    // one lane covers four columns; with sub-byte containers 8/c lanes share an output word, and the words up
+    // to the pitch are written (as zero) by the lanes past the last column
+    const int64_t lanes_cols = cols / 4, lanes_pitch = (out->pitch_bytes / 4) * (8 / c);
+    const int64_t lanes = lanes_cols > lanes_pitch ? lanes_cols : lanes_pitch;
+    int qn, qp;
+    code_range(out->bits, out->is_signed, &qn, &qp);
+    cudaStream_t st = (cudaStream_t)stream;
+    launch_kernel(ln_running_stats_kernel, dim3((unsigned)((rows + 31) / 32)), dim3(32), 0, st, x, rows, (int)cols, ldx,
+                  n_eps, stats);
+    if (int rc = cuda_status(cudaGetLastError())) return rc;
+    const int64_t row_groups = (rows + 4 * LNC_ROWS_PER_THREAD - 1) / (4 * LNC_ROWS_PER_THREAD);
+    if (row_groups > 65535) return VITINT_ERR_UNSUPPORTED;
+    const dim3 grid((unsigned)((lanes + 31) / 32), (unsigned)row_groups);
+    uint8_t* o = (uint8_t*)out->data;
+    switch (out->bits) {
+        case 2: return launch_ln_compare<2>(c, grid, st, x, rows, (int)cols, ldx, refs, flip, stats, o, out->pitch_bytes, qn);
+        case 3: return launch_ln_compare<3>(c, grid, st, x, rows, (int)cols, ldx, refs, flip, stats, o, out->pitch_bytes, qn);
+        default: return launch_ln_compare<4>(c, grid, st, x, rows, (int)cols, ldx, refs, flip, stats, o, out->pitch_bytes, qn);
+    }
+}

@@ -25,7 +25,7 @@ def _dev(a, device):
 class EncoderLayer:
     def __init__(self, batch: int, tokens: int, heads: int, mlp_dim: int, bits: int, prm: dict, device="cuda",
                  eps: float = 1e-6, widen_weights: bool = True, fused_attention: bool = True,
-                 wide_activations: bool = True, softmax: str = "exp"):
+                 wide_activations: bool = True, softmax: str = "exp", layernorm: str = "fp32"):
         self.batch, self.tokens, self.heads, self.bits, self.eps = batch, tokens, heads, bits, eps
         self.dim = D = heads * 64
         self.mlp_dim = F = mlp_dim
@@ -34,6 +34,10 @@ class EncoderLayer:
         if softmax not in ("exp", "shift"):
             raise ValueError("softmax must be 'exp' (Eq. 3) or 'shift' (Eq. 4 with the comparator quantizer)")
         self.softmax = softmax
+        if layernorm not in ("fp32", "compare"):
+            raise ValueError("layernorm must be 'fp32' (LayerNorm, then round) or 'compare' (Eq. 5 statistics with the "
+                             "division- and square-root-free comparator quantizer)")
+        self.layernorm = layernorm
         # the shift-based softmax is a separate kernel: it runs in the unfused attention pipeline
         self.fused_attention = fused_attention and bits != 8 and tokens <= 256 and softmax == "exp"
         self.stages = STAGES_FUSED if self.fused_attention else STAGES_UNFUSED
@@ -42,6 +46,13 @@ class EncoderLayer:
         self.s_ln, self.s_q, self.s_k, self.s_v = f("s_ln"), f("s_q"), f("s_k"), f("s_v")
         self.s_p, self.s_o, self.s_g = f("s_p"), f("s_o"), f("s_g")
         self.ln1_g, self.ln1_b, self.ln2_g, self.ln2_b = d(prm["ln1_g"]), d(prm["ln1_b"]), d(prm["ln2_g"]), d(prm["ln2_b"])
+        if layernorm == "compare":
+            self.ln_refs = []
+            for gk, bk in (("ln1_g", "ln1_b"), ("ln2_g", "ln2_b")):
+                r, fl = B.fold_layernorm_references(prm[gk], prm[bk], prm["s_ln"], bits, True, D)
+                self.ln_refs.append((d(r), d(fl)))
+            self.n_eps = float(np.float32(np.float64(D) * np.float64(np.float32(eps))))
+            self.ln_stats = torch.empty((M, 2), dtype=torch.float32, device=device)
         # weights: quantized once by the library's own quantizer (per-output-channel steps)
         self.w = {}
         for name in ("qkv", "proj", "fc1", "fc2"):
@@ -94,7 +105,11 @@ class EncoderLayer:
                 events.append(e)
         b, t, h = self.batch, self.tokens, self.heads
         mark()
-        B.vitint_layernorm_quantize(x, self.ln1_g, self.ln1_b, self.eps, self.s_ln, self.bits, True, out=self.x1)
+        if self.layernorm == "compare":
+            B.vitint_layernorm_compare_quantize(x, self.ln_refs[0][0], self.ln_refs[0][1], self.n_eps, self.bits, True,
+                                                out=self.x1, stats=self.ln_stats)
+        else:
+            B.vitint_layernorm_quantize(x, self.ln1_g, self.ln1_b, self.eps, self.s_ln, self.bits, True, out=self.x1)
         mark()
         B.vitint_linear(self.x1, self.s_ln, self.w["qkv"], None, None, self.epi_qkv, out=self.qkv)
         mark()
@@ -114,7 +129,11 @@ class EncoderLayer:
         B.vitint_linear(self.O, self.s_o, self.w["proj"], self.s_w["proj"], self.bias["proj"],
                         B.Epilogue(mode=B.EPI_DEQUANT_F32, residual=x), out=self.h)
         mark()
-        B.vitint_layernorm_quantize(self.h, self.ln2_g, self.ln2_b, self.eps, self.s_ln, self.bits, True, out=self.x2)
+        if self.layernorm == "compare":
+            B.vitint_layernorm_compare_quantize(self.h, self.ln_refs[1][0], self.ln_refs[1][1], self.n_eps, self.bits,
+                                                True, out=self.x2, stats=self.ln_stats)
+        else:
+            B.vitint_layernorm_quantize(self.h, self.ln2_g, self.ln2_b, self.eps, self.s_ln, self.bits, True, out=self.x2)
         mark()
         B.vitint_linear(self.x2, self.s_ln, self.w["fc1"], self.s_w["fc1"], self.bias["fc1"], self.epi_fc1, out=self.g)
         mark()

@@ -227,3 +227,34 @@ def test_twelve_layer_encoder_sampled_images():
     assert vt.vitint_device_status() == 0
     assert rel_rms < 0.25 and corr > 0.97 and ref.std() > 0.5, (rel_rms, corr)
     print(f"12 layers: relative rms difference {rel_rms:.4f}, correlation {corr:.5f}")
+
+
+@pytest.mark.parametrize("bits", [4, 2])
+def test_encoder_layer_comparator_layernorm_and_shift_softmax_bit_exact_up_to_gelu(bits):
+    """With the comparator LayerNorm quantizer (Eq. 5, Fig. 5(b)) and the Eq. 4 softmax no stage before the GELU
+    decides a level after an fp32 island: LayerNorm levels, QKV, P, O, the fp32 residual stream and the second
+    LayerNorm's levels must equal the oracle's bit for bit, for every image and token, with no band."""
+    from paper_2504_18547_b200.encoder import EncoderLayer
+    cfg = si.VIT_BASE_LAYER.with_(batch=2, bits=bits)
+    prm = si.layer_parameters(cfg)
+    x = si.activations(cfg)
+    st = vp.encoder_layer(x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits, softmax="shift", layernorm="compare")
+    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, softmax="shift",
+                         layernorm="compare")
+    out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
+    layer.forward(dev(x), out)
+    assert vt.vitint_device_status() == 0
+    T, H = cfg.tokens, cfg.heads
+    g = gpu_stages(layer, out, range(cfg.batch), T, H)
+    att = st["attn"]
+    assert np.array_equal(g["x1"], st["x1_codes"])
+    assert np.array_equal(g["qkv"], att["qkv_codes"])
+    assert np.array_equal(g["P"], att["p_codes"])
+    assert np.array_equal(g["O"], att["o_codes"])
+    assert np.array_equal(g["h"].view(np.uint32), st["h"].view(np.uint32))
+    assert np.array_equal(g["x2"], st["x2_codes"])
+    # GELU is the one remaining fp32 island: its levels stay inside the oracle's band
+    assert np.all(g["g"] >= st["g_lo"]) and np.all(g["g"] <= st["g_hi"])
+    tok = (g["g"] == st["g_codes"]).all(axis=1)
+    assert tok.mean() > 0.5
+    assert np.array_equal(g["out"][tok].view(np.uint32), st["out"][tok].view(np.uint32))

@@ -363,6 +363,47 @@ def test_layernorm_quantize(cols, bits):
     assert padding_is_zero(got)
 
 
+@pytest.mark.parametrize("rows,cols", [(197, 192), (197, 768), (70, 64), (1, 4), (133, 1024), (37, 100)])
+@pytest.mark.parametrize("bits,container", [(4, 0), (4, 8), (3, 0), (2, 0), (2, 8)])
+def test_layernorm_compare_quantize_bit_exact(rows, cols, bits, container):
+    """Eq. 5 statistics + the comparator of Fig. 5(b): single fp32 operations in a fixed order on both
+    sides, so the row statistics and every level are compared bit for bit (no band)."""
+    x = si.normal(900 + cols + rows, (rows, cols), 0.7, 1.9)
+    if rows > 5:
+        x[5] += 50.0                                 # |mean| >> sigma
+        x[3] *= 1e-3
+    g = si.normal(901 + cols, (cols,), 1.0, 0.3)
+    g[cols // 3] = -0.8                               # a negative gain flips the comparison
+    b = si.normal(902 + cols, (cols,), 0.0, 0.3)
+    step = si.gaussian_lsq_step(1.0, bits)
+    eps = 1e-6
+    ref, neg, flip = vo.layernorm_references(g, b, step, bits, True, cols)
+    q_ref, mu_ref, v_ref = vo.layernorm_compare_quantize(x, ref, neg, flip, eps, bits, True, want_stats=True)
+    refs_g, flip_g = vt.fold_layernorm_references(g, b, step, bits, True, cols)
+    # the library's own folding gives the oracle's references (magnitude, sign, flip)
+    assert np.array_equal(np.abs(refs_g), ref) and np.array_equal(flip_g, flip)
+    assert np.array_equal(np.signbit(refs_g) & (refs_g != 0), (neg != 0) & (ref != 0))
+    n_eps = float(np.float32(np.float64(cols) * np.float64(np.float32(eps))))
+    out = vt.Codes.empty(rows, cols, bits, True, "cuda", container=container)
+    got, stats = vt.vitint_layernorm_compare_quantize(dev(x), dev(refs_g), dev(flip_g), n_eps, bits, True, out=out)
+    st = stats.cpu().numpy()
+    assert np.array_equal(st[:, 0].view(np.uint32), mu_ref.view(np.uint32))
+    assert np.array_equal(st[:, 1].view(np.uint32), v_ref.view(np.uint32))
+    assert np.array_equal(from_codes(got), q_ref)
+    assert padding_is_zero(got)
+
+
+def test_layernorm_compare_quantize_argument_checks():
+    x = torch.zeros((8, 64), dtype=torch.float32, device="cuda")
+    refs, flip = vt.fold_layernorm_references(np.ones(64), np.zeros(64), 0.5, 4, True, 64)
+    with pytest.raises(vt.VitintError):               # eps must be positive: V > 0 keeps the reference order
+        vt.vitint_layernorm_compare_quantize(x, dev(refs), dev(flip), 0.0, 4, True)
+    with pytest.raises(vt.VitintError):               # 255 references per column are not supported
+        vt.vitint_layernorm_compare_quantize(x, dev(refs), dev(flip), 1e-4, 8, True)
+    with pytest.raises(vt.VitintError):               # columns must come in fours
+        vt.vitint_layernorm_compare_quantize(x[:, :62], dev(refs), dev(flip), 1e-4, 4, True)
+
+
 # ---------------------------------------------------------------------------
 # a7: composed block, staged
 # ---------------------------------------------------------------------------

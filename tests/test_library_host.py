@@ -21,7 +21,7 @@ def test_every_declared_symbol_is_exported(L):
     header = (ROOT / "include" / "vitint.h").read_text()
     names = set(re.findall(r"\b(vitint_[a-z_0-9]+)\s*\(", header))
     assert {"vitint_quantize", "vitint_linear", "vitint_qk", "vitint_pv", "vitint_softmax_quantize",
-            "vitint_attention_block", "vitint_layernorm_quantize"} <= names
+            "vitint_attention_block", "vitint_layernorm_quantize", "vitint_layernorm_compare_quantize"} <= names
     lib = L.lib()
     for n in sorted(names):
         assert hasattr(lib, n), n
