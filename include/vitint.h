@@ -279,7 +279,7 @@ int vitint_layernorm_quantize(const float* x, int64_t rows, int64_t cols, int64_
  * x: device fp32 [rows, ldx], 16-byte aligned, ldx a multiple of 4, finite values.  refs: device fp32
  * [cols][2^bits - 1], ascending along t (the bisection in the kernel relies on it).  flip: device bytes
  * [cols] or NULL (no negative gain).  n_eps > 0.  out: codes [rows, cols] of 2, 3 or 4 bits in any
- * container, cols a multiple of 4; padding bytes up to the pitch are written as zero.  stats: device fp32
+ * container, cols a multiple of 4 and at most 4096; padding bytes up to the pitch are written as zero.  stats: device fp32
  * [rows][2], receives (mu, V) of every row (it also carries them from the first kernel to the second).
  * Returns VITINT_ERR_UNSUPPORTED for 8-bit codes, VITINT_ERR_ALIGNMENT / VITINT_ERR_INVALID_ARG otherwise.
  * Asynchronous on `stream`; nothing is allocated. */

@@ -19,45 +19,89 @@ namespace vitint {
 namespace {
 
 constexpr int LNC_ROWS_PER_THREAD = 16;
+constexpr int LNC_BATCH = 4;            // rows whose loads are issued together
+
+constexpr int LNS_PREFETCH_LINES = 6; // 128-byte lines of a row requested into L2 ahead of the register loads
+constexpr int LNS_MAX_COLS = 4096;    // (float(i), RN(1/i)) pairs tabulated in shared memory
+
+// One step of Eq. 5 for element xi, i = fi: every operation a single rounded fp32 one.  The update of S
+// belonging to the PREVIOUS element (its delta in pd, its value in px; mu is still that element's mean) is
+// written between the operations of this element's dependent chain delta -> quotient -> mu, so the two
+// interleave in issue order; operands and operations are exactly those of the recurrence.
+__device__ __forceinline__ void running_step(float xi, float fi, float r, float& mu, float& S, float& pd, float& px) {
+    const float delta = __fadd_rn(xi, -mu);
+    const float tt = __fadd_rn(px, -mu);
+    // RN(delta / i): q0 = RN(delta*r), remainder exact in one FMA, one correction
+    const float q0 = __fmul_rn(delta, r);
+    const float pp = __fmul_rn(pd, tt);
+    const float rem = __fmaf_rn(-q0, fi, delta);
+    S = __fadd_rn(S, pp);
+    const float q = __fmaf_rn(rem, r, q0);
+    mu = __fadd_rn(mu, q);
+    pd = delta;
+    px = xi;
+}
 
 __global__ void __launch_bounds__(32)
 ln_running_stats_kernel(const float* __restrict__ x, int64_t rows, int cols, int64_t ldx, float n_eps,
                         float* __restrict__ stats) {
+    // (float(i), RN(1/i)) for every column: one broadcast shared-memory read per element instead of a
+    // conversion and a reciprocal (both run on the quarter-rate unit) in front of the dependent chain
+    extern __shared__ float2 inv_tab[];
+    for (int i = threadIdx.x; i < cols; i += 32) {
+        const float fi = (float)(i + 1);
+        inv_tab[i] = make_float2(fi, __frcp_rn(fi));
+    }
+    __syncwarp();
     grid_dependency_wait();        // x may come from the previous kernel of the stream
     grid_dependency_launch();
     const int64_t row = (int64_t)blockIdx.x * 32 + threadIdx.x;
     if (row >= rows) return;
     const float4* xr = reinterpret_cast<const float4*>(x + row * ldx);
-    const int nv = cols >> 2;
-    float mu = 0.0f, S = 0.0f;
-    // one 128-byte line of the row (eight 16-byte loads) is requested while the previous one is walked
+    const int nv = cols >> 2, nv_full = nv & ~7;
+    float mu = 0.0f, S = 0.0f, pd = 0.0f, px = 0.0f;
+    // With one thread per row only a few megabytes would be in flight; the lines further ahead are therefore
+    // requested into L2 (one prefetch per 128-byte line), so the register loads below find them there.
+#pragma unroll
+    for (int a = 1; a < 1 + LNS_PREFETCH_LINES; ++a)
+        if (8 * a < nv) asm volatile("prefetch.global.L2 [%0];" ::"l"(xr + 8 * a));
+    // whole 128-byte lines: eight 16-byte loads are requested while the previous line is walked
     float4 cur[8], nxt[8];
+    if (nv_full > 0) {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) cur[k] = k < nv ? __ldg(xr + k) : make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int v0 = 0; v0 < nv; v0 += 8) {
+        for (int k = 0; k < 8; ++k) cur[k] = __ldg(xr + k);
+    }
+    for (int v0 = 0; v0 < nv_full; v0 += 8) {
+        if (v0 + 8 * (1 + LNS_PREFETCH_LINES) < nv)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(xr + v0 + 8 * (1 + LNS_PREFETCH_LINES)));
+        if (v0 + 8 < nv_full) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) nxt[k] = v0 + 8 + k < nv ? __ldg(xr + v0 + 8 + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int k = 0; k < 8; ++k) nxt[k] = __ldg(xr + v0 + 8 + k);
+        }
+        const float2* tab = inv_tab + 4 * v0;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            if (v0 + k < nv) {
-                const float e[4] = {cur[k].x, cur[k].y, cur[k].z, cur[k].w};
+            const float e[4] = {cur[k].x, cur[k].y, cur[k].z, cur[k].w};
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float fi = (float)(4 * (v0 + k) + j + 1);
-                    const float r = __frcp_rn(fi);                    // off the dependent chain
-                    const float delta = __fadd_rn(e[j], -mu);
-                    // RN(delta / i): q0 = RN(delta*r), remainder exact in one FMA, one correction
-                    const float q0 = __fmul_rn(delta, r);
-                    const float rem = __fmaf_rn(-q0, fi, delta);
-                    const float q = __fmaf_rn(rem, r, q0);
-                    mu = __fadd_rn(mu, q);
-                    S = __fadd_rn(S, __fmul_rn(delta, __fadd_rn(e[j], -mu)));
-                }
+            for (int j = 0; j < 4; ++j) {
+                const float2 t = tab[4 * k + j];
+                running_step(e[j], t.x, t.y, mu, S, pd, px);
             }
         }
 #pragma unroll
         for (int k = 0; k < 8; ++k) cur[k] = nxt[k];
     }
+    // the last, partial line
+    for (int v = nv_full; v < nv; ++v) {
+        const float4 c4 = __ldg(xr + v);
+        const float e[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 t = inv_tab[4 * v + j];
+            running_step(e[j], t.x, t.y, mu, S, pd, px);
+        }
+    }
+    S = __fadd_rn(S, __fmul_rn(pd, __fadd_rn(px, -mu)));      // the last element's term
     stats[2 * row] = mu;
     stats[2 * row + 1] = __fadd_rn(S, n_eps);
 }
@@ -86,11 +130,31 @@ ln_compare_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, 
     const int words_per_row = (int)(pitch / 4);
     const int word = (blockIdx.x * 32 + lane) / LANES_PER_WORD;
     const int64_t row0 = ((int64_t)blockIdx.y * 4 + threadIdx.y) * LNC_ROWS_PER_THREAD;
-    for (int rr = 0; rr < LNC_ROWS_PER_THREAD; ++rr) {
-        const int64_t row = row0 + rr;
+    // Rows go in batches of LNC_BATCH: the loads of the next batch are in flight while this batch's levels are
+    // found (a single row per thread would leave too few bytes in flight to keep HBM busy).
+    float4 xb[LNC_BATCH], xb_next[LNC_BATCH];
+    float2 mb[LNC_BATCH], mb_next[LNC_BATCH];
+    auto load_batch = [&](int64_t first, float4 (&xv)[LNC_BATCH], float2 (&mv)[LNC_BATCH]) {
+#pragma unroll
+        for (int k = 0; k < LNC_BATCH; ++k) {
+            const int64_t row = first + k;
+            const bool ok = row < rows && row < row0 + LNC_ROWS_PER_THREAD;
+            mv[k] = ok ? __ldg(reinterpret_cast<const float2*>(stats) + row) : make_float2(0.f, 1.f);
+            xv[k] = (ok && col_ok) ? __ldg(reinterpret_cast<const float4*>(x + row * ldx + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    load_batch(row0, xb_next, mb_next);
+    for (int rb = 0; rb < LNC_ROWS_PER_THREAD; rb += LNC_BATCH) {
+        if (row0 + rb >= rows) break;                            // uniform across the warp
+#pragma unroll
+        for (int k = 0; k < LNC_BATCH; ++k) { xb[k] = xb_next[k]; mb[k] = mb_next[k]; }
+        load_batch(row0 + rb + LNC_BATCH, xb_next, mb_next);
+#pragma unroll
+      for (int k = 0; k < LNC_BATCH; ++k) {
+        const int64_t row = row0 + rb + k;
         if (row >= rows) break;                                  // uniform across the warp
-        const float mu = __ldg(stats + 2 * row), V = __ldg(stats + 2 * row + 1);
-        const float4 xv = col_ok ? __ldg(reinterpret_cast<const float4*>(x + row * ldx + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 xv = xb[k];
+        const float mu = mb[k].x, V = mb[k].y;
         const float e[4] = {xv.x, xv.y, xv.z, xv.w};
         uint32_t bits = 0;
 #pragma unroll
@@ -125,6 +189,7 @@ ln_compare_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, 
         }
         if ((lane % LANES_PER_WORD) == 0 && word < words_per_row)
             *reinterpret_cast<uint32_t*>(out + row * pitch + (int64_t)word * 4) = bits;
+      }
     }
 }
 
@@ -153,7 +218,7 @@ extern "C" int vitint_layernorm_compare_quantize(const float* x, int64_t rows, i
     if (int rc = check_codes(out)) return rc;
     if (rows <= 0 || cols <= 0 || ldx < cols || out->rows != rows || out->cols != cols) return VITINT_ERR_INVALID_ARG;
     if (!(n_eps > 0.0f && n_eps < INFINITY)) return VITINT_ERR_INVALID_ARG;
-    if (out->bits == 8 || cols % 4 != 0 || cols > (1 << 22)) return VITINT_ERR_UNSUPPORTED;
+    if (out->bits == 8 || cols % 4 != 0 || cols > LNS_MAX_COLS) return VITINT_ERR_UNSUPPORTED;
     if (!aligned16(x) || ldx % 4 != 0 || (reinterpret_cast<uintptr_t>(stats) & 7u) != 0) return VITINT_ERR_ALIGNMENT;
     const int c = codes_container(out);
     // one lane covers four columns; with sub-byte containers 8/c lanes share an output word, and the words up
@@ -163,7 +228,7 @@ extern "C" int vitint_layernorm_compare_quantize(const float* x, int64_t rows, i
     int qn, qp;
     code_range(out->bits, out->is_signed, &qn, &qp);
     cudaStream_t st = (cudaStream_t)stream;
-    launch_kernel(ln_running_stats_kernel, dim3((unsigned)((rows + 31) / 32)), dim3(32), 0, st, x, rows, (int)cols, ldx,
+    launch_kernel(ln_running_stats_kernel, dim3((unsigned)((rows + 31) / 32)), dim3(32), (size_t)cols * sizeof(float2), st, x, rows, (int)cols, ldx,
                   n_eps, stats);
     if (int rc = cuda_status(cudaGetLastError())) return rc;
     const int64_t row_groups = (rows + 4 * LNC_ROWS_PER_THREAD - 1) / (4 * LNC_ROWS_PER_THREAD);
