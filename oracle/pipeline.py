@@ -109,6 +109,51 @@ def attention_block(x_codes, s_x, prm: dict, batch: int, tokens: int, heads: int
     return st
 
 
+def normed_attention(x_codes, s_x, prm: dict, qkn: dict, batch: int, tokens: int, heads: int, bits: int,
+                     head_dim: int = 64, eps: float = 1e-6) -> dict:
+    """The self-attention module as the paper's power table lays it out (Section V-B): separate Q, K and V linear
+    layers; Q and K pass a LayerNorm over each head's channels whose quantizer is the comparator of Fig. 5(b)
+    (statistics by Eq. 5); V is requantized directly; Q K^T; the Eq. 4 softmax with its division-free
+    quantizer; P V, requantized.  No level is decided after a floating-point island, so every stage is unique."""
+    D = heads * head_dim
+    M = batch * tokens
+    st: dict = {}
+    w = vo.quantize(prm["w_qkv"], 0.0, bits, True, row_steps=prm["s_w_qkv"])
+    st["w_qkv_codes"] = w
+    for i, name in enumerate(("q", "k")):
+        sl = slice(i * D, (i + 1) * D)
+        acc = vo.matmul_i32(x_codes, w[sl])
+        y = vo.epilogue_dequant(acc, s_x, prm["s_w_qkv"][sl], prm["b_qkv"][sl])
+        st[name + "_f32"] = y
+        ref, neg, flip = vo.layernorm_references(qkn[name + "n_g"], qkn[name + "n_b"], qkn["s_" + name + "n"], bits,
+                                                 True, head_dim)
+        st[name + "_refs"] = (ref, neg, flip)
+        codes, mu, v = vo.layernorm_compare_quantize(y.reshape(M * heads, head_dim), ref, neg, flip, eps, bits, True,
+                                                     want_stats=True)
+        st[name + "_codes"] = codes.reshape(M, D)
+        st[name + "_stats"] = np.stack([mu, v], axis=1)
+    sl = slice(2 * D, 3 * D)
+    a_v, b_v = fold(s_x, prm["s_w_qkv"][sl], prm["b_qkv"][sl], prm["s_v"])
+    st["alpha_v"], st["beta_v"] = a_v, b_v
+    st["v_codes"] = vo.epilogue_requant(vo.matmul_i32(x_codes, w[sl]), a_v, b_v, bits, True)
+    q = split_heads(st["q_codes"], batch, tokens, heads, head_dim, 0)
+    k = split_heads(st["k_codes"], batch, tokens, heads, head_dim, 0)
+    v = split_heads(st["v_codes"], batch, tokens, heads, head_dim, 0)
+    st["S"] = vo.qk(q, k)
+    c = softmax_scale(qkn["s_qn"], qkn["s_kn"], head_dim)
+    c2 = np.float32(np.float64(c) * np.log2(np.e))
+    st["c"], st["c2"] = c, c2
+    n = batch * heads
+    st["p_codes"] = vo.softmax_shift_quantize(st["S"].reshape(n * tokens, tokens), c2, prm["s_p"], bits).reshape(
+        n, tokens, tokens)
+    st["acc_o"] = vo.pv(st["p_codes"], v)
+    a_o, b_o = fold(prm["s_p"], np.full(head_dim, prm["s_v"], np.float32), None, prm["s_o"])
+    st["alpha_o"] = a_o
+    o_slabs = vo.epilogue_requant(st["acc_o"].reshape(n * tokens, head_dim), a_o, b_o, bits, True)
+    st["o_codes"] = merge_heads(o_slabs.reshape(n, tokens, head_dim), batch, tokens, heads, head_dim)
+    return st
+
+
 def encoder_layer(x, prm: dict, batch: int, tokens: int, heads: int, bits: int, head_dim: int = 64,
                   eps: float = 1e-6, softmax: str = "exp", layernorm: str = "fp32") -> dict:
     """LN1 -> quantize -> attention (+residual) -> LN2 -> quantize -> fc1 -> GELU -> quantize -> fc2 (+residual).

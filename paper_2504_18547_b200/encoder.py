@@ -181,3 +181,75 @@ class EncoderStack:
 
     def ops(self) -> int:
         return sum(sum(v for k, v in l.stage_ops().items() if k in l.stages) for l in self.layers)
+
+
+class NormedAttention:
+    """The self-attention module laid out as in the paper's power table (Section V-B): separate Q, K and V
+    linear layers, a LayerNorm over each head's 64 channels in front of the Q and K quantizers (statistics by
+    Eq. 5, comparator quantizer of Fig. 5(b)), Q K^T, the Eq. 4 softmax with its division-free quantizer, P V.
+    A fixed sequence of C-ABI calls over preallocated buffers; `qkn` holds the per-head LayerNorm parameters
+    (qn_g, qn_b, kn_g, kn_b over 64 channels) and the steps s_qn, s_kn of the normalised values."""
+
+    def __init__(self, batch: int, tokens: int, heads: int, bits: int, prm: dict, qkn: dict, device="cuda",
+                 eps: float = 1e-6):
+        self.batch, self.tokens, self.heads, self.bits = batch, tokens, heads, bits
+        self.dim = D = heads * 64
+        self.rows = M = batch * tokens
+        d = lambda a: _dev(a, device)
+        w = B.vitint_widen(B.vitint_quantize(d(prm["w_qkv"]), 0.0, bits, True, row_steps=d(prm["s_w_qkv"])))
+        part = lambda i: B.Codes(w.data[i * D:(i + 1) * D], D, D, bits, True, 8)
+        self.w_q, self.w_k, self.w_v = part(0), part(1), part(2)
+        self.s_w = [d(prm["s_w_qkv"][i * D:(i + 1) * D]) for i in range(2)]
+        self.bias = [d(prm["b_qkv"][i * D:(i + 1) * D]) for i in range(2)]
+        a, b = B.fold_requant(1.0, prm["s_w_qkv"][2 * D:], prm["b_qkv"][2 * D:], prm["s_v"])
+        self._alpha_v_unit, self.beta_v = a, d(b)             # alpha scales with the input step given to forward()
+        self.refs = []
+        for n in ("q", "k"):
+            r, fl = B.fold_layernorm_references(qkn[n + "n_g"], qkn[n + "n_b"], qkn["s_" + n + "n"], bits, True, 64)
+            self.refs.append((d(r), d(fl)))
+        self.n_eps = float(np.float32(np.float64(64) * np.float64(np.float32(eps))))
+        self.s_v, self.s_p, self.s_o = float(prm["s_v"]), float(prm["s_p"]), float(prm["s_o"])
+        c = np.float32(float(qkn["s_qn"]) * float(qkn["s_kn"]) / 8.0)
+        self.c2 = float(np.float32(np.float64(c) * np.log2(np.e)))
+        a_o, _ = B.fold_requant(prm["s_p"], np.full(D, prm["s_v"], np.float32), None, prm["s_o"])
+        self.alpha_o = d(a_o)
+        self._prm = prm
+        self._alpha_v_for = None
+        c_bits = 4 if bits == 3 else bits
+        self.f32 = [torch.empty((M, D), dtype=torch.float32, device=device) for _ in range(2)]
+        self.qk_codes = [B.Codes.empty(M * heads, 64, bits, True, device) for _ in range(2)]
+        self.stats = [torch.empty((M * heads, 2), dtype=torch.float32, device=device) for _ in range(2)]
+        pitch = D * c_bits // 8
+        self.slabs = [B.Slabs(c.data, 0, pitch, pitch * tokens, 64 * c_bits // 8, bits, True) for c in self.qk_codes]
+        self.v = B.Codes.empty(M, D, bits, True, device)
+        self.v_slabs = B.Slabs(self.v.data, 0, self.v.pitch, self.v.pitch * tokens, 64 * c_bits // 8, bits, True)
+        self.ld_s = (tokens + 3) // 4 * 4
+        self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
+        self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
+        self.O = B.Codes.empty(M, D, bits, True, device)
+        self.epi_o = B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_o, out_bits=bits, out_signed=True)
+
+    def forward(self, x: "B.Codes", s_x: float) -> "B.Codes":
+        """x: codes [batch*tokens, dim] with step s_x.  Returns the O codes [batch*tokens, dim]."""
+        if self._alpha_v_for != float(s_x):
+            D = self.dim
+            a, _ = B.fold_requant(s_x, self._prm["s_w_qkv"][2 * D:], None, self._prm["s_v"])
+            self.alpha_v = _dev(a, self.O.data.device)
+            self._alpha_v_for = float(s_x)
+        b, t, h = self.batch, self.tokens, self.heads
+        for i, w in enumerate((self.w_q, self.w_k)):
+            B.vitint_linear(x, s_x, w, self.s_w[i], self.bias[i], B.Epilogue(mode=B.EPI_DEQUANT_F32), out=self.f32[i])
+            B.vitint_layernorm_compare_quantize(self.f32[i].view(self.rows * h, 64), self.refs[i][0], self.refs[i][1],
+                                                self.n_eps, self.bits, True, out=self.qk_codes[i], stats=self.stats[i])
+        B.vitint_linear(x, s_x, self.w_v, None, None,
+                        B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_v, beta=self.beta_v, out_bits=self.bits,
+                                   out_signed=True), out=self.v)
+        B.vitint_qk(self.slabs[0], self.slabs[1], b, h, t, out=self.S, ld_s=self.ld_s)
+        B.vitint_softmax_shift_quantize(self.S, t, self.c2, self.s_p, self.bits, out=self.P)
+        B.vitint_pv(self.P, self.v_slabs, b, h, t, self.s_p, self.s_v, self.epi_o, out=self.O)
+        return self.O
+
+    def ops(self) -> int:
+        """Integer operations (2 per multiply-accumulate) of the five contractions."""
+        M, D, T = self.rows, self.dim, self.tokens
+        return 2 * (3 * M * D * D + 2 * self.batch * self.heads * T * T * 64)

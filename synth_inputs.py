@@ -144,7 +144,10 @@ VIT_TINY_BLOCK = BlockConfig("vit_tiny_attn_b1", 1, 197, 192, 3, 4, seed_index=1
 VIT_SMALL_BLOCK = BlockConfig("vit_small_attn_b64", 64, 197, 384, 6, 4, outlier_frac=0.01, seed_index=2)
 VIT_BASE_LAYER = BlockConfig("vit_base_layer_b128", 128, 197, 768, 12, 4, mlp_dim=3072, seed_index=3)
 VIT_BASE_ENCODER = BlockConfig("vit_base_12layer_b256", 256, 197, 768, 12, 4, mlp_dim=3072, layers=12, seed_index=4)
-CONFIGS = {c.name: c for c in (VIT_TINY_BLOCK, VIT_SMALL_BLOCK, VIT_BASE_LAYER, VIT_BASE_ENCODER)}
+# The self-attention module of the paper's power table: DeiT-S width, 198 tokens (class + distillation + 196
+# patches), 3-bit, with a LayerNorm over each head's 64 channels in front of the Q and K quantizers.
+DEIT_S_ATTENTION = BlockConfig("deit_s_attn_n198_b64", 64, 198, 384, 6, 3, seed_index=5)
+CONFIGS = {c.name: c for c in (VIT_TINY_BLOCK, VIT_SMALL_BLOCK, VIT_BASE_LAYER, VIT_BASE_ENCODER, DEIT_S_ATTENTION)}
 
 
 def activations(cfg: BlockConfig, batch: int | None = None, first_image: int = 0) -> np.ndarray:
@@ -214,6 +217,16 @@ def layer_parameters(cfg: BlockConfig, layer: int = 0) -> dict:
         p["s_ln"] = gaussian_lsq_step(1.0, b)
         p["s_g"] = gelu_lsq_step(ws * math.sqrt(D), b, sd("gelu_mc"))
     return p
+
+
+def qk_norm_parameters(cfg: BlockConfig, layer: int = 0) -> dict:
+    """Parameters of the per-head LayerNorm in front of the Q and K quantizers (gain ~ N(1, 0.02), offset
+    ~ N(0, 0.02) over the head's channels, shared by the heads) and the step of the normalised values."""
+    sd = lambda tag: substream(cfg.seed, f"L{layer}/{tag}")
+    d = cfg.head_dim
+    return {"qn_g": normal(sd("qn_g"), (d,), 1.0, 0.02), "qn_b": normal(sd("qn_b"), (d,), 0.0, 0.02),
+            "kn_g": normal(sd("kn_g"), (d,), 1.0, 0.02), "kn_b": normal(sd("kn_b"), (d,), 0.0, 0.02),
+            "s_qn": gaussian_lsq_step(1.0, cfg.bits), "s_kn": gaussian_lsq_step(1.0, cfg.bits)}
 
 
 # ---------------------------------------------------------------------------

@@ -258,3 +258,35 @@ def test_encoder_layer_comparator_layernorm_and_shift_softmax_bit_exact_up_to_ge
     tok = (g["g"] == st["g_codes"]).all(axis=1)
     assert tok.mean() > 0.5
     assert np.array_equal(g["out"][tok].view(np.uint32), st["out"][tok].view(np.uint32))
+
+
+@pytest.mark.parametrize("bits", [3, 4])
+def test_normed_attention_module_bit_exact(bits):
+    """The attention module of the paper's power table at its shapes (198 tokens, 384 channels, 6 heads of 64):
+    Q, K, V linears, per-head comparator LayerNorm on Q and K, Q K^T, Eq. 4 softmax, P V.  Every stage is integer
+    or single-rounding arithmetic, so every buffer equals the oracle's bit for bit."""
+    from paper_2504_18547_b200.encoder import NormedAttention
+    cfg = si.DEIT_S_ATTENTION.with_(batch=2, bits=bits)
+    prm, qkn = si.layer_parameters(cfg), si.qk_norm_parameters(cfg)
+    x = si.activations(cfg)
+    s_x = si.lsq_step(x, cfg.bits, True)
+    xq = vo.quantize(x, s_x, cfg.bits, True)
+    st = vp.normed_attention(xq, s_x, prm, qkn, cfg.batch, cfg.tokens, cfg.heads, cfg.bits)
+    mod = NormedAttention(cfg.batch, cfg.tokens, cfg.heads, cfg.bits, prm, qkn)
+    xg = vt.vitint_quantize(dev(x), float(s_x), cfg.bits, True)
+    O = mod.forward(xg, float(s_x))
+    assert vt.vitint_device_status() == 0
+    M, D, T, H = cfg.rows, cfg.dim, cfg.tokens, cfg.heads
+    for i, n in enumerate(("q", "k")):
+        assert np.array_equal(mod.f32[i].cpu().numpy().view(np.uint32), st[n + "_f32"].view(np.uint32)), n
+        assert np.array_equal(mod.stats[i].cpu().numpy().view(np.uint32), st[n + "_stats"].view(np.uint32)), n
+        assert np.array_equal(from_codes(mod.qk_codes[i]).reshape(M, D), st[n + "_codes"]), n
+    assert np.array_equal(from_codes(mod.v), st["v_codes"])
+    S = mod.S.cpu().numpy()[:, :T].reshape(cfg.batch * H, T, T)
+    assert np.array_equal(S, st["S"])
+    assert np.array_equal(from_codes(mod.P).reshape(-1, T, T), st["p_codes"])
+    assert np.array_equal(from_codes(O), st["o_codes"])
+    # the module's contractions are those of the paper's table: per head 198*384*64 = 4.87 M multiply-accumulates
+    # per linear layer and 198*198*64 = 2.51 M per attention matmul
+    per_image = mod.ops() // (2 * cfg.batch)
+    assert per_image == H * (3 * 198 * 384 * 64 + 2 * 198 * 198 * 64)
