@@ -314,6 +314,19 @@ def run_ours(args, cfg):
             standalone[name] = {"ms": round(ms, 4), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
                                 "frac_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks_early["hbm_gbs"], 4)}
         del S, Pq, xq
+        # the attention module of the paper's power table at its own shapes (DeiT-S width, 198 tokens, 3-bit,
+        # per-head comparator LayerNorm on Q and K, Eq. 4 softmax), batch 64
+        from paper_2504_18547_b200.encoder import NormedAttention
+        dcfg = si.DEIT_S_ATTENTION
+        dprm, dqkn = si.layer_parameters(dcfg), si.qk_norm_parameters(dcfg)
+        mod = NormedAttention(dcfg.batch, dcfg.tokens, dcfg.heads, dcfg.bits, dprm, dqkn, device)
+        dx = torch.from_numpy(si.activations(dcfg)).to(device)
+        ds_x = float(si.lsq_step(dx[:dcfg.tokens].cpu().numpy(), dcfg.bits, True))
+        dxq = vt.vitint_quantize(dx, ds_x, dcfg.bits, True)
+        ms = timed(lambda: mod.forward(dxq, ds_x))
+        standalone["deit_s_attention_n198_b64"] = {"ms": round(ms, 4), "tops": round(mod.ops() / (ms * 1e-3) / 1e12, 1),
+                                                   "images_per_s": round(dcfg.batch / (ms * 1e-3), 1), "launches": 10}
+        del mod, dx, dxq
 
     # ---- CPU oracle on a bounded sample (rank 0, single-GPU runs only) -----------------
     cpu = None
