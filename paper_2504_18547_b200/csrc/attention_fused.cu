@@ -231,6 +231,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
         const int sh_idx = DIRECT ? 0 : 2 * (8 - C) - 2;            // scaled score -> byte offset 4*S
         const int chunks = P.kv_rows / 32;
         const int tab_half = 4 * P.smax;
+        const char* const tab_lo = tab_mid - tab_half;
         const double inv_p_step = 1.0 / (double)P.p_step;
         bool ok = true;
         int n = 0;
@@ -279,10 +280,21 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                         // every table entry is a positive normal float (exp of a bounded argument), so its
                         // double is formed from the bits with two integer operations instead of a conversion
                         // (the conversion unit runs at a quarter of the fp64 adder's rate)
-                        int off = DIRECT ? ((int)v[i] << 2) : ((int)v[i] >> sh_idx);
-                        if (DIRECT) off = max(-tab_half, min(tab_half, off));   // raw bytes: keep any value inside the table
-                        const uint32_t eb = *reinterpret_cast<const uint32_t*>(tab_mid + off);
-                        zp[i & 3] += __hiloint2double((int)((eb >> 3) + 0x38000000u), (int)(eb << 29));
+                        // Integer multiply-adds run beside the compare / shift / permute unit, which is the busier
+                        // one in this kernel: the byte offset, its clamp (one unsigned minimum after biasing) and
+                        // both words of the double are formed with them.
+                        uint32_t eb;
+                        if (DIRECT) {
+                            // raw bytes: 4*S + 4*smax, kept inside the table for any operand value
+                            const uint32_t off = min((uint32_t)((int)v[i] * 4 + tab_half), (uint32_t)(2 * tab_half));
+                            eb = *reinterpret_cast<const uint32_t*>(tab_lo + off);
+                        } else {
+                            eb = *reinterpret_cast<const uint32_t*>(tab_mid + ((int)v[i] >> sh_idx));
+                        }
+                        uint32_t hi, lo;
+                        asm("mad.hi.u32 %0, %1, 536870912, 939524096;" : "=r"(hi) : "r"(eb));    // (eb >> 3) + 0x38000000
+                        asm("mul.lo.u32 %0, %1, 536870912;" : "=r"(lo) : "r"(eb));                // eb << 29
+                        zp[i & 3] += __hiloint2double((int)hi, (int)lo);
                         v[i] = eb;
                     }
                 } else {
