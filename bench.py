@@ -327,6 +327,17 @@ def run_ours(args, cfg):
         standalone["deit_s_attention_n198_b64"] = {"ms": round(ms, 4), "tops": round(mod.ops() / (ms * 1e-3) / 1e12, 1),
                                                    "images_per_s": round(dcfg.batch / (ms * 1e-3), 1), "launches": 10}
         del mod, dx, dxq
+        # the whole DeiT-S-shaped model (patch embedding, 198 tokens, 12 layers, final LayerNorm, two heads), batch 128
+        from paper_2504_18547_b200.encoder import DeitModel
+        mcfg = si.DEIT_S_MODEL
+        model = DeitModel(si.model_end_parameters(mcfg), [si.layer_parameters(mcfg, layer=l) for l in range(mcfg.layers)],
+                          mcfg.batch, mcfg.tokens, mcfg.heads, mcfg.mlp_dim, mcfg.bits, device)
+        mp = torch.from_numpy(si.patch_rows(mcfg, batch=8)).to(device).repeat(mcfg.batch // 8, 1)
+        ms = timed(lambda: model.forward(mp), reps=5)
+        standalone["deit_s_model_n198_b128"] = {"ms": round(ms, 4), "tops": round(model.ops() / (ms * 1e-3) / 1e12, 1),
+                                                "images_per_s": round(mcfg.batch / (ms * 1e-3), 1),
+                                                "launches": 2 + 8 * mcfg.layers + 4}
+        del model, mp
 
     # ---- CPU oracle on a bounded sample (rank 0, single-GPU runs only) -----------------
     cpu = None

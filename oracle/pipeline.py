@@ -199,3 +199,32 @@ def encoder_stack(x, layer_params: list, batch: int, tokens: int, heads: int, bi
         stages.append(st)
         cur = st["out"]
     return stages
+
+
+def deit_forward(patches, ends: dict, layer_params: list, batch: int, tokens: int, heads: int, bits: int,
+                 eps: float = 1e-6, **layer_modes) -> dict:
+    """Whole model: patch embedding as an integerized linear over flattened patches (class / distillation rows are
+    zero) plus the token table, the encoder layers, final LayerNorm + quantizer on the class and distillation
+    rows, two integerized classifier heads whose logits are summed."""
+    st: dict = {}
+    xq = vo.quantize(patches, ends["s_patch"], bits, True)
+    w_pe = vo.quantize(ends["w_pe"], 0.0, bits, True, row_steps=ends["s_w_pe"])
+    table = np.tile(np.asarray(ends["tokens"], np.float32), (batch, 1))
+    st["x0"] = vo.epilogue_dequant(vo.matmul_i32(xq, w_pe), ends["s_patch"], ends["s_w_pe"], ends["b_pe"], table)
+    cur = st["x0"]
+    st["layers"] = []
+    for prm in layer_params:
+        ls = encoder_layer(cur, prm, batch, tokens, heads, bits, eps=eps, **layer_modes)
+        st["layers"].append(ls)
+        cur = ls["out"]
+    st["x_final"] = cur
+    logits = None
+    for name, row in (("head", 0), ("head_dist", 1)):
+        rows = np.ascontiguousarray(cur[row::tokens])
+        y, tol = vo.layernorm(rows, ends["lnf_g"], ends["lnf_b"], eps)
+        q, lo, hi = vo.quantize_band(y, tol, ends["s_lnf"], bits, True)
+        st[name + "_codes"], st[name + "_lo"], st[name + "_hi"] = q, lo, hi
+        w = vo.quantize(ends["w_" + name], 0.0, bits, True, row_steps=ends["s_w_" + name])
+        logits = vo.epilogue_dequant(vo.matmul_i32(q, w), ends["s_lnf"], ends["s_w_" + name], ends["b_" + name], logits)
+    st["logits"] = logits
+    return st

@@ -253,3 +253,51 @@ class NormedAttention:
         """Integer operations (2 per multiply-accumulate) of the five contractions."""
         M, D, T = self.rows, self.dim, self.tokens
         return 2 * (3 * M * D * D + 2 * self.batch * self.heads * T * T * 64)
+
+
+class DeitModel:
+    """The whole DeiT-S-shaped model as C-ABI calls: quantize the flattened patches, patch embedding as an
+    integerized linear whose fp32 epilogue adds the token table (class / distillation tokens and position
+    embeddings; the two token rows of every image carry zero patches), the encoder layers, final LayerNorm +
+    quantizer on the class and distillation rows, two classifier heads (the second adds onto the first's logits)."""
+
+    def __init__(self, ends: dict, layer_params: list, batch: int, tokens: int, heads: int, mlp_dim: int, bits: int,
+                 device="cuda", eps: float = 1e-6, **layer_kw):
+        self.batch, self.tokens, self.bits, self.eps = batch, tokens, bits, eps
+        self.dim = D = heads * 64
+        M = batch * tokens
+        d = lambda a: _dev(a, device)
+        self.stack = EncoderStack(layer_params, batch, tokens, heads, mlp_dim, bits, device, eps=eps, **layer_kw)
+        q = lambda w, s: B.vitint_widen(B.vitint_quantize(d(w), 0.0, bits, True, row_steps=d(s)))
+        self.w_pe, self.s_w_pe, self.b_pe = q(ends["w_pe"], ends["s_w_pe"]), d(ends["s_w_pe"]), d(ends["b_pe"])
+        self.table = d(np.tile(np.asarray(ends["tokens"], np.float32), (batch, 1)))
+        self.s_patch, self.s_lnf = float(ends["s_patch"]), float(ends["s_lnf"])
+        self.lnf_g, self.lnf_b = d(ends["lnf_g"]), d(ends["lnf_b"])
+        self.heads_w = [(q(ends["w_" + n], ends["s_w_" + n]), d(ends["s_w_" + n]), d(ends["b_" + n]))
+                        for n in ("head", "head_dist")]
+        n_cls = ends["w_head"].shape[0]
+        self.xq = B.Codes.empty(M, ends["w_pe"].shape[1], bits, True, device, container=8)
+        self.x0 = torch.empty((M, D), dtype=torch.float32, device=device)
+        self.x_final = torch.empty((M, D), dtype=torch.float32, device=device)
+        self.head_codes = [B.Codes.empty(batch, D, bits, True, device, container=8) for _ in range(2)]
+        self.logits = [torch.empty((batch, n_cls), dtype=torch.float32, device=device) for _ in range(2)]
+
+    def forward(self, patches: torch.Tensor) -> torch.Tensor:
+        """patches: fp32 [batch*tokens, patch_dim] on the device.  Returns the summed logits [batch, classes]."""
+        B.vitint_quantize(patches, self.s_patch, self.bits, True, out=self.xq)
+        B.vitint_linear(self.xq, self.s_patch, self.w_pe, self.s_w_pe, self.b_pe,
+                        B.Epilogue(mode=B.EPI_DEQUANT_F32, residual=self.table), out=self.x0)
+        self.stack.forward(self.x0, self.x_final)
+        for i, (w, s_w, b) in enumerate(self.heads_w):
+            rows = self.x_final[i::self.tokens]                 # class rows (i = 0), distillation rows (i = 1)
+            B.vitint_layernorm_quantize(rows, self.lnf_g, self.lnf_b, self.eps, self.s_lnf, self.bits, True,
+                                        out=self.head_codes[i])
+            B.vitint_linear(self.head_codes[i], self.s_lnf, w, s_w, b,
+                            B.Epilogue(mode=B.EPI_DEQUANT_F32, residual=self.logits[0] if i else None),
+                            out=self.logits[i])
+        return self.logits[1]
+
+    def ops(self) -> int:
+        M, D = self.batch * self.tokens, self.dim
+        ends = 2 * M * D * self.xq.cols + 2 * 2 * self.batch * D * self.logits[0].shape[1]
+        return ends + self.stack.ops()

@@ -147,7 +147,13 @@ VIT_BASE_ENCODER = BlockConfig("vit_base_12layer_b256", 256, 197, 768, 12, 4, ml
 # The self-attention module of the paper's power table: DeiT-S width, 198 tokens (class + distillation + 196
 # patches), 3-bit, with a LayerNorm over each head's 64 channels in front of the Q and K quantizers.
 DEIT_S_ATTENTION = BlockConfig("deit_s_attn_n198_b64", 64, 198, 384, 6, 3, seed_index=5)
-CONFIGS = {c.name: c for c in (VIT_TINY_BLOCK, VIT_SMALL_BLOCK, VIT_BASE_LAYER, VIT_BASE_ENCODER, DEIT_S_ATTENTION)}
+# The whole DeiT-S model the paper evaluates (Section V-A): 16x16x3 patches -> 384 channels, class and distillation
+# tokens (198 tokens), 12 encoder layers with a 1536-wide MLP, final LayerNorm, two classifier heads (10 classes).
+DEIT_S_MODEL = BlockConfig("deit_s_model_n198_b128", 128, 198, 384, 6, 4, mlp_dim=1536, layers=12, seed_index=6)
+PATCH_DIM = 16 * 16 * 3
+NUM_CLASSES = 10
+CONFIGS = {c.name: c for c in (VIT_TINY_BLOCK, VIT_SMALL_BLOCK, VIT_BASE_LAYER, VIT_BASE_ENCODER, DEIT_S_ATTENTION,
+                               DEIT_S_MODEL)}
 
 
 def activations(cfg: BlockConfig, batch: int | None = None, first_image: int = 0) -> np.ndarray:
@@ -216,6 +222,37 @@ def layer_parameters(cfg: BlockConfig, layer: int = 0) -> dict:
         p["s_w_fc2"] = lsq_step_rows(p["w_fc2"], b)
         p["s_ln"] = gaussian_lsq_step(1.0, b)
         p["s_g"] = gelu_lsq_step(ws * math.sqrt(D), b, sd("gelu_mc"))
+    return p
+
+
+def patch_rows(cfg: BlockConfig, batch: int | None = None, first_image: int = 0) -> np.ndarray:
+    """Flattened, normalised image patches ~ N(0,1), fp32 [batch*tokens, PATCH_DIM].  The rows of the class and
+    distillation tokens (the first two of every image) are zero: their embeddings come from the token table."""
+    b = cfg.batch if batch is None else batch
+    out = np.zeros((b * cfg.tokens, PATCH_DIM), dtype=np.float32)
+    for i in range(b):
+        s = substream(cfg.seed, f"patches/{first_image + i}")
+        out[i * cfg.tokens + 2:(i + 1) * cfg.tokens] = normal(s, (cfg.tokens - 2, PATCH_DIM))
+    return out
+
+
+def model_end_parameters(cfg: BlockConfig) -> dict:
+    """Random-init parameters of the model's two ends: patch embedding (a linear layer over flattened patches),
+    the token table (class / distillation token and position embeddings, one fp32 row per token, added after the
+    patch embedding), final LayerNorm, and the two classifier heads whose logits are summed."""
+    sd = lambda tag: substream(cfg.seed, f"ends/{tag}")
+    D, b = cfg.dim, cfg.bits
+    p = {"w_pe": normal(sd("w_pe"), (D, PATCH_DIM), 0.0, cfg.w_std), "b_pe": normal(sd("b_pe"), (D,), 0.0, 0.01),
+         "tokens": normal(sd("tokens"), (cfg.tokens, D), 0.0, 0.02),
+         "lnf_g": normal(sd("lnf_g"), (D,), 1.0, 0.02), "lnf_b": normal(sd("lnf_b"), (D,), 0.0, 0.02),
+         "w_head": normal(sd("w_head"), (NUM_CLASSES, D), 0.0, cfg.w_std),
+         "b_head": normal(sd("b_head"), (NUM_CLASSES,), 0.0, 0.01),
+         "w_head_dist": normal(sd("w_head_dist"), (NUM_CLASSES, D), 0.0, cfg.w_std),
+         "b_head_dist": normal(sd("b_head_dist"), (NUM_CLASSES,), 0.0, 0.01)}
+    for n in ("w_pe", "w_head", "w_head_dist"):
+        p["s_" + n] = lsq_step_rows(p[n], b)
+    p["s_patch"] = gaussian_lsq_step(1.0, b)
+    p["s_lnf"] = gaussian_lsq_step(1.0, b)
     return p
 
 

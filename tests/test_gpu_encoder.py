@@ -290,3 +290,56 @@ def test_normed_attention_module_bit_exact(bits):
     # per linear layer and 198*198*64 = 2.51 M per attention matmul
     per_image = mod.ops() // (2 * cfg.batch)
     assert per_image == H * (3 * 198 * 384 * 64 + 2 * 198 * 198 * 64)
+
+
+def test_deit_s_model_forward():
+    """Whole DeiT-S-shaped model (patch embedding, 198 tokens, 12 layers, final LayerNorm, two heads) against the
+    oracle on sampled images.  The patch embedding is one fixed IEEE sequence (bit-exact); after twelve layers the
+    legitimate one-level differences on near-ties have spread, so the residual stream and the logits are compared
+    statistically; the heads are checked exactly by feeding them the oracle's own final activations."""
+    from paper_2504_18547_b200.encoder import DeitModel
+    cfg = si.DEIT_S_MODEL.with_(batch=4)
+    T, H, D = cfg.tokens, cfg.heads, cfg.dim
+    ends = si.model_end_parameters(cfg)
+    lps = [si.layer_parameters(cfg, layer=l) for l in range(cfg.layers)]
+    patches = si.patch_rows(cfg)
+    model = DeitModel(ends, lps, cfg.batch, T, H, cfg.mlp_dim, cfg.bits)
+    logits = model.forward(dev(patches)).cpu().numpy()
+    assert vt.vitint_device_status() == 0
+    images = [0, 3]
+    st = vp.deit_forward(_rows(patches, images, T), ends, lps, len(images), T, H, cfg.bits)
+    # patch embedding + token table
+    x0 = _rows(model.x0.cpu().numpy(), images, T)
+    assert np.array_equal(x0.view(np.uint32), st["x0"].view(np.uint32))
+    # the class and distillation rows received no patch contribution: bias + token table only
+    tok = np.asarray(ends["tokens"], np.float32)
+    assert np.array_equal(x0[:2], (ends["b_pe"][None, :] + tok[:2]).astype(np.float32))
+    # residual stream after 12 layers
+    xf = _rows(model.x_final.cpu().numpy(), images, T)
+    err = (xf - st["x_final"]).astype(np.float64)
+    rel_rms = np.sqrt((err ** 2).mean()) / st["x_final"].std()
+    corr = np.corrcoef(xf.ravel(), st["x_final"].ravel())[0, 1]
+    assert rel_rms < 0.3 and corr > 0.95, (rel_rms, corr)
+    # heads, exactly: the oracle's final activations through the library's final LayerNorm + heads
+    xfin = np.zeros((cfg.rows, D), np.float32)
+    for j, b in enumerate(images):
+        xfin[b * T:(b + 1) * T] = st["x_final"][j * T:(j + 1) * T]
+    model.x_final.copy_(dev(xfin))
+    for i, (w, s_w, bias) in enumerate(model.heads_w):
+        rows = model.x_final[i::T]
+        vt.vitint_layernorm_quantize(rows, model.lnf_g, model.lnf_b, model.eps, model.s_lnf, cfg.bits, True,
+                                     out=model.head_codes[i])
+        vt.vitint_linear(model.head_codes[i], model.s_lnf, w, s_w, bias,
+                         vt.Epilogue(mode=vt.EPI_DEQUANT_F32, residual=model.logits[0] if i else None),
+                         out=model.logits[i])
+    hc = [from_codes(c)[images] for c in model.head_codes]
+    ok = np.ones(len(images), bool)
+    for name, c in zip(("head", "head_dist"), hc):
+        assert np.all(c >= st[name + "_lo"]) and np.all(c <= st[name + "_hi"])
+        ok &= (c == st[name + "_codes"]).all(axis=1)
+    got = model.logits[1].cpu().numpy()[images]
+    assert ok.any()
+    assert np.array_equal(got[ok].view(np.uint32), st["logits"][ok].view(np.uint32))
+    # end to end the logits stay close
+    assert np.abs(logits[images] - st["logits"]).max() < 0.25 * max(1.0, np.abs(st["logits"]).max())
+    print(f"DeiT-S model: residual stream relative rms {rel_rms:.4f}, correlation {corr:.5f}")
