@@ -338,6 +338,18 @@ def run_ours(args, cfg):
                                                 "images_per_s": round(mcfg.batch / (ms * 1e-3), 1),
                                                 "launches": 2 + 8 * mcfg.layers + 4}
         del model, mp
+        # the 12-layer ViT-Base encoder at batch 256 (the multi-layer configuration): whole forward, images/s
+        from paper_2504_18547_b200.encoder import EncoderStack
+        ecfg = si.VIT_BASE_ENCODER.with_(bits=cfg.bits)
+        stack = EncoderStack([si.layer_parameters(ecfg, layer=l) for l in range(ecfg.layers)], ecfg.batch, ecfg.tokens,
+                             ecfg.heads, ecfg.mlp_dim, ecfg.bits, device)
+        ex = torch.cat([xs[0], xs[1]])                       # 256 images of synthetic patch embeddings ~ N(0,1)
+        eout = torch.empty_like(ex)
+        ms = timed(lambda: stack.forward(ex, eout), reps=5)
+        standalone["vit_base_encoder12_b256"] = {"ms": round(ms, 4), "tops": round(stack.ops() / (ms * 1e-3) / 1e12, 1),
+                                                 "images_per_s": round(ecfg.batch / (ms * 1e-3), 1),
+                                                 "launches": 8 * ecfg.layers}
+        del stack, ex, eout
 
     # ---- CPU oracle on a bounded sample (rank 0, single-GPU runs only) -----------------
     cpu = None
