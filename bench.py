@@ -280,7 +280,7 @@ def run_ours(args, cfg):
 
     # ---- streaming kernels that the fused step does not launch, timed alone (HBM roofline) -------------
     standalone = {}
-    if world == 1:
+    if world == 1 and not args.no_standalone:
         def timed(fn, reps=10):
             for _ in range(3):
                 fn()
@@ -412,6 +412,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="images per GPU (default: the configuration's 128)")
     ap.add_argument("--ref-images", type=int, default=None, help="images per step of the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-standalone", action="store_true",
+                    help="skip the kernels and composed workloads that are timed alone after the step")
     ap.add_argument("--packed-activations", action="store_true",
                     help="keep every activation code matrix bit-packed (default: one code per byte where only a linear layer reads it)")
     ap.add_argument("--unfused-attention", action="store_true", help="run Q K^T, softmax and P V as separate kernels")
