@@ -402,6 +402,107 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+# ---------------------------------------------------------------------------
+# sweep: integer linear over K, N, tokens and bits; streaming kernels at the same sizes
+# ---------------------------------------------------------------------------
+
+SWEEP_KN = (192, 384, 768, 1024, 3072, 4096)
+SWEEP_TOKENS_BATCH = ((197, 256), (577, 64), (785, 32))
+
+
+def run_sweep(args):
+    """Times vitint_linear (requantizing epilogue) for every K, N of SWEEP_KN at M = tokens x batch, 4-bit codes
+    stored one per byte and 8-bit codes, against the int8 tensor roofline, and the quantize and softmax kernels at
+    the same token counts against the HBM roofline.  Prints ONE JSON line; operands are seeded and synthetic
+    (uniform random codes, which is all the timing depends on)."""
+    import torch
+
+    import paper_2504_18547_b200 as vt
+
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+    gen = torch.Generator(device=device)
+    gen.manual_seed(si.BASE_SEED)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)       # larger than L2
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn()
+        t = 0.0
+        for _ in range(reps):
+            flush.zero_()                                                   # L2 flushed between timed iterations
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            t += a.elapsed_time(b)
+        return t / reps
+
+    def codes(rows, cols, bits):
+        qn, qp = si.code_range(bits, True)
+        t = torch.randint(qn, qp + 1, (rows, cols), dtype=torch.int8, device=device, generator=gen)
+        return vt.Codes(t.view(torch.uint8), rows, cols, bits, True, 8)
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    linear = []
+    for tokens, batch in SWEEP_TOKENS_BATCH:
+        M = tokens * batch
+        for bits in (4, 8):
+            for K in SWEEP_KN:
+                x = codes(M, K, bits)
+                for N in SWEEP_KN:
+                    w = codes(N, K, bits)
+                    alpha = torch.full((N,), 1.0 / (K ** 0.5 * 2.0 ** (bits - 1)), dtype=torch.float32, device=device)
+                    beta = torch.zeros((N,), dtype=torch.float32, device=device)
+                    epi = vt.Epilogue(mode=vt.EPI_REQUANT, alpha=alpha, beta=beta, out_bits=bits, out_signed=True,
+                                      out_container=8)
+                    out = vt.Codes.empty(M, N, bits, True, device, container=8)
+                    ms = timed(lambda: vt.vitint_linear(x, 1.0, w, None, None, epi, out=out), args.steps)
+                    tops = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+                    linear.append({"tokens": tokens, "batch": batch, "bits": bits, "K": K, "N": N, "ms": round(ms, 4),
+                                   "tops": round(tops, 1), "frac_int8_peak": round(tops / int8_peak, 4)})
+                    del w, out
+                del x
+    streaming = []
+    for tokens, batch in SWEEP_TOKENS_BATCH:
+        M = tokens * batch
+        for bits in (2, 4, 8):
+            cb = bits
+            xf = torch.randn((M, 768), dtype=torch.float32, device=device, generator=gen)
+            xq = vt.Codes.empty(M, 768, bits, True, device)
+            ms = timed(lambda: vt.vitint_quantize(xf, 0.25, bits, True, out=xq), args.steps)
+            nbytes = M * 768 * 4 + M * 768 * cb // 8
+            streaming.append({"kernel": "quantize", "rows": M, "cols": 768, "bits": bits, "ms": round(ms, 4),
+                              "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                              "frac_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
+            rows = min(batch, 32) * 12 * tokens                     # attention rows of up to 32 images, 12 heads
+            S = torch.randint(-300, 300, (rows, (tokens + 3) // 4 * 4), dtype=torch.int32, device=device, generator=gen)
+            Pq = vt.Codes.empty(rows, tokens, bits, False, device)
+            nbytes = rows * tokens * 4 + rows * ((tokens * cb + 7) // 8)
+            for name, fn in (("softmax_quantize", lambda: vt.vitint_softmax_quantize(S, tokens, 0.01, 0.02, bits, out=Pq)),
+                             ("softmax_shift_quantize", lambda: vt.vitint_softmax_shift_quantize(S, tokens, 0.0144, 0.02, bits, out=Pq))):
+                ms = timed(fn, args.steps)
+                streaming.append({"kernel": name, "rows": rows, "cols": tokens, "bits": bits, "ms": round(ms, 4),
+                                  "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                                  "frac_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
+            del xf, xq, S, Pq
+    clocks = sampler.stop()
+    if vt.vitint_device_status() != 0:
+        raise RuntimeError("device-side timeout during the sweep")
+    best = max(linear, key=lambda r: r["tops"])
+    print(json.dumps({"metric": "integerized linear sweep, effective TOPS", "value": best["tops"], "unit": "TOPS",
+                      "n_gpus": 1, "steps": args.steps, "warmup": 3, "higher_is_better": True, "dtype": "int8",
+                      "data": "synthetic", "config": {"workload": "linear_and_streaming_sweep", "K_N": list(SWEEP_KN),
+                                                      "tokens_batch": [list(t) for t in SWEEP_TOKENS_BATCH],
+                                                      "l2": "256 MB written between timed iterations"},
+                      "peaks": {"int8_tops": int8_peak, "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]},
+                      "clocks": clocks, "best": best, "linear": linear, "streaming": streaming}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -412,6 +513,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="images per GPU (default: the configuration's 128)")
     ap.add_argument("--ref-images", type=int, default=None, help="images per step of the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time the integer linear over K, N, tokens and bits, and the streaming kernels (one JSON line)")
     ap.add_argument("--no-standalone", action="store_true",
                     help="skip the kernels and composed workloads that are timed alone after the step")
     ap.add_argument("--packed-activations", action="store_true",
@@ -425,7 +528,10 @@ def main():
     if args.ref_images is None:
         args.ref_images = 64 if args.impl == "ours" else 8
     args.ref_images = min(args.ref_images, cfg.batch)
-    if args.impl == "reference":
+    if args.sweep:
+        if dist_env()[0] == 0:
+            run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         run_ours(args, cfg)
