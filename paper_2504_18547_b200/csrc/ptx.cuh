@@ -81,6 +81,13 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
 
+// One 32-byte store by the calling thread (address 32-byte aligned): lo to the first 16 bytes, hi to the rest.
+__device__ __forceinline__ void st_global_32B(void* dst, const uint32_t (&lo)[4], const uint32_t (&hi)[4]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]),
+                 "r"(lo[3]), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3])
+                 : "memory");
+}
+
 // ---- tcgen05 ------------------------------------------------------------------
 // Whole-warp, converged.  ncols: power of two in [32, 512].
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
