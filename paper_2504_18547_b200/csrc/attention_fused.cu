@@ -393,6 +393,10 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     *reinterpret_cast<uint4*>(o) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                 } else if (P.out_c == 2) {
                     *reinterpret_cast<uint2*>(o) = make_uint2(ow[0], ow[1]);
+                } else if ((reinterpret_cast<uintptr_t>(o) & 31u) == 0) {
+                    // one 32-byte store: a warp's store touches 32 different rows whatever its width
+                    const uint32_t lo[4] = {ow[0], ow[1], ow[2], ow[3]}, hi[4] = {ow[4], ow[5], ow[6], ow[7]};
+                    ptx::st_global_32B(o, lo, hi);
                 } else {
                     reinterpret_cast<uint4*>(o)[0] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                     reinterpret_cast<uint4*>(o)[1] = make_uint4(ow[4], ow[5], ow[6], ow[7]);
