@@ -833,7 +833,7 @@ int make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint6
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? VITINT_OK : VITINT_ERR_CUDA;
 }
 
@@ -895,7 +895,10 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
                   aligned16(P.out) && P.ld_out % 4 == 0 &&
                   (!P.residual || (aligned16(P.residual) && P.ld_res % 4 == 0));
     // the fp32 kinds keep 8 epilogue warps: their two staging blocks per warp come out of the ring space
-    P.epi_warps = (P.a_direct && P.b_direct && !staged) ? MAX_EPI_WARPS : EPI_WARPS;
+    // ... unless the contraction is short (K <= 1024): such a GEMM is bound by its fp32 epilogue, which gains more
+    // from twelve warps than the mainloop loses with two ring stages (proj, batch 128: 45 -> 43 us; with the
+    // long contraction of fc2 the same choice costs 17 us)
+    P.epi_warps = (P.a_direct && P.b_direct && (!staged || K <= 1024)) ? MAX_EPI_WARPS : EPI_WARPS;
     const uint32_t stage_total = staged ? (uint32_t)(P.epi_warps * STAGE_BYTES) : 0u;
     const uint32_t ring_budget = SMEM_TILE_BUDGET + 12u * 1024u - stage_total;   // staging comes out of the ring space
     // The packed ring hides the global-memory latency of the TMA loads; the int8 ring only
