@@ -275,12 +275,15 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
 // all of them real columns; col_begin and col_end are multiples of 16.  Whole-warp call: the TMEM
 // load is a warp-wide instruction, so lanes whose row lies past M run the arithmetic too and only
 // their stores are masked.
-template <int KIND, int SMALL, bool UNIT>
+// BYTES: the output container is one byte per code, known at compile time, so the packing of each group of four
+// codes can be scheduled right behind their arithmetic instead of after all sixteen (fewer live registers, more
+// independent work in flight: fc1 94 -> 91 us).
+template <int KIND, int SMALL, bool UNIT, bool BYTES>
 __device__ __forceinline__ void epilogue_requant_blocks(const GemmParams& P, const EpiParams& ep, int buf,
                                                        uint32_t t_row, bool row_ok, long long orow, long long col0,
                                                        int col_begin, int col_end) {
     const bool sgn = P.out_qn < 0.0f;
-    const float magic = 12582912.0f + (sgn ? (float)(1 << (P.out_c - 1)) : 0.0f);
+    const float magic = 12582912.0f + (sgn ? (float)(1 << ((BYTES ? 8 : P.out_c) - 1)) : 0.0f);
     uint8_t* const o_row = (uint8_t*)P.out + orow * P.ld_out;
     // Byte codes without an activation: the 16 bytes of an even block wait in registers for the odd block and
     // the two leave as ONE 32-byte store.  A warp's store touches 32 different rows whatever its width, so this
@@ -342,7 +345,7 @@ __device__ __forceinline__ void epilogue_requant_blocks(const GemmParams& P, con
         }
         // offset-binary packing as in epilogue_chunk: 16 codes = 2 * out_c bytes
         const long long c = col0 + col;
-        if (P.out_c == 8) {
+        if (BYTES) {
             uint32_t w[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -478,9 +481,11 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiPara
         // every column of the tile is real: rolled 16-column blocks
         const long long col0 = colbase + (long long)n_tile * P.bn;
         if (KIND == EK_REQUANT_GELU && P.unit_out)
-            epilogue_requant_blocks<EK_REQUANT_GELU, SMALL, true>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+            if (P.out_c == 8) epilogue_requant_blocks<EK_REQUANT_GELU, SMALL, true, true>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+            else epilogue_requant_blocks<EK_REQUANT_GELU, SMALL, true, false>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
         else
-            epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL, false>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+            if (P.out_c == 8) epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL, false, true>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+            else epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL, false, false>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
         // row padding behind the last column of the matrix
         if (row_ok && P.col_off_inner == 0 && n_tile * P.bn + c_end * 32 >= P.N && c_end > c_begin) {
             for (long long off = ((long long)P.N * P.out_c) >> 3; off + 4 <= P.ld_out; off += 4)
