@@ -387,7 +387,7 @@ def run_ours(args, cfg):
         "clocks": clocks,
         "e2e": {"value": e2e_tops, "unit": "TOPS", "h2d_bytes_per_step": M * D * 4, "d2h_bytes_per_step": M * D * 4,
                 "ms_per_step": ms_e2e / args.steps},
-        "gpu_launches": (len(STAGES) + (1 if layer.fused_attention else 0)) * args.steps,
+        "gpu_launches": len(STAGES) * args.steps,
         "roofline": {"bound": "tensor", "kernel": f"gemm_i8_kernel ({len(gemm_stages)} launches per step)", "achieved": achieved,
                      "peak": int8_peak, "unit": "TOPS", "frac": achieved / int8_peak, "traffic": traffic,
                      "timing": "CUDA events around every call, second pass over the same K steps (the timed K steps carry no events)",

@@ -198,6 +198,18 @@ int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int32_t heads,
                           float k_step, float p_step, int32_t p_bits, const float* alpha_o, const float* beta_o,
                           const vitint_codes* o_out, void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same core with the exp table prepared once: the table depends only on the code width and on the steps of
+ * Q and K (Eq. 3's scale), which are fixed per layer, so a caller that runs the layer many times fills it once
+ *   vitint_attention_exp_table(bits, q_step, k_step, table, table_bytes, stream)
+ * (table: device memory, 256-byte aligned, >= vitint_attention_core_workspace_bytes(bits) bytes) and then calls
+ * vitint_attention_core_prepared with that table and the SAME bits, q_step and k_step: one kernel launch instead
+ * of two, results identical to vitint_attention_core.  The table is only read by the prepared call. */
+int vitint_attention_exp_table(int32_t bits, float q_step, float k_step, void* table, size_t table_bytes, void* stream);
+int vitint_attention_core_prepared(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens, float q_step,
+                                   float k_step, float p_step, int32_t p_bits, const float* alpha_o,
+                                   const float* beta_o, const vitint_codes* o_out, const void* table,
+                                   size_t table_bytes, void* stream);
+
 /* vitint_attention_core without caller-provided scratch.  (No counterpart in the paper: this is
  *   a packaging variant, not a step of the method.)
  *   Who needs it: code that is not allowed to obtain device memory when it runs the attention

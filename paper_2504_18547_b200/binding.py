@@ -77,6 +77,10 @@ def lib():
         L.vitint_attention_core_workspace_bytes.argtypes = [c_int32]
         L.vitint_attention_core.argtypes = [POINTER(_Codes), c_int32, c_int32, c_int32, c_float, c_float, c_float,
                                             c_int32, c_void_p, c_void_p, POINTER(_Codes), c_void_p, c_size_t, c_void_p]
+        L.vitint_attention_exp_table.argtypes = [c_int32, c_float, c_float, c_void_p, c_size_t, c_void_p]
+        L.vitint_attention_core_prepared.argtypes = [POINTER(_Codes), c_int32, c_int32, c_int32, c_float, c_float, c_float,
+                                                     c_int32, c_void_p, c_void_p, POINTER(_Codes), c_void_p, c_size_t,
+                                                     c_void_p]
         L.vitint_attention_core_noalloc.argtypes = [POINTER(_Codes), c_int32, c_int32, c_int32, c_float, c_float, c_float,
                                                     c_int32, c_void_p, c_void_p, POINTER(_Codes), c_void_p]
         L.vitint_attention_block_workspace_bytes.restype = c_size_t
@@ -335,6 +339,29 @@ def vitint_attention_core(qkv: Codes, batch: int, heads: int, tokens: int, q_ste
     _check(lib().vitint_attention_core(byref(dq), batch, heads, tokens, float(q_step), float(k_step), float(p_step),
                                        p_bits, _ptr(alpha_o), _ptr(beta_o), byref(do), workspace.data_ptr(),
                                        workspace.numel(), _stream()), "vitint_attention_core")
+    return out
+
+
+def vitint_attention_exp_table(bits: int, q_step: float, k_step: float, table: torch.Tensor | None = None,
+                               device="cuda") -> torch.Tensor:
+    """Fills (and returns) the exp table of the fused attention core for these steps; see
+    vitint_attention_core_prepared."""
+    if table is None:
+        table = torch.empty(vitint_attention_core_workspace_bytes(bits), dtype=torch.uint8, device=device)
+    _check(lib().vitint_attention_exp_table(bits, float(q_step), float(k_step), table.data_ptr(), table.numel(),
+                                            _stream()), "vitint_attention_exp_table")
+    return table
+
+
+def vitint_attention_core_prepared(qkv: Codes, batch: int, heads: int, tokens: int, q_step: float, k_step: float,
+                                   p_step: float, p_bits: int, alpha_o: torch.Tensor, beta_o: torch.Tensor | None,
+                                   out: Codes, table: torch.Tensor) -> Codes:
+    """vitint_attention_core with a table filled once by vitint_attention_exp_table (same bits and steps)."""
+    dq, do = qkv.desc(), out.desc()
+    _check(lib().vitint_attention_core_prepared(byref(dq), batch, heads, tokens, float(q_step), float(k_step),
+                                                float(p_step), p_bits, _ptr(alpha_o), _ptr(beta_o), byref(do),
+                                                table.data_ptr(), table.numel(), _stream()),
+           "vitint_attention_core_prepared")
     return out
 
 

@@ -430,10 +430,12 @@ extern "C" size_t vitint_attention_core_workspace_bytes(int32_t bits) {
     return (size_t)(2 * 64 * m * m + 1) * sizeof(float) + 256;
 }
 
-extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
-                                     float q_step, float k_step, float p_step, int32_t p_bits, const float* alpha_o,
-                                     const float* beta_o, const vitint_codes* o_out, void* workspace,
-                                     size_t workspace_bytes, void* stream) {
+// Shared by the three entry points below.  build_table: fill `workspace` with the exp table first (one more
+// small launch); otherwise the caller has filled it for exactly these steps and bits (vitint_attention_exp_table).
+static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
+                                 float q_step, float k_step, float p_step, int32_t p_bits, const float* alpha_o,
+                                 const float* beta_o, const vitint_codes* o_out, void* workspace,
+                                 size_t workspace_bytes, bool build_table, void* stream) {
     if (int rc = check_codes(qkv)) return rc;
     if (int rc = check_codes(o_out)) return rc;
     if (batch <= 0 || heads <= 0 || tokens <= 0 || !alpha_o) return VITINT_ERR_INVALID_ARG;
@@ -516,8 +518,10 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return VITINT_ERR_CUDA;
     }
-    launch_kernel(exp_table_kernel, dim3((2 * smax + 1 + 255) / 256), dim3(256), 0, st, (float*)workspace, smax, cs);
-    if (cudaGetLastError() != cudaSuccess) return VITINT_ERR_CUDA;
+    if (build_table) {
+        launch_kernel(exp_table_kernel, dim3((2 * smax + 1 + 255) / 256), dim3(256), 0, st, (float*)workspace, smax, cs);
+        if (cudaGetLastError() != cudaSuccess) return VITINT_ERR_CUDA;
+    }
     int grid = sm_count();
     const int want = (P.total_items + AT_GROUPS - 1) / AT_GROUPS;
     if (grid > want) grid = want;
@@ -537,6 +541,36 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
     else VITINT_ATTN_LAUNCH(2, 0)
 #undef VITINT_ATTN_LAUNCH
     return cuda_status(cudaGetLastError());
+}
+
+extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
+                                     float q_step, float k_step, float p_step, int32_t p_bits, const float* alpha_o,
+                                     const float* beta_o, const vitint_codes* o_out, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+    return attention_core_launch(qkv, batch, heads, tokens, q_step, k_step, p_step, p_bits, alpha_o, beta_o, o_out,
+                                 workspace, workspace_bytes, true, stream);
+}
+
+extern "C" int vitint_attention_exp_table(int32_t bits, float q_step, float k_step, void* table, size_t table_bytes,
+                                          void* stream) {
+    if (!valid_bits(bits) || bits == 8) return VITINT_ERR_UNSUPPORTED;
+    if (!(q_step > 0.0f && q_step < INFINITY) || !(k_step > 0.0f && k_step < INFINITY)) return VITINT_ERR_INVALID_ARG;
+    if (!table || (reinterpret_cast<uintptr_t>(table) & 255u) || table_bytes < vitint_attention_core_workspace_bytes(bits))
+        return VITINT_ERR_WORKSPACE;
+    const int m = 1 << (container_bits(bits) - 1);
+    const int smax = 64 * m * m;
+    const float cs = (float)((double)q_step * (double)k_step / 8.0);
+    launch_kernel(exp_table_kernel, dim3((2 * smax + 1 + 255) / 256), dim3(256), 0, (cudaStream_t)stream, (float*)table,
+                  smax, cs);
+    return cuda_status(cudaGetLastError());
+}
+
+extern "C" int vitint_attention_core_prepared(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
+                                              float q_step, float k_step, float p_step, int32_t p_bits,
+                                              const float* alpha_o, const float* beta_o, const vitint_codes* o_out,
+                                              const void* table, size_t table_bytes, void* stream) {
+    return attention_core_launch(qkv, batch, heads, tokens, q_step, k_step, p_step, p_bits, alpha_o, beta_o, o_out,
+                                 const_cast<void*>(table), table_bytes, false, stream);
 }
 
 // ---------------------------------------------------------------------------------------

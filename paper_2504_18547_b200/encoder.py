@@ -80,7 +80,8 @@ class EncoderLayer:
         self.qkv = B.Codes.empty(M, 3 * D, bits, True, device, container=cq)
         self.ld_s = (tokens + 3) // 4 * 4
         if self.fused_attention:
-            self.attn_ws = torch.empty(B.vitint_attention_core_workspace_bytes(bits), dtype=torch.uint8, device=device)
+            # the exp table of the fused core depends only on the code width and the steps of Q and K: filled once
+            self.attn_table = B.vitint_attention_exp_table(bits, self.s_q, self.s_k, device=device)
         else:
             self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
             self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
@@ -114,8 +115,8 @@ class EncoderLayer:
         B.vitint_linear(self.x1, self.s_ln, self.w["qkv"], None, None, self.epi_qkv, out=self.qkv)
         mark()
         if self.fused_attention:
-            B.vitint_attention_core(self.qkv, b, h, t, self.s_q, self.s_k, self.s_p, self.bits, self.alpha_o, None,
-                                    out=self.O, workspace=self.attn_ws)
+            B.vitint_attention_core_prepared(self.qkv, b, h, t, self.s_q, self.s_k, self.s_p, self.bits, self.alpha_o,
+                                             None, out=self.O, table=self.attn_table)
         else:
             B.vitint_qk(self.slabs[0], self.slabs[1], b, h, t, out=self.S, ld_s=self.ld_s)
             mark()

@@ -339,6 +339,14 @@ def test_attention_core_fused(batch, tokens, heads, bits, scale, byte_codes):
     assert len(np.unique(want)) >= 3
     if scale >= 1.0:
         assert len(np.unique(pc)) >= 3
+    # the same call with the exp table filled once beforehand gives the same codes, bit for bit, also when the
+    # table is reused by a second call
+    table = vt.vitint_attention_exp_table(bits, s_q, s_k)
+    for _ in range(2):
+        out2 = vt.Codes.empty(batch * tokens, D, bits, True)
+        vt.vitint_attention_core_prepared(qkv_dev, batch, heads, tokens, s_q, s_k, s_p, bits, dev(alpha), dev(beta),
+                                          out=out2, table=table)
+        assert np.array_equal(from_codes(out2), got)
 
 
 # ---------------------------------------------------------------------------
