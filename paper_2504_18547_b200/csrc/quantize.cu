@@ -63,45 +63,54 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
     const float* xr = x + row * ldx;
-    float4 f[NV];
-    float sum = 0.0f;
+    // The row is held as packed pairs: adds, multiplies and fused multiply-adds below run two elements per
+    // instruction (each half is the scalar IEEE result), which is what this issue-bound kernel needs.
+    f32x2 f[NV][2];
+    f32x2 sum2 = f2_dup(0.0f);
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
         const int col = (v * 32 + lane) * 4;
-        f[v] = (col < cols) ? __ldg(reinterpret_cast<const float4*>(xr + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        sum += (f[v].x + f[v].y) + (f[v].z + f[v].w);
+        const float4 t = (col < cols) ? __ldg(reinterpret_cast<const float4*>(xr + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        f[v][0] = f2_pack(t.x, t.y);
+        f[v][1] = f2_pack(t.z, t.w);
+        sum2 = f2_add(sum2, f2_add(f[v][0], f[v][1]));
     }
+    float s_lo, s_hi;
+    f2_unpack(sum2, s_lo, s_hi);
+    float sum = s_lo + s_hi;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     const float inv_n = 1.0f / (float)cols;
-    // corrected two-pass mean: centre on the fp32 estimate, then remove the mean of the
-    // residuals, which carries the estimate's rounding error even when |mean| >> sigma
+    // Centre on the fp32 estimate of the mean; one more pass gives both the mean of the residuals (which carries
+    // the estimate's rounding error even when |mean| >> sigma) and their sum of squares.  The variance is
+    // sum(d^2)/n - corr^2 with corr the residual mean: exact algebra, and corr is a rounding-level quantity.
     const float mean0 = sum * inv_n;
-    float rsum = 0.0f;
+    const f32x2 nmean2 = f2_dup(-mean0);
+    f32x2 rs2 = f2_dup(0.0f), m22 = f2_dup(0.0f);
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
         const int col = (v * 32 + lane) * 4;
         if (col < cols) {
-            f[v].x -= mean0; f[v].y -= mean0; f[v].z -= mean0; f[v].w -= mean0;
-            rsum += (f[v].x + f[v].y) + (f[v].z + f[v].w);
+            f[v][0] = f2_add(f[v][0], nmean2);
+            f[v][1] = f2_add(f[v][1], nmean2);
+            rs2 = f2_add(rs2, f2_add(f[v][0], f[v][1]));
+            m22 = f2_fma(f[v][0], f[v][0], m22);
+            m22 = f2_fma(f[v][1], f[v][1], m22);
         }
     }
+    float r_lo, r_hi, q_lo, q_hi;
+    f2_unpack(rs2, r_lo, r_hi);
+    f2_unpack(m22, q_lo, q_hi);
+    float rsum = r_lo + r_hi, m2 = q_lo + q_hi;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
+    for (int o = 16; o > 0; o >>= 1) {
+        rsum += __shfl_xor_sync(0xffffffffu, rsum, o);
+        m2 += __shfl_xor_sync(0xffffffffu, m2, o);
+    }
     const float corr = rsum * inv_n;
-    float m2 = 0.0f;
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        const int col = (v * 32 + lane) * 4;
-        if (col < cols) {
-            f[v].x -= corr; f[v].y -= corr; f[v].z -= corr; f[v].w -= corr;
-            m2 += fmaf(f[v].x, f[v].x, f[v].y * f[v].y) + fmaf(f[v].z, f[v].z, f[v].w * f[v].w);
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
+    const f32x2 ncorr2 = f2_dup(-corr);
     // 1/sqrt(var + eps): hardware estimate plus one Newton step (about 1 ulp), all in fp32
-    const float var = fmaf(m2, inv_n, eps);
+    const float var = fmaf(m2, inv_n, eps) - corr * corr;
     float rstd = rsqrtf(var);
     rstd = rstd * fmaf(-0.5f * var, rstd * rstd, 1.5f);
     // y / step as y * RN(1/step): at most 1.5 ulp from the exact quotient, far inside the tolerance
@@ -121,16 +130,21 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
         if (col < cols) {
             const float4 g = __ldg(reinterpret_cast<const float4*>(gamma + col));
             const float4 b = __ldg(reinterpret_cast<const float4*>(beta + col));
+            const f32x2 rstd2 = f2_dup(rstd), rstep2 = f2_dup(rstep), magic2 = f2_dup(magic);
+            const f32x2 y01 = f2_fma(f2_mul(f2_add(f[v][0], ncorr2), rstd2), f2_pack(g.x, g.y), f2_pack(b.x, b.y));
+            const f32x2 y23 = f2_fma(f2_mul(f2_add(f[v][1], ncorr2), rstd2), f2_pack(g.z, g.w), f2_pack(b.z, b.w));
             float4 y;
-            y.x = fmaf(f[v].x * rstd, g.x, b.x);
-            y.y = fmaf(f[v].y * rstd, g.y, b.y);
-            y.z = fmaf(f[v].z * rstd, g.z, b.z);
-            y.w = fmaf(f[v].w * rstd, g.w, b.w);
+            f2_unpack(y01, y.x, y.y);
+            f2_unpack(y23, y.z, y.w);
             if (y_out) *reinterpret_cast<float4*>(y_out + row * ld_y + col) = y;
             // clamp, then add 1.5*2^23 (+ 2^(C-1) for signed codes): the low mantissa bits hold the code in
             // offset binary, so the four codes combine by shift-add without masking
-            const float cx = fminf(fmaxf(y.x * rstep, qn), qp) + magic, cy = fminf(fmaxf(y.y * rstep, qn), qp) + magic;
-            const float cz = fminf(fmaxf(y.z * rstep, qn), qp) + magic, cw = fminf(fmaxf(y.w * rstep, qn), qp) + magic;
+            float u0, u1, u2, u3;
+            f2_unpack(f2_mul(y01, rstep2), u0, u1);
+            f2_unpack(f2_mul(y23, rstep2), u2, u3);
+            float cx, cy, cz, cw;
+            f2_unpack(f2_add(f2_pack(fminf(fmaxf(u0, qn), qp), fminf(fmaxf(u1, qn), qp)), magic2), cx, cy);
+            f2_unpack(f2_add(f2_pack(fminf(fmaxf(u2, qn), qp), fminf(fmaxf(u3, qn), qp)), magic2), cz, cw);
             bits = (__float_as_uint(cx) + (__float_as_uint(cy) << C) + (__float_as_uint(cz) << (2 * C)) +
                     (__float_as_uint(cw) << (3 * C)) - 0x4B400000u * (1u + (1u << C) + (1u << (2 * C)) + (1u << (3 * C))));
             bits = (bits ^ flip) & (C == 8 ? 0xFFFFFFFFu : ((1u << ((4 * C) & 31)) - 1u));
