@@ -325,6 +325,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             const double rz = warp_live ? inv_p_step / z : 0.0;
             const float rzh = (float)rz;
             const float rzl = (float)(rz - (double)rzh);
+            const f32x2 rzh2 = f2_dup(rzh), rzl2 = f2_dup(rzl), magic2 = f2_dup(12582912.0f);
             uint8_t* const prow = ggen + P.off_p + row * 128;
             const int sw = row & 7;
             // pass 2: code = min(rint(e_j / (Z s_P)), Qp) (p >= 0: no lower clamp)
@@ -337,9 +338,14 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 for (int i4 = 0; i4 < 8; ++i4) {
                     uint32_t cb[4];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float e = __uint_as_float(v[4 * i4 + j]);
-                        cb[j] = __float_as_uint(fminf(fmaf(e, rzh, e * rzl), P.p_qp) + 12582912.0f);   // code in the low byte
+                    for (int j = 0; j < 4; j += 2) {
+                        // two scores per instruction (each half is the scalar IEEE result): e*r_hi + RN(e*r_lo)
+                        const f32x2 e2 = f2_pack(__uint_as_float(v[4 * i4 + j]), __uint_as_float(v[4 * i4 + j + 1]));
+                        float a0, a1, c0, c1;
+                        f2_unpack(f2_fma(e2, rzh2, f2_mul(e2, rzl2)), a0, a1);
+                        f2_unpack(f2_add(f2_pack(fminf(a0, P.p_qp), fminf(a1, P.p_qp)), magic2), c0, c1);
+                        cb[j] = __float_as_uint(c0);                                           // code in the low byte
+                        cb[j + 1] = __float_as_uint(c1);
                     }
                     wd[i4] = __byte_perm(__byte_perm(cb[0], cb[1], 0x4040), __byte_perm(cb[2], cb[3], 0x4040), 0x5410);
                 }
