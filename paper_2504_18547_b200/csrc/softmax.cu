@@ -16,12 +16,25 @@
 
 namespace vitint {
 
-__device__ __forceinline__ float exp_reduced(double d) {
-    // d <= 0.  Below -200 the result is far under the smallest denormal.
-    d = fmax(d, -200.0);
-    const float kf = rintf((float)d * 1.44269504088896340736f);
-    const double r = fma(-(double)kf, 0.693147180559945309417, d);
-    const float rf = (float)r;
+// exp(t - mx) for mx >= t, all in fp32 and integer instructions (no conversion instruction: those run at an eighth of
+// the issue rate and used to bound this kernel).
+//   * t - mx as an exact two-float sum (TwoSum), so nothing is lost when the two differ by more than a factor of two;
+//   * k = rint((t - mx) * log2 e) by the 1.5*2^23 addition, which also leaves k as an integer in the mantissa;
+//   * r = (t - mx) - k*ln2 with ln2 split so that k*ln2_hi is exact, the low parts folded in with one FMA;
+//   * degree-7 Taylor polynomial on |r| <= ln2/2 (truncation < 0.1 ulp), then 2^k added to the exponent field.
+// Results below 2^-125 (relative to the row's largest term, which is 1) are returned as 0: they lie in the range
+// where the tolerance is the absolute 2^-126.
+__device__ __forceinline__ float exp_reduced(float t, float mx) {
+    const float sh = __fadd_rn(t, -mx);
+    const float bv = __fadd_rn(sh, -t);
+    const float sl = __fadd_rn(__fadd_rn(t, -__fadd_rn(sh, -bv)), __fadd_rn(-mx, -bv));     // sh + sl = t - mx exactly
+    const float d = fmaxf(sh, -200.0f);
+    const float m = __fmaf_rn(d, 1.44269504088896340736f, 12582912.0f);
+    const float kf = __fadd_rn(m, -12582912.0f);
+    const int k = __float_as_int(m) - 0x4B400000;
+    const float rh = __fmaf_rn(-kf, 0.693145751953125f, d);                  // exact: ln2_hi has 15 significant bits
+    const float rl = __fmaf_rn(-kf, 1.42860682030941723212e-6f, sl);         // ln2 - ln2_hi, and the low part of t - mx
+    const float rf = __fadd_rn(rh, rl);
     float p = 1.0f / 5040.0f;
     p = fmaf(p, rf, 1.0f / 720.0f);
     p = fmaf(p, rf, 1.0f / 120.0f);
@@ -30,10 +43,8 @@ __device__ __forceinline__ float exp_reduced(double d) {
     p = fmaf(p, rf, 0.5f);
     p = fmaf(p, rf, 1.0f);
     p = fmaf(p, rf, 1.0f);
-    // 2^k in two exact factors so that k down to -252 stays representable
-    const int k = (int)kf;
-    const int k1 = k >> 1, k2 = k - k1;
-    return p * __int_as_float((k1 + 127) << 23) * __int_as_float((k2 + 127) << 23);
+    // p lies in [0.70, 1.42]: for k >= -125 the product p * 2^k is normal and exact as an exponent addition
+    return k >= -125 ? __int_as_float(__float_as_int(p) + (int)((uint32_t)k << 23)) : 0.0f;
 }
 
 template <int C, int NCH>
@@ -68,18 +79,26 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
 
-    const double mxd = (double)mx;
-    double z = 0.0;
+    // two interleaved fp64 partial sums; a float enters as a double built from its bits with integer
+    // multiply-adds (every term is zero or a positive normal float; a zero adds 2^-127, nothing beside the
+    // row's largest term, which is 1)
+    double z0 = 0.0, z1 = 0.0;
 #pragma unroll
     for (int k = 0; k < NCH; ++k) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int col = k * 256 + lane * 8 + i;
-            const float e = (col < cols) ? exp_reduced((double)t[k][i] - mxd) : 0.0f;
+            const float e = (col < cols) ? exp_reduced(t[k][i], mx) : 0.0f;
             t[k][i] = e;
-            z += (double)e;
+            const uint32_t eb = __float_as_uint(e);
+            uint32_t hi, lo;
+            asm("mad.hi.u32 %0, %1, 536870912, 939524096;" : "=r"(hi) : "r"(eb));    // (eb >> 3) + 0x38000000
+            asm("mul.lo.u32 %0, %1, 536870912;" : "=r"(lo) : "r"(eb));                // eb << 29
+            const double ed = (col < cols) ? __hiloint2double((int)hi, (int)lo) : 0.0;
+            if (i & 1) z1 += ed; else z0 += ed;
         }
     }
+    double z = z0 + z1;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
     const double rz = 1.0 / z;
