@@ -44,7 +44,7 @@ __device__ __forceinline__ float exp_reduced(float t, float mx) {
     p = fmaf(p, rf, 1.0f);
     p = fmaf(p, rf, 1.0f);
     // p lies in [0.70, 1.42]: for k >= -125 the product p * 2^k is normal and exact as an exponent addition
-    return k >= -125 ? __int_as_float(__float_as_int(p) + (int)((uint32_t)k << 23)) : 0.0f;
+    return k >= -125 ? __int_as_float(k * 8388608 + __float_as_int(p)) : 0.0f;
 }
 
 template <int C, int NCH>
@@ -59,16 +59,23 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
     if (row >= rows) return;
     const int32_t* sr = s + row * ld_s;
 
+    // Columns past the row's end take t = -inf.  Their exponential is exactly 0, so they add nothing to the row
+    // sum and quantize to code 0 (the padding value) without any per-element masking further down.
     float t[NCH][8];
     float mx = -INFINITY;
 #pragma unroll
     for (int k = 0; k < NCH; ++k) {
         const int col = k * 256 + lane * 8;
-        if (vec_in && col + 8 <= cols) {
+        if (vec_in && col + 8 <= ld_s) {
+            // whole 32 bytes inside the row's storage (the leading dimension may exceed the column count)
             const int4 a = __ldg(reinterpret_cast<const int4*>(sr + col));
             const int4 b = __ldg(reinterpret_cast<const int4*>(sr + col) + 1);
             t[k][0] = (float)a.x * c; t[k][1] = (float)a.y * c; t[k][2] = (float)a.z * c; t[k][3] = (float)a.w * c;
             t[k][4] = (float)b.x * c; t[k][5] = (float)b.y * c; t[k][6] = (float)b.z * c; t[k][7] = (float)b.w * c;
+            if (col + 8 > cols) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) if (col + i >= cols) t[k][i] = -INFINITY;
+            }
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) t[k][i] = (col + i < cols) ? (float)__ldg(sr + col + i) * c : -INFINITY;
@@ -87,14 +94,13 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
     for (int k = 0; k < NCH; ++k) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const int col = k * 256 + lane * 8 + i;
-            const float e = (col < cols) ? exp_reduced(t[k][i], mx) : 0.0f;
+            const float e = exp_reduced(t[k][i], mx);
             t[k][i] = e;
             const uint32_t eb = __float_as_uint(e);
             uint32_t hi, lo;
             asm("mad.hi.u32 %0, %1, 536870912, 939524096;" : "=r"(hi) : "r"(eb));    // (eb >> 3) + 0x38000000
             asm("mul.lo.u32 %0, %1, 536870912;" : "=r"(lo) : "r"(eb));                // eb << 29
-            const double ed = (col < cols) ? __hiloint2double((int)hi, (int)lo) : 0.0;
+            const double ed = __hiloint2double((int)hi, (int)lo);
             if (i & 1) z1 += ed; else z0 += ed;
         }
     }
@@ -105,7 +111,6 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
     const float rzh = (float)rz, rzl = (float)(rz - (double)(float)rz);   // 1/Z as two floats
     const Divisor dv = make_divisor(p_step);
 
-    constexpr uint32_t MASK = (1u << C) - 1u;
     const int chunk_bytes = 32 * C;                                   // 256 codes
     const int n_out_chunks = (int)((pitch + chunk_bytes - 1) / chunk_bytes);
     for (int k = 0; k < n_out_chunks; ++k) {
@@ -129,11 +134,23 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
                     for (int i = 0; i < 8; ++i) if (col + i < cols) pr[i] = p[i];
                 }
             }
+            // p >= 0, so only the upper clamp is needed; adding 1.5*2^23 rounds to nearest even and leaves the
+            // (unsigned) code in the low mantissa bits, and the codes combine by shift-add without masking
+            uint32_t cb[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t q = (col + i < cols) ? (round_clamp_bits(div_rn(p[i], dv), 0.0f, qp) & 0xFFu) : 0u;
-                if (C == 8) { if (i < 4) w0 |= q << (8 * i); else w1 |= q << (8 * (i - 4)); }
-                else w0 |= (q & MASK) << (C * i);
+            for (int i = 0; i < 8; ++i) cb[i] = __float_as_uint(fminf(div_rn(p[i], dv), qp) + 12582912.0f);
+            if (C == 8) {
+                w0 = cb[0] + (cb[1] << 8) + (cb[2] << 16) + (cb[3] << 24) - 0x4B400000u * 0x01010101u;
+                w1 = cb[4] + (cb[5] << 8) + (cb[6] << 16) + (cb[7] << 24) - 0x4B400000u * 0x01010101u;
+            } else {
+                uint32_t acc = cb[0];
+#pragma unroll
+                for (int i = 1; i < 8; ++i) acc += cb[i] << (C * i);
+                uint32_t ones = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) ones += 1u << (C * i);
+                w0 = acc - 0x4B400000u * ones;
+                if (C == 2) w0 &= 0xFFFFu;
             }
         }
         uint8_t* orow = out + row * pitch;
