@@ -76,9 +76,14 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
 #pragma unroll
                 for (int i = 0; i < 8; ++i) if (col + i >= cols) t[k][i] = -INFINITY;
             }
-        } else {
+        } else if (col < cols) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) t[k][i] = (col + i < cols) ? (float)__ldg(sr + col + i) * c : -INFINITY;
+        } else {
+            // lanes wholly past the row: nothing to load (kept apart so that a warp whose other lanes all took the
+            // vector path does not walk the scalar one as well)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) t[k][i] = -INFINITY;
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) mx = fmaxf(mx, t[k][i]);
