@@ -211,13 +211,19 @@ softmax_shift_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int c
     for (int k = 0; k < NCH; ++k) {
         const int col = k * 256 + lane * 8;
         int sv[8];
-        if (vec_in && col + 8 <= cols) {
+        if (vec_in && col + 8 <= ld_s) {
+            // whole 32 bytes inside the row's storage; values past the last column are masked below
             const int4 a = __ldg(reinterpret_cast<const int4*>(sr + col));
             const int4 b = __ldg(reinterpret_cast<const int4*>(sr + col) + 1);
             sv[0] = a.x; sv[1] = a.y; sv[2] = a.z; sv[3] = a.w; sv[4] = b.x; sv[5] = b.y; sv[6] = b.z; sv[7] = b.w;
-        } else {
+        } else if (col < cols) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) sv[i] = (col + i < cols) ? __ldg(sr + col + i) : 0;
+        } else {
+            // lanes wholly past the row: nothing to load (kept apart so that a warp whose other lanes all took the
+            // vector path does not walk the scalar one as well)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sv[i] = 0;
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
