@@ -258,6 +258,12 @@ softmax_shift_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int c
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sigma += __shfl_xor_sync(0xffffffffu, sigma, o);
     const float sig_f = __ull2float_rn(sigma);
+    // The comparator references fl32(fl32((t - 1/2) * step) * Sigma), t = 1 .. 2^bits - 1, depend on the row only:
+    // formed once per row and kept in registers (entries past the code range stay +inf and are never exceeded).
+    float thr[16];
+#pragma unroll
+    for (int tcode = 1; tcode < 16; ++tcode)
+        thr[tcode] = tcode < (1 << code_bits) ? __fmul_rn(__fmul_rn(__fsub_rn((float)tcode, 0.5f), p_step), sig_f) : INFINITY;
 
     constexpr uint32_t MASK = (1u << C) - 1u;
     const int chunk_bytes = 32 * C;
@@ -272,11 +278,28 @@ softmax_shift_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int c
                     for (int i = 0; i < 8; ++i) {
                         const unsigned long long e = ((unsigned long long)(uint32_t)fi[u][i] << 32) | mant[u][i];
                         const float e_f = __ull2float_rn(e);
+                        // the references ascend, so the number exceeded is found bit by bit; with the candidates in
+                        // registers each step is one comparison and a halving of the candidate list by selects
                         uint32_t code = 0;
-                        for (int b = code_bits - 1; b >= 0; --b) {
-                            const uint32_t t = code | (1u << b);
-                            const float thr = __fmul_rn(__fmul_rn(__fsub_rn((float)t, 0.5f), p_step), sig_f);
-                            code = (e_f > thr) ? t : code;
+                        if (code_bits > 4) {
+                            // wide codes: the references are formed on the fly, one comparison per code bit
+                            for (int b = code_bits - 1; b >= 0; --b) {
+                                const uint32_t tc = code | (1u << b);
+                                const float th = __fmul_rn(__fmul_rn(__fsub_rn((float)tc, 0.5f), p_step), sig_f);
+                                code = (e_f > th) ? tc : code;
+                            }
+                        } else {
+                        float cand[7];
+                        const bool p3 = e_f > thr[8];
+#pragma unroll
+                        for (int j = 0; j < 7; ++j) cand[j] = p3 ? thr[9 + j] : thr[1 + j];
+                        const bool p2 = e_f > cand[3];
+#pragma unroll
+                        for (int j = 0; j < 3; ++j) cand[j] = p2 ? cand[4 + j] : cand[j];
+                        const bool p1 = e_f > cand[1];
+                        cand[0] = p1 ? cand[2] : cand[0];
+                        const bool p0 = e_f > cand[0];
+                        code = (p3 ? 8u : 0u) + (p2 ? 4u : 0u) + (p1 ? 2u : 0u) + (p0 ? 1u : 0u);
                         }
                         const int col = k * 256 + lane * 8 + i;
                         if (col >= cols) code = 0;
