@@ -129,3 +129,23 @@ def test_product_fold_matches_definition(L):
     assert np.allclose(be, b / 0.25, rtol=1e-6)
     a2, be2 = L.fold_requant(np.float32(0.3), s_w, None, np.float32(0.25))
     assert np.array_equal(a, a2) and not be2.any()
+
+
+def test_layernorm_reference_folding_matches_the_oracle_side(L):
+    """The binding's host-side folding of the comparator references (Fig. 5(b)) and the oracle's are two separate
+    pieces of code that must hand their sides the same numbers: magnitude, sign and flip flag, bit for bit."""
+    import numpy as np
+    import oracle as vo
+    rng = np.random.default_rng(5)
+    cols = 48
+    gamma = rng.normal(1.0, 0.4, cols).astype(np.float32)
+    gamma[[3, 17]] *= -1.0
+    beta = rng.normal(0.0, 0.5, cols).astype(np.float32)
+    for bits, signed in ((2, True), (3, True), (4, True), (4, False)):
+        ref, neg, flip = vo.layernorm_references(gamma, beta, 0.31, bits, signed, cols)
+        refs, flip_b = L.fold_layernorm_references(gamma, beta, 0.31, bits, signed, cols)
+        assert refs.shape == (cols, 2 ** bits - 1) and refs.dtype == np.float32
+        assert np.array_equal(np.abs(refs).view(np.uint32), ref.view(np.uint32))
+        assert np.array_equal(np.signbit(refs) & (refs != 0), (neg != 0) & (ref != 0))
+        assert np.array_equal(flip_b, flip) and flip_b.sum() == 2
+        assert np.all(np.diff(refs.astype(np.float64), axis=1) >= 0)      # ascending along the thresholds
