@@ -401,6 +401,43 @@ def test_layernorm_compare_quantize_bit_exact(rows, cols, bits, container):
     assert padding_is_zero(got)
 
 
+def test_layernorm_compare_quantize_widest_row_and_single_row():
+    """The widest supported row (4096 columns: the reciprocal table fills 32 KB of shared memory) and a single row."""
+    rows, cols, bits = 3, 4096, 3
+    x = si.normal(77, (rows, cols), -0.2, 1.1)
+    g = si.normal(78, (cols,), 1.0, 0.1)
+    b = si.normal(79, (cols,), 0.0, 0.1)
+    step = si.gaussian_lsq_step(1.0, bits)
+    ref, neg, flip = vo.layernorm_references(g, b, step, bits, True, cols)
+    q_ref, mu_ref, v_ref = vo.layernorm_compare_quantize(x, ref, neg, flip, 1e-6, bits, True, want_stats=True)
+    refs_g, flip_g = vt.fold_layernorm_references(g, b, step, bits, True, cols)
+    n_eps = float(np.float32(np.float64(cols) * np.float64(np.float32(1e-6))))
+    for r0, r1 in ((0, rows), (1, 2)):
+        got, stats = vt.vitint_layernorm_compare_quantize(dev(x[r0:r1]), dev(refs_g), dev(flip_g), n_eps, bits, True)
+        st = stats.cpu().numpy()
+        assert np.array_equal(st[:, 0].view(np.uint32), mu_ref[r0:r1].view(np.uint32))
+        assert np.array_equal(st[:, 1].view(np.uint32), v_ref[r0:r1].view(np.uint32))
+        assert np.array_equal(from_codes(got), q_ref[r0:r1])
+    with pytest.raises(vt.VitintError):               # one more group of four columns is beyond the table
+        wide = torch.zeros((2, 4100), dtype=torch.float32, device="cuda")
+        r2, f2 = vt.fold_layernorm_references(np.ones(4100), np.zeros(4100), step, bits, True, 4100)
+        vt.vitint_layernorm_compare_quantize(wide, dev(r2), dev(f2), 1e-3, bits, True)
+
+
+def test_attention_core_prepared_argument_checks():
+    qkv = vt.Codes.empty(197, 3 * 64, 4, True)
+    qkv.data.zero_()
+    out = vt.Codes.empty(197, 64, 4, True)
+    alpha = torch.ones(64, dtype=torch.float32, device="cuda")
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(vt.VitintError):               # table too small for 4-bit codes
+        vt.vitint_attention_core_prepared(qkv, 1, 1, 197, 0.1, 0.1, 0.01, 4, alpha, None, out=out, table=small)
+    with pytest.raises(vt.VitintError):               # no table-driven kernel for 8-bit codes
+        vt.vitint_attention_exp_table(8, 0.1, 0.1, table=small)
+    with pytest.raises(vt.VitintError):               # steps must be positive and finite
+        vt.vitint_attention_exp_table(4, 0.0, 0.1)
+
+
 def test_layernorm_compare_quantize_argument_checks():
     x = torch.zeros((8, 64), dtype=torch.float32, device="cuda")
     refs, flip = vt.fold_layernorm_references(np.ones(64), np.zeros(64), 0.5, 4, True, 64)
