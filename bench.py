@@ -327,6 +327,16 @@ def run_ours(args, cfg):
         standalone["deit_s_attention_n198_b64"] = {"ms": round(ms, 4), "tops": round(mod.ops() / (ms * 1e-3) / 1e12, 1),
                                                    "images_per_s": round(dcfg.batch / (ms * 1e-3), 1), "launches": 10}
         del mod, dx, dxq
+        # the same encoder layer with the paper's own quantizers throughout (Eq. 4 softmax with the division-free
+        # comparator, Eq. 5 statistics with the comparator LayerNorm quantizer): unfused attention, 11 launches
+        from paper_2504_18547_b200.encoder import EncoderLayer as _Layer
+        plain = _Layer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, device, softmax="shift",
+                       layernorm="compare")
+        ms = timed(lambda: plain.forward(xs[0], out), reps=5)
+        standalone["layer_with_comparator_quantizers"] = {"ms": round(ms, 4), "tops": round(ops_step / (ms * 1e-3) / 1e12, 1),
+                                                          "images_per_s": round(cfg.batch / (ms * 1e-3), 1),
+                                                          "launches": len(plain.stages) + 2}
+        del plain
         # the whole DeiT-S-shaped model (patch embedding, 198 tokens, 12 layers, final LayerNorm, two heads), batch 128
         from paper_2504_18547_b200.encoder import DeitModel
         mcfg = si.DEIT_S_MODEL
