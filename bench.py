@@ -49,36 +49,83 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples the SM clock and the clock-event (throttle) reasons of one GPU while timed regions run.
+
+    Readings come from NVML (the library nvidia-smi itself reads; read-only queries) every ~2 ms on a thread of
+    this process, each with a host timestamp, so that a region only a few milliseconds long still gets samples
+    taken INSIDE it: window(t0, t1) summarises the samples whose timestamps fall between two perf_counter()
+    readings.  Without NVML it falls back to polling `nvidia-smi -lms 20`."""
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+    MASKS = (0x8, 0x40, 0x20, 0x4)      # NVML clock-event reason bits, in the order of NAMES
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, index: int, pci_bus_id: str | None = None):
+        self.index, self.pci, self.samples, self.source = index, pci_bus_id, [], None
+        self._stop = threading.Event()
+        self._thread = self._proc = None
+        self.max_mhz = None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
-            threading.Thread(target=self._read, daemon=True).start()
+            import pynvml
+            pynvml.nvmlInit()
+            try:
+                h = pynvml.nvmlDeviceGetHandleByPciBusId(self.pci.encode()) if self.pci else None
+            except Exception:
+                h = None
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            reasons_fn = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
+
+            def poll():
+                while not self._stop.is_set():
+                    try:
+                        mhz = float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                        mask = int(reasons_fn(h))
+                        self.samples.append((time.perf_counter(), mhz, mask))
+                    except Exception:
+                        pass
+                    time.sleep(0.002)
+            self.source = "nvml"
+            self._thread = threading.Thread(target=poll, daemon=True)
+            self._thread.start()
+            return
+        except Exception:
+            pass
+        try:
+            self._proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                           "-i", str(self.index), "-lms", "20"], stdout=subprocess.PIPE, text=True)
+
+            def read():
+                for line in self._proc.stdout:
+                    c = [v.strip() for v in line.split(",")]
+                    if len(c) >= 6 and c[0].replace(".", "").isdigit():
+                        mask = sum(m for m, v in zip(self.MASKS, c[2:6]) if v.lower() == "active")
+                        self.samples.append((time.perf_counter(), float(c[0]), mask))
+                        if c[1].replace(".", "").isdigit():
+                            self.max_mhz = float(c[1])
+            self.source = "nvidia-smi"
+            self._thread = threading.Thread(target=read, daemon=True)
+            self._thread.start()
         except OSError:
-            self.proc = None
+            self.source = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+    def window(self, t0: float, t1: float) -> dict:
+        """Median SM clock and the union of the reasons over the samples taken in [t0, t1]."""
+        if self.source is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source"], "samples": 0}
+        sel = [x for x in list(self.samples) if t0 <= x[0] <= t1]
+        reasons = sorted({n for _, _, mask in sel for n, m in zip(self.NAMES, self.MASKS) if mask & m})
+        return {"sm_mhz": float(np.median([x[1] for x in sel])) if sel else None, "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(sel), "source": self.source}
 
-    def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        mhz = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
-        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = sorted({n for r in self.rows if len(r) >= 6 for n, v in zip(names, r[2:6]) if v.lower() == "active"})
-        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(mhz)}
+    def stop(self):
+        self._stop.set()
+        if self._proc is not None:
+            self._proc.terminate()
 
 
 def dist_env():
@@ -178,37 +225,61 @@ def run_ours(args, cfg):
     if vt.vitint_device_status() != 0:
         raise RuntimeError("device-side timeout during warm-up")
 
-    sampler = ClockSampler(local_rank)
+    pci = None
+    try:
+        pr = torch.cuda.get_device_properties(local_rank)
+        pci = "%08x:%02x:%02x.0" % (pr.pci_domain_id, pr.pci_bus_id, pr.pci_device_id)
+    except Exception:
+        pass
+    sampler = ClockSampler(local_rank, pci)
     if rank == 0:
         sampler.start()
-        time.sleep(0.25)
+        time.sleep(0.05)
 
-    # ---- device-resident timing: exactly K steps back to back ---------------------------
-    # No event sits between two kernels here: each kernel is launched as a programmatic dependent of the
-    # one before it, and a stream operation in between would put the plain launch gap back.
-    barrier()
-    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for i in range(args.steps):
-        layer.forward(xs[i % N_INPUT_BUFFERS], out)
-    t_end.record()
-    barrier()
-    ms_total = max_over_ranks(t_start.elapsed_time(t_end), world, device)
-    clocks = sampler.stop() if rank == 0 else None
+    def timed_steps(n):
+        """n steps back to back, timed with CUDA events on the launching stream, max over ranks; also returns
+        the host-clock window of the region for the clock samples."""
+        # No event sits between two kernels here: each kernel is launched as a programmatic dependent of the
+        # one before it, and a stream operation in between would put the plain launch gap back.
+        barrier()
+        w0 = time.perf_counter()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(n):
+            layer.forward(xs[i % N_INPUT_BUFFERS], out)
+        b.record()
+        barrier()
+        return max_over_ranks(a.elapsed_time(b), world, device), (w0, time.perf_counter())
 
-    # ---- per-stage breakdown: the same K steps again, with an event around every call ---
-    ev_steps = []
-    for i in range(args.steps):
-        ev = []
-        layer.forward(xs[i % N_INPUT_BUFFERS], out, events=ev)
-        ev_steps.append(ev)
-    torch.cuda.synchronize()
+    def stage_breakdown(n):
+        """The same steps again with an event around every call: per-stage milliseconds."""
+        ev_steps = []
+        for i in range(n):
+            ev = []
+            layer.forward(xs[i % N_INPUT_BUFFERS], out, events=ev)
+            ev_steps.append(ev)
+        torch.cuda.synchronize()
+        acc = {s: 0.0 for s in STAGES}
+        for ev in ev_steps:
+            for j, s in enumerate(STAGES):
+                acc[s] += ev[j].elapsed_time(ev[j + 1])
+        return {s: v / n for s, v in acc.items()}
 
-    stage_ms = {s: 0.0 for s in STAGES}
-    for ev in ev_steps:
-        for j, s in enumerate(STAGES):
-            stage_ms[s] += ev[j].elapsed_time(ev[j + 1])
-    stage_ms = {s: v / args.steps for s, v in stage_ms.items()}
+    # ---- device-resident timing: exactly K steps back to back (a burst: a few milliseconds) ------------
+    ms_total, win = timed_steps(args.steps)
+    clocks = sampler.window(*win) if rank == 0 else None
+    stage_ms = stage_breakdown(args.steps)
+
+    # ---- sustained leg: the same step repeated for several seconds, clock sampled inside the loop -------
+    sustained = None
+    if args.sustain_seconds > 0:
+        n_sus = max(args.steps, int(np.ceil(args.sustain_seconds * 1e3 / (ms_total / args.steps))))
+        ms_sus, win_s = timed_steps(n_sus)
+        stage_ms_sus = stage_breakdown(min(50, n_sus))          # taken right behind the loop, still at its clocks
+        sustained = {"steps": n_sus, "seconds": ms_sus * 1e-3, "ms_per_step": ms_sus / n_sus,
+                     "clocks": sampler.window(*win_s) if rank == 0 else None, "stage_ms": stage_ms_sus}
+    if rank == 0:
+        sampler.stop()
 
     # ---- end to end: host -> device, step, device -> host, every step -----------------
     # Three streams, double-buffered device input and output: the copy of step i+1's input and the read-back
@@ -264,8 +335,19 @@ def run_ours(args, cfg):
     sops = layer.stage_ops()
     gemm_ms = sum(stage_ms[s] for s in gemm_stages)
     gemm_ops = sum(sops[s] for s in gemm_stages)
-    int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+    # The K timed steps are a burst (milliseconds at the boost clock): their fractions are taken against the
+    # burst figure of the measured bf16 peak; the sustained leg's against the sustained figure.
+    int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
+    int8_peak_sustained = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
+    if sustained is not None:
+        g_ms = sum(sustained["stage_ms"][s] for s in gemm_stages)
+        sus_tops = world * ops_step / (sustained["ms_per_step"] * 1e-3) / 1e12
+        sustained.update({"value": sus_tops, "unit": "TOPS",
+                          "images_per_s": world * cfg.batch / (sustained["ms_per_step"] * 1e-3),
+                          "gemm_achieved": gemm_ops / (g_ms * 1e-3) / 1e12, "gemm_peak": int8_peak_sustained,
+                          "gemm_frac": gemm_ops / (g_ms * 1e-3) / 1e12 / int8_peak_sustained,
+                          "stage_ms": {k: round(v, 4) for k, v in sustained["stage_ms"].items()}})
     sbytes = layer.stage_bytes()
     kernels = {}
     for s in STAGES:
@@ -361,6 +443,26 @@ def run_ours(args, cfg):
                                                  "launches": 8 * ecfg.layers}
         del stack, ex, eout
 
+    # ---- a library int8 GEMM in the same run, as context for the int8 ceiling (never on the product path) ----
+    library_int8 = None
+    if world == 1 and not args.no_standalone and hasattr(torch, "_int_mm"):
+        try:
+            n = 8192
+            la = torch.randint(-8, 8, (n, n), dtype=torch.int8, device=device)
+            lb = torch.randint(-8, 8, (n, n), dtype=torch.int8, device=device).t()
+            for _ in range(3):
+                torch._int_mm(la, lb)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                torch._int_mm(la, lb)
+            e1.record()
+            torch.cuda.synchronize()
+            library_int8 = 2.0 * n ** 3 * 10 / (e0.elapsed_time(e1) * 1e-3) / 1e12
+            del la, lb
+        except Exception:
+            library_int8 = None
+
     # ---- CPU oracle on a bounded sample (rank 0, single-GPU runs only) -----------------
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -401,8 +503,14 @@ def run_ours(args, cfg):
         "roofline": {"bound": "tensor", "kernel": f"gemm_i8_kernel ({len(gemm_stages)} launches per step)", "achieved": achieved,
                      "peak": int8_peak, "unit": "TOPS", "frac": achieved / int8_peak, "traffic": traffic,
                      "timing": "CUDA events around every call, second pass over the same K steps (the timed K steps carry no events)",
-                     "peak_source": f"{peaks['source']} sustained bf16 cuBLAS x {INT8_OVER_BF16:g} (nominal int8:bf16)",
-                     "frac_of_nominal_4500": achieved / 4500.0},
+                     "peak_source": f"{peaks['source']} burst bf16 cuBLAS x {INT8_OVER_BF16:g} (nominal int8:bf16); the K steps are a burst",
+                     "frac_of_nominal_4500": achieved / 4500.0,
+                     "achieved_sustained": sustained["gemm_achieved"] if sustained else None,
+                     "peak_sustained": int8_peak_sustained,
+                     "frac_sustained": sustained["gemm_frac"] if sustained else None,
+                     "library_int8_tops": library_int8,
+                     "library_int8_note": "torch._int_mm 8192^3 in this run: context for the int8 ceiling, not on the product path"},
+        "sustained": sustained,
         "kernels": kernels,
         "kernels_standalone": standalone,
         "cpu_baseline": cpu,
@@ -418,12 +526,22 @@ def run_ours(args, cfg):
 
 SWEEP_KN = (192, 384, 768, 1024, 3072, 4096)
 SWEEP_TOKENS_BATCH = ((197, 256), (577, 64), (785, 32))
+SWEEP_BATCHES = {197: (1, 8, 64, 256), 577: (1, 8, 64), 785: (1, 8, 32)}
+SWEEP_KN_THIN = ((192, 192), (768, 768), (768, 3072), (3072, 768), (4096, 4096))
 
 
 def run_sweep(args):
-    """Times vitint_linear (requantizing epilogue) for every K, N of SWEEP_KN at M = tokens x batch, 4-bit codes
-    stored one per byte and 8-bit codes, against the int8 tensor roofline, and the quantize and softmax kernels at
-    the same token counts against the HBM roofline.  Prints ONE JSON line; operands are seeded and synthetic
+    """The scaling study over K, N, tokens, batch and bit width.  ONE JSON line with five tables:
+    linear          vitint_linear, requantizing epilogue, every K, N of SWEEP_KN at M = tokens x batch (the largest
+                    batch per token count), 4-bit codes stored one per byte and 8-bit codes;
+    linear_batch    the same call at batch 1 ... 256 on a thinned K, N grid;
+    linear_formats  bit-packed 2-, 3- and 4-bit operands (activations packed, weights packed or widened once) and the
+                    fp32 (dequantizing) epilogue;
+    attention       the fused core (up to 256 tokens) and the unfused Q K^T -> softmax -> P V sequence (577 and 785
+                    tokens), 12 heads, batch 1 ... 256;
+    streaming       quantize and the two softmax kernels against the HBM roofline.
+    GEMM-shaped points are given against the int8 tensor roofline.  Every point is timed alone with the L2 flushed
+    before each timed call (a burst), so the tensor peak is the burst figure.  Operands are seeded and synthetic
     (uniform random codes, which is all the timing depends on)."""
     import torch
 
@@ -432,7 +550,7 @@ def run_sweep(args):
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
     peaks = measured_peaks()
-    int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+    int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
     gen = torch.Generator(device=device)
     gen.manual_seed(si.BASE_SEED)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)       # larger than L2
@@ -451,13 +569,34 @@ def run_sweep(args):
             t += a.elapsed_time(b)
         return t / reps
 
-    def codes(rows, cols, bits):
-        qn, qp = si.code_range(bits, True)
+    def codes(rows, cols, bits, signed=True, container=8):
+        """Random codes of the declared range, one per byte (container 8) or bit-packed."""
+        qn, qp = si.code_range(bits, signed)
         t = torch.randint(qn, qp + 1, (rows, cols), dtype=torch.int8, device=device, generator=gen)
-        return vt.Codes(t.view(torch.uint8), rows, cols, bits, True, 8)
+        if container == 8:
+            return vt.Codes(t.view(torch.uint8), rows, cols, bits, signed, 8)
+        c = 4 if bits == 3 else bits
+        per = 8 // c
+        v = (t.to(torch.int32) & ((1 << c) - 1)).view(rows, cols // per, per)
+        sh = torch.arange(per, device=device, dtype=torch.int32) * c
+        return vt.Codes((v << sh).sum(dim=2).to(torch.uint8).contiguous(), rows, cols, bits, signed, 0)
 
+    def requant_epi(N, K, bits, container=8):
+        alpha = torch.full((N,), 1.0 / (K ** 0.5 * 2.0 ** (bits - 1)), dtype=torch.float32, device=device)
+        beta = torch.zeros((N,), dtype=torch.float32, device=device)
+        return vt.Epilogue(mode=vt.EPI_REQUANT, alpha=alpha, beta=beta, out_bits=bits, out_signed=True,
+                           out_container=container)
+
+    def lin_point(M, K, N, bits, x, w, epi, out, **tags):
+        ms = timed(lambda: vt.vitint_linear(x, 1.0, w, epi_args.get("w_step"), epi_args.get("bias"), epi, out=out), args.steps)
+        tops = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+        return dict(tags, bits=bits, K=K, N=N, M=M, ms=round(ms, 4), tops=round(tops, 1),
+                    frac_int8_peak=round(tops / int8_peak, 4))
+
+    epi_args = {}
     sampler = ClockSampler(0)
     sampler.start()
+    w_start = time.perf_counter()
     linear = []
     for tokens, batch in SWEEP_TOKENS_BATCH:
         M = tokens * batch
@@ -466,17 +605,79 @@ def run_sweep(args):
                 x = codes(M, K, bits)
                 for N in SWEEP_KN:
                     w = codes(N, K, bits)
-                    alpha = torch.full((N,), 1.0 / (K ** 0.5 * 2.0 ** (bits - 1)), dtype=torch.float32, device=device)
-                    beta = torch.zeros((N,), dtype=torch.float32, device=device)
-                    epi = vt.Epilogue(mode=vt.EPI_REQUANT, alpha=alpha, beta=beta, out_bits=bits, out_signed=True,
-                                      out_container=8)
                     out = vt.Codes.empty(M, N, bits, True, device, container=8)
-                    ms = timed(lambda: vt.vitint_linear(x, 1.0, w, None, None, epi, out=out), args.steps)
-                    tops = 2.0 * M * N * K / (ms * 1e-3) / 1e12
-                    linear.append({"tokens": tokens, "batch": batch, "bits": bits, "K": K, "N": N, "ms": round(ms, 4),
-                                   "tops": round(tops, 1), "frac_int8_peak": round(tops / int8_peak, 4)})
+                    linear.append(lin_point(M, K, N, bits, x, w, requant_epi(N, K, bits), out, tokens=tokens, batch=batch))
                     del w, out
                 del x
+    linear_batch = []
+    for tokens, batches in SWEEP_BATCHES.items():
+        for batch in batches:
+            M = tokens * batch
+            for K, N in SWEEP_KN_THIN:
+                x, w = codes(M, K, 4), codes(N, K, 4)
+                out = vt.Codes.empty(M, N, 4, True, device, container=8)
+                linear_batch.append(lin_point(M, K, N, 4, x, w, requant_epi(N, K, 4), out, tokens=tokens, batch=batch))
+                del x, w, out
+    linear_formats = []
+    M = 197 * 64
+    for K, N in ((768, 768), (768, 3072), (3072, 768)):
+        for bits in (2, 3, 4):
+            xp = codes(M, K, bits, container=0)
+            for wname, w in (("packed", codes(N, K, bits, container=0)), ("one per byte", codes(N, K, bits))):
+                out = vt.Codes.empty(M, N, bits, True, device)
+                linear_formats.append(lin_point(M, K, N, bits, xp, w, requant_epi(N, K, bits, 0), out, activations="packed",
+                                                weights=wname, epilogue="requantize, packed output"))
+                del out
+            del xp
+        # fp32 epilogue (scale, bias, no residual) on codes stored one per byte
+        x, w = codes(M, K, 4), codes(N, K, 4)
+        epi_args = {"w_step": torch.full((N,), 0.01, dtype=torch.float32, device=device),
+                    "bias": torch.zeros((N,), dtype=torch.float32, device=device)}
+        outf = torch.empty((M, N), dtype=torch.float32, device=device)
+        linear_formats.append(lin_point(M, K, N, 4, x, w, vt.Epilogue(mode=vt.EPI_DEQUANT_F32), outf, activations="one per byte",
+                                        weights="one per byte", epilogue="fp32 (scale + bias)"))
+        epi_args = {}
+        del x, w, outf
+    attention = []
+    heads, D = 12, 768
+    for tokens, batches in SWEEP_BATCHES.items():
+        for batch in batches:
+            M = tokens * batch
+            ops = 4.0 * batch * heads * tokens * tokens * 64
+            for bits in ((4, 2) if tokens <= 256 else (4,)):
+                qmax = 1 << (bits - 1)
+                s_qk = float(np.float32((3.0 / (qmax * qmax)) ** 0.5))
+                s_p = float(np.float32(2.0 / (tokens * (2 ** bits - 1) ** 0.5)))
+                alpha = torch.full((D,), 0.01, dtype=torch.float32, device=device)
+                if tokens <= 256:
+                    qkv = codes(M, 3 * D, bits)
+                    o = vt.Codes.empty(M, D, bits, True, device, container=8)
+                    table = vt.vitint_attention_exp_table(bits, s_qk, s_qk, device=device)
+                    ms = timed(lambda: vt.vitint_attention_core_prepared(qkv, batch, heads, tokens, s_qk, s_qk, s_p, bits,
+                                                                         alpha, None, out=o, table=table), args.steps)
+                    attention.append({"path": "fused core", "tokens": tokens, "batch": batch, "bits": bits,
+                                      "ms": round(ms, 4), "tops": round(ops / (ms * 1e-3) / 1e12, 1)})
+                    del qkv, o
+                else:
+                    qkv = codes(M, 3 * D, bits, container=0)
+                    sl = [vt.Slabs.of_qkv(qkv, tokens, D, i) for i in range(3)]
+                    ld_s = (tokens + 3) // 4 * 4
+                    S = torch.empty((batch * heads * tokens, ld_s), dtype=torch.int32, device=device)
+                    P = vt.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
+                    o = vt.Codes.empty(M, D, bits, True, device)
+                    epi = vt.Epilogue(mode=vt.EPI_REQUANT, alpha=alpha, out_bits=bits, out_signed=True)
+                    c = float(np.float32(s_qk * s_qk / 8.0))
+                    parts = {"qk": lambda: vt.vitint_qk(sl[0], sl[1], batch, heads, tokens, out=S, ld_s=ld_s),
+                             "softmax_quantize": lambda: vt.vitint_softmax_quantize(S, tokens, c, s_p, bits, out=P),
+                             "pv": lambda: vt.vitint_pv(P, sl[2], batch, heads, tokens, s_p, 0.1, epi, out=o)}
+                    pm = {k: round(timed(f, args.steps), 4) for k, f in parts.items()}
+                    ms = timed(lambda: [f() for f in parts.values()], args.steps)
+                    sm_bytes = S.shape[0] * tokens * 4 + S.shape[0] * ((tokens * (4 if bits == 3 else bits) + 7) // 8)
+                    attention.append({"path": "unfused qk -> softmax -> pv", "tokens": tokens, "batch": batch, "bits": bits,
+                                      "ms": round(ms, 4), "tops": round(ops / (ms * 1e-3) / 1e12, 1), "kernel_ms": pm,
+                                      "softmax_gbs": round(sm_bytes / (pm["softmax_quantize"] * 1e-3) / 1e9, 1),
+                                      "softmax_frac_hbm_peak": round(sm_bytes / (pm["softmax_quantize"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
+                    del qkv, S, P, o
     streaming = []
     for tokens, batch in SWEEP_TOKENS_BATCH:
         M = tokens * batch
@@ -500,17 +701,21 @@ def run_sweep(args):
                                   "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
                                   "frac_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
             del xf, xq, S, Pq
-    clocks = sampler.stop()
+    clocks = sampler.window(w_start, time.perf_counter())
+    sampler.stop()
     if vt.vitint_device_status() != 0:
         raise RuntimeError("device-side timeout during the sweep")
     best = max(linear, key=lambda r: r["tops"])
     print(json.dumps({"metric": "integerized linear sweep, effective TOPS", "value": best["tops"], "unit": "TOPS",
                       "n_gpus": 1, "steps": args.steps, "warmup": 3, "higher_is_better": True, "dtype": "int8",
-                      "data": "synthetic", "config": {"workload": "linear_and_streaming_sweep", "K_N": list(SWEEP_KN),
+                      "data": "synthetic", "config": {"workload": "linear_and_attention_sweep", "K_N": list(SWEEP_KN),
                                                       "tokens_batch": [list(t) for t in SWEEP_TOKENS_BATCH],
+                                                      "batches": {str(k): list(v) for k, v in SWEEP_BATCHES.items()},
                                                       "l2": "256 MB written between timed iterations"},
-                      "peaks": {"int8_tops": int8_peak, "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]},
-                      "clocks": clocks, "best": best, "linear": linear, "streaming": streaming}))
+                      "peaks": {"int8_tops": int8_peak, "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"],
+                                "int8_note": "burst bf16 cuBLAS x 2 (nominal int8 : bf16)"},
+                      "clocks": clocks, "best": best, "linear": linear, "linear_batch": linear_batch,
+                      "linear_formats": linear_formats, "attention": attention, "streaming": streaming}))
 
 
 def main():
@@ -523,6 +728,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="images per GPU (default: the configuration's 128)")
     ap.add_argument("--ref-images", type=int, default=None, help="images per step of the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustain-seconds", type=float, default=3.0,
+                    help="length of the sustained leg that follows the K timed steps (0 = skip it)")
     ap.add_argument("--sweep", action="store_true",
                     help="time the integer linear over K, N, tokens and bits, and the streaming kernels (one JSON line)")
     ap.add_argument("--no-standalone", action="store_true",
@@ -538,6 +745,20 @@ def main():
     if args.ref_images is None:
         args.ref_images = 64 if args.impl == "ours" else 8
     args.ref_images = min(args.ref_images, cfg.batch)
+    rank, _, world = dist_env()
+    if args.impl == "ours" and not args.sweep and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain process: start one rank per GPU of this node and let rank 0 print the line
+        import socket
+        sk = socket.socket()
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+        sk.close()
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve())] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
+    if args.impl == "ours" and not args.sweep and world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but {world} rank(s) were started (WORLD_SIZE); "
+                         "start it with one rank per GPU or let bench.py start them itself")
     if args.sweep:
         if dist_env()[0] == 0:
             run_sweep(args)

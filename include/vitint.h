@@ -101,13 +101,22 @@ int vitint_version(void);
  * the device.  Returns VITINT_OK, VITINT_ERR_TIMEOUT or VITINT_ERR_CUDA. */
 int vitint_device_status(void);
 
+/* Self-test of the bounded wait: launches one warp that waits on a barrier nothing ever completes, with a limit of
+ * `limit_cycles` SM clock cycles (1 .. 2e9; about a millisecond at 2e6).  When the limit passes the kernel records
+ * VITINT_ERR_TIMEOUT in the device status word, writes 1 to *gave_up (device int32, may be NULL) and returns; the
+ * context stays usable and the next vitint_device_status() reports (and clears) the timeout.  Asynchronous on
+ * `stream`.  Nothing faults, traps or spins without bound. */
+int vitint_selftest_wait_timeout(int64_t limit_cycles, int32_t* gave_up, void* stream);
+
 /* Bytes a packed row of `cols` b-bit codes needs, rounded up to 16. */
 int64_t vitint_packed_pitch(int64_t cols, int32_t bits);
 
 /* a1. Quantize and pack (Section IV-B comparator quantizer, round-to-nearest-even):
  *   q[m][k] = clamp(rint(x[m*ldx + k] / s_m)), s_m = row_steps[m] if row_steps != NULL
  *   (per-output-channel weight steps, Eq. 1's Delta_W) else `step` (the single input
- *   step of Eq. 2).  One IEEE fp32 division per element.
+ *   step of Eq. 2).  One IEEE fp32 division per element; non-finite inputs follow that definition (+-inf and any
+ *   quotient beyond the range clamp to the end levels, NaN gives Qn).  The steps in row_steps are the caller's
+ *   responsibility: a step that is zero, negative or not finite yields whatever the IEEE quotient rounds and clamps to.
  *   x: device fp32 [rows, ldx] (ldx >= cols, elements).  out: descriptor whose data,
  *   rows (== rows), cols (== cols), pitch_bytes, bits, is_signed are set by the caller;
  *   the whole pitch of every row is written (padding as zero).
@@ -220,12 +229,13 @@ int vitint_attention_core_prepared(const vitint_codes* qkv, int32_t batch, int32
  *   of exp(fl32(s*c)) over all integer scores -- comes from the library: a fixed device array of
  *   33,280 bytes that every GPU loading the library holds until the process exits.
  *   The function allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.
- *   Limit: the table must fit the array, i.e. 2-, 3- and 4-bit codes (at most 8193 entries);
- *   anything larger is rejected with VITINT_ERR_WORKSPACE (8-bit codes: VITINT_ERR_UNSUPPORTED,
- *   as in vitint_attention_core).  All other arguments, results and errors are those of
- *   vitint_attention_core.
+ *   Limit: the array holds the table of the widest codes the table-driven kernel takes (2-, 3- and
+ *   4-bit codes, at most 8193 entries); 8-bit codes are rejected with VITINT_ERR_UNSUPPORTED, as
+ *   in vitint_attention_core.  All other arguments, results and errors are those of
+ *   vitint_attention_core, argument errors being reported first.
  *   The first call on each device looks up the array's device address (with that device
- *   current); make that first call outside any stream capture.
+ *   current; concurrent first calls from several host threads are safe); make that first call
+ *   outside any stream capture.
  *   Every call on a device uses the same array and rewrites all the entries it needs, so nothing
  *   carries over between calls -- but two calls that overlap on the GPU (different streams) race
  *   on it: serialize calls per device. */
@@ -298,6 +308,20 @@ int vitint_layernorm_quantize(const float* x, int64_t rows, int64_t cols, int64_
 int vitint_layernorm_compare_quantize(const float* x, int64_t rows, int64_t cols, int64_t ldx, const float* refs,
                                       const uint8_t* flip, float n_eps, const vitint_codes* out, float* stats,
                                       void* stream);
+
+/* Host-side helpers (no device work, HOST pointers): the constants that the method absorbs into the stage behind a
+ * contraction, computed in fp64 and rounded once to fp32.
+ *   vitint_fold_requant (Eq. 2, "equivalent bias" and "post-scaling factor" followed by a quantizer of step
+ *     out_step[i]):  alpha[i] = x_step * w_step[i] / out_step[i],  beta[i] = bias[i] / out_step[i] (0 when bias is
+ *     NULL), i < n: the arguments of the REQUANT epilogue.  Steps must be positive and finite.
+ *   vitint_fold_layernorm_references (Fig. 5(b)):  for column j and threshold k = Qn+1 .. Qp,
+ *     c = ((k - 1/2) step - beta[j]) / gamma[j], negated where gamma[j] < 0 (then flip[j] = 1, else 0);
+ *     refs[j][k - Qn - 1] = sgn(c) c^2 / cols: the arguments of vitint_layernorm_compare_quantize.  gamma[j] != 0.
+ * Return VITINT_OK or VITINT_ERR_INVALID_ARG. */
+int vitint_fold_requant(float x_step, const float* w_step, const float* bias, const float* out_step, int64_t n,
+                        float* alpha, float* beta);
+int vitint_fold_layernorm_references(const float* gamma, const float* beta, float step, int32_t bits,
+                                     int32_t is_signed, int64_t cols, float* refs, uint8_t* flip);
 
 #ifdef __cplusplus
 }

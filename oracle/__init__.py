@@ -20,8 +20,7 @@ _SRC = _HERE / "vitint_oracle.cpp"
 _LIB = _HERE / "libvitint_oracle.so"
 _lib = None
 
-GELU_TOL_REL = float(2.0 ** -21)   # absolute tolerance of an fp32 GELU, as a fraction of |y|
-SOFTMAX_ULP_BAND = 2               # fp32 softmax probabilities may differ by this many ulp
+SOFTMAX_ULP_BAND = 2               # fp32 softmax probabilities may differ by this many ulp (the path's stated bound)
 
 
 def build(force: bool = False) -> Path:
@@ -156,8 +155,10 @@ def epilogue_requant(acc, alpha, beta, bits: int, signed: bool) -> np.ndarray:
     return q
 
 
-def epilogue_gelu_requant(acc, s_x, s_w, bias, inv_s, bits: int, signed: bool = False, tol_rel: float = GELU_TOL_REL):
-    """Returns (codes, lowest acceptable code, highest acceptable code)."""
+def epilogue_gelu_requant(acc, s_x, s_w, bias, inv_s, bits: int, signed: bool = False, tol_rel: float = 0.0):
+    """Returns (codes, lowest, highest): the codes of GELU(y) by the erf definition (fp64, rounded once), and the
+    codes reached when that value moves by -/+ tol_rel*|y|.  The tolerance belongs to whoever checks an fp32
+    implementation against this and is passed in; with the default 0 the three arrays are equal."""
     acc = np.ascontiguousarray(acc, dtype=np.int32)
     M, N = acc.shape
     s_w, bias, inv_s = _f32(s_w), _f32(bias), _f32(inv_s)

@@ -155,7 +155,7 @@ def normed_attention(x_codes, s_x, prm: dict, qkn: dict, batch: int, tokens: int
 
 
 def encoder_layer(x, prm: dict, batch: int, tokens: int, heads: int, bits: int, head_dim: int = 64,
-                  eps: float = 1e-6, softmax: str = "exp", layernorm: str = "fp32") -> dict:
+                  eps: float = 1e-6, softmax: str = "exp", layernorm: str = "fp32", gelu_tol_rel: float = 0.0) -> dict:
     """LN1 -> quantize -> attention (+residual) -> LN2 -> quantize -> fc1 -> GELU -> quantize -> fc2 (+residual).
     layernorm="compare": both LayerNorm + quantize stages run as Eq. 5 statistics with the comparator quantizer of
     Fig. 5(b); their levels are then unique (the band collapses to the code itself)."""
@@ -184,7 +184,8 @@ def encoder_layer(x, prm: dict, batch: int, tokens: int, heads: int, bits: int, 
     inv_g = inv_step(np.full(w_fc1.shape[0], prm["s_g"], np.float32))
     st["inv_s_g"] = inv_g
     st["g_codes"], st["g_lo"], st["g_hi"] = vo.epilogue_gelu_requant(st["acc_fc1"], prm["s_ln"], prm["s_w_fc1"],
-                                                                     prm["b_fc1"], inv_g, bits, False)
+                                                                     prm["b_fc1"], inv_g, bits, False,
+                                                                     tol_rel=gelu_tol_rel)
     st["acc_fc2"] = vo.matmul_i32(st["g_codes"], w_fc2)
     st["out"] = vo.epilogue_dequant(st["acc_fc2"], prm["s_g"], prm["s_w_fc2"], prm["b_fc2"], h)
     return st
@@ -227,4 +228,92 @@ def deit_forward(patches, ends: dict, layer_params: list, batch: int, tokens: in
         w = vo.quantize(ends["w_" + name], 0.0, bits, True, row_steps=ends["s_w_" + name])
         logits = vo.epilogue_dequant(vo.matmul_i32(q, w), ends["s_lnf"], ends["s_w_" + name], ends["b_" + name], logits)
     st["logits"] = logits
+    return st
+
+
+def o_band_from_p_band(p_lo, p_hi, v, alpha_o, bits: int):
+    """Codes of O = requant(P V) reachable when every P code may lie anywhere in [p_lo, p_hi] (Section IV-B's
+    W_attn V followed by its absorbing quantizer).  The requantizer is monotone in the accumulator (alpha_o > 0),
+    so the extremes are reached by taking, per term, the end of the P interval that the sign of V favours.
+    p_lo, p_hi: [n, T, T]; v: [n, T, d] signed codes; returns (o_lo, o_hi) as [n*T, d] codes."""
+    assert np.all(np.asarray(alpha_o) > 0)
+    vp_, vn_ = np.maximum(v, 0).astype(np.int16), np.minimum(v, 0).astype(np.int16)
+    n, T, d = v.shape
+    acc_lo = vo.pv(p_lo, vp_) + vo.pv(p_hi, vn_)
+    acc_hi = vo.pv(p_hi, vp_) + vo.pv(p_lo, vn_)
+    zero = np.zeros_like(np.asarray(alpha_o, np.float32))
+    o_lo = vo.epilogue_requant(acc_lo.reshape(n * T, d), alpha_o, zero, bits, True)
+    o_hi = vo.epilogue_requant(acc_hi.reshape(n * T, d), alpha_o, zero, bits, True)
+    return o_lo, o_hi
+
+
+def encoder_layer_stagewise(x, prm: dict, batch: int, tokens: int, heads: int, bits: int, given: dict,
+                            head_dim: int = 64, eps: float = 1e-6, softmax: str = "exp",
+                            layernorm: str = "fp32") -> dict:
+    """The stages of encoder_layer(), each computed from GIVEN upstream values instead of from this function's own
+    previous stage: given["x1"], ["qkv"], ["O"], ["x2"], ["g"] are code matrices, given["h"] the fp32 residual
+    stream after the attention block, given["P"] (optional, [batch*heads, T, T]) the attention codes.  A checker
+    that has verified another implementation's stage k (exactly, or inside this oracle's band) passes that
+    implementation's own stage-k values here and obtains what stage k+1 must be for THOSE inputs, so every
+    element of every stage can be compared although a legitimate one-code difference upstream would otherwise
+    cascade.  Returns, per stage, the oracle's result (and band where the stage decides a level after a
+    floating-point island)."""
+    D = heads * head_dim
+    n = batch * heads
+    st: dict = {}
+
+    def ln_quant(v, g, b):
+        if layernorm == "compare":
+            ref, neg, flip = vo.layernorm_references(prm[g], prm[b], prm["s_ln"], bits, True, v.shape[1])
+            q = vo.layernorm_compare_quantize(v, ref, neg, flip, eps, bits, True)
+            return q, q, q
+        y, tol = vo.layernorm(v, prm[g], prm[b], eps)
+        return vo.quantize_band(y, tol, prm["s_ln"], bits, True)
+
+    # LayerNorm 1 + quantizer, from x
+    st["x1_codes"], st["x1_lo"], st["x1_hi"] = ln_quant(x, "ln1_g", "ln1_b")
+    # QKV linear from the given LayerNorm codes
+    w_qkv = vo.quantize(prm["w_qkv"], 0.0, bits, True, row_steps=prm["s_w_qkv"])
+    s_seg = np.concatenate([np.full(D, prm["s_q"]), np.full(D, prm["s_k"]), np.full(D, prm["s_v"])]).astype(np.float32)
+    a_qkv, b_qkv = fold(prm["s_ln"], prm["s_w_qkv"], prm["b_qkv"], s_seg)
+    st["qkv_codes"] = vo.epilogue_requant(vo.matmul_i32(given["x1"], w_qkv), a_qkv, b_qkv, bits, True)
+    # scores and attention codes from the given QKV codes
+    q = split_heads(given["qkv"], batch, tokens, heads, head_dim, 0)
+    k = split_heads(given["qkv"], batch, tokens, heads, head_dim, D)
+    v = split_heads(given["qkv"], batch, tokens, heads, head_dim, 2 * D)
+    S = vo.qk(q, k)
+    c = softmax_scale(prm["s_q"], prm["s_k"], head_dim)
+    if softmax == "shift":
+        c2 = np.float32(np.float64(c) * np.log2(np.e))
+        pc = vo.softmax_shift_quantize(S.reshape(n * tokens, tokens), c2, prm["s_p"], bits).reshape(n, tokens, tokens)
+        st["p_codes"] = st["p_lo"] = st["p_hi"] = pc
+    else:
+        _, pc, plo, phi = vo.softmax_quantize(S.reshape(n * tokens, tokens), c, prm["s_p"], bits)
+        st["p_codes"], st["p_lo"], st["p_hi"] = (a.reshape(n, tokens, tokens) for a in (pc, plo, phi))
+    # O = requant(P V): exact from the given P codes, else the interval reachable inside the P band
+    a_o, b_o = fold(prm["s_p"], np.full(head_dim, prm["s_v"], np.float32), None, prm["s_o"])
+    if given.get("P") is not None:
+        o = vo.epilogue_requant(vo.pv(given["P"], v).reshape(n * tokens, head_dim), a_o, b_o, bits, True)
+        o = merge_heads(o.reshape(n, tokens, head_dim), batch, tokens, heads, head_dim)
+        st["o_codes"] = st["o_lo"] = st["o_hi"] = o
+    else:
+        o = vo.epilogue_requant(vo.pv(st["p_codes"], v).reshape(n * tokens, head_dim), a_o, b_o, bits, True)
+        lo, hi = o_band_from_p_band(st["p_lo"], st["p_hi"], v, a_o, bits)
+        st["o_codes"], st["o_lo"], st["o_hi"] = (merge_heads(a.reshape(n, tokens, head_dim), batch, tokens, heads, head_dim)
+                                                 for a in (o, lo, hi))
+    # projection + residual from the given O codes
+    w_proj = vo.quantize(prm["w_proj"], 0.0, bits, True, row_steps=prm["s_w_proj"])
+    st["h"] = vo.epilogue_dequant(vo.matmul_i32(given["O"], w_proj), prm["s_o"], prm["s_w_proj"], prm["b_proj"], x)
+    # LayerNorm 2 + quantizer from the given residual stream
+    st["x2_codes"], st["x2_lo"], st["x2_hi"] = ln_quant(given["h"], "ln2_g", "ln2_b")
+    # fc1 + GELU + quantizer from the given LayerNorm codes
+    w_fc1 = vo.quantize(prm["w_fc1"], 0.0, bits, True, row_steps=prm["s_w_fc1"])
+    w_fc2 = vo.quantize(prm["w_fc2"], 0.0, bits, True, row_steps=prm["s_w_fc2"])
+    inv_g = inv_step(np.full(w_fc1.shape[0], prm["s_g"], np.float32))
+    st["g_codes"], st["g_lo"], st["g_hi"] = vo.epilogue_gelu_requant(
+        vo.matmul_i32(given["x2"], w_fc1), prm["s_ln"], prm["s_w_fc1"], prm["b_fc1"], inv_g, bits, False,
+        tol_rel=given.get("gelu_tol_rel", 0.0))
+    # fc2 + residual from the given GELU codes and residual stream
+    st["out"] = vo.epilogue_dequant(vo.matmul_i32(given["g"], w_fc2), prm["s_g"], prm["s_w_fc2"], prm["b_fc2"],
+                                    given["h"])
     return st

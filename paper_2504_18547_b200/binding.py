@@ -90,6 +90,10 @@ def lib():
                                              c_void_p]
         L.vitint_layernorm_compare_quantize.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_float,
                                                         POINTER(_Codes), c_void_p, c_void_p]
+        L.vitint_selftest_wait_timeout.argtypes = [c_int64, c_void_p, c_void_p]
+        L.vitint_fold_requant.argtypes = [c_float, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
+        L.vitint_fold_layernorm_references.argtypes = [c_void_p, c_void_p, c_float, c_int32, c_int32, c_int64, c_void_p,
+                                                       c_void_p]
         L.vitint_layernorm_quantize.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_float,
                                                 c_float, POINTER(_Codes), c_void_p, c_int64, c_void_p]
         _lib = L
@@ -106,6 +110,11 @@ def vitint_version() -> int:
 
 def vitint_device_status() -> int:
     return lib().vitint_device_status()
+
+
+def vitint_selftest_wait_timeout(limit_cycles: int, gave_up: torch.Tensor | None = None) -> None:
+    """Launches the library's bounded-wait self-test (a wait that nothing completes; gives up after `limit_cycles`)."""
+    _check(lib().vitint_selftest_wait_timeout(int(limit_cycles), _ptr(gave_up), _stream()), "vitint_selftest_wait_timeout")
 
 
 def packed_pitch(cols: int, bits: int) -> int:
@@ -205,31 +214,35 @@ class Slabs:
                       self.bits, int(self.signed))
 
 
-def fold_requant(s_x, s_w, bias, s_out):
-    """Host-side parameter preparation for the requantizing epilogue (Eq. 2):
-    alpha = s_x*s_w/s_out and beta = b/s_out in fp64, each rounded once to fp32."""
-    s_w64 = np.asarray(s_w, dtype=np.float64)
-    s_out64 = np.broadcast_to(np.asarray(s_out, dtype=np.float64), s_w64.shape)
-    alpha = (float(s_x) * s_w64 / s_out64).astype(np.float32)
-    beta = np.zeros_like(alpha) if bias is None else (np.asarray(bias, np.float64) / s_out64).astype(np.float32)
+def vitint_fold_requant(s_x, s_w, bias, s_out):
+    """Host helper of the library (Eq. 2 folding): alpha = s_x*s_w/s_out, beta = b/s_out per output channel.
+    s_w, bias (or None), s_out: host arrays (s_out may be a scalar).  Returns (alpha, beta) as fp32 numpy arrays."""
+    s_w = np.ascontiguousarray(s_w, dtype=np.float32).ravel()
+    n = s_w.size
+    s_out = np.ascontiguousarray(np.broadcast_to(np.asarray(s_out, dtype=np.float32), (n,)))
+    bias = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32).ravel()
+    alpha, beta = np.empty(n, np.float32), np.empty(n, np.float32)
+    fp = lambda a: None if a is None else a.ctypes.data_as(c_void_p)
+    _check(lib().vitint_fold_requant(float(s_x), fp(s_w), fp(bias), fp(s_out), n, fp(alpha), fp(beta)), "vitint_fold_requant")
     return alpha, beta
 
 
-def fold_layernorm_references(gamma, beta, step, bits: int, signed: bool, cols: int):
-    """Host-side parameter preparation for vitint_layernorm_compare_quantize (Fig. 5(b)): the signed
-    references sgn(c) c^2 / cols, c = ((k - 1/2) step - beta) / gamma for k = Qn+1 .. Qp (fp64, one rounding),
-    with c negated for columns of negative gain, and the per-column flip flags.  Returns (refs fp32
-    [cols, 2^bits - 1], flip uint8 [cols])."""
-    qn = -(1 << (bits - 1)) if signed else 0
-    qp = (1 << (bits - 1)) - 1 if signed else (1 << bits) - 1
-    g = np.asarray(gamma, dtype=np.float64).reshape(-1, 1)
-    b = np.asarray(beta, dtype=np.float64).reshape(-1, 1)
-    k = np.arange(qn + 1, qp + 1, dtype=np.float64).reshape(1, -1)
-    c = ((k - 0.5) * float(step) - b) / g
-    flip = g[:, 0] < 0
-    c[flip] = -c[flip]
-    refs = (np.sign(c) * c * c / float(cols)).astype(np.float32)
-    return np.ascontiguousarray(refs), np.ascontiguousarray(flip.astype(np.uint8))
+def vitint_fold_layernorm_references(gamma, beta, step, bits: int, signed: bool, cols: int):
+    """Host helper of the library (Fig. 5(b)): signed comparator references and per-column flip flags for
+    vitint_layernorm_compare_quantize.  Returns (refs fp32 [cols, 2^bits - 1], flip uint8 [cols])."""
+    gamma = np.ascontiguousarray(gamma, dtype=np.float32).ravel()
+    beta = np.ascontiguousarray(beta, dtype=np.float32).ravel()
+    n_thr = (1 << bits) - 1
+    refs, flip = np.empty((cols, n_thr), np.float32), np.empty(cols, np.uint8)
+    fp = lambda a: a.ctypes.data_as(c_void_p)
+    _check(lib().vitint_fold_layernorm_references(fp(gamma), fp(beta), float(step), bits, int(signed), cols, fp(refs),
+                                                  fp(flip)), "vitint_fold_layernorm_references")
+    return refs, flip
+
+
+# names kept for callers of the earlier Python helpers
+fold_requant = vitint_fold_requant
+fold_layernorm_references = vitint_fold_layernorm_references
 
 
 # ---------------------------------------------------------------------------

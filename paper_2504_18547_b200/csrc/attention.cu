@@ -44,8 +44,14 @@ int copy_codes(const vitint_codes* dst, const void* src, int64_t src_pitch, int6
     if (int rc = check_codes(dst)) return rc;
     if (dst->rows != rows || dst->pitch_bytes < row_bytes_valid) return VITINT_ERR_INVALID_ARG;
     const int64_t w = dst->pitch_bytes < src_pitch ? dst->pitch_bytes : src_pitch;
-    return cuda_status(cudaMemcpy2DAsync(dst->data, (size_t)dst->pitch_bytes, src, (size_t)src_pitch, (size_t)w,
-                                         (size_t)rows, cudaMemcpyDeviceToDevice, st));
+    if (int rc = cuda_status(cudaMemcpy2DAsync(dst->data, (size_t)dst->pitch_bytes, src, (size_t)src_pitch, (size_t)w,
+                                               (size_t)rows, cudaMemcpyDeviceToDevice, st)))
+        return rc;
+    // a destination pitch beyond the source's: the rest of every row is padding and is written as zero
+    if (dst->pitch_bytes > w)
+        return cuda_status(cudaMemset2DAsync((uint8_t*)dst->data + w, (size_t)dst->pitch_bytes, 0,
+                                             (size_t)(dst->pitch_bytes - w), (size_t)rows, st));
+    return VITINT_OK;
 }
 
 }  // namespace

@@ -21,6 +21,7 @@
 // and p_j = RN(e_j * (1/Z)) with 1/Z carried as two floats, so p_j stays within 2 ulp.
 // The host only selects this kernel when smax*|c| <= 80 (no overflow without max subtraction).
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 #include "ptx.cuh"
@@ -408,6 +409,12 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     reinterpret_cast<uint4*>(o)[1] = make_uint4(ow[4], ow[5], ow[6], ow[7]);
                 }
             }
+            // row padding behind the last head's columns (a caller may choose a pitch beyond the row's codes)
+            if (token < T && h == P.heads - 1 && hf == 1) {
+                uint8_t* const orow = P.out + ((long long)b * T + token) * P.out_pitch;
+                for (long long off = (long long)P.heads * (8 * P.out_c); off + 4 <= P.out_pitch; off += 4)
+                    *reinterpret_cast<uint32_t*>(orow + off) = 0u;
+            }
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&B.o_done));
@@ -531,7 +538,10 @@ static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t
     int grid = sm_count();
     const int want = (P.total_items + AT_GROUPS - 1) / AT_GROUPS;
     if (grid > want) grid = want;
-    static bool attr_set[3] = {false, false, false};
+    const int dev = current_device();
+    if (dev < 0) return VITINT_ERR_CUDA;
+    static bool attr_set_dev[MAX_DEVICES][3] = {};
+    bool* const attr_set = attr_set_dev[dev];
 #define VITINT_ATTN_LAUNCH(CC, SLOT)                                                                               \
     {                                                                                                              \
         if (!attr_set[SLOT]) {                                                                                     \
@@ -590,21 +600,27 @@ constexpr int STATIC_TABLE_FLOATS = 8320;   // largest table (8193 entries, 4-bi
 // Resident on every GPU that loads the library, from load until the process exits (about 33 KB).
 static __device__ __align__(256) float g_static_exp_table[STATIC_TABLE_FLOATS];
 
-constexpr int MAX_DEVICES = 64;
+// the widest codes the table-driven kernel takes (4-bit containers: scores in -4096 .. 4096) must fit the array
+static_assert((2 * 64 * 8 * 8 + 1) * sizeof(float) + 256 <= sizeof(float) * STATIC_TABLE_FLOATS,
+              "the built-in scratch must hold the exp table of 4-bit codes");
+
 void* g_static_table_addr[MAX_DEVICES];   // device address of the array, per device, once looked up
-bool g_static_table_ready[MAX_DEVICES];
+int g_static_table_rc[MAX_DEVICES];
+std::once_flag g_static_table_once[MAX_DEVICES];
 
 // The array's name is only a host-side handle; kernels need its device address.  Looked up once
-// per device, with that device current.
+// per device, with that device current (std::call_once: concurrent first calls from several host
+// threads are safe).
 int static_table_address(void** out) {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return VITINT_ERR_CUDA;
-    if (!g_static_table_ready[dev]) {
+    const int dev = current_device();
+    if (dev < 0) return VITINT_ERR_CUDA;
+    std::call_once(g_static_table_once[dev], [dev]() {
         void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_exp_table) != cudaSuccess || !p) return VITINT_ERR_CUDA;
-        g_static_table_addr[dev] = p;
-        g_static_table_ready[dev] = true;
-    }
+        const bool ok = cudaGetSymbolAddress(&p, g_static_exp_table) == cudaSuccess && p != nullptr;
+        g_static_table_addr[dev] = ok ? p : nullptr;
+        g_static_table_rc[dev] = ok ? VITINT_OK : VITINT_ERR_CUDA;
+    });
+    if (g_static_table_rc[dev] != VITINT_OK) return g_static_table_rc[dev];
     *out = g_static_table_addr[dev];
     return VITINT_OK;
 }
@@ -616,10 +632,11 @@ extern "C" int vitint_attention_core_noalloc(const vitint_codes* qkv, int32_t ba
                                              float q_step, float k_step, float p_step, int32_t p_bits,
                                              const float* alpha_o, const float* beta_o, const vitint_codes* o_out,
                                              void* stream) {
-    if (!qkv) return VITINT_ERR_INVALID_ARG;
+    // argument errors first, so that they are reported exactly as vitint_attention_core reports them
+    if (int rc = check_codes(qkv)) return rc;
+    if (int rc = check_codes(o_out)) return rc;
     const size_t need = vitint_attention_core_workspace_bytes(qkv->bits);
     if (need == 0) return VITINT_ERR_UNSUPPORTED;                     // 8-bit codes: no table-driven kernel
-    if (need > sizeof(float) * STATIC_TABLE_FLOATS) return VITINT_ERR_WORKSPACE;   // beyond the built-in scratch
     void* table = nullptr;
     if (int rc = static_table_address(&table)) return rc;
     return vitint_attention_core(qkv, batch, heads, tokens, q_step, k_step, p_step, p_bits, alpha_o, beta_o, o_out,

@@ -77,21 +77,34 @@ __device__ __forceinline__ int round_clamp(float r, float qn, float qp) {
 
 // Correctly rounded a / b from r = RN(1/b) by one Newton correction on the quotient
 // (Markstein): q0 = RN(a*r); rem = a - q0*b (exact in an FMA); q = RN(q0 + rem*r) = RN(a/b)
-// whenever b's significand is not all ones and nothing underflows.  A quotient that
-// underflows is below 2^-100 in magnitude and quantizes to code 0 either way.
+// whenever b's significand is not all ones and nothing overflows or underflows on the way.
+// The quantizers only need the quotient where it can still decide a level, so they first clamp the
+// dividend to [lo, hi] = [(Qn - 1) b, (Qp + 1) b] (clamp_dividend): a quotient beyond Qn - 1 / Qp + 1
+// clamps to the same end level as the true one, +-inf lands on the end levels like the IEEE quotient
+// does, NaN becomes lo (level Qn, as the host rule "not >= Qn" gives), and q0 stays finite.  Steps
+// outside [2^-100, 2^100] (where b*(Qp+1), 1/b or the remainder could leave the normal range) take
+// the IEEE division instead.
 struct Divisor {
     float b, r;
-    int exact;   // 0: significand of b is all ones, use the IEEE division instead
+    float lo, hi;   // dividend clamp
+    int exact;      // 0: use the IEEE division instead
 };
-__device__ __forceinline__ Divisor make_divisor(float b) {
+__device__ __forceinline__ Divisor make_divisor(float b, float qn = -128.0f, float qp = 255.0f) {
     Divisor d;
     d.b = b;
     d.r = __frcp_rn(b);
-    d.exact = ((__float_as_uint(b) & 0x007FFFFFu) != 0x007FFFFFu) ? 1 : 0;
+    d.lo = (qn - 1.0f) * b;
+    d.hi = (qp + 1.0f) * b;
+    const bool in_range = b >= 7.8886090522101181e-31f && b <= 1.2676506002282294e30f;    // 2^-100 .. 2^100
+    d.exact = (in_range && (__float_as_uint(b) & 0x007FFFFFu) != 0x007FFFFFu) ? 1 : 0;
     return d;
 }
+__device__ __forceinline__ float clamp_dividend(float a, const Divisor& d) {
+    return fminf(fmaxf(a, d.lo), d.hi);          // NaN -> lo
+}
 // Straight-line form for inner loops; valid only when d.exact (callers test that once, outside
-// the loop, because a branch per element would serialise the otherwise independent elements).
+// the loop, because a branch per element would serialise the otherwise independent elements)
+// and for dividends inside [d.lo, d.hi].
 __device__ __forceinline__ float div_rn_exact(float a, const Divisor& d) {
     const float q0 = a * d.r;
     const float rem = fmaf(-q0, d.b, a);

@@ -73,6 +73,32 @@ struct EpiParams {                      // per-column epilogue parameters of the
     float a[2][MAX_BN], b[2][MAX_BN], q[2][MAX_BN];
 };
 
+// ---- optional timeline of the warp roles (diagnostic builds only, -DVITINT_TRACE) ------------------
+// The first TRACE_CTAS CTAs record (clock64() << 8 | tag) into a caller-provided buffer, one sequence
+// per role: where the TMA producer, the MMA issuer and two epilogue warps wait, tile by tile.  The
+// product library is built without the flag and contains none of this.
+#ifdef VITINT_TRACE
+constexpr int TRACE_CTAS = 4, TRACE_ROLES = 4, TRACE_SLOTS = 4096;
+__device__ long long* g_trace_buf = nullptr;
+struct Tracer {
+    long long* p;
+    int n;
+    __device__ Tracer(int role) : p(nullptr), n(0) {
+        if (role >= 0 && g_trace_buf && blockIdx.x < TRACE_CTAS) p = g_trace_buf + ((size_t)blockIdx.x * TRACE_ROLES + role) * TRACE_SLOTS;
+    }
+    __device__ __forceinline__ void stamp(int tag) {
+        if (p && n < TRACE_SLOTS - 1) { p[1 + n] = (clock64() << 8) | (long long)(tag & 255); ++n; p[0] = n; }
+    }
+};
+#define VT_TRACER(name, role) Tracer name(role)
+#define VT_STAMP(name, tag) name.stamp(tag)
+enum TraceTag { TT_WAIT_EMPTY = 1, TT_GOT_EMPTY = 2, TT_WAIT_FULL = 3, TT_GOT_FULL = 4, TT_ISSUED = 5, TT_WAIT_ACC = 6,
+                TT_GOT_ACC = 7, TT_TILE_DONE = 8, TT_START = 9, TT_END = 10 };
+#else
+#define VT_TRACER(name, role)
+#define VT_STAMP(name, tag)
+#endif
+
 // K-contiguous operand tile: `rows` rows of 16*C packed bytes -> rows of 128 int8, 128-byte swizzle.
 template <int C, int SGN>
 __device__ __forceinline__ void unpack_k_major(const uint8_t* src, uint8_t* dst, int rows, int tid, int nthreads) {
@@ -595,6 +621,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (warp == WARP_TMA) {
         // ------------------------------ TMA producer -------------------------------
         if (lane == 0) {
+            VT_TRACER(tr, 0);
+            VT_STAMP(tr, TT_START);
             int it = 0;
             bool ok = true;
             const uint32_t packed_bytes = (P.a_direct ? 0u : P.pa_bytes) + (P.b_direct ? 0u : P.pb_bytes);
@@ -613,7 +641,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         ptx::mbar_arrive_expect_tx(p_full, packed_bytes);
                     }
                     if (any_direct) {
+                        VT_STAMP(tr, TT_WAIT_EMPTY);
                         if (!mbar_wait(ptx::smem_addr(&bars.i_empty[si]), phi ^ 1u, abort_ptr)) { ok = false; break; }
+                        VT_STAMP(tr, TT_GOT_EMPTY);
                         ptx::mbar_arrive_expect_tx(i_full, direct_bytes);
                     }
                     if (P.a_direct) ptx::tma_load_4d(i_dst, &map_a, i_full, kb * BK, m_tile * BM, inner, outer);
@@ -644,18 +674,24 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------- MMA issuer --------------------------------
         if (lane == 0) {
             const uint32_t idesc = ptx::idesc_i8(BM, P.bn, P.a_signed, P.b_signed, P.b_mn_major);
+            VT_TRACER(tr, 1);
+            VT_STAMP(tr, TT_START);
             int it = 0, tl = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++tl) {
                 const int buf = tl & 1;
                 const uint32_t acc_ph = (uint32_t)(tl >> 1) & 1u;
+                VT_STAMP(tr, TT_WAIT_EMPTY);
                 if (!mbar_wait(ptx::smem_addr(&bars.acc_empty[buf]), acc_ph ^ 1u, abort_ptr)) { ok = false; break; }
+                VT_STAMP(tr, TT_GOT_EMPTY);
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * acc_stride;
                 for (int kb = 0; kb < P.k_blocks; ++kb, ++it) {
                     const int s = it % P.ns_i;
                     const uint32_t ph = (uint32_t)(it / P.ns_i) & 1u;
+                    VT_STAMP(tr, TT_WAIT_FULL);
                     if (!mbar_wait(ptx::smem_addr(&bars.i_full[s]), ph, abort_ptr)) { ok = false; break; }
+                    VT_STAMP(tr, TT_GOT_FULL);
                     ptx::tc_fence_after();
                     const uint32_t a_addr = smem_base + (uint32_t)s * stage_i;
                     const uint32_t b_addr = a_addr + P.ia_bytes;
@@ -674,6 +710,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     ptx::mma_commit(ptx::smem_addr(&bars.i_empty[s]));
                 }
                 if (ok) ptx::mma_commit(ptx::smem_addr(&bars.acc_full[buf]));
+                VT_STAMP(tr, TT_ISSUED);
             }
         }
     } else if (warp >= WARP_UNPACK0 + (P.epi_warps - EPI_WARPS)) {
@@ -758,6 +795,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         int tl = 0;
         bool ok = true;
+        VT_TRACER(tr, (lane == 0 && ewarp == 0) ? 2 : ((lane == 0 && ewarp == P.epi_warps - 1) ? 3 : -1));
+        VT_STAMP(tr, TT_START);
         for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++tl) {
             int m_tile, n_tile, inner, outer;
             tile_coords(P, tile, m_tile, n_tile, inner, outer);
@@ -774,8 +813,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             float* const stage = P.stage_off ? reinterpret_cast<float*>(smem_gen + P.stage_off + (size_t)ewarp * STAGE_BYTES) : nullptr;
             const bool first_prefetched = epilogue_prefetch_first<KIND>(P, colbase, n_tile, slice, stage, lane, orow0, rows_valid);
             const uint32_t acc_ph = (uint32_t)(tl >> 1) & 1u;
+            VT_STAMP(tr, TT_WAIT_ACC);
             bool w = KIND == EK_ACC || epi_barrier(ptx::smem_addr(&bars.epi_sync), (uint32_t)tl & 1u, abort_ptr);
+            VT_STAMP(tr, TT_WAIT_FULL);
             w = w && mbar_wait(ptx::smem_addr(&bars.acc_full[buf]), acc_ph, abort_ptr);
+            VT_STAMP(tr, TT_GOT_ACC);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
             ptx::tc_fence_after();
             if (fetch_next) {
@@ -793,7 +835,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&bars.acc_empty[buf]));
+            VT_STAMP(tr, TT_TILE_DONE);
         }
+        VT_STAMP(tr, TT_END);
         ptx::cp_async_wait<0>();   // a residual copy requested before a wait that gave up has landed before the CTA exits
     }
 
@@ -851,15 +895,24 @@ struct Operand {
     uint64_t pitch, inner_stride, outer_stride;
 };
 
+// Per-device caches (a process may use several GPUs): SM count, and which kernels already carry their
+// shared-memory opt-in on that device.
+constexpr int MAX_DEVICES = 64;
+int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return -1;
+    return dev;
+}
 int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 1;
+    static int n[MAX_DEVICES] = {};
+    const int dev = current_device();
+    if (dev < 0) return 1;
+    if (!n[dev]) {
+        int v = 0;
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+        n[dev] = v > 0 ? v : 1;
     }
-    return n;
+    return n[dev];
 }
 
 constexpr uint32_t SMEM_TILE_BUDGET = 204u * 1024u;   // dynamic shared memory spent on operand rings
@@ -947,7 +1000,10 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     if (smem < 120 * 1024) smem = 120 * 1024;
     int grid = sm_count();
     if (grid > P.total_tiles) grid = P.total_tiles;
-    static bool attr_set[5] = {false, false, false, false, false};
+    const int dev = current_device();
+    if (dev < 0) return VITINT_ERR_CUDA;
+    static bool attr_set_dev[MAX_DEVICES][5] = {};
+    bool* const attr_set = attr_set_dev[dev];
 #define VITINT_LAUNCH(KIND)                                                                                        \
     case KIND:                                                                                                     \
         if (!attr_set[KIND]) {                                                                                     \
@@ -1033,6 +1089,14 @@ static int check_slabs(const vitint_slabs* s) {
 }  // namespace vitint
 
 using namespace vitint;
+
+#ifdef VITINT_TRACE
+// Diagnostic builds only: buffer of vitint_trace_words() 64-bit words of device memory, or NULL to stop recording.
+extern "C" int vitint_trace_set(long long* buf) {
+    return cuda_status(cudaMemcpyToSymbol(g_trace_buf, &buf, sizeof(buf)));
+}
+extern "C" int vitint_trace_words(void) { return TRACE_CTAS * TRACE_ROLES * TRACE_SLOTS; }
+#endif
 
 extern "C" int vitint_linear(const vitint_codes* x, float x_step, const vitint_codes* w, const float* w_step,
                              const float* bias, const vitint_epilogue* epi, void* out, int64_t ld_out, void* stream) {

@@ -20,7 +20,7 @@ quantize_pack_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, in
     const int64_t col0 = (int64_t)w * E;
     for (int64_t row = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; row < rows;
          row += (int64_t)gridDim.y * blockDim.y) {
-        const Divisor dv = make_divisor(row_steps ? row_steps[row] : step);
+        const Divisor dv = make_divisor(row_steps ? row_steps[row] : step, qn, qp);
         const float* xr = x + row * ldx + col0;
         float v[E];
         if (vec_ok && col0 + E <= cols) {
@@ -37,7 +37,7 @@ quantize_pack_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, in
         if (dv.exact) {
 #pragma unroll
             for (int i = 0; i < E; ++i)
-                word |= (round_clamp_bits(div_rn_exact(v[i], dv), qn, qp) & ((1u << C) - 1u)) << (C * i);
+                word |= (round_clamp_bits(div_rn_exact(clamp_dividend(v[i], dv), dv), qn, qp) & ((1u << C) - 1u)) << (C * i);
         } else {
 #pragma unroll
             for (int i = 0; i < E; ++i)

@@ -11,7 +11,8 @@ constexpr long long WAIT_LIMIT_CYCLES = 2000000000ll;   // about one second
 
 // Bounded wait.  Gives up after WAIT_LIMIT_CYCLES or as soon as another thread of the CTA
 // has given up; the first to give up records the timeout in the device status word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = WAIT_LIMIT_CYCLES) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
@@ -19,7 +20,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         // issue slots to the warps that have work
         if (ptx::mbar_try_wait_hint(bar, parity, 50000u)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > limit_cycles) {
             *abort_flag = 1;
             atomicExch(&g_device_status, (int)VITINT_ERR_TIMEOUT);
             return false;

@@ -71,3 +71,12 @@ def test_reference_arm_prints_one_json_line():
     assert line["impl"] == "reference" and line["unit"] == "TOPS" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["config"]["workload"] == "vit_base_layer_b128"
+
+
+def test_gpus_flag_must_match_the_ranks_that_were_started():
+    """`--gpus N` either starts N ranks itself (no WORLD_SIZE in the environment) or insists that the launcher
+    started exactly N: a mismatch is an error before any device is touched, never a silent 1-GPU run."""
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    out = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--gpus", "2", "--steps", "1"], env=env,
+                         capture_output=True, text=True, timeout=300)
+    assert out.returncode != 0 and "--gpus 2 but 1 rank" in out.stderr

@@ -15,7 +15,7 @@ from oracle import pipeline as vp
 
 pytestmark = pytest.mark.gpu
 vt = pytest.importorskip("paper_2504_18547_b200")
-from gpu_util import dev, from_codes  # noqa: E402
+from gpu_util import GELU_TOL_REL, dev, from_codes  # noqa: E402
 
 
 def _rows(a, images, T):
@@ -23,61 +23,73 @@ def _rows(a, images, T):
     return np.concatenate([a[b * T:(b + 1) * T] for b in images])
 
 
+def _code_rows(c, images, T):
+    """Codes of the selected images' token rows (sliced on the device, unpacked by the oracle's unpacker)."""
+    import paper_2504_18547_b200 as vt_
+    idx = torch.cat([torch.arange(b * T, (b + 1) * T) for b in images]).to(c.data.device)
+    sub = vt_.Codes(c.data.index_select(0, idx).contiguous(), len(idx), c.cols, c.bits, c.signed, c.container)
+    return from_codes(sub)
+
+
+def _f32_rows(t, images, T):
+    idx = torch.cat([torch.arange(b * T, (b + 1) * T) for b in images]).to(t.device)
+    return t.index_select(0, idx).cpu().numpy()
+
+
 def gpu_stages(layer, out, images, T, H):
     """Intermediate buffers of an EncoderLayer after forward(), restricted to the given images."""
-    g = {"x1": _rows(from_codes(layer.x1), images, T), "qkv": _rows(from_codes(layer.qkv), images, T),
-         "O": _rows(from_codes(layer.O), images, T), "h": _rows(layer.h.cpu().numpy(), images, T),
-         "x2": _rows(from_codes(layer.x2), images, T), "g": _rows(from_codes(layer.g), images, T),
-         "out": _rows(out.cpu().numpy(), images, T)}
+    g = {"x1": _code_rows(layer.x1, images, T), "qkv": _code_rows(layer.qkv, images, T),
+         "O": _code_rows(layer.O, images, T), "h": _f32_rows(layer.h, images, T),
+         "x2": _code_rows(layer.x2, images, T), "g": _code_rows(layer.g, images, T),
+         "out": _f32_rows(out, images, T)}
     if not layer.fused_attention:
-        P = from_codes(layer.P).reshape(-1, T, T)
-        g["P"] = np.concatenate([P[b * H:(b + 1) * H] for b in images])
+        heads = [b * H + h for b in images for h in range(H)]
+        g["P"] = _code_rows(layer.P, heads, T).reshape(-1, T, T)
     return g
 
 
-def compare_stages(g, st, B, T, H, D, fused, min_images_ok):
-    """Stage-by-stage comparison of GPU buffers `g` with the oracle stages `st` for B images."""
-    att = st["attn"]
-    x1 = g["x1"]
-    assert np.all(x1 >= st["x1_lo"]) and np.all(x1 <= st["x1_hi"])
-    img_ok = np.array([(x1[b * T:(b + 1) * T] == st["x1_codes"][b * T:(b + 1) * T]).all() for b in range(B)])
-    assert img_ok.sum() >= min_images_ok
-    rows_img = np.repeat(img_ok, T)
-    assert np.array_equal(g["qkv"][rows_img], att["qkv_codes"][rows_img])
+FLIP_LIMIT = 1e-3      # largest share of a stage's codes that may sit on the other side of a near-tie
 
-    prob_ok = np.repeat(img_ok, H)
-    if fused:
-        # P never leaves the SM: rows whose every code is unique under the 2-ulp band must agree downstream
-        p_row_ok = (att["p_lo"] == att["p_hi"]).all(axis=2) & prob_ok[:, None]
+
+def compare_stages(g, x, prm, B, T, H, bits, tag="", **modes):
+    """Every element of every stage of the GPU's layer against the oracle.
+
+    Stage k of the oracle is recomputed from the GPU's own stage k-1 values (handed over as data), so a
+    legitimate one-code difference on a near-tie upstream does not cascade: stages that are a fixed IEEE /
+    integer sequence (QKV, O given P, the residual stream h, the output) must then agree bit for bit on 100 %
+    of their elements, and stages that decide a level after an fp32 island (LayerNorm, softmax, GELU) must lie
+    inside the oracle's band everywhere, with at most FLIP_LIMIT of them off the oracle's own code.  The
+    fused attention kernel keeps P on the SM; its O codes must lie inside the interval that the oracle's P band
+    can reach (its P codes themselves are compared element by element in test_fused_attention_p_codes)."""
+    given = {k: g[k] for k in ("x1", "qkv", "O", "h", "x2", "g")}
+    given["P"] = g.get("P")
+    given["gelu_tol_rel"] = GELU_TOL_REL
+    st = vp.encoder_layer_stagewise(x, prm, B, T, H, bits, given, **modes)
+    flips = {}
+
+    def in_band(name, got, code, lo, hi):
+        assert np.all(got >= lo) and np.all(got <= hi), f"{tag}{name}: code outside the oracle's band"
+        flips[name] = float((got != code).mean())
+
+    in_band("x1", g["x1"], st["x1_codes"], st["x1_lo"], st["x1_hi"])
+    assert np.array_equal(g["qkv"], st["qkv_codes"]), f"{tag}qkv"
+    if given["P"] is not None:
+        in_band("P", g["P"], st["p_codes"], st["p_lo"], st["p_hi"])
+        assert np.array_equal(g["O"], st["o_codes"]), f"{tag}O from the GPU's P codes"
     else:
-        P = g["P"]
-        assert np.all(P[prob_ok] >= att["p_lo"][prob_ok]) and np.all(P[prob_ok] <= att["p_hi"][prob_ok])
-        p_row_ok = (P == att["p_codes"]).all(axis=2) & prob_ok[:, None]           # [B*H, T]
-    assert p_row_ok[prob_ok].mean() > 0.97
-
-    O = g["O"]
-    tok_ok = np.ones(B * T, bool)
-    for b in range(B):
-        for h in range(H):
-            sel = p_row_ok[b * H + h]
-            blk = slice(b * T, (b + 1) * T)
-            assert np.array_equal(O[blk, h * 64:(h + 1) * 64][sel], att["o_codes"][blk, h * 64:(h + 1) * 64][sel])
-            tok_ok[blk] &= sel
-    assert tok_ok.mean() > 0.4
-
-    assert np.array_equal(g["h"][tok_ok].view(np.uint32), st["h"][tok_ok].view(np.uint32))
-    x2 = g["x2"]
-    assert np.all(x2[tok_ok] >= st["x2_lo"][tok_ok]) and np.all(x2[tok_ok] <= st["x2_hi"][tok_ok])
-    tok_ok2 = tok_ok & (x2 == st["x2_codes"]).all(axis=1)
-    gg = g["g"]
-    assert np.all(gg[tok_ok2] >= st["g_lo"][tok_ok2]) and np.all(gg[tok_ok2] <= st["g_hi"][tok_ok2])
-    tok_ok3 = tok_ok2 & (gg == st["g_codes"]).all(axis=1)
-    assert tok_ok3.mean() > 0.3
-    o = g["out"]
-    assert np.array_equal(o[tok_ok3].view(np.uint32), st["out"][tok_ok3].view(np.uint32))
-    # everything else stays close: one code flip moves an output by a few steps at most
-    assert np.abs(o - st["out"]).max() < 0.5
-    return tok_ok3.mean()
+        in_band("O", g["O"], st["o_codes"], st["o_lo"], st["o_hi"])
+        # the band of O is narrow: at most one code wide for all but a sliver of the elements
+        assert ((st["o_hi"] - st["o_lo"]) <= 1).mean() > 0.999
+    assert np.array_equal(g["h"].view(np.uint32), st["h"].view(np.uint32)), f"{tag}h"
+    in_band("x2", g["x2"], st["x2_codes"], st["x2_lo"], st["x2_hi"])
+    in_band("g", g["g"], st["g_codes"], st["g_lo"], st["g_hi"])
+    assert np.array_equal(g["out"].view(np.uint32), st["out"].view(np.uint32)), f"{tag}out"
+    print(f"{tag}off-centre share per stage (of {g['x1'].size} / {g['g'].size} codes): " +
+          ", ".join(f"{k} {v:.2e}" for k, v in flips.items()))
+    for k, v in flips.items():
+        # O inherits every P flip of its row through 197 products, so its share is that of P times the row length
+        assert v <= (FLIP_LIMIT if k != "O" else 0.05), (k, v)
+    return st, flips
 
 
 @pytest.mark.parametrize("wide", [True, False], ids=["byte_codes", "packed_codes"])
@@ -88,7 +100,6 @@ def test_encoder_layer_staged(bits, fused, wide):
     cfg = si.VIT_BASE_LAYER.with_(batch=3, bits=bits)
     prm = si.layer_parameters(cfg)
     x = si.activations(cfg)
-    st = vp.encoder_layer(x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits)
     layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, fused_attention=fused,
                          wide_activations=wide)
     assert layer.fused_attention == fused
@@ -96,21 +107,20 @@ def test_encoder_layer_staged(bits, fused, wide):
     layer.forward(dev(x), out)
     assert vt.vitint_device_status() == 0
     # weights quantized by the library equal the oracle's
-    assert np.array_equal(from_codes(layer.w["qkv"]), st["attn"]["w_qkv_codes"])
-    assert np.array_equal(from_codes(layer.w["fc2"]), st["w_fc2_codes"])
+    assert np.array_equal(from_codes(layer.w["qkv"]), vo.quantize(prm["w_qkv"], 0.0, bits, True, row_steps=prm["s_w_qkv"]))
+    assert np.array_equal(from_codes(layer.w["fc2"]), vo.quantize(prm["w_fc2"], 0.0, bits, True, row_steps=prm["s_w_fc2"]))
     g = gpu_stages(layer, out, range(cfg.batch), cfg.tokens, cfg.heads)
-    compare_stages(g, st, cfg.batch, cfg.tokens, cfg.heads, cfg.dim, fused, min_images_ok=2)
+    compare_stages(g, x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits, tag=f"{bits}-bit: ")
 
 
 @pytest.mark.parametrize("bits", [4, 3])
 def test_encoder_layer_shift_softmax_attention_bit_exact(bits):
     """Encoder layer with the Eq. 4 softmax and the comparator quantizer: the attention stage has no fp32 island,
-    so in every image whose LayerNorm codes agree, P and O must equal the oracle's bit for bit."""
+    so P and O must equal what the oracle computes from the same QKV codes bit for bit, with no band."""
     from paper_2504_18547_b200.encoder import EncoderLayer
     cfg = si.VIT_BASE_LAYER.with_(batch=3, bits=bits)
     prm = si.layer_parameters(cfg)
     x = si.activations(cfg)
-    st = vp.encoder_layer(x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits, softmax="shift")
     layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, softmax="shift")
     assert not layer.fused_attention
     out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
@@ -118,22 +128,16 @@ def test_encoder_layer_shift_softmax_attention_bit_exact(bits):
     assert vt.vitint_device_status() == 0
     T, H = cfg.tokens, cfg.heads
     g = gpu_stages(layer, out, range(cfg.batch), T, H)
-    att = st["attn"]
-    img_ok = np.array([(g["x1"][b * T:(b + 1) * T] == st["x1_codes"][b * T:(b + 1) * T]).all() for b in range(cfg.batch)])
-    assert img_ok.sum() >= 2
-    heads_ok = np.repeat(img_ok, H)
-    rows_ok = np.repeat(img_ok, T)
-    assert np.array_equal(g["P"][heads_ok], att["p_codes"][heads_ok])
-    assert np.array_equal(g["O"][rows_ok], att["o_codes"][rows_ok])
-    assert len(np.unique(att["p_codes"])) >= 4
-    # the rest of the layer as in the exp mode
-    compare_stages(g, st, cfg.batch, T, H, cfg.dim, False, min_images_ok=2)
+    st, flips = compare_stages(g, x, prm, cfg.batch, T, H, cfg.bits, softmax="shift")
+    assert flips["P"] == 0.0 and np.array_equal(st["p_lo"], st["p_hi"])
+    assert len(np.unique(st["p_codes"])) >= 4
 
 
-@pytest.mark.parametrize("bits", [4, 2])
+@pytest.mark.parametrize("bits", [4, 3, 2])
 def test_encoder_layer_full_size_sampled_images(bits):
-    """The benchmark's own launch configuration (ViT-Base layer, batch 128): the GPU runs the full batch, the
-    oracle recomputes a sample of the images on its own (images are independent), stage by stage."""
+    """The benchmark's own launch configuration (ViT-Base layer, batch 128) at all three widths: the GPU runs the
+    full batch, the oracle follows a sample of the images on its own (images are independent), every element of
+    every stage of those images."""
     from paper_2504_18547_b200.encoder import EncoderLayer
     cfg = si.VIT_BASE_LAYER.with_(bits=bits)
     prm = si.layer_parameters(cfg)
@@ -144,10 +148,8 @@ def test_encoder_layer_full_size_sampled_images(bits):
     assert vt.vitint_device_status() == 0
     images = [0, 63, 64, 127]
     T = cfg.tokens
-    xs = _rows(x, images, T)
-    st = vp.encoder_layer(xs, prm, len(images), T, cfg.heads, cfg.bits)
     g = gpu_stages(layer, out, images, T, cfg.heads)
-    compare_stages(g, st, len(images), T, cfg.heads, cfg.dim, True, min_images_ok=2)
+    compare_stages(g, _rows(x, images, T), prm, len(images), T, cfg.heads, cfg.bits, tag=f"batch 128, {bits}-bit: ")
     # a property that holds for every image at any size: output rows are finite and their spread is that of
     # the residual stream plus the MLP branch
     o = out.cpu().numpy()
@@ -155,15 +157,20 @@ def test_encoder_layer_full_size_sampled_images(bits):
 
 
 def test_attention_block_full_size_sampled_images():
-    """ViT-Small attention block at its full batch of 64 (with the x10 outlier channels): sampled images."""
+    """ViT-Small attention block at its full batch of 64 (with the x10 outlier channels): sampled images, every
+    element of every stage, each stage recomputed by the oracle from the GPU's previous stage."""
     cfg = si.VIT_SMALL_BLOCK
+    _attention_block_sampled(cfg, [0, 31, 63])
+
+
+def _attention_block_sampled(cfg, images, want_p=False, tag=""):
     prm = si.layer_parameters(cfg)
     x = si.activations(cfg)
     s_x = si.lsq_step(x, cfg.bits, True)
     T, H, D = cfg.tokens, cfg.heads, cfg.dim
-    images = [0, 31, 63]
+    B = len(images)
     xq = vo.quantize(_rows(x, images, T), s_x, cfg.bits, True)
-    st = vp.attention_block(xq, s_x, prm, len(images), T, H, cfg.bits, proj="requant")
+    st = vp.attention_block(xq, s_x, prm, B, T, H, cfg.bits, proj="requant")
     from gpu_util import to_codes
     aw = vt.AttentionWeights(
         batch=cfg.batch, tokens=T, heads=H, bits=cfg.bits, w_qkv=to_codes(st["w_qkv_codes"], cfg.bits, True),
@@ -176,57 +183,74 @@ def test_attention_block_full_size_sampled_images():
     xg = vt.vitint_quantize(dev(x), float(s_x), cfg.bits, True)
     dq = vt.Codes.empty(cfg.rows, 3 * D, cfg.bits, True)
     do = vt.Codes.empty(cfg.rows, D, cfg.bits, True)
-    outc = vt.vitint_attention_block(xg, aw, dbg_qkv=dq, dbg_o=do)
+    dp = vt.Codes.empty(cfg.batch * H * T, T, cfg.bits, False) if want_p else None
+    outc = vt.vitint_attention_block(xg, aw, dbg_qkv=dq, dbg_p=dp, dbg_o=do)
     assert vt.vitint_device_status() == 0
-    assert np.array_equal(_rows(from_codes(xg), images, T), xq)
-    assert np.array_equal(_rows(from_codes(dq), images, T), st["qkv_codes"])
-    unique_row = (st["p_lo"] == st["p_hi"]).all(axis=2)                      # [len(images)*H, T]
-    go = _rows(from_codes(do), images, T)
-    tok_ok = np.ones(len(images) * T, bool)
-    for b in range(len(images)):
-        for h in range(H):
-            sel = unique_row[b * H + h]
-            blk = slice(b * T, (b + 1) * T)
-            assert np.array_equal(go[blk, h * 64:(h + 1) * 64][sel], st["o_codes"][blk, h * 64:(h + 1) * 64][sel])
-            tok_ok[blk] &= sel
-    assert tok_ok.mean() > 0.5
-    assert np.array_equal(_rows(from_codes(outc), images, T)[tok_ok], st["out_codes"][tok_ok])
+    assert np.array_equal(_code_rows(xg, images, T), xq)
+    # QKV: a fixed integer / IEEE sequence, bit for bit
+    gq = _code_rows(dq, images, T)
+    assert np.array_equal(gq, st["qkv_codes"])
+    n = B * H
+    v = vp.split_heads(gq, B, T, H, 64, 2 * D)
+    go = _code_rows(do, images, T)
+    a_o = st["alpha_o"]
+    if want_p:
+        # P inside the band everywhere; O recomputed from the GPU's own P codes, bit for bit
+        heads = [b * H + h for b in images for h in range(H)]
+        gp = _code_rows(dp, heads, T).reshape(n, T, T)
+        assert np.all(gp >= st["p_lo"]) and np.all(gp <= st["p_hi"])
+        flip_p = float((gp != st["p_codes"]).mean())
+        o = vo.epilogue_requant(vo.pv(gp, v).reshape(n * T, 64), a_o, np.zeros_like(a_o), cfg.bits, True)
+        assert np.array_equal(go, vp.merge_heads(o.reshape(n, T, 64), B, T, H, 64))
+        assert flip_p <= FLIP_LIMIT, flip_p
+    else:
+        # P stays on the SM: O inside the interval that the oracle's P band can reach
+        lo, hi = vp.o_band_from_p_band(st["p_lo"], st["p_hi"], v, a_o, cfg.bits)
+        lo, hi = (vp.merge_heads(a.reshape(n, T, 64), B, T, H, 64) for a in (lo, hi))
+        assert np.all(go >= lo) and np.all(go <= hi)
+        assert (lo == hi).mean() > 0.9
+        flip_p = float((go != st["o_codes"]).mean())
+    # projection recomputed from the GPU's own O codes, bit for bit on every element
+    want = vo.epilogue_requant(vo.matmul_i32(go, st["w_proj_codes"]), st["alpha_proj"], st["beta_proj"], cfg.bits, True)
+    assert np.array_equal(_code_rows(outc, images, T), want)
+    print(f"{tag}{cfg.name}: off-centre share {'P' if want_p else 'O'} {flip_p:.2e}")
 
 
-def test_twelve_layer_encoder_sampled_images():
-    """12 integerized ViT-Base layers (the 12-layer configuration at a reduced batch; the oracle follows two of
-    the images through all layers).  Near-tie code flips accumulate with depth, so the end-to-end check is a
-    closeness bound, while the first layer is checked stage by stage and bit-exactly where codes agree."""
+@pytest.mark.parametrize("tokens,bits", [(577, 4), (785, 4), (785, 2), (577, 3)])
+def test_attention_block_long_sequences_batch_32(tokens, bits):
+    """The token counts of the scaling study beyond one accumulator tile (577 and 785 tokens) at batch 32, through
+    vitint_attention_block (which runs Q K^T, the softmax kernel and P V unfused there): QKV, P (inside the
+    band), O from the GPU's own P codes and the projection, every element of the sampled images."""
+    cfg = si.VIT_SMALL_BLOCK.with_(batch=32, tokens=tokens, bits=bits, name=f"vit_small_attn_b32_t{tokens}")
+    _attention_block_sampled(cfg, [0, 31], want_p=True)
+
+
+def test_twelve_layer_encoder_batch_256_all_layers_staged():
+    """12 integerized ViT-Base layers at the full batch of 256 (4-bit): the GPU runs the whole stack on its own
+    activations; for four sampled images the oracle recomputes every stage of every layer from the GPU's previous
+    stage (the layer input included), so all 12 layers are compared on 100 % of the sampled images' elements."""
     from paper_2504_18547_b200.encoder import EncoderStack
-    cfg = si.VIT_BASE_ENCODER.with_(batch=8)
+    cfg = si.VIT_BASE_ENCODER
     T, H = cfg.tokens, cfg.heads
     prms = [si.layer_parameters(cfg, layer=l) for l in range(cfg.layers)]
-    x = si.activations(cfg)
+    images = [0, 100, 101, 255]
+    x = np.concatenate([si.activations(cfg, batch=64, first_image=f) for f in range(0, cfg.batch, 64)])
     stack = EncoderStack(prms, cfg.batch, T, H, cfg.mlp_dim, cfg.bits)
-    out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
-    stack.forward(dev(x), out)
-    assert vt.vitint_device_status() == 0
-    images = [0, 7]
-    sts = vp.encoder_stack(_rows(x, images, T), prms, len(images), T, H, cfg.bits)
-    # Every layer, fed with the ORACLE's previous-layer output for the sampled images (tiled to the batch), is
-    # checked stage by stage: this exercises each layer's own weights and steps without any cascade.
-    for l in (0, 5, 11):
-        xin = _rows(x, images, T) if l == 0 else sts[l - 1]["out"]
-        xin_b = np.concatenate([xin] * (cfg.batch // len(images)))
-        out_l = torch.empty_like(out)
-        stack.layers[l].forward(dev(xin_b), out_l)
-        g = gpu_stages(stack.layers[l], out_l, range(len(images)), T, H)
-        compare_stages(g, sts[l], len(images), T, H, cfg.dim, True, min_images_ok=1)
-    # End to end, near-tie code flips (legitimate one-code differences) spread through attention and are
-    # re-quantized twelve times, so the two results are compared statistically.
-    o = _rows(out.cpu().numpy(), images, T)
-    ref = sts[-1]["out"]
-    err = (o - ref).astype(np.float64)
-    rel_rms = np.sqrt((err ** 2).mean()) / ref.std()
-    corr = np.corrcoef(o.ravel(), ref.ravel())[0, 1]
-    assert vt.vitint_device_status() == 0
-    assert rel_rms < 0.25 and corr > 0.97 and ref.std() > 0.5, (rel_rms, corr)
-    print(f"12 layers: relative rms difference {rel_rms:.4f}, correlation {corr:.5f}")
+    cur = dev(x)
+    cur_host = _rows(x, images, T)
+    worst = {}
+    for l, layer in enumerate(stack.layers):
+        dst = stack.buf[l & 1]
+        layer.forward(cur, dst)
+        assert vt.vitint_device_status() == 0
+        g = gpu_stages(layer, dst, images, T, H)
+        _, flips = compare_stages(g, cur_host, prms[l], len(images), T, H, cfg.bits, tag=f"layer {l}: ")
+        for k, v in flips.items():
+            worst[k] = max(worst.get(k, 0.0), v)
+        cur, cur_host = dst, g["out"]
+    o = cur.cpu().numpy()
+    assert np.isfinite(o).all() and o.std() > 0.5
+    print("12 layers, batch 256: largest off-centre share per stage " + ", ".join(f"{k} {v:.2e}" for k, v in worst.items()))
 
 
 @pytest.mark.parametrize("bits", [4, 2])
@@ -247,17 +271,16 @@ def test_encoder_layer_comparator_layernorm_and_shift_softmax_bit_exact_up_to_ge
     T, H = cfg.tokens, cfg.heads
     g = gpu_stages(layer, out, range(cfg.batch), T, H)
     att = st["attn"]
+    # the oracle's own free-running chain: identical up to the GELU
     assert np.array_equal(g["x1"], st["x1_codes"])
     assert np.array_equal(g["qkv"], att["qkv_codes"])
     assert np.array_equal(g["P"], att["p_codes"])
     assert np.array_equal(g["O"], att["o_codes"])
     assert np.array_equal(g["h"].view(np.uint32), st["h"].view(np.uint32))
     assert np.array_equal(g["x2"], st["x2_codes"])
-    # GELU is the one remaining fp32 island: its levels stay inside the oracle's band
-    assert np.all(g["g"] >= st["g_lo"]) and np.all(g["g"] <= st["g_hi"])
-    tok = (g["g"] == st["g_codes"]).all(axis=1)
-    assert tok.mean() > 0.5
-    assert np.array_equal(g["out"][tok].view(np.uint32), st["out"][tok].view(np.uint32))
+    # GELU is the one remaining fp32 island: band for its levels, and the output from the GPU's own levels
+    _, flips = compare_stages(g, x, prm, cfg.batch, T, H, cfg.bits, softmax="shift", layernorm="compare")
+    assert flips["x1"] == 0.0 and flips["P"] == 0.0 and flips["x2"] == 0.0
 
 
 @pytest.mark.parametrize("bits", [3, 4])
@@ -294,9 +317,10 @@ def test_normed_attention_module_bit_exact(bits):
 
 def test_deit_s_model_forward():
     """Whole DeiT-S-shaped model (patch embedding, 198 tokens, 12 layers, final LayerNorm, two heads) against the
-    oracle on sampled images.  The patch embedding is one fixed IEEE sequence (bit-exact); after twelve layers the
-    legitimate one-level differences on near-ties have spread, so the residual stream and the logits are compared
-    statistically; the heads are checked exactly by feeding them the oracle's own final activations."""
+    oracle on sampled images.  The patch embedding is one fixed IEEE sequence (bit-exact); each of the twelve
+    layers is compared stage by stage on every element, the oracle recomputing a stage from the GPU's previous one;
+    the final LayerNorm's levels lie inside the oracle's band and the logits are recomputed from the GPU's own
+    levels, bit for bit."""
     from paper_2504_18547_b200.encoder import DeitModel
     cfg = si.DEIT_S_MODEL.with_(batch=4)
     T, H, D = cfg.tokens, cfg.heads, cfg.dim
@@ -307,39 +331,35 @@ def test_deit_s_model_forward():
     logits = model.forward(dev(patches)).cpu().numpy()
     assert vt.vitint_device_status() == 0
     images = [0, 3]
-    st = vp.deit_forward(_rows(patches, images, T), ends, lps, len(images), T, H, cfg.bits)
     # patch embedding + token table
-    x0 = _rows(model.x0.cpu().numpy(), images, T)
-    assert np.array_equal(x0.view(np.uint32), st["x0"].view(np.uint32))
+    xq = vo.quantize(_rows(patches, images, T), ends["s_patch"], cfg.bits, True)
+    w_pe = vo.quantize(ends["w_pe"], 0.0, cfg.bits, True, row_steps=ends["s_w_pe"])
+    table = np.tile(np.asarray(ends["tokens"], np.float32), (len(images), 1))
+    x0_ref = vo.epilogue_dequant(vo.matmul_i32(xq, w_pe), ends["s_patch"], ends["s_w_pe"], ends["b_pe"], table)
+    x0 = _f32_rows(model.x0, images, T)
+    assert np.array_equal(x0.view(np.uint32), x0_ref.view(np.uint32))
     # the class and distillation rows received no patch contribution: bias + token table only
     tok = np.asarray(ends["tokens"], np.float32)
     assert np.array_equal(x0[:2], (ends["b_pe"][None, :] + tok[:2]).astype(np.float32))
-    # residual stream after 12 layers
-    xf = _rows(model.x_final.cpu().numpy(), images, T)
-    err = (xf - st["x_final"]).astype(np.float64)
-    rel_rms = np.sqrt((err ** 2).mean()) / st["x_final"].std()
-    corr = np.corrcoef(xf.ravel(), st["x_final"].ravel())[0, 1]
-    assert rel_rms < 0.3 and corr > 0.95, (rel_rms, corr)
-    # heads, exactly: the oracle's final activations through the library's final LayerNorm + heads
-    xfin = np.zeros((cfg.rows, D), np.float32)
-    for j, b in enumerate(images):
-        xfin[b * T:(b + 1) * T] = st["x_final"][j * T:(j + 1) * T]
-    model.x_final.copy_(dev(xfin))
-    for i, (w, s_w, bias) in enumerate(model.heads_w):
-        rows = model.x_final[i::T]
-        vt.vitint_layernorm_quantize(rows, model.lnf_g, model.lnf_b, model.eps, model.s_lnf, cfg.bits, True,
-                                     out=model.head_codes[i])
-        vt.vitint_linear(model.head_codes[i], model.s_lnf, w, s_w, bias,
-                         vt.Epilogue(mode=vt.EPI_DEQUANT_F32, residual=model.logits[0] if i else None),
-                         out=model.logits[i])
-    hc = [from_codes(c)[images] for c in model.head_codes]
-    ok = np.ones(len(images), bool)
-    for name, c in zip(("head", "head_dist"), hc):
-        assert np.all(c >= st[name + "_lo"]) and np.all(c <= st[name + "_hi"])
-        ok &= (c == st[name + "_codes"]).all(axis=1)
-    got = model.logits[1].cpu().numpy()[images]
-    assert ok.any()
-    assert np.array_equal(got[ok].view(np.uint32), st["logits"][ok].view(np.uint32))
-    # end to end the logits stay close
-    assert np.abs(logits[images] - st["logits"]).max() < 0.25 * max(1.0, np.abs(st["logits"]).max())
-    print(f"DeiT-S model: residual stream relative rms {rel_rms:.4f}, correlation {corr:.5f}")
+    # the twelve layers, each on the GPU's own input
+    cur, cur_host = model.x0, x0
+    for l, layer in enumerate(model.stack.layers):
+        dst = model.x_final if l == cfg.layers - 1 else model.stack.buf[l & 1]
+        layer.forward(cur, dst)
+        g = gpu_stages(layer, dst, images, T, H)
+        compare_stages(g, cur_host, lps[l], len(images), T, H, cfg.bits, tag=f"DeiT-S layer {l}: ")
+        cur, cur_host = dst, g["out"]
+    # the forward pass above left the same final activations (same kernels, same inputs)
+    xf = cur_host
+    # final LayerNorm + heads from the GPU's final activations
+    want = None
+    for i, name in enumerate(("head", "head_dist")):
+        rows = np.ascontiguousarray(xf[i::T])
+        y, tol = vo.layernorm(rows, ends["lnf_g"], ends["lnf_b"], model.eps)
+        q, lo, hi = vo.quantize_band(y, tol, ends["s_lnf"], cfg.bits, True)
+        c = from_codes(model.head_codes[i])[images]
+        assert np.all(c >= lo) and np.all(c <= hi)
+        w = vo.quantize(ends["w_" + name], 0.0, cfg.bits, True, row_steps=ends["s_w_" + name])
+        want = vo.epilogue_dequant(vo.matmul_i32(c, w), ends["s_lnf"], ends["s_w_" + name], ends["b_" + name], want)
+    assert np.array_equal(logits[images].view(np.uint32), want.view(np.uint32))
+    assert vt.vitint_device_status() == 0

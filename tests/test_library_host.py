@@ -124,15 +124,15 @@ def test_product_fold_matches_definition(L):
     import numpy as np
     s_w = np.array([0.01, 0.02, 0.5], np.float32)
     b = np.array([0.1, -0.2, 0.0], np.float32)
-    a, be = L.fold_requant(np.float32(0.3), s_w, b, np.float32(0.25))
+    a, be = L.vitint_fold_requant(np.float32(0.3), s_w, b, np.float32(0.25))
     assert a.dtype == np.float32 and np.allclose(a, 0.3 * s_w / 0.25, rtol=1e-6)
     assert np.allclose(be, b / 0.25, rtol=1e-6)
-    a2, be2 = L.fold_requant(np.float32(0.3), s_w, None, np.float32(0.25))
+    a2, be2 = L.vitint_fold_requant(np.float32(0.3), s_w, None, np.float32(0.25))
     assert np.array_equal(a, a2) and not be2.any()
 
 
 def test_layernorm_reference_folding_matches_the_oracle_side(L):
-    """The binding's host-side folding of the comparator references (Fig. 5(b)) and the oracle's are two separate
+    """The library's host-side folding of the comparator references (Fig. 5(b), a C entry point) and the oracle's are two separate
     pieces of code that must hand their sides the same numbers: magnitude, sign and flip flag, bit for bit."""
     import numpy as np
     import oracle as vo
@@ -142,8 +142,9 @@ def test_layernorm_reference_folding_matches_the_oracle_side(L):
     gamma[[3, 17]] *= -1.0
     beta = rng.normal(0.0, 0.5, cols).astype(np.float32)
     for bits, signed in ((2, True), (3, True), (4, True), (4, False)):
-        ref, neg, flip = vo.layernorm_references(gamma, beta, 0.31, bits, signed, cols)
-        refs, flip_b = L.fold_layernorm_references(gamma, beta, 0.31, bits, signed, cols)
+        step = np.float32(0.31)
+        ref, neg, flip = vo.layernorm_references(gamma, beta, step, bits, signed, cols)
+        refs, flip_b = L.vitint_fold_layernorm_references(gamma, beta, step, bits, signed, cols)
         assert refs.shape == (cols, 2 ** bits - 1) and refs.dtype == np.float32
         assert np.array_equal(np.abs(refs).view(np.uint32), ref.view(np.uint32))
         assert np.array_equal(np.signbit(refs) & (refs != 0), (neg != 0) & (ref != 0))

@@ -301,7 +301,11 @@ def test_gelu_requant_band_brackets_code():
     s_w = np.full(N, 1e-3, np.float32)
     bias = si.normal(42, (N,), 0.0, 0.01)
     inv_s = np.full(N, np.float32(1.0 / 0.05), np.float32)
-    q, lo, hi = vo.epilogue_gelu_requant(acc.astype(np.int32), np.float32(0.6), s_w, bias, inv_s, 4, False)
+    q0, lo0, hi0 = vo.epilogue_gelu_requant(acc.astype(np.int32), np.float32(0.6), s_w, bias, inv_s, 4, False)
+    assert np.array_equal(q0, lo0) and np.array_equal(q0, hi0)          # no tolerance given: the band is the code
+    q, lo, hi = vo.epilogue_gelu_requant(acc.astype(np.int32), np.float32(0.6), s_w, bias, inv_s, 4, False,
+                                         tol_rel=2.0 ** -23)
+    assert np.array_equal(q, q0)
     assert np.all(lo <= q) and np.all(q <= hi) and np.all(hi - lo <= 1)
     assert (hi != lo).mean() < 1e-3
     # independent evaluation of the code in fp64 agrees wherever the band is a single code
@@ -696,3 +700,92 @@ def test_layernorm_comparator_brute_force_tiny_rows():
             assert q[r].tolist() == want, rows[r]
             n_checked += 1
     assert n_checked > 100
+
+
+# ---------------------------------------------------------------------------
+# band helpers: the tolerances the GPU tests grant must be the stated ones, and narrow
+# ---------------------------------------------------------------------------
+
+def test_quantize_band_hand_rows_exact_rationals():
+    """vo_quantize_band against exact rational arithmetic: codes of y, y - tol and y + tol under the a1 rule
+    (one fp32 subtraction / addition, one fp32 division, ties to even, clamp), including a tie that sits exactly
+    at y + tol and one exactly at y - tol."""
+    step = np.float32(0.25)
+    #            y       tol      (y - tol)/s   (y + tol)/s
+    rows = [(0.300, 0.000, ),   # 1.2 -> 1, band 1..1
+            (0.350, 0.025, ),   # 1.3 .. 1.5: upper end exactly on the tie 1.5 -> even 2
+            (0.400, 0.025, ),   # 1.5 (tie -> 2) .. 1.7 -> 2
+            (0.650, 0.025, ),   # 2.5 (tie -> 2) .. 2.7 -> 3
+            (-0.13, 0.010, ),   # -0.56 -> -1 .. -0.48 -> 0
+            (5.000, 0.500, ),   # clamps at +7
+            (-9.00, 4.000, )]   # clamps at -8 on both ends
+    y = np.array([[r[0] for r in rows]], np.float32)
+    tol = np.array([[r[1] for r in rows]], np.float32)
+    q, lo, hi = vo.quantize_band(y, tol, step, 4, True)
+
+    def code(fr):
+        v = f32_from_fraction(fr / Fraction(float(step)))
+        n = int(np.rint(np.float64(v)))                      # rint of an fp32 value: ties to even
+        return max(-8, min(7, n))
+
+    for j in range(len(rows)):
+        yj, tj = Fraction(float(y[0, j])), Fraction(float(tol[0, j]))
+        lo_in = Fraction(float(f32_from_fraction(yj - tj)))
+        hi_in = Fraction(float(f32_from_fraction(yj + tj)))
+        assert int(q[0, j]) == code(yj), j
+        assert int(lo[0, j]) == code(lo_in), j
+        assert int(hi[0, j]) == code(hi_in), j
+    # with power-of-two friendly numbers the ties are exact: 0.375/0.25 = 1.5 -> 2 and 0.625/0.25 = 2.5 -> 2
+    yy = np.array([[0.25, 0.75]], np.float32)
+    tt = np.array([[0.125, 0.125]], np.float32)
+    q, lo, hi = vo.quantize_band(yy, tt, step, 4, True)
+    assert q.tolist() == [[1, 3]] and lo.tolist() == [[0, 2]] and hi.tolist() == [[2, 4]]
+
+
+def test_layernorm_tolerance_formula_and_band_is_narrow():
+    """The tolerance array of vo_layernorm is 8 * 2^-24 * (|gamma| * max_row|x - mu| / sigma + |beta|), evaluated
+    here in Python on two rows; on ViT-Base-shaped rows the band of codes it induces is at most one code wide and
+    touches fewer than one code in a thousand."""
+    cols = 8
+    x = np.array([[1.0, 2.0, 3.0, 4.0, -2.0, 0.5, 7.0, 0.5], [10.0, 10.5, 9.5, 10.25, 9.75, 10.0, 11.0, 9.0]], np.float32)
+    g = np.array([1.0, -0.5, 2.0, 0.25, 1.5, 1.0, 0.75, 3.0], np.float32)
+    b = np.array([0.0, 0.1, -0.2, 0.3, 0.0, -1.0, 0.5, 0.05], np.float32)
+    eps = 1e-6
+    y, tol = vo.layernorm(x, g, b, eps)
+    for r in range(2):
+        xs = [Fraction(float(v)) for v in x[r]]
+        mu = sum(xs) / cols
+        var = sum((v - mu) ** 2 for v in xs) / cols
+        sigma = math.sqrt(float(var) + float(np.float32(eps)))
+        maxdev = max(abs(float(v - mu)) for v in xs)
+        for k in range(cols):
+            want = 8.0 * 2.0 ** -24 * (abs(float(g[k])) * maxdev / sigma + abs(float(b[k])))
+            assert abs(float(tol[r, k]) - want) <= 2e-7 * want, (r, k)
+            yk = float(xs[k] - mu) / sigma * float(g[k]) + float(b[k])
+            assert abs(float(y[r, k]) - yk) <= 1e-6 * max(1.0, abs(yk))
+    cfg = si.VIT_BASE_LAYER.with_(batch=2)
+    prm = si.layer_parameters(cfg)
+    xa = si.activations(cfg)
+    ya, ta = vo.layernorm(xa, prm["ln1_g"], prm["ln1_b"], 1e-6)
+    assert ta.max() < 1e-5 and ta.min() > 0
+    for bits in (4, 3, 2):
+        q, lo, hi = vo.quantize_band(ya, ta, si.gaussian_lsq_step(1.0, bits), bits, True)
+        assert np.all(lo <= q) and np.all(q <= hi) and np.all(hi - lo <= 1)
+        assert (hi != lo).mean() < 1e-3
+
+
+def test_softmax_band_is_the_two_ulp_neighbourhood():
+    """q_lo / q_hi of vo_softmax_quantize are the codes of p moved by two units in the last place, nothing wider:
+    recomputed here with numpy's nextafter and an fp32 division."""
+    rows, cols = 16, 197
+    S = ((si.splitmix64(91, rows * cols) % np.uint64(801)).astype(np.int64) - 400).astype(np.int32).reshape(rows, cols)
+    c, s_p = np.float32(0.0123), np.float32(2.0 / (cols * math.sqrt(15.0)))
+    p, q, lo, hi = vo.softmax_quantize(S, c, s_p, 4)
+    dn, up = p.copy(), p.copy()
+    for _ in range(2):
+        dn = np.nextafter(dn, np.float32(-np.inf))
+        up = np.nextafter(up, np.float32(np.inf))
+    dn = np.maximum(dn, np.float32(0))
+    code = lambda v: np.clip(np.rint((v / s_p).astype(np.float32)), 0, 15).astype(np.int16)
+    assert np.array_equal(lo, code(dn)) and np.array_equal(hi, code(up)) and np.array_equal(q, code(p))
+    assert np.all(hi - lo <= 1) and (hi != lo).mean() < 2e-3
