@@ -144,6 +144,18 @@ int vitint_widen(const vitint_codes* in, const vitint_codes* out, void* stream);
 int vitint_linear(const vitint_codes* x, float x_step, const vitint_codes* w, const float* w_step,
                   const float* bias, const vitint_epilogue* epi, void* out, int64_t ld_out, void* stream);
 
+/* a2 through the FP4 tensor-core kind (Section V-B: fewer bits, cheaper multiply-accumulate).  e2m1 represents
+ *   0, 1/2, 1, 3/2, 2, 3, 4, 6 and their negatives, so signed codes of at most 3 bits (-4 .. 3) and unsigned codes of
+ *   at most 2 bits (0 .. 3) are exact operands of tcgen05 kind::mxf4 with unit block scales; their products are
+ *   integers and the fp32 accumulators hold the sums exactly (checked by brute force in the tests).
+ *   acc[m][n] = sum_k q_x[m][k] * q_w[n][k], written as int32.
+ *   x: codes [M, K], w: codes [N, K], both stored one code per byte (container_bits = 8), K <= 2^20;
+ *   out: device int32 [M, ld_out], ld_out >= N;  inexact_flag: device int32, set to 1 if any accumulator was not an
+ *   integer (the caller clears it beforehand).  This kernel establishes exactness; it is not tuned for speed.
+ *   Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED (packed containers, or codes e2m1 cannot represent), CUDA. */
+int vitint_linear_e2m1(const vitint_codes* x, const vitint_codes* w, int32_t* out, int64_t ld_out,
+                       int32_t* inexact_flag, void* stream);
+
 /* Strided set of [tokens, head_dim] code slabs inside a larger code matrix (the Q, K
  * or V part of a QKV activation).  Slab (image b, head h) starts at
  * data + b*image_stride_bytes + h*head_stride_bytes; rows are pitch_bytes apart.

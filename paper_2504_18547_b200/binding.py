@@ -90,6 +90,7 @@ def lib():
                                              c_void_p]
         L.vitint_layernorm_compare_quantize.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_float,
                                                         POINTER(_Codes), c_void_p, c_void_p]
+        L.vitint_linear_e2m1.argtypes = [POINTER(_Codes), POINTER(_Codes), c_void_p, c_int64, c_void_p, c_void_p]
         L.vitint_selftest_wait_timeout.argtypes = [c_int64, c_void_p, c_void_p]
         L.vitint_fold_requant.argtypes = [c_float, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
         L.vitint_fold_layernorm_references.argtypes = [c_void_p, c_void_p, c_float, c_int32, c_int32, c_int64, c_void_p,
@@ -289,6 +290,18 @@ def vitint_linear(x: Codes, x_step: float, w: Codes, w_step: torch.Tensor | None
     _check(lib().vitint_linear(byref(dx), float(x_step), byref(dw), _ptr(w_step), _ptr(bias), byref(de), ptr, ld,
                                _stream()), "vitint_linear")
     return out
+
+
+def vitint_linear_e2m1(x: Codes, w: Codes, out: torch.Tensor | None = None, inexact: torch.Tensor | None = None):
+    """Raw accumulators of the integer linear layer computed through the FP4 (e2m1) tensor-core kind.  x, w: codes
+    stored one per byte, signed of at most 3 bits or unsigned of at most 2.  Returns (int32 [M, N], flag): the flag
+    (device int32) becomes 1 if any fp32 accumulator was not an integer."""
+    out = torch.empty((x.rows, w.rows), dtype=torch.int32, device=x.data.device) if out is None else out
+    inexact = torch.zeros(1, dtype=torch.int32, device=x.data.device) if inexact is None else inexact
+    dx, dw = x.desc(), w.desc()
+    _check(lib().vitint_linear_e2m1(byref(dx), byref(dw), out.data_ptr(), _ld(out), inexact.data_ptr(), _stream()),
+           "vitint_linear_e2m1")
+    return out, inexact
 
 
 def vitint_qk(q: Slabs, k: Slabs, batch: int, heads: int, tokens: int, out: torch.Tensor | None = None,

@@ -168,7 +168,8 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& P, const uint32
     const int nvalid = FULL ? 32 : (P.N - n0 < 32 ? P.N - n0 : 32);
     if (KIND == EK_ACC) {
         int32_t* o = (int32_t*)P.out + orow * P.ld_out + colbase + n0;
-        if (FULL) {
+        // 16-byte stores only where the row really starts on a 16-byte boundary (any leading dimension is allowed)
+        if (FULL && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
 #pragma unroll
             for (int i = 0; i < 8; ++i)
                 reinterpret_cast<int4*>(o)[i] = make_int4((int)v[4 * i] >> P.shift, (int)v[4 * i + 1] >> P.shift,
