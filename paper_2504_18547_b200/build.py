@@ -33,5 +33,16 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
     return LIB
 
 
+TRACE_LIB = PKG / "libvitint_trace.so"
+
+
+def build_trace_library() -> Path:
+    """Diagnostic build (-DVITINT_TRACE): the GEMM kernel records a timeline of its warp roles (see trace_gemm.py).
+    A separate file; the product library is never built with the flag."""
+    cmd = ["nvcc", *NVCC_FLAGS, "-DVITINT_TRACE", f"-I{INCLUDE}", str(CSRC / "vitint_lib.cu"), "-o", str(TRACE_LIB)]
+    subprocess.run(cmd, check=True)
+    return TRACE_LIB
+
+
 if __name__ == "__main__":
     print(build_library(force=True, verbose=True))

@@ -507,12 +507,14 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiPara
     if (is_req && (n_tile + 1) * P.bn <= P.N && (P.bn & 31) == 0 && (colbase & 15) == 0) {
         // every column of the tile is real: rolled 16-column blocks
         const long long col0 = colbase + (long long)n_tile * P.bn;
-        if (KIND == EK_REQUANT_GELU && P.unit_out)
-            if (P.out_c == 8) epilogue_requant_blocks<EK_REQUANT_GELU, SMALL, true, true>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
-            else epilogue_requant_blocks<EK_REQUANT_GELU, SMALL, true, false>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
-        else
-            if (P.out_c == 8) epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL, false, true>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
-            else epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL, false, false>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+        if (c_begin < c_end) {
+            if (KIND == EK_REQUANT_GELU && P.unit_out)
+                if (P.out_c == 8) epilogue_requant_blocks<EK_REQUANT_GELU, SMALL, true, true>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+                else epilogue_requant_blocks<EK_REQUANT_GELU, SMALL, true, false>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+            else
+                if (P.out_c == 8) epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL, false, true>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+                else epilogue_requant_blocks<is_req ? KIND : EK_REQUANT, SMALL, false, false>(P, ep, buf, t_row, row_ok, orow, col0, c_begin * 32, c_end * 32);
+        }
         // row padding behind the last column of the matrix
         if (row_ok && P.col_off_inner == 0 && n_tile * P.bn + c_end * 32 >= P.N && c_end > c_begin) {
             for (long long off = ((long long)P.N * P.out_c) >> 3; off + 4 <= P.ld_out; off += 4)
@@ -628,6 +630,28 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             bool ok = true;
             const uint32_t packed_bytes = (P.a_direct ? 0u : P.pa_bytes) + (P.b_direct ? 0u : P.pb_bytes);
             const uint32_t direct_bytes = (P.a_direct ? P.ia_bytes : 0u) + (P.b_direct ? P.ib_bytes : 0u);
+            if (P.a_direct && P.b_direct) {
+                // both operands go straight into the operand ring: slot and phase advance by increments
+                const uint32_t full0 = ptx::smem_addr(&bars.i_full[0]), empty0 = ptx::smem_addr(&bars.i_empty[0]);
+                const int k_blocks = P.k_blocks, ns = P.ns_i;
+                int s = 0;
+                uint32_t ph = 1u, dst = smem_base;
+                for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+                    int m_tile, n_tile, inner, outer;
+                    tile_coords(P, tile, m_tile, n_tile, inner, outer);
+                    const int m0 = m_tile * BM, n0 = n_tile * P.bn;
+                    for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                        VT_STAMP(tr, TT_WAIT_EMPTY);
+                        if (!mbar_wait(empty0 + 8u * (uint32_t)s, ph, abort_ptr)) { ok = false; break; }
+                        VT_STAMP(tr, TT_GOT_EMPTY);
+                        const uint32_t full = full0 + 8u * (uint32_t)s;
+                        ptx::mbar_arrive_expect_tx(full, direct_bytes);
+                        ptx::tma_load_4d(dst, &map_a, full, kb * BK, m0, inner, outer);
+                        ptx::tma_load_4d(dst + P.ia_bytes, &map_b, full, kb * BK, n0, inner, outer);
+                        if (++s == ns) { s = 0; ph ^= 1u; dst = smem_base; } else dst += stage_i;
+                    }
+                }
+            } else
             for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
                 int m_tile, n_tile, inner, outer;
                 tile_coords(P, tile, m_tile, n_tile, inner, outer);
@@ -677,7 +701,21 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t idesc = ptx::idesc_i8(BM, P.bn, P.a_signed, P.b_signed, P.b_mn_major);
             VT_TRACER(tr, 1);
             VT_STAMP(tr, TT_START);
-            int it = 0, tl = 0;
+            // This one thread feeds the tensor core, and a lone thread runs its dependent scalar instructions a few
+            // cycles apart: everything the loop needs is therefore kept in registers and advanced by additions (no
+            // division for the ring slot, no descriptor rebuilt per K block); the four MMAs of a whole K block are
+            // issued back to back.
+            const uint64_t a_desc0 = ptx::smem_desc(smem_base, 16, 1024, ptx::SWIZZLE_128B);
+            const uint64_t b_desc0 = P.b_mn_major ? ptx::smem_desc(smem_base + P.ia_bytes, 16, 512, ptx::SWIZZLE_64B)
+                                                  : ptx::smem_desc(smem_base + P.ia_bytes, 16, 1024, ptx::SWIZZLE_128B);
+            const uint64_t stage_step = (uint64_t)(stage_i >> 4);            // descriptor address field counts 16-byte units
+            const uint64_t b_kstep = P.b_mn_major ? 128u : 2u;
+            const uint32_t full0 = ptx::smem_addr(&bars.i_full[0]), empty0 = ptx::smem_addr(&bars.i_empty[0]);
+            const int k_blocks = P.k_blocks, ns = P.ns_i;
+            const int last_steps = (P.K - (k_blocks - 1) * BK + 31) / 32;     // MMAs of the last (possibly partial) K block
+            int s = 0, tl = 0;
+            uint32_t ph = 0;
+            uint64_t a_desc = a_desc0, b_desc = b_desc0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++tl) {
                 const int buf = tl & 1;
@@ -687,28 +725,25 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 VT_STAMP(tr, TT_GOT_EMPTY);
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * acc_stride;
-                for (int kb = 0; kb < P.k_blocks; ++kb, ++it) {
-                    const int s = it % P.ns_i;
-                    const uint32_t ph = (uint32_t)(it / P.ns_i) & 1u;
+                for (int kb = 0; kb < k_blocks; ++kb) {
                     VT_STAMP(tr, TT_WAIT_FULL);
-                    if (!mbar_wait(ptx::smem_addr(&bars.i_full[s]), ph, abort_ptr)) { ok = false; break; }
+                    if (!mbar_wait(full0 + 8u * (uint32_t)s, ph, abort_ptr)) { ok = false; break; }
                     VT_STAMP(tr, TT_GOT_FULL);
                     ptx::tc_fence_after();
-                    const uint32_t a_addr = smem_base + (uint32_t)s * stage_i;
-                    const uint32_t b_addr = a_addr + P.ia_bytes;
-                    const uint64_t a_desc = ptx::smem_desc(a_addr, 16, 1024, ptx::SWIZZLE_128B);
-                    const uint64_t b_desc = P.b_mn_major ? ptx::smem_desc(b_addr, 16, 512, ptx::SWIZZLE_64B)
-                                                         : ptx::smem_desc(b_addr, 16, 1024, ptx::SWIZZLE_128B);
-                    const int k_left = P.K - kb * BK;
-                    const int k_steps = k_left >= BK ? BK / 32 : (k_left + 31) / 32;
-                    for (int k = 0; k < k_steps; ++k) {
-                        // 32 int8 of K per MMA: 32 bytes along a swizzled row, or four 8-row
-                        // groups (4 * 512 bytes) when K is the slow axis of the B tile
-                        const uint64_t a_k = a_desc + (uint64_t)(k * 2);
-                        const uint64_t b_k = b_desc + (uint64_t)(P.b_mn_major ? k * 128 : k * 2);
-                        ptx::mma_i8(d_tmem, a_k, b_k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    // 32 int8 of K per MMA: 32 bytes along a swizzled row, or four 8-row
+                    // groups (4 * 512 bytes) when K is the slow axis of the B tile
+                    if (kb + 1 < k_blocks || last_steps == 4) {
+                        ptx::mma_i8(d_tmem, a_desc, b_desc, idesc, kb != 0 ? 1u : 0u);
+                        ptx::mma_i8(d_tmem, a_desc + 2u, b_desc + b_kstep, idesc, 1u);
+                        ptx::mma_i8(d_tmem, a_desc + 4u, b_desc + 2u * b_kstep, idesc, 1u);
+                        ptx::mma_i8(d_tmem, a_desc + 6u, b_desc + 3u * b_kstep, idesc, 1u);
+                    } else {
+                        for (int k = 0; k < last_steps; ++k)
+                            ptx::mma_i8(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)k * b_kstep, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
-                    ptx::mma_commit(ptx::smem_addr(&bars.i_empty[s]));
+                    ptx::mma_commit(empty0 + 8u * (uint32_t)s);
+                    if (++s == ns) { s = 0; ph ^= 1u; a_desc = a_desc0; b_desc = b_desc0; }
+                    else { a_desc += stage_step; b_desc += stage_step; }
                 }
                 if (ok) ptx::mma_commit(ptx::smem_addr(&bars.acc_full[buf]));
                 VT_STAMP(tr, TT_ISSUED);

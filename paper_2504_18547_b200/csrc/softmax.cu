@@ -1,8 +1,7 @@
-// a5: scale + row softmax + quantize (Eq. 3), one warp per row.
+// a5: scale + row softmax + quantize (Eq. 3), half a warp per row.
 //
-// HBM-bound: 4 bytes read and c/8 bytes written per element.  The row lives in
-// registers (lane l owns columns 256*k + 8*l .. +7 of chunk k); the maximum and
-// the normaliser are reduced with warp shuffles.
+// HBM-bound by bytes: 4 bytes read and c/8 bytes written per element.  The row lives in
+// registers; the maximum and the normaliser are reduced with shuffles inside the half-warp.
 //
 // Accuracy target: probabilities within 2 ulp of the exactly rounded softmax.
 //   * t_j - max is formed exactly in fp64 (a rounded fp32 difference would already
@@ -16,175 +15,253 @@
 
 namespace vitint {
 
-// exp(t - mx) for mx >= t, all in fp32 and integer instructions (no conversion instruction: those run at an eighth of
-// the issue rate and used to bound this kernel).
+// exp(t - mx) for mx >= t, two elements at a time, in fp32 and integer instructions (no special-function unit;
+// every packed operation gives each half the IEEE result of the scalar one).
 //   * t - mx as an exact two-float sum (TwoSum), so nothing is lost when the two differ by more than a factor of two;
 //   * k = rint((t - mx) * log2 e) by the 1.5*2^23 addition, which also leaves k as an integer in the mantissa;
 //   * r = (t - mx) - k*ln2 with ln2 split so that k*ln2_hi is exact, the low parts folded in with one FMA;
 //   * degree-7 Taylor polynomial on |r| <= ln2/2 (truncation < 0.1 ulp), then 2^k added to the exponent field.
 // Results below 2^-125 (relative to the row's largest term, which is 1) are returned as 0: they lie in the range
-// where the tolerance is the absolute 2^-126.
-__device__ __forceinline__ float exp_reduced(float t, float mx) {
-    const float sh = __fadd_rn(t, -mx);
-    const float bv = __fadd_rn(sh, -t);
-    const float sl = __fadd_rn(__fadd_rn(t, -__fadd_rn(sh, -bv)), __fadd_rn(-mx, -bv));     // sh + sl = t - mx exactly
-    const float d = fmaxf(sh, -200.0f);
-    const float m = __fmaf_rn(d, 1.44269504088896340736f, 12582912.0f);
-    const float kf = __fadd_rn(m, -12582912.0f);
-    const int k = __float_as_int(m) - 0x4B400000;
-    const float rh = __fmaf_rn(-kf, 0.693145751953125f, d);                  // exact: ln2_hi has 15 significant bits
-    const float rl = __fmaf_rn(-kf, 1.42860682030941723212e-6f, sl);         // ln2 - ln2_hi, and the low part of t - mx
-    const float rf = __fadd_rn(rh, rl);
-    float p = 1.0f / 5040.0f;
-    p = fmaf(p, rf, 1.0f / 720.0f);
-    p = fmaf(p, rf, 1.0f / 120.0f);
-    p = fmaf(p, rf, 1.0f / 24.0f);
-    p = fmaf(p, rf, 1.0f / 6.0f);
-    p = fmaf(p, rf, 0.5f);
-    p = fmaf(p, rf, 1.0f);
-    p = fmaf(p, rf, 1.0f);
-    // p lies in [0.70, 1.42]: for k >= -125 the product p * 2^k is normal and exact as an exponent addition
-    return k >= -125 ? __int_as_float(k * 8388608 + __float_as_int(p)) : 0.0f;
+// where the tolerance is the absolute 2^-126.  t = -inf (a column past the row's end) gives exactly 0.
+__device__ __forceinline__ f32x2 exp_reduced2(f32x2 t, f32x2 nmx) {
+    const f32x2 neg1 = f2_dup(-1.0f);
+    const f32x2 sh = f2_add(t, nmx);
+    const f32x2 bv = f2_fma(t, neg1, sh);                         // sh - t
+    const f32x2 u = f2_fma(bv, neg1, sh);                         // sh - bv
+    const f32x2 v = f2_fma(u, neg1, t);                           // t - (sh - bv)
+    const f32x2 w = f2_fma(bv, neg1, nmx);                        // -mx - bv
+    const f32x2 sl = f2_add(v, w);                                // sh + sl = t - mx exactly
+    // m = 1.5*2^23 + k for every difference down to about -2^21; further down (and for -inf or NaN) m falls below the
+    // threshold tested at the end and the result is 0 whatever the polynomial made of it
+    const f32x2 m = f2_fma(sh, f2_dup(1.44269504088896340736f), f2_dup(12582912.0f));
+    const f32x2 kf = f2_add(m, f2_dup(-12582912.0f));
+    const f32x2 rh = f2_fma(kf, f2_dup(-0.693145751953125f), sh);              // exact: ln2_hi has 15 significant bits
+    const f32x2 rl = f2_fma(kf, f2_dup(-1.42860682030941723212e-6f), sl);      // ln2 - ln2_hi, and the low part of t - mx
+    const f32x2 rf = f2_add(rh, rl);
+    f32x2 p = f2_dup(1.0f / 5040.0f);
+    p = f2_fma(p, rf, f2_dup(1.0f / 720.0f));
+    p = f2_fma(p, rf, f2_dup(1.0f / 120.0f));
+    p = f2_fma(p, rf, f2_dup(1.0f / 24.0f));
+    p = f2_fma(p, rf, f2_dup(1.0f / 6.0f));
+    p = f2_fma(p, rf, f2_dup(0.5f));
+    p = f2_fma(p, rf, f2_dup(1.0f));
+    p = f2_fma(p, rf, f2_dup(1.0f));
+    // p lies in [0.70, 1.42]: for k >= -125 the product p * 2^k is normal and exact as an exponent addition.  The
+    // float m holds 1.5*2^23 + k exactly, and its low 9 bits shifted up by 23 are k's (0x4B400000 << 23 is 0 mod 2^32).
+    float m0, m1, p0, p1;
+    f2_unpack(m, m0, m1);
+    f2_unpack(p, p0, p1);
+    const float e0 = m0 >= 12582912.0f - 125.0f ? __int_as_float(__float_as_int(m0) * 8388608 + __float_as_int(p0)) : 0.0f;
+    const float e1 = m1 >= 12582912.0f - 125.0f ? __int_as_float(__float_as_int(m1) * 8388608 + __float_as_int(p1)) : 0.0f;
+    return f2_pack(e0, e1);
 }
 
-template <int C, int NCH>
-__global__ void __launch_bounds__(256)
-softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, int64_t ld_s, float c, float p_step,
-                        uint8_t* __restrict__ out, int64_t pitch, float* __restrict__ p_out, int64_t ld_p, float qp,
-                        int vec_in, int vec_p) {
-    grid_dependency_wait();        // inputs may come from the previous kernel of the stream
-    grid_dependency_launch();
-    const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (row >= rows) return;
-    const int32_t* sr = s + row * ld_s;
+constexpr int SM_ROWS_PER_BLOCK = 16;      // half a warp per row, eight warps
+constexpr int SM_TAIL_SLOTS = 4;           // up to 63 columns behind the last whole 64-column chunk, 16 per slot
 
-    // Columns past the row's end take t = -inf.  Their exponential is exactly 0, so they add nothing to the row
-    // sum and quantize to code 0 (the padding value) without any per-element masking further down.
-    float t[NCH][8];
+// One row by half a warp.  Lane h (0..15) of the row owns columns 64 j + 4 h .. + 3 of every whole 64-column chunk j
+// (one 16-byte load each) and, of the up to 63 columns behind the last whole chunk, column 64 nv + 16 s + h of slot
+// s: a row of 197 columns costs 13 element slots per lane instead of the 16 that whole vectors would take.
+// NVT is the compiled number of chunk slots (>= the row's whole chunks nv; a surplus slot carries t = -inf and stores
+// nothing); NTT the compiled number of tail slots.  The loops are straight-line code: loads and stores are
+// predicated, nothing branches per element.  VEC: 16-byte loads are legal; DIV3: the step admits the three-operation
+// exact quotient.
+template <int C, int NVT, int NTT, bool VEC, bool DIV3>
+__device__ __forceinline__ void softmax_row(const int32_t* __restrict__ sr, int cols, float c, const Divisor dv, float qp,
+                                            uint8_t* crow, float* pr, bool vec_p, int hl) {
+    const int nv = cols >> 6;
+    const int tail0 = nv << 6, n_tail = cols - tail0;
+    const f32x2 c2 = f2_dup(c);
+    constexpr int NP = 2 * NVT + (NTT + 1) / 2;          // register pairs: two per chunk, one per two tail slots
+    f32x2 t[NP > 0 ? NP : 1];
     float mx = -INFINITY;
+    // Columns past the row's end take t = -inf: their exponential is exactly 0, so they add nothing to the row
+    // sum and quantize to code 0 without any masking further down.
 #pragma unroll
-    for (int k = 0; k < NCH; ++k) {
-        const int col = k * 256 + lane * 8;
-        if (vec_in && col + 8 <= ld_s) {
-            // whole 32 bytes inside the row's storage (the leading dimension may exceed the column count)
-            const int4 a = __ldg(reinterpret_cast<const int4*>(sr + col));
-            const int4 b = __ldg(reinterpret_cast<const int4*>(sr + col) + 1);
-            t[k][0] = (float)a.x * c; t[k][1] = (float)a.y * c; t[k][2] = (float)a.z * c; t[k][3] = (float)a.w * c;
-            t[k][4] = (float)b.x * c; t[k][5] = (float)b.y * c; t[k][6] = (float)b.z * c; t[k][7] = (float)b.w * c;
-            if (col + 8 > cols) {
+    for (int j = 0; j < NVT; ++j) {
+        const int col = j * 64 + hl * 4;
+        const bool have = j < nv;
+        int4 a = make_int4(0, 0, 0, 0);
+        if (have) {
+            if (VEC) a = __ldg(reinterpret_cast<const int4*>(sr + col));
+            else a = make_int4(__ldg(sr + col), __ldg(sr + col + 1), __ldg(sr + col + 2), __ldg(sr + col + 3));
+        }
+        const f32x2 lo = f2_mul(f2_pack((float)a.x, (float)a.y), c2), hi = f2_mul(f2_pack((float)a.z, (float)a.w), c2);
+        t[2 * j] = have ? lo : f2_dup(-INFINITY);
+        t[2 * j + 1] = have ? hi : f2_dup(-INFINITY);
+        float x0, x1, x2, x3;
+        f2_unpack(t[2 * j], x0, x1);
+        f2_unpack(t[2 * j + 1], x2, x3);
+        mx = fmaxf(fmaxf(mx, fmaxf(x0, x1)), fmaxf(x2, x3));
+    }
+    {
+        float x[NTT > 0 ? NTT + 1 : 2];
+        x[NTT > 0 ? NTT : 1] = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) if (col + i >= cols) t[k][i] = -INFINITY;
-            }
-        } else if (col < cols) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) t[k][i] = (col + i < cols) ? (float)__ldg(sr + col + i) * c : -INFINITY;
-        } else {
-            // lanes wholly past the row: nothing to load (kept apart so that a warp whose other lanes all took the
-            // vector path does not walk the scalar one as well)
-#pragma unroll
-            for (int i = 0; i < 8; ++i) t[k][i] = -INFINITY;
+        for (int q = 0; q < NTT; ++q) {
+            const int o = q * 16 + hl;
+            int v = 0;
+            if (o < n_tail) v = __ldg(sr + tail0 + o);
+            x[q] = o < n_tail ? __fmul_rn((float)v, c) : -INFINITY;
+            mx = fmaxf(mx, x[q]);
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) mx = fmaxf(mx, t[k][i]);
+        for (int q = 0; q < NTT; q += 2) t[2 * NVT + q / 2] = f2_pack(x[q], x[q + 1]);
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
 
-    // two interleaved fp64 partial sums; a float enters as a double built from its bits with integer
-    // multiply-adds (every term is zero or a positive normal float; a zero adds 2^-127, nothing beside the
-    // row's largest term, which is 1)
+    // exponentials (kept in the registers of t) and the fp64 row sum
+    const f32x2 nmx = f2_dup(-mx);
     double z0 = 0.0, z1 = 0.0;
 #pragma unroll
-    for (int k = 0; k < NCH; ++k) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float e = exp_reduced(t[k][i], mx);
-            t[k][i] = e;
-            const uint32_t eb = __float_as_uint(e);
-            uint32_t hi, lo;
-            asm("mad.hi.u32 %0, %1, 536870912, 939524096;" : "=r"(hi) : "r"(eb));    // (eb >> 3) + 0x38000000
-            asm("mul.lo.u32 %0, %1, 536870912;" : "=r"(lo) : "r"(eb));                // eb << 29
-            const double ed = __hiloint2double((int)hi, (int)lo);
-            if (i & 1) z1 += ed; else z0 += ed;
-        }
+    for (int i = 0; i < NP; ++i) {
+        t[i] = exp_reduced2(t[i], nmx);
+        float e0, e1;
+        f2_unpack(t[i], e0, e1);
+        z0 += (double)e0;
+        z1 += (double)e1;
     }
     double z = z0 + z1;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-    const double rz = 1.0 / z;
-    const float rzh = (float)rz, rzl = (float)(rz - (double)(float)rz);   // 1/Z as two floats
-    const Divisor dv = make_divisor(p_step);
+    for (int o = 8; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    // 1/Z to about 2^-45 from the fp32 reciprocal and one Newton step in fp64 (Z lies in [1, cols]: no range issue),
+    // then split into two floats
+    const double r0 = (double)__frcp_rn((float)z);
+    const double rz = r0 * (2.0 - z * r0);
+    const float rzh = (float)rz, rzl = (float)(rz - (double)(float)rz);
+    const f32x2 rzh2 = f2_dup(rzh), rzl2 = f2_dup(rzl);
+    const f32x2 dr2 = f2_dup(dv.r), ndb2 = f2_dup(-dv.b), magic2 = f2_dup(12582912.0f);
 
-    const int chunk_bytes = 32 * C;                                   // 256 codes
-    const int n_out_chunks = (int)((pitch + chunk_bytes - 1) / chunk_bytes);
-    for (int k = 0; k < n_out_chunks; ++k) {
-        uint32_t w0 = 0, w1 = 0;
-        if (k < NCH) {
-            float p[8];
-#pragma unroll
-            for (int u = 0; u < NCH; ++u)
-                if (u == k) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) p[i] = fmaf(t[u][i], rzh, t[u][i] * rzl);
-                }
-            const int col = k * 256 + lane * 8;
-            if (p_out && col < cols) {
-                float* pr = p_out + row * ld_p + col;
-                if (vec_p && col + 8 <= cols) {
-                    reinterpret_cast<float4*>(pr)[0] = make_float4(p[0], p[1], p[2], p[3]);
-                    reinterpret_cast<float4*>(pr)[1] = make_float4(p[4], p[5], p[6], p[7]);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) if (col + i < cols) pr[i] = p[i];
-                }
-            }
-            // p >= 0, so only the upper clamp is needed; adding 1.5*2^23 rounds to nearest even and leaves the
-            // (unsigned) code in the low mantissa bits, and the codes combine by shift-add without masking
-            uint32_t cb[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) cb[i] = __float_as_uint(fminf(div_rn(p[i], dv), qp) + 12582912.0f);
-            if (C == 8) {
-                w0 = cb[0] + (cb[1] << 8) + (cb[2] << 16) + (cb[3] << 24) - 0x4B400000u * 0x01010101u;
-                w1 = cb[4] + (cb[5] << 8) + (cb[6] << 16) + (cb[7] << 24) - 0x4B400000u * 0x01010101u;
-            } else {
-                uint32_t acc = cb[0];
-#pragma unroll
-                for (int i = 1; i < 8; ++i) acc += cb[i] << (C * i);
-                uint32_t ones = 0;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) ones += 1u << (C * i);
-                w0 = acc - 0x4B400000u * ones;
-                if (C == 2) w0 &= 0xFFFFu;
-            }
-        }
-        uint8_t* orow = out + row * pitch;
-        const int64_t off = (int64_t)k * chunk_bytes + lane * C;       // this lane's C bytes
-        if (C == 8) {
-            if (off + 8 <= pitch) *reinterpret_cast<uint2*>(orow + off) = make_uint2(w0, w1);
-        } else if (C == 4) {
-            if (off + 4 <= pitch) *reinterpret_cast<uint32_t*>(orow + off) = w0;
+    // p = e / Z, code = min(rint(p / p_step), Qp) (p >= 0: no lower clamp); adding 1.5*2^23 rounds to nearest even and
+    // leaves the unsigned code in the low mantissa bits.  b0, b1: the two codes' float bits.
+    auto quantize_pair = [&](f32x2 e, f32x2& p, uint32_t& b0, uint32_t& b1) {
+        p = f2_fma(e, rzh2, f2_mul(e, rzl2));
+        float q0, q1;
+        if (DIV3) {
+            const f32x2 qa = f2_mul(p, dr2);                            // Markstein: RN(p / step) in three operations
+            const f32x2 rem = f2_fma(qa, ndb2, p);
+            f2_unpack(f2_fma(rem, dr2, qa), q0, q1);
         } else {
-            w0 |= __shfl_xor_sync(0xffffffffu, w0, 1) << 16;
-            if ((lane & 1) == 0 && off + 4 <= pitch) *reinterpret_cast<uint32_t*>(orow + off) = w0;
+            float p0, p1;
+            f2_unpack(p, p0, p1);
+            q0 = __fdiv_rn(p0, dv.b);
+            q1 = __fdiv_rn(p1, dv.b);
+        }
+        float c0, c1;
+        f2_unpack(f2_add(f2_pack(fminf(q0, qp), fminf(q1, qp)), magic2), c0, c1);
+        b0 = __float_as_uint(c0);
+        b1 = __float_as_uint(c1);
+    };
+#pragma unroll
+    for (int j = 0; j < NVT; ++j) {
+        f32x2 pa, pb;
+        uint32_t b0, b1, b2, b3;
+        quantize_pair(t[2 * j], pa, b0, b1);
+        quantize_pair(t[2 * j + 1], pb, b2, b3);
+        const int col = j * 64 + hl * 4;
+        const bool have = j < nv;
+        if (pr != nullptr && have) {
+            float f0, f1, f2, f3;
+            f2_unpack(pa, f0, f1);
+            f2_unpack(pb, f2, f3);
+            if (vec_p) *reinterpret_cast<float4*>(pr + col) = make_float4(f0, f1, f2, f3);
+            else { pr[col] = f0; pr[col + 1] = f1; pr[col + 2] = f2; pr[col + 3] = f3; }
+        }
+        // four codes = C/2 bytes, combined by shift-add (the constant high bits of the four floats are removed at once)
+        const uint32_t w = b0 + (b1 << C) + (b2 << (2 * C)) + (b3 << (3 * C)) -
+                           0x4B400000u * (1u + (1u << C) + (1u << (2 * C)) + (1u << (3 * C)));
+        if (have) {
+            if (C == 8) *reinterpret_cast<uint32_t*>(crow + col) = w;
+            else if (C == 4) *reinterpret_cast<uint16_t*>(crow + (col >> 1)) = (uint16_t)w;
+            else crow[col >> 2] = (uint8_t)w;
+        }
+    }
+#pragma unroll
+    for (int q2 = 0; q2 < NTT; q2 += 2) {
+        f32x2 pa;
+        uint32_t b[2];
+        quantize_pair(t[2 * NVT + q2 / 2], pa, b[0], b[1]);
+        float f[2];
+        f2_unpack(pa, f[0], f[1]);
+#pragma unroll
+        for (int i = 0; i < 2 && q2 + i < NTT; ++i) {
+            const int o = (q2 + i) * 16 + hl;
+            // neighbouring lanes hold neighbouring columns: 8/C of them share a byte (every lane takes part in the
+            // shuffles; lanes past the tail hold code 0)
+            uint32_t code = b[i] - 0x4B400000u;
+            if (C == 4) code |= __shfl_xor_sync(0xffffffffu, code, 1) << 4;
+            if (C == 2) {
+                code |= __shfl_xor_sync(0xffffffffu, code, 1) << 2;
+                code |= __shfl_xor_sync(0xffffffffu, code, 2) << 4;
+            }
+            if (o < n_tail) {
+                if (pr != nullptr) pr[tail0 + o] = f[i];
+                const int col = tail0 + o;
+                if (C == 8) crow[col] = (uint8_t)code;
+                else if (C == 4) { if ((hl & 1) == 0) crow[col >> 1] = (uint8_t)code; }
+                else { if ((hl & 3) == 0) crow[col >> 2] = (uint8_t)code; }
+            }
         }
     }
 }
 
+template <int C, int NVT, int NTT, bool VEC>
+__global__ void __launch_bounds__(32 * SM_ROWS_PER_BLOCK / 2)
+softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, int64_t ld_s, float c, float p_step,
+                        uint8_t* __restrict__ out, int64_t pitch, float* __restrict__ p_out, int64_t ld_p, float qp,
+                        int vec_p) {
+    extern __shared__ __align__(16) uint8_t sm_codes[];   // one output row (pitch bytes) per half-warp
+    grid_dependency_wait();        // inputs may come from the previous kernel of the stream
+    grid_dependency_launch();
+    const int hl = threadIdx.x & 15;
+    const int hw = threadIdx.x >> 4;                                   // half-warp of the block
+    const int64_t row_raw = (int64_t)blockIdx.x * SM_ROWS_PER_BLOCK + hw;
+    const bool row_ok = row_raw < rows;
+    const int64_t row = row_ok ? row_raw : rows - 1;                   // a surplus half-warp repeats the last row, stores nothing
+    uint8_t* const crow = sm_codes + (size_t)hw * pitch;
+    // padding behind the last code (and the unused part of a shared byte) is zero: clear the row buffer first
+    for (int o = hl * 16; o < pitch; o += 256) *reinterpret_cast<uint4*>(crow + o) = make_uint4(0u, 0u, 0u, 0u);
+    __syncwarp();
+    float* const pr = (p_out != nullptr && row_ok) ? p_out + row * ld_p : nullptr;
+    const Divisor dv = make_divisor(p_step);
+    if (dv.exact) softmax_row<C, NVT, NTT, VEC, true>(s + row * ld_s, cols, c, dv, qp, crow, pr, vec_p != 0, hl);
+    else softmax_row<C, NVT, NTT, VEC, false>(s + row * ld_s, cols, c, dv, qp, crow, pr, vec_p != 0, hl);
+    __syncwarp();
+    // the finished row leaves in 16-byte pieces
+    if (row_ok) {
+        uint8_t* const orow = out + row * pitch;
+        for (int o = hl * 16; o < pitch; o += 256) *reinterpret_cast<uint4*>(orow + o) = *reinterpret_cast<const uint4*>(crow + o);
+    }
+}
+
+template <int C, int NVT, int NTT>
+static int launch_softmax_nv(const int32_t* s, int64_t rows, int cols, int64_t ld_s, float c, float p_step, uint8_t* out,
+                             int64_t pitch, float* p, int64_t ld_p, float qp, int vec_in, int vec_p, cudaStream_t st) {
+    dim3 grid((unsigned)((rows + SM_ROWS_PER_BLOCK - 1) / SM_ROWS_PER_BLOCK)), block(16 * SM_ROWS_PER_BLOCK);
+    const size_t smem = (size_t)SM_ROWS_PER_BLOCK * (size_t)pitch;
+    if (smem > 48 * 1024) return VITINT_ERR_UNSUPPORTED;
+    if (vec_in) launch_kernel(softmax_quantize_kernel<C, NVT, NTT, true>, grid, block, smem, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_p);
+    else launch_kernel(softmax_quantize_kernel<C, NVT, NTT, false>, grid, block, smem, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_p);
+    return cuda_status(cudaGetLastError());
+}
+
 template <int C>
-static int launch_softmax(int nch, const int32_t* s, int64_t rows, int cols, int64_t ld_s, float c, float p_step,
+static int launch_softmax(const int32_t* s, int64_t rows, int cols, int64_t ld_s, float c, float p_step,
                           uint8_t* out, int64_t pitch, float* p, int64_t ld_p, float qp, int vec_in, int vec_p,
                           cudaStream_t st) {
-    const int warps = 8;
-    dim3 grid((unsigned)((rows + warps - 1) / warps)), block(32 * warps);
-    switch (nch) {
-        case 1: launch_kernel(softmax_quantize_kernel<C, 1>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
-        case 2: launch_kernel(softmax_quantize_kernel<C, 2>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
-        case 3: launch_kernel(softmax_quantize_kernel<C, 3>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
-        case 4: launch_kernel(softmax_quantize_kernel<C, 4>, dim3(grid), dim3(block), 0, st, s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p); break;
-        default: return VITINT_ERR_UNSUPPORTED;
+    const int nv = cols >> 6, n_tail = cols & 63;
+    const bool short_tail = n_tail <= 32;           // two tail slots are enough
+#define VITINT_SM_CASE(NVT)                                                                                                       \
+    if (nv <= NVT) {                                                                                                              \
+        if (n_tail == 0) return launch_softmax_nv<C, NVT, 0>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p, st); \
+        if (short_tail) return launch_softmax_nv<C, NVT, 2>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p, st); \
+        return launch_softmax_nv<C, NVT, 4>(s, rows, cols, ld_s, c, p_step, out, pitch, p, ld_p, qp, vec_in, vec_p, st);           \
     }
-    return cuda_status(cudaGetLastError());
+    VITINT_SM_CASE(0) VITINT_SM_CASE(1) VITINT_SM_CASE(2) VITINT_SM_CASE(3) VITINT_SM_CASE(4) VITINT_SM_CASE(6) VITINT_SM_CASE(9)
+    VITINT_SM_CASE(12) VITINT_SM_CASE(16)
+#undef VITINT_SM_CASE
+    return VITINT_ERR_UNSUPPORTED;
 }
 
 // Shift-based softmax with the division-free quantizer (Eq. 4 and the comparator of Section IV-B),
@@ -354,14 +431,13 @@ extern "C" int vitint_softmax_quantize(const int32_t* s, int64_t rows, int32_t c
     const int cb = codes_container(p_out);
     int qn, qp;
     code_range(p_out->bits, 0, &qn, &qp);
-    const int nch = (cols + 255) / 256;
     const int vec_in = (aligned16(s) && ld_s % 4 == 0) ? 1 : 0;
     const int vec_p = (p_f32 && aligned16(p_f32) && ld_p % 4 == 0) ? 1 : 0;
     cudaStream_t st = (cudaStream_t)stream;
     uint8_t* o = (uint8_t*)p_out->data;
-    if (cb == 2) return launch_softmax<2>(nch, s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
-    if (cb == 4) return launch_softmax<4>(nch, s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
-    return launch_softmax<8>(nch, s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
+    if (cb == 2) return launch_softmax<2>(s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
+    if (cb == 4) return launch_softmax<4>(s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
+    return launch_softmax<8>(s, rows, cols, ld_s, c, p_step, o, p_out->pitch_bytes, p_f32, ld_p, (float)qp, vec_in, vec_p, st);
 }
 
 extern "C" int vitint_softmax_shift_quantize(const int32_t* s, int64_t rows, int32_t cols, int64_t ld_s, float c2,

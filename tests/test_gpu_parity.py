@@ -136,7 +136,8 @@ def test_byte_containers_for_low_bit_codes():
     assert np.array_equal(from_codes(q8), vo.epilogue_requant(acc, alpha, beta, 4, True)) and padding_is_zero(q8)
 
 
-BYTE_SHAPES = [(129, 64, 256), (256, 192, 512), (300, 768, 768), (1000, 1000, 1000), (515, 3072, 264), (2049, 384, 2304)]
+BYTE_SHAPES = [(129, 64, 256), (256, 192, 512), (300, 768, 768), (1000, 1000, 1000), (515, 3072, 264), (2049, 384, 2304),
+               (257, 1024, 128), (1000, 1008, 1000), (400, 16, 200), (5000, 768, 264)]
 
 
 @pytest.mark.parametrize("M,K,N", BYTE_SHAPES)
