@@ -401,14 +401,24 @@ def run_ours(args, cfg):
         from paper_2504_18547_b200.encoder import NormedAttention
         dcfg = si.DEIT_S_ATTENTION
         dprm, dqkn = si.layer_parameters(dcfg), si.qk_norm_parameters(dcfg)
-        mod = NormedAttention(dcfg.batch, dcfg.tokens, dcfg.heads, dcfg.bits, dprm, dqkn, device)
         dx = torch.from_numpy(si.activations(dcfg)).to(device)
         ds_x = float(si.lsq_step(dx[:dcfg.tokens].cpu().numpy(), dcfg.bits, True))
         dxq = vt.vitint_quantize(dx, ds_x, dcfg.bits, True)
-        ms = timed(lambda: mod.forward(dxq, ds_x))
-        standalone["deit_s_attention_n198_b64"] = {"ms": round(ms, 4), "tops": round(mod.ops() / (ms * 1e-3) / 1e12, 1),
-                                                   "images_per_s": round(dcfg.batch / (ms * 1e-3), 1), "launches": 10}
-        del mod, dx, dxq
+        # fused: the per-head LayerNorm + comparator quantizer runs in the QKV GEMM's epilogue (4 launches);
+        # unfused: fp32 Q and K rows through memory and a LayerNorm kernel each (10 launches)
+        for name, fused, launches in (("deit_s_attention_n198_b64", True, 4), ("deit_s_attention_n198_b64_unfused", False, 10)):
+            mod = NormedAttention(dcfg.batch, dcfg.tokens, dcfg.heads, dcfg.bits, dprm, dqkn, device, fused=fused)
+            ms = timed(lambda: mod.forward(dxq, ds_x))
+            standalone[name] = {"ms": round(ms, 4), "tops": round(mod.ops() / (ms * 1e-3) / 1e12, 1),
+                                "images_per_s": round(dcfg.batch / (ms * 1e-3), 1), "launches": launches}
+            if fused:
+                ms_q = timed(lambda: vt.vitint_linear_qkv_norm(dxq, ds_x, mod.w_qkv, mod.s_w_all, mod.bias_all, mod.refs_all,
+                                                               mod.flip_all, mod.n_eps, mod.alpha_v, mod.beta_v, mod.bits,
+                                                               out=mod.qkv, stats=mod.stats_all))
+                standalone["qkv_linear_with_head_layernorm_deit_s_b64"] = {
+                    "ms": round(ms_q, 4), "tops": round(2 * 3 * mod.rows * mod.dim * mod.dim / (ms_q * 1e-3) / 1e12, 1)}
+            del mod
+        del dx, dxq
         # the same encoder layer with the paper's own quantizers throughout (Eq. 4 softmax with the division-free
         # comparator, Eq. 5 statistics with the comparator LayerNorm quantizer): unfused attention, 11 launches
         from paper_2504_18547_b200.encoder import EncoderLayer as _Layer

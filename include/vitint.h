@@ -144,6 +144,25 @@ int vitint_widen(const vitint_codes* in, const vitint_codes* out, void* stream);
 int vitint_linear(const vitint_codes* x, float x_step, const vitint_codes* w, const float* w_step,
                   const float* bias, const vitint_epilogue* epi, void* out, int64_t ld_out, void* stream);
 
+/* QKV projection with the per-head quantizing LayerNorm in its epilogue (the self-attention module of Section V-B:
+ *   a LayerNorm over each head's 64 channels in front of the Q and K quantizers, statistics by Eq. 5, comparator
+ *   quantizer of Fig. 5(b); Section IV-C).  One GEMM over the stacked weights w_qkv [3D, K], D = heads*64:
+ *     columns [0, D) (Q) and [D, 2D) (K): y = fma(float(acc), fl32(x_step * w_step[n]), bias[n]); over every group of
+ *       64 consecutive columns (a head) the running statistics of Eq. 5 in channel order, V = S + n_eps, and the level
+ *       Qn + #{t : copysign(d*d, d) > V * refs[s][j][t]}, d = y - mu negated where flip[s][j] != 0 -- exactly the
+ *       arithmetic of vitint_layernorm_compare_quantize on the fp32 rows, which here never reach memory;
+ *     columns [2D, 3D) (V): clamp(rint(fma(float(acc), alpha_v[n-2D], beta_v[n-2D]))) as in the REQUANT epilogue.
+ *   w_step, bias: device [3D] (the first 2D entries are read; bias may be NULL).  refs: device
+ *   [2][64][2^bits - 1] ascending per channel, flip: device [2][64] bytes or NULL (s = 0 for Q, 1 for K; the
+ *   arrays vitint_fold_layernorm_references produces, Q's then K's).  n_eps = 64 * eps.
+ *   out: signed codes [M, 3D] of at most 4 bits (any container), every byte of every row written.
+ *   stats: device fp32 [2][M*heads][2] receiving (mu, V) of every Q and K head row, or NULL.
+ *   Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED (codes wider than 4 bits), OVERFLOW_BOUND, CUDA. */
+int vitint_linear_qkv_norm(const vitint_codes* x, float x_step, const vitint_codes* w_qkv, const float* w_step,
+                           const float* bias, const float* refs, const uint8_t* flip, float n_eps,
+                           const float* alpha_v, const float* beta_v, const vitint_codes* out, float* stats,
+                           void* stream);
+
 /* a2 through the FP4 tensor-core kind (Section V-B: fewer bits, cheaper multiply-accumulate).  e2m1 represents
  *   0, 1/2, 1, 3/2, 2, 3, 4, 6 and their negatives, so signed codes of at most 3 bits (-4 .. 3) and unsigned codes of
  *   at most 2 bits (0 .. 3) are exact operands of tcgen05 kind::mxf4 with unit block scales; their products are

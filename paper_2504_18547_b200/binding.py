@@ -91,6 +91,8 @@ def lib():
         L.vitint_layernorm_compare_quantize.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_float,
                                                         POINTER(_Codes), c_void_p, c_void_p]
         L.vitint_linear_e2m1.argtypes = [POINTER(_Codes), POINTER(_Codes), c_void_p, c_int64, c_void_p, c_void_p]
+        L.vitint_linear_qkv_norm.argtypes = [POINTER(_Codes), c_float, POINTER(_Codes), c_void_p, c_void_p, c_void_p, c_void_p,
+                                             c_float, c_void_p, c_void_p, POINTER(_Codes), c_void_p, c_void_p]
         L.vitint_selftest_wait_timeout.argtypes = [c_int64, c_void_p, c_void_p]
         L.vitint_fold_requant.argtypes = [c_float, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
         L.vitint_fold_layernorm_references.argtypes = [c_void_p, c_void_p, c_float, c_int32, c_int32, c_int64, c_void_p,
@@ -290,6 +292,23 @@ def vitint_linear(x: Codes, x_step: float, w: Codes, w_step: torch.Tensor | None
     _check(lib().vitint_linear(byref(dx), float(x_step), byref(dw), _ptr(w_step), _ptr(bias), byref(de), ptr, ld,
                                _stream()), "vitint_linear")
     return out
+
+
+def vitint_linear_qkv_norm(x: Codes, x_step: float, w_qkv: Codes, w_step: torch.Tensor, bias: torch.Tensor | None,
+                           refs: torch.Tensor, flip: torch.Tensor | None, n_eps: float, alpha_v: torch.Tensor,
+                           beta_v: torch.Tensor | None, bits: int, out: Codes | None = None,
+                           stats: torch.Tensor | None = None):
+    """QKV projection whose epilogue normalises and quantizes every Q and K head (Eq. 5 statistics, comparator
+    quantizer of Fig. 5(b)) and requantizes V.  refs: [2, 64, 2^bits - 1], flip: [2, 64] uint8 or None (Q's then
+    K's).  Returns (codes [M, 3D], stats [2, M*heads, 2])."""
+    M, N = x.rows, w_qkv.rows
+    out = Codes.empty(M, N, bits, True, x.data.device) if out is None else out
+    stats = torch.empty((2, M * (N // 192), 2), dtype=torch.float32, device=x.data.device) if stats is None else stats
+    dx, dw, do = x.desc(), w_qkv.desc(), out.desc()
+    _check(lib().vitint_linear_qkv_norm(byref(dx), float(x_step), byref(dw), w_step.data_ptr(), _ptr(bias), refs.data_ptr(),
+                                        _ptr(flip), float(n_eps), alpha_v.data_ptr(), _ptr(beta_v), byref(do),
+                                        stats.data_ptr(), _stream()), "vitint_linear_qkv_norm")
+    return out, stats
 
 
 def vitint_linear_e2m1(x: Codes, w: Codes, out: torch.Tensor | None = None, inexact: torch.Tensor | None = None):

@@ -40,7 +40,8 @@ constexpr int NUM_THREADS = (WARP_UNPACK0 + UNPACK_WARPS) * 32;
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_BN = 256;
 
-enum EpiKind { EK_ACC = 0, EK_DEQUANT = 1, EK_DEQUANT_GELU = 2, EK_REQUANT = 3, EK_REQUANT_GELU = 4 };
+enum EpiKind { EK_ACC = 0, EK_DEQUANT = 1, EK_DEQUANT_GELU = 2, EK_REQUANT = 3, EK_REQUANT_GELU = 4, EK_QKV_NORM = 5 };
+constexpr int NUM_KINDS = 6;
 
 struct GemmParams {
     int M, N, K;
@@ -62,6 +63,14 @@ struct GemmParams {
     const float* inv_s;
     const float* residual;
     long long ld_res;
+    // EK_QKV_NORM: the QKV projection whose Q and K heads pass the quantizing LayerNorm of Section IV-C in the epilogue
+    const float* norm_refs;            // [2][64][2^bits - 1] comparator references of the Q and the K norm
+    const uint8_t* norm_flip;          // [2][64] or null
+    float n_eps;
+    int norm_bits, norm_qn, norm_dim;  // code width and lowest level of Q/K; D = heads * 64 (columns per segment)
+    float* norm_stats;                 // [2][M * heads][2] (mu, V) or null
+    const float* v_alpha;              // [D] requantization of the V segment
+    const float* v_beta;               // [D] or null
 };
 
 struct Bars {
@@ -474,6 +483,140 @@ __device__ __forceinline__ void epilogue_chunk_staged(const GemmParams& P, const
     __syncwarp();                                               // the buffer is free for the next chunk
 }
 
+// NG consecutive 64-channel heads of one accumulator row, starting at tile column `col` (their recurrences are
+// independent dependency chains, stepped side by side when NG > 1).
+template <int SMALL, int NG>
+__device__ __forceinline__ void norm_heads(const GemmParams& P, const EpiParams& ep, int buf, uint32_t t_row, bool row_ok,
+                                           long long orow, int tile_col0, int col, const float* refs_s, const float* sgn_s) {
+    uint8_t* const o_row = (uint8_t*)P.out + orow * P.ld_out;
+    const int heads = P.norm_dim >> 6;
+    const uint32_t mask = (1u << P.out_c) - 1u;
+    auto to_float = [&](uint32_t v) -> float {
+        return SMALL == 2 ? small_int_to_float((int)v) : SMALL == 1 ? small_int_to_float((int)v >> P.shift) : (float)(int)v;
+    };
+    const float* pa = &ep.a[buf][col];
+    const float* pb = &ep.b[buf][col];
+    // pass 1: running statistics over each head's 64 channels, in order
+    float mu[NG], S[NG];
+#pragma unroll
+    for (int u = 0; u < NG; ++u) { mu[u] = 0.0f; S[u] = 0.0f; }
+#pragma unroll
+    for (int blk = 0; blk < 4; ++blk) {
+        uint32_t v[NG][16];
+#pragma unroll
+        for (int u = 0; u < NG; ++u) ptx::tmem_ld16(t_row + (uint32_t)(col + 64 * u + 16 * blk), v[u]);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int idx = 16 * blk + i;
+            const float fi = (float)(idx + 1), ri = 1.0f / (float)(idx + 1);       // compile-time constants: i and RN(1/i)
+#pragma unroll
+            for (int u = 0; u < NG; ++u) {
+                const float y = fmaf(to_float(v[u][i]), pa[64 * u + idx], pb[64 * u + idx]);
+                const float delta = __fadd_rn(y, -mu[u]);
+                // RN(delta / i): quotient estimate, exact remainder in one FMA, one correction
+                const float q0 = __fmul_rn(delta, ri);
+                const float rem = __fmaf_rn(-q0, fi, delta);
+                mu[u] = __fadd_rn(mu[u], __fmaf_rn(rem, ri, q0));
+                S[u] = __fadd_rn(S[u], __fmul_rn(delta, __fadd_rn(y, -mu[u])));
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < NG; ++u) {
+        const int gcol = tile_col0 + col + 64 * u;
+        const int seg = gcol / P.norm_dim;
+        const float V = __fadd_rn(S[u], P.n_eps);
+        if (P.norm_stats != nullptr && row_ok) {
+            const int head = (gcol - seg * P.norm_dim) >> 6;
+            float* st = P.norm_stats + ((long long)seg * P.M * heads + orow * heads + head) * 2;
+            st[0] = mu[u];
+            st[1] = V;
+        }
+        // pass 2: levels
+        const float* rs = refs_s + (size_t)seg * 64 * 16;
+        const float* sg = sgn_s + seg * 64;
+#pragma unroll
+        for (int blk = 0; blk < 4; ++blk) {
+            uint32_t v[16];
+            ptx::tmem_ld16(t_row + (uint32_t)(col + 64 * u + 16 * blk), v);
+            ptx::tmem_ld_wait();
+            uint32_t code[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int idx = 16 * blk + i;
+                const float y = fmaf(to_float(v[i]), pa[64 * u + idx], pb[64 * u + idx]);
+                const float d = __fmul_rn(__fadd_rn(y, -mu[u]), sg[idx]);             // exact sign change
+                const float ds = copysignf(__fmul_rn(d, d), d);
+                const float* r = rs + idx * 16;
+                // four bisection steps whatever the code width: entries past the last reference are +inf and never
+                // counted, and a fixed depth lets the sixteen columns' dependent loads interleave
+                int cnt = 0;
+#pragma unroll
+                for (int step = 8; step > 0; step >>= 1)
+                    cnt += ds > __fmul_rn(V, r[cnt + step - 1]) ? step : 0;
+                code[i] = (uint32_t)(P.norm_qn + cnt) & mask;
+            }
+            const long long c = gcol + 16 * blk;
+            if (P.out_c == 8) {
+                uint32_t w[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) w[k] = code[4 * k] | (code[4 * k + 1] << 8) | (code[4 * k + 2] << 16) | (code[4 * k + 3] << 24);
+                if (row_ok) *reinterpret_cast<uint4*>(o_row + c) = make_uint4(w[0], w[1], w[2], w[3]);
+            } else if (P.out_c == 4) {
+                uint32_t w[2] = {0u, 0u};
+#pragma unroll
+                for (int k = 0; k < 16; ++k) w[k >> 3] |= code[k] << (4 * (k & 7));
+                if (row_ok) *reinterpret_cast<uint2*>(o_row + (c >> 1)) = make_uint2(w[0], w[1]);
+            } else {
+                uint32_t w = 0u;
+#pragma unroll
+                for (int k = 0; k < 16; ++k) w |= code[k] << (2 * k);
+                if (row_ok) *reinterpret_cast<uint32_t*>(o_row + (c >> 2)) = w;
+            }
+        }
+    }
+}
+
+// Epilogue of the QKV projection with the per-head quantizing LayerNorm of Section IV-C (Eq. 5 statistics, comparator of
+// Fig. 5(b)) on the Q and K heads; the V heads are requantized as usual.  A thread owns an accumulator ROW, so the 64
+// channels of a head are its own: it walks them in order through the recurrence of Eq. 5
+//     delta = y_i - mu;  mu += delta / i;  S += delta * (y_i - mu)          (one rounded fp32 operation each)
+// with y_i = fma(float(acc_i), s_x s_w[i], b_i), forms V = S + n*eps, reads the accumulators a second time and finds each
+// level as Qn + number of references r with copysign(d*d, d) > V*r, d = y - mu (negated where the gain is negative) by
+// bisection over the column's ascending references in shared memory.  The fp32 Q and K never exist in memory.
+// refs_s: [2][64][16] (Q then K; entries past 2^bits - 1 unused), sgn_s: [2][64] (+1 / -1).
+template <int SMALL>
+__device__ __forceinline__ void epilogue_qkv_norm(const GemmParams& P, const EpiParams& ep, int buf, uint32_t t_row, bool row_ok,
+                                                  long long orow, int n_tile, int slice, const float* refs_s, const float* sgn_s) {
+    const int tile_col0 = n_tile * P.bn;
+    const int valid = P.N - tile_col0 < P.bn ? P.N - tile_col0 : P.bn;      // a multiple of 64
+    const int groups = valid >> 6, half = (groups + 1) >> 1;
+    const int g_begin = slice == 0 ? 0 : half, g_end = slice == 0 ? half : groups;
+    const int v_col0 = 2 * P.norm_dim;
+    for (int g = g_begin; g < g_end;) {
+        const int col = g << 6, gcol = tile_col0 + col;
+        if (gcol >= v_col0) {
+            // V head: plain requantization of its 64 columns
+            if (P.out_c == 8) epilogue_requant_blocks<EK_REQUANT, SMALL, false, true>(P, ep, buf, t_row, row_ok, orow, tile_col0, col, col + 64);
+            else epilogue_requant_blocks<EK_REQUANT, SMALL, false, false>(P, ep, buf, t_row, row_ok, orow, tile_col0, col, col + 64);
+            g += 1;
+        } else {
+            // (stepping two heads' recurrences side by side was measured slower: 67 against 53 us at DeiT-S width,
+            // batch 64 -- the second chain's registers spill)
+            norm_heads<SMALL, 1>(P, ep, buf, t_row, row_ok, orow, tile_col0, col, refs_s, sgn_s);
+            g += 1;
+        }
+    }
+    // row padding behind the last column of the matrix
+    if (row_ok && slice == 1 && tile_col0 + valid >= P.N) {
+        uint8_t* const o_row = (uint8_t*)P.out + orow * P.ld_out;
+        for (long long off = ((long long)P.N * P.out_c) >> 3; off + 4 <= P.ld_out; off += 4)
+            *reinterpret_cast<uint32_t*>(o_row + off) = 0u;
+    }
+    __syncwarp();
+}
+
 // The warps of a lane quarter split the tile's 32-column chunks into contiguous shares.
 __device__ __forceinline__ void chunk_share(const GemmParams& P, int slice, int& c_begin, int& c_end) {
     const int n_slices = P.epi_warps >> 2;
@@ -500,7 +643,12 @@ __device__ __forceinline__ bool epilogue_prefetch_first(const GemmParams& P, lon
 template <int KIND, int SMALL>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& P, const EpiParams& ep, int buf, uint32_t t_row,
                                               bool row_ok, long long orow, long long colbase, int n_tile, int slice,
-                                              float* stage, int lane, int rows_valid, bool first_prefetched) {
+                                              float* stage, int lane, int rows_valid, bool first_prefetched,
+                                              const float* refs_s, const float* sgn_s) {
+    if constexpr (KIND == EK_QKV_NORM) {
+        epilogue_qkv_norm<SMALL>(P, ep, buf, t_row, row_ok, orow, n_tile, slice, refs_s, sgn_s);
+        return;
+    }
     int c_begin, c_end;
     chunk_share(P, slice, c_begin, c_end);
     constexpr bool is_req = (KIND == EK_REQUANT || KIND == EK_REQUANT_GELU);
@@ -580,6 +728,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __shared__ __align__(16) EpiParams epi_params;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ __align__(16) float norm_refs_s[KIND == EK_QKV_NORM ? 2 * 64 * 16 : 4];   // comparator references of the Q and K norms
+    __shared__ float norm_sgn_s[KIND == EK_QKV_NORM ? 2 * 64 : 1];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -808,6 +958,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const long long cidx = (long long)inner * P.col_off_inner + n;
                 if (KIND == EK_REQUANT) {
                     a = __ldg(P.col_a + cidx);
+                } else if (KIND == EK_QKV_NORM && n >= 2 * P.norm_dim) {
+                    a = __ldg(P.v_alpha + (n - 2 * P.norm_dim));                       // V segment: folded requantization
                 } else {
                     a = P.col_a ? __fmul_rn(P.x_step, __ldg(P.col_a + cidx)) : P.x_step;
                     if (KIND == EK_REQUANT_GELU) {                                  // folds GELU's 1/2 (and 1/Qp)
@@ -815,7 +967,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         if (P.unit_out) q = __fdiv_rn(q, P.out_qp);
                     }
                 }
-                b = P.col_b ? __ldg(P.col_b + cidx) : 0.0f;
+                if (KIND == EK_QKV_NORM && n >= 2 * P.norm_dim) b = P.v_beta ? __ldg(P.v_beta + (n - 2 * P.norm_dim)) : 0.0f;
+                else b = P.col_b ? __ldg(P.col_b + cidx) : 0.0f;
                 a *= down;
             }
         };
@@ -828,6 +981,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             epi_params.a[0][tid_e] = a;
             epi_params.b[0][tid_e] = b;
             epi_params.q[0][tid_e] = q;
+        }
+        if constexpr (KIND == EK_QKV_NORM) {
+            // comparator references and gain signs of the Q and K norms: read by every epilogue warp after the first tile's
+            // group barrier
+            const int nt = (1 << P.norm_bits) - 1;
+            for (int i = tid_e; i < 2 * 64 * 16; i += P.epi_warps * 32) {
+                const int set = i >> 10, c = (i >> 4) & 63, t = i & 15;
+                norm_refs_s[i] = t < nt ? __ldg(P.norm_refs + ((size_t)set * 64 + c) * nt + t) : INFINITY;
+            }
+            for (int i = tid_e; i < 2 * 64; i += P.epi_warps * 32)
+                norm_sgn_s[i] = (P.norm_flip != nullptr && __ldg(P.norm_flip + i)) ? -1.0f : 1.0f;
         }
         int tl = 0;
         bool ok = true;
@@ -865,9 +1029,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool row_ok = row0_in_problem + lane < P.M;
             const long long orow = orow0 + lane;
             const uint32_t t_row = tmem_base + (uint32_t)buf * acc_stride + ((uint32_t)(q4 * 32) << 16);
-            if (P.small_acc == 2) epilogue_tile<KIND, 2>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid, first_prefetched);
-            else if (P.small_acc == 1) epilogue_tile<KIND, 1>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid, first_prefetched);
-            else epilogue_tile<KIND, 0>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid, first_prefetched);
+            if (P.small_acc == 2) epilogue_tile<KIND, 2>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid, first_prefetched, norm_refs_s, norm_sgn_s);
+            else if (P.small_acc == 1) epilogue_tile<KIND, 1>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid, first_prefetched, norm_refs_s, norm_sgn_s);
+            else epilogue_tile<KIND, 0>(P, epi_params, buf, t_row, row_ok, orow, colbase, n_tile, slice, stage, lane, rows_valid, first_prefetched, norm_refs_s, norm_sgn_s);
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&bars.acc_empty[buf]));
@@ -993,8 +1157,10 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     // from twelve warps than the mainloop loses with two ring stages (proj, batch 128: 45 -> 43 us; with the
     // long contraction of fc2 the same choice costs 17 us)
     P.epi_warps = (P.a_direct && P.b_direct && (!staged || K <= 1024)) ? MAX_EPI_WARPS : EPI_WARPS;
+    if (P.kind == EK_QKV_NORM) P.epi_warps = EPI_WARPS;        // two warps per lane quarter, each taking whole 64-channel heads
     const uint32_t stage_total = staged ? (uint32_t)(P.epi_warps * STAGE_BYTES) : 0u;
-    const uint32_t ring_budget = SMEM_TILE_BUDGET + 12u * 1024u - stage_total;   // staging comes out of the ring space
+    // staging comes out of the ring space; the norm kind keeps 9 KB of reference tables in static shared memory
+    const uint32_t ring_budget = SMEM_TILE_BUDGET + 12u * 1024u - stage_total - (P.kind == EK_QKV_NORM ? 16u * 1024u : 0u);
     // The packed ring hides the global-memory latency of the TMA loads; the int8 ring only
     // decouples unpack from MMA issue, unless TMA writes it directly.
     int ns_i, ns_p;
@@ -1038,13 +1204,13 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     if (grid > P.total_tiles) grid = P.total_tiles;
     const int dev = current_device();
     if (dev < 0) return VITINT_ERR_CUDA;
-    static bool attr_set_dev[MAX_DEVICES][5] = {};
+    static bool attr_set_dev[MAX_DEVICES][NUM_KINDS] = {};
     bool* const attr_set = attr_set_dev[dev];
 #define VITINT_LAUNCH(KIND)                                                                                        \
     case KIND:                                                                                                     \
         if (!attr_set[KIND]) {                                                                                     \
             if (cudaFuncSetAttribute(gemm_i8_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,            \
-                                     (int)SMEM_TILE_BUDGET + 14 * 1024) != cudaSuccess)                                 \
+                                     (int)SMEM_TILE_BUDGET + (KIND == EK_QKV_NORM ? 0 : 14 * 1024)) != cudaSuccess)      \
                 return VITINT_ERR_CUDA;                                                                            \
             attr_set[KIND] = true;                                                                                 \
         }                                                                                                          \
@@ -1056,6 +1222,7 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
         VITINT_LAUNCH(EK_DEQUANT_GELU)
         VITINT_LAUNCH(EK_REQUANT)
         VITINT_LAUNCH(EK_REQUANT_GELU)
+        VITINT_LAUNCH(EK_QKV_NORM)
         default: return VITINT_ERR_INVALID_ARG;
     }
 #undef VITINT_LAUNCH
@@ -1152,6 +1319,38 @@ extern "C" int vitint_linear(const vitint_codes* x, float x_step, const vitint_c
               (uint64_t)w->pitch_bytes, (uint64_t)w->pitch_bytes * (uint64_t)w->rows,
               (uint64_t)w->pitch_bytes * (uint64_t)w->rows};
     return launch_gemm(A, B, (int)x->rows, (int)w->rows, (int)x->cols, 1, 1, 0, P, (cudaStream_t)stream);
+}
+
+extern "C" int vitint_linear_qkv_norm(const vitint_codes* x, float x_step, const vitint_codes* w_qkv, const float* w_step,
+                                      const float* bias, const float* refs, const uint8_t* flip, float n_eps,
+                                      const float* alpha_v, const float* beta_v, const vitint_codes* out, float* stats,
+                                      void* stream) {
+    if (int rc = check_codes(x)) return rc;
+    if (int rc = check_codes(w_qkv)) return rc;
+    if (int rc = check_codes(out)) return rc;
+    if (!w_step || !refs || !alpha_v) return VITINT_ERR_INVALID_ARG;
+    if (x->cols != w_qkv->cols || w_qkv->rows % 192 != 0 || w_qkv->rows <= 0) return VITINT_ERR_INVALID_ARG;
+    if (out->rows != x->rows || out->cols != w_qkv->rows || !out->is_signed) return VITINT_ERR_INVALID_ARG;
+    if (!(x_step > 0.0f && x_step < INFINITY) || !(n_eps >= 0.0f && n_eps < INFINITY)) return VITINT_ERR_INVALID_ARG;
+    if (out->bits > 4) return VITINT_ERR_UNSUPPORTED;               // the reference table holds at most 15 thresholds a channel
+    if (x->rows > 0x7fffffff || w_qkv->rows > 0x7fffffff || x->cols > 0x7fffffff) return VITINT_ERR_UNSUPPORTED;
+    GemmParams P{};
+    int qn, qp;
+    code_range(out->bits, 1, &qn, &qp);
+    P.kind = EK_QKV_NORM;
+    P.out = out->data; P.ld_out = out->pitch_bytes; P.out_c = codes_container(out);
+    P.out_qn = (float)qn; P.out_qp = (float)qp;
+    P.x_step = x_step; P.col_a = w_step; P.col_b = bias; P.inv_s = nullptr; P.residual = nullptr; P.ld_res = 0;
+    P.norm_refs = refs; P.norm_flip = flip; P.n_eps = n_eps; P.norm_bits = out->bits; P.norm_qn = qn;
+    P.norm_dim = (int)(w_qkv->rows / 3); P.norm_stats = stats; P.v_alpha = alpha_v; P.v_beta = beta_v;
+    P.row_off_outer = 0; P.row_off_inner = 0; P.col_off_inner = 0;
+    Operand A{x->data, x->bits, x->is_signed, codes_container(x), (uint64_t)codes_row_bytes(x, x->cols), (uint64_t)x->rows,
+              (uint64_t)x->pitch_bytes, (uint64_t)x->pitch_bytes * (uint64_t)x->rows,
+              (uint64_t)x->pitch_bytes * (uint64_t)x->rows};
+    Operand B{w_qkv->data, w_qkv->bits, w_qkv->is_signed, codes_container(w_qkv), (uint64_t)codes_row_bytes(w_qkv, w_qkv->cols),
+              (uint64_t)w_qkv->rows, (uint64_t)w_qkv->pitch_bytes, (uint64_t)w_qkv->pitch_bytes * (uint64_t)w_qkv->rows,
+              (uint64_t)w_qkv->pitch_bytes * (uint64_t)w_qkv->rows};
+    return launch_gemm(A, B, (int)x->rows, (int)w_qkv->rows, (int)x->cols, 1, 1, 0, P, (cudaStream_t)stream);
 }
 
 extern "C" int vitint_qk(const vitint_slabs* q, const vitint_slabs* k, int32_t batch, int32_t heads, int32_t tokens,

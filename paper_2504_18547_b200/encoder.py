@@ -189,25 +189,32 @@ class NormedAttention:
     linear layers, a LayerNorm over each head's 64 channels in front of the Q and K quantizers (statistics by
     Eq. 5, comparator quantizer of Fig. 5(b)), Q K^T, the Eq. 4 softmax with its division-free quantizer, P V.
     A fixed sequence of C-ABI calls over preallocated buffers; `qkn` holds the per-head LayerNorm parameters
-    (qn_g, qn_b, kn_g, kn_b over 64 channels) and the steps s_qn, s_kn of the normalised values."""
+    (qn_g, qn_b, kn_g, kn_b over 64 channels) and the steps s_qn, s_kn of the normalised values.
+    fused=True (default): one QKV GEMM whose epilogue normalises and quantizes the Q and K heads and requantizes V
+    (4 launches); fused=False: separate Q, K, V linears with fp32 Q and K rows and a LayerNorm kernel pass each
+    (10 launches, the fp32 rows and their statistics left in `f32` / `stats` for inspection)."""
 
     def __init__(self, batch: int, tokens: int, heads: int, bits: int, prm: dict, qkn: dict, device="cuda",
-                 eps: float = 1e-6):
+                 eps: float = 1e-6, fused: bool = True):
+        self.fused = fused
         self.batch, self.tokens, self.heads, self.bits = batch, tokens, heads, bits
         self.dim = D = heads * 64
         self.rows = M = batch * tokens
         d = lambda a: _dev(a, device)
         w = B.vitint_widen(B.vitint_quantize(d(prm["w_qkv"]), 0.0, bits, True, row_steps=d(prm["s_w_qkv"])))
         part = lambda i: B.Codes(w.data[i * D:(i + 1) * D], D, D, bits, True, 8)
-        self.w_q, self.w_k, self.w_v = part(0), part(1), part(2)
-        self.s_w = [d(prm["s_w_qkv"][i * D:(i + 1) * D]) for i in range(2)]
-        self.bias = [d(prm["b_qkv"][i * D:(i + 1) * D]) for i in range(2)]
+        self.w_qkv, self.w_q, self.w_k, self.w_v = w, part(0), part(1), part(2)
+        self.s_w_all, self.bias_all = d(prm["s_w_qkv"]), d(prm["b_qkv"])
+        self.s_w = [self.s_w_all[i * D:(i + 1) * D] for i in range(2)]
+        self.bias = [self.bias_all[i * D:(i + 1) * D] for i in range(2)]
         a, b = B.fold_requant(1.0, prm["s_w_qkv"][2 * D:], prm["b_qkv"][2 * D:], prm["s_v"])
         self._alpha_v_unit, self.beta_v = a, d(b)             # alpha scales with the input step given to forward()
         self.refs = []
         for n in ("q", "k"):
             r, fl = B.fold_layernorm_references(qkn[n + "n_g"], qkn[n + "n_b"], qkn["s_" + n + "n"], bits, True, 64)
             self.refs.append((d(r), d(fl)))
+        self.refs_all = torch.stack([r for r, _ in self.refs]).contiguous()
+        self.flip_all = torch.stack([f for _, f in self.refs]).contiguous()
         self.n_eps = float(np.float32(np.float64(64) * np.float64(np.float32(eps))))
         self.s_v, self.s_p, self.s_o = float(prm["s_v"]), float(prm["s_p"]), float(prm["s_o"])
         c = np.float32(float(qkn["s_qn"]) * float(qkn["s_kn"]) / 8.0)
@@ -217,13 +224,20 @@ class NormedAttention:
         self._prm = prm
         self._alpha_v_for = None
         c_bits = 4 if bits == 3 else bits
-        self.f32 = [torch.empty((M, D), dtype=torch.float32, device=device) for _ in range(2)]
-        self.qk_codes = [B.Codes.empty(M * heads, 64, bits, True, device) for _ in range(2)]
-        self.stats = [torch.empty((M * heads, 2), dtype=torch.float32, device=device) for _ in range(2)]
+        self.stats_all = torch.empty((2, M * heads, 2), dtype=torch.float32, device=device)
+        self.stats = [self.stats_all[0], self.stats_all[1]]
         pitch = D * c_bits // 8
-        self.slabs = [B.Slabs(c.data, 0, pitch, pitch * tokens, 64 * c_bits // 8, bits, True) for c in self.qk_codes]
-        self.v = B.Codes.empty(M, D, bits, True, device)
-        self.v_slabs = B.Slabs(self.v.data, 0, self.v.pitch, self.v.pitch * tokens, 64 * c_bits // 8, bits, True)
+        if fused:
+            self.qkv = B.Codes.empty(M, 3 * D, bits, True, device)
+            qp = self.qkv.pitch
+            self.slabs = [B.Slabs(self.qkv.data, i * pitch, qp, qp * tokens, 64 * c_bits // 8, bits, True) for i in range(2)]
+            self.v_slabs = B.Slabs(self.qkv.data, 2 * pitch, qp, qp * tokens, 64 * c_bits // 8, bits, True)
+        else:
+            self.f32 = [torch.empty((M, D), dtype=torch.float32, device=device) for _ in range(2)]
+            self.qk_codes = [B.Codes.empty(M * heads, 64, bits, True, device) for _ in range(2)]
+            self.slabs = [B.Slabs(c.data, 0, pitch, pitch * tokens, 64 * c_bits // 8, bits, True) for c in self.qk_codes]
+            self.v = B.Codes.empty(M, D, bits, True, device)
+            self.v_slabs = B.Slabs(self.v.data, 0, self.v.pitch, self.v.pitch * tokens, 64 * c_bits // 8, bits, True)
         self.ld_s = (tokens + 3) // 4 * 4
         self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
         self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
@@ -238,13 +252,17 @@ class NormedAttention:
             self.alpha_v = _dev(a, self.O.data.device)
             self._alpha_v_for = float(s_x)
         b, t, h = self.batch, self.tokens, self.heads
-        for i, w in enumerate((self.w_q, self.w_k)):
-            B.vitint_linear(x, s_x, w, self.s_w[i], self.bias[i], B.Epilogue(mode=B.EPI_DEQUANT_F32), out=self.f32[i])
-            B.vitint_layernorm_compare_quantize(self.f32[i].view(self.rows * h, 64), self.refs[i][0], self.refs[i][1],
-                                                self.n_eps, self.bits, True, out=self.qk_codes[i], stats=self.stats[i])
-        B.vitint_linear(x, s_x, self.w_v, None, None,
-                        B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_v, beta=self.beta_v, out_bits=self.bits,
-                                   out_signed=True), out=self.v)
+        if self.fused:
+            B.vitint_linear_qkv_norm(x, s_x, self.w_qkv, self.s_w_all, self.bias_all, self.refs_all, self.flip_all,
+                                     self.n_eps, self.alpha_v, self.beta_v, self.bits, out=self.qkv, stats=self.stats_all)
+        else:
+            for i, w in enumerate((self.w_q, self.w_k)):
+                B.vitint_linear(x, s_x, w, self.s_w[i], self.bias[i], B.Epilogue(mode=B.EPI_DEQUANT_F32), out=self.f32[i])
+                B.vitint_layernorm_compare_quantize(self.f32[i].view(self.rows * h, 64), self.refs[i][0], self.refs[i][1],
+                                                    self.n_eps, self.bits, True, out=self.qk_codes[i], stats=self.stats[i])
+            B.vitint_linear(x, s_x, self.w_v, None, None,
+                            B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_v, beta=self.beta_v, out_bits=self.bits,
+                                       out_signed=True), out=self.v)
         B.vitint_qk(self.slabs[0], self.slabs[1], b, h, t, out=self.S, ld_s=self.ld_s)
         B.vitint_softmax_shift_quantize(self.S, t, self.c2, self.s_p, self.bits, out=self.P)
         B.vitint_pv(self.P, self.v_slabs, b, h, t, self.s_p, self.s_v, self.epi_o, out=self.O)

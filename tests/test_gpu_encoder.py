@@ -295,7 +295,7 @@ def test_normed_attention_module_bit_exact(bits):
     s_x = si.lsq_step(x, cfg.bits, True)
     xq = vo.quantize(x, s_x, cfg.bits, True)
     st = vp.normed_attention(xq, s_x, prm, qkn, cfg.batch, cfg.tokens, cfg.heads, cfg.bits)
-    mod = NormedAttention(cfg.batch, cfg.tokens, cfg.heads, cfg.bits, prm, qkn)
+    mod = NormedAttention(cfg.batch, cfg.tokens, cfg.heads, cfg.bits, prm, qkn, fused=False)
     xg = vt.vitint_quantize(dev(x), float(s_x), cfg.bits, True)
     O = mod.forward(xg, float(s_x))
     assert vt.vitint_device_status() == 0
@@ -313,6 +313,43 @@ def test_normed_attention_module_bit_exact(bits):
     # per linear layer and 198*198*64 = 2.51 M per attention matmul
     per_image = mod.ops() // (2 * cfg.batch)
     assert per_image == H * (3 * 198 * 384 * 64 + 2 * 198 * 198 * 64)
+
+
+@pytest.mark.parametrize("bits,batch,negate", [(4, 2, False), (3, 2, True), (2, 1, False), (4, 5, True)])
+def test_normed_attention_fused_qkv_epilogue_bit_exact(bits, batch, negate):
+    """The same module with the per-head LayerNorm + comparator quantizer run inside the QKV GEMM's epilogue (one
+    launch instead of seven): Q, K and V codes, the (mu, V) statistics of every head row and everything downstream
+    equal the oracle bit for bit, although the fp32 Q and K never reach memory.  batch 5 gives 990 rows: seven full
+    128-row tiles and a ragged one.  negate: every third gain of both norms made negative, which flips those
+    channels' comparators."""
+    from paper_2504_18547_b200.encoder import NormedAttention
+    cfg = si.DEIT_S_ATTENTION.with_(batch=batch, bits=bits)
+    prm, qkn = si.layer_parameters(cfg), si.qk_norm_parameters(cfg)
+    if negate:
+        for n in ("qn_g", "kn_g"):
+            qkn[n] = qkn[n].copy()
+            qkn[n][::3] *= -1.0
+    x = si.activations(cfg)
+    s_x = si.lsq_step(x, cfg.bits, True)
+    xq = vo.quantize(x, s_x, cfg.bits, True)
+    st = vp.normed_attention(xq, s_x, prm, qkn, cfg.batch, cfg.tokens, cfg.heads, cfg.bits)
+    mod = NormedAttention(cfg.batch, cfg.tokens, cfg.heads, cfg.bits, prm, qkn)
+    assert mod.fused
+    xg = vt.vitint_quantize(dev(x), float(s_x), cfg.bits, True)
+    mod.qkv.data.fill_(0x5A)
+    O = mod.forward(xg, float(s_x))
+    assert vt.vitint_device_status() == 0
+    M, D, T, H = cfg.rows, cfg.dim, cfg.tokens, cfg.heads
+    qkv = from_codes(mod.qkv)
+    stats = mod.stats_all.cpu().numpy()
+    for i, n in enumerate(("q", "k")):
+        assert np.array_equal(stats[i].view(np.uint32), st[n + "_stats"].view(np.uint32)), n
+        assert np.array_equal(qkv[:, i * D:(i + 1) * D], st[n + "_codes"]), n
+    assert np.array_equal(qkv[:, 2 * D:], st["v_codes"])
+    assert any(st[n + "_refs"][2].any() for n in ("q", "k")) == negate
+    assert np.array_equal(mod.S.cpu().numpy()[:, :T].reshape(cfg.batch * H, T, T), st["S"])
+    assert np.array_equal(from_codes(mod.P).reshape(-1, T, T), st["p_codes"])
+    assert np.array_equal(from_codes(O), st["o_codes"])
 
 
 def test_deit_s_model_forward():

@@ -128,6 +128,30 @@ def test_outputs_stay_inside_their_buffers():
             out2, stats = guarded_codes(rows, cols, bits, True, cont), guarded_tensor((rows, 2), torch.float32)
             vt.vitint_layernorm_compare_quantize(dev(x), dev(refs), dev(flip), 1e-4, bits, True, out=out2, stats=stats)
             assert padding_is_zero(out2)
+    # QKV projection with the per-head LayerNorm in its epilogue: one head (a 192-column tile) and three heads
+    # (three 256-column tiles, the last ragged), odd row counts, packed and byte containers, over-wide pitch
+    for M, K, heads in ((1, 64, 1), (197, 128, 1), (131, 192, 3)):
+        D = 64 * heads
+        qx, qw = rand_codes(41 + M, (M, K), 4, True), rand_codes(42, (3 * D, K), 4, True)
+        s_w, bias = np.full(3 * D, 0.01, np.float32), si.normal(43, (3 * D,), 0.0, 0.05)
+        g, b = si.normal(44, (64,), 1.0, 0.1), si.normal(45, (64,), 0.0, 0.1)
+        g[::5] *= -1.0
+        alpha_v, beta_v = np.full(D, 0.02, np.float32), si.normal(46, (D,), 0.0, 0.5)
+        for bits, cont, pitch in ((4, 0, None), (4, 8, None), (3, 0, 3 * D // 2 + 48), (2, 0, None)):
+            ref, neg, flip = vo.layernorm_references(g, b, np.float32(0.4), bits, True, 64)
+            refs, fl = vt.vitint_fold_layernorm_references(g, b, np.float32(0.4), bits, True, 64)
+            want = []
+            for i in range(2):
+                y = vo.epilogue_dequant(vo.matmul_i32(qx, qw[i * D:(i + 1) * D]), np.float32(0.5), s_w[i * D:(i + 1) * D], bias[i * D:(i + 1) * D])
+                want.append(vo.layernorm_compare_quantize(y.reshape(M * heads, 64), ref, neg, flip, 1e-6, bits, True).reshape(M, D))
+            want.append(vo.epilogue_requant(vo.matmul_i32(qx, qw[2 * D:]), alpha_v, beta_v, bits, True))
+            out = guarded_codes(M, 3 * D, bits, True, cont, pitch)
+            stats = guarded_tensor((2, M * heads, 2), torch.float32)
+            n_eps = float(np.float32(np.float64(64) * np.float64(np.float32(1e-6))))
+            vt.vitint_linear_qkv_norm(vt.vitint_widen(to_codes(qx, 4, True)), 0.5, vt.vitint_widen(to_codes(qw, 4, True)), dev(s_w),
+                                      dev(bias), torch.stack([dev(refs)] * 2).contiguous(), torch.stack([dev(fl)] * 2).contiguous(),
+                                      n_eps, dev(alpha_v), dev(beta_v), bits, out=out, stats=stats)
+            assert np.array_equal(from_codes(out), np.concatenate(want, axis=1)) and padding_is_zero(out)
     torch.cuda.synchronize()
     assert vt.vitint_device_status() == 0
     assert check_guards() > 100
