@@ -379,6 +379,7 @@ def run_ours(args, cfg):
         Pq = vt.Codes.empty(n_rows, T, cfg.bits, False, device)
         xq = vt.Codes.empty(M, D, cfg.bits, True, device)
         sm_bytes = n_rows * T * 4 + n_rows * ((T * cb + 7) // 8)
+        sm_ws = torch.empty(vt.vitint_softmax_table_workspace_bytes(64 * (1 << (cb - 1)) ** 2), dtype=torch.uint8, device=device)
         q_bytes = M * D * 4 + M * D * cb // 8
         # the paper's own LayerNorm quantizer (Eq. 5 statistics + comparator), which the default step does not use
         lrefs, lflip = vt.fold_layernorm_references(prm["ln1_g"], prm["ln1_b"], prm["s_ln"], cfg.bits, True, D)
@@ -390,12 +391,14 @@ def run_ours(args, cfg):
                 ("layernorm_compare_quant", lambda: vt.vitint_layernorm_compare_quantize(
                     xs[2], lrefs, lflip, n_eps, cfg.bits, True, out=xq, stats=lstats), q_bytes),
                 ("softmax_quant", lambda: vt.vitint_softmax_quantize(S, T, layer.c, layer.s_p, cfg.bits, out=Pq), sm_bytes),
+                ("softmax_quant_bounded", lambda: vt.vitint_softmax_quantize_bounded(
+                    S, T, layer.c, layer.s_p, cfg.bits, 64 * (1 << (cb - 1)) ** 2, out=Pq, workspace=sm_ws), sm_bytes),
                 ("softmax_shift_quant", lambda: vt.vitint_softmax_shift_quantize(S, T, layer.c * 1.4426950408889634,
                                                                                  layer.s_p, cfg.bits, out=Pq), sm_bytes)):
             ms = timed(fn)
             standalone[name] = {"ms": round(ms, 4), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
                                 "frac_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks_early["hbm_gbs"], 4)}
-        del S, Pq, xq
+        del S, Pq, xq, sm_ws
         # the attention module of the paper's power table at its own shapes (DeiT-S width, 198 tokens, 3-bit,
         # per-head comparator LayerNorm on Q and K, Eq. 4 softmax), batch 64
         from paper_2504_18547_b200.encoder import NormedAttention

@@ -98,7 +98,8 @@ const char* vitint_status_string(int status);
 int vitint_version(void);
 
 /* Reads (and clears) the device status word of the current device; synchronizes
- * the device.  Returns VITINT_OK, VITINT_ERR_TIMEOUT or VITINT_ERR_CUDA. */
+ * the device.  Returns VITINT_OK, VITINT_ERR_TIMEOUT, VITINT_ERR_INVALID_ARG (a kernel met data that contradicts what
+ * its caller declared: vitint_softmax_quantize_bounded) or VITINT_ERR_CUDA. */
 int vitint_device_status(void);
 
 /* Self-test of the bounded wait: launches one warp that waits on a barrier nothing ever completes, with a limit of
@@ -198,6 +199,23 @@ int vitint_qk(const vitint_slabs* q, const vitint_slabs* k, int32_t batch, int32
  *   cols <= 1024. */
 int vitint_softmax_quantize(const int32_t* s, int64_t rows, int32_t cols, int64_t ld_s, float c, float p_step,
                             const vitint_codes* p_out, float* p_f32, int64_t ld_p, void* stream);
+
+/* a5 for scores of known range (the scores Q K^T of b-bit codes satisfy |S| <= 64 * max|q| * max|k|): the same
+ *   result as vitint_softmax_quantize -- Eq. 3's softmax of t_j = fl32(S_j * c), probabilities within 2 ulp, codes
+ *   clamp(rint(p / p_step), 0, 2^bits - 1) -- with exp(t_j) read from a table of exp(fl32(s * c)), s = -score_bound
+ *   .. score_bound (fp64 exp, rounded once), so the kernel is bound by memory traffic instead of arithmetic.
+ *   exp(t_j) / sum_k exp(t_k) is the softmax exactly; no maximum is subtracted, hence score_bound * |c| <= 80.
+ *   workspace: device memory, 256-byte aligned, at least vitint_softmax_table_workspace_bytes(score_bound) bytes;
+ *   it receives the table (one more small launch) unless table_ready != 0, in which case it already holds the table
+ *   an earlier call with the same c and score_bound wrote.  s must be 16-byte aligned with ld_s % 4 == 0.
+ *   A score outside the declared range cannot touch memory outside the table; it makes that row's codes meaningless
+ *   and the next vitint_device_status() returns VITINT_ERR_INVALID_ARG.
+ *   Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED (cols > 895, score_bound > 8192, score_bound*|c| > 80:
+ *   use vitint_softmax_quantize), CUDA. */
+size_t vitint_softmax_table_workspace_bytes(int32_t score_bound);
+int vitint_softmax_quantize_bounded(const int32_t* s, int64_t rows, int32_t cols, int64_t ld_s, float c, float p_step,
+                                    int32_t score_bound, const vitint_codes* p_out, float* p_f32, int64_t ld_p,
+                                    void* workspace, size_t workspace_bytes, int32_t table_ready, void* stream);
 
 /* a5, shift form (Eq. 4 with the division-free comparator quantizer of Section IV-B).  Integer and
  *   single-rounding fp32 operations only, so the codes are unique (bit-exact against the definition):

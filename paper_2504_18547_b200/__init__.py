@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     vitint_attention_core_noalloc, vitint_attention_core_prepared, vitint_attention_core_workspace_bytes,
     vitint_attention_exp_table, vitint_device_status, vitint_selftest_wait_timeout,
     vitint_layernorm_compare_quantize, vitint_layernorm_quantize, vitint_linear, vitint_linear_e2m1, vitint_linear_qkv_norm, vitint_pv, vitint_qk, vitint_quantize,
-    vitint_softmax_quantize, vitint_softmax_shift_quantize, vitint_status_string, vitint_version, vitint_widen, EPI_ACC_I32, EPI_DEQUANT_F32, EPI_REQUANT,
+    vitint_softmax_quantize, vitint_softmax_quantize_bounded, vitint_softmax_table_workspace_bytes, vitint_softmax_shift_quantize, vitint_status_string, vitint_version, vitint_widen, EPI_ACC_I32, EPI_DEQUANT_F32, EPI_REQUANT,
 )

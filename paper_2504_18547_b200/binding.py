@@ -93,6 +93,11 @@ def lib():
         L.vitint_linear_e2m1.argtypes = [POINTER(_Codes), POINTER(_Codes), c_void_p, c_int64, c_void_p, c_void_p]
         L.vitint_linear_qkv_norm.argtypes = [POINTER(_Codes), c_float, POINTER(_Codes), c_void_p, c_void_p, c_void_p, c_void_p,
                                              c_float, c_void_p, c_void_p, POINTER(_Codes), c_void_p, c_void_p]
+        L.vitint_softmax_table_workspace_bytes.restype = c_size_t
+        L.vitint_softmax_table_workspace_bytes.argtypes = [c_int32]
+        L.vitint_softmax_quantize_bounded.argtypes = [c_void_p, c_int64, c_int32, c_int64, c_float, c_float, c_int32,
+                                                      POINTER(_Codes), c_void_p, c_int64, c_void_p, c_size_t, c_int32,
+                                                      c_void_p]
         L.vitint_selftest_wait_timeout.argtypes = [c_int64, c_void_p, c_void_p]
         L.vitint_fold_requant.argtypes = [c_float, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
         L.vitint_fold_layernorm_references.argtypes = [c_void_p, c_void_p, c_float, c_int32, c_int32, c_int64, c_void_p,
@@ -342,6 +347,28 @@ def vitint_softmax_quantize(s: torch.Tensor, cols: int, c: float, p_step: float,
     d = out.desc()
     _check(lib().vitint_softmax_quantize(s.data_ptr(), rows, cols, ld_s, float(c), float(p_step), byref(d), _ptr(p),
                                          cols if want_p else 0, _stream()), "vitint_softmax_quantize")
+    return (out, p) if want_p else out
+
+
+def vitint_softmax_table_workspace_bytes(score_bound: int) -> int:
+    return int(lib().vitint_softmax_table_workspace_bytes(int(score_bound)))
+
+
+def vitint_softmax_quantize_bounded(s: torch.Tensor, cols: int, c: float, p_step: float, bits: int, score_bound: int,
+                                    want_p: bool = False, out: Codes | None = None,
+                                    workspace: torch.Tensor | None = None, table_ready: bool = False):
+    """vitint_softmax_quantize for scores known to lie in -score_bound .. score_bound (exp from a table).
+    workspace: uint8 device tensor of vitint_softmax_table_workspace_bytes(score_bound) bytes (allocated if None)."""
+    rows, ld_s = s.shape[0], _ld(s)
+    out = Codes.empty(rows, cols, bits, False, s.device) if out is None else out
+    p = torch.empty((rows, cols), dtype=torch.float32, device=s.device) if want_p else None
+    if workspace is None:
+        workspace = torch.empty(vitint_softmax_table_workspace_bytes(score_bound), dtype=torch.uint8, device=s.device)
+    d = out.desc()
+    _check(lib().vitint_softmax_quantize_bounded(s.data_ptr(), rows, cols, ld_s, float(c), float(p_step), int(score_bound),
+                                                 byref(d), _ptr(p), cols if want_p else 0, workspace.data_ptr(),
+                                                 workspace.numel(), int(table_ready), _stream()),
+           "vitint_softmax_quantize_bounded")
     return (out, p) if want_p else out
 
 

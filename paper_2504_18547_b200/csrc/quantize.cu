@@ -51,7 +51,9 @@ quantize_pack_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, in
 // normalisation.  Lane l owns float4 number v*32 + l of the row, v < NV.
 // All per-element arithmetic is fp32 on the FMA pipe (no conversions); the corrected
 // two-pass mean keeps the result inside a few ulp of the exact normalisation.
-template <int C, int NV>
+// FULL: the row is exactly NV*128 columns and no fp32 copy is written, so no access needs a guard (the guards
+// otherwise become branches around every vector: a third of the instructions at 768 columns).
+template <int C, int NV, bool FULL>
 __global__ void __launch_bounds__(128)
 layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, int64_t ldx,
                           const float* __restrict__ gamma, const float* __restrict__ beta, float eps, float step,
@@ -70,7 +72,7 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
         const int col = (v * 32 + lane) * 4;
-        const float4 t = (col < cols) ? __ldg(reinterpret_cast<const float4*>(xr + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 t = (FULL || col < cols) ? __ldg(reinterpret_cast<const float4*>(xr + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
         f[v][0] = f2_pack(t.x, t.y);
         f[v][1] = f2_pack(t.z, t.w);
         sum2 = f2_add(sum2, f2_add(f[v][0], f[v][1]));
@@ -90,7 +92,7 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
         const int col = (v * 32 + lane) * 4;
-        if (col < cols) {
+        if (FULL || col < cols) {
             f[v][0] = f2_add(f[v][0], nmean2);
             f[v][1] = f2_add(f[v][1], nmean2);
             rs2 = f2_add(rs2, f2_add(f[v][0], f[v][1]));
@@ -127,7 +129,7 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
     for (int v = 0; v < NV; ++v) {
         uint32_t bits = 0;
         const int col = (v * 32 + lane) * 4;
-        if (col < cols) {
+        if (FULL || col < cols) {
             const float4 g = __ldg(reinterpret_cast<const float4*>(gamma + col));
             const float4 b = __ldg(reinterpret_cast<const float4*>(beta + col));
             const f32x2 rstd2 = f2_dup(rstd), rstep2 = f2_dup(rstep), magic2 = f2_dup(magic);
@@ -136,7 +138,7 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
             float4 y;
             f2_unpack(y01, y.x, y.y);
             f2_unpack(y23, y.z, y.w);
-            if (y_out) *reinterpret_cast<float4*>(y_out + row * ld_y + col) = y;
+            if (!FULL && y_out) *reinterpret_cast<float4*>(y_out + row * ld_y + col) = y;
             // clamp, then add 1.5*2^23 (+ 2^(C-1) for signed codes): the low mantissa bits hold the code in
             // offset binary, so the four codes combine by shift-add without masking
             float u0, u1, u2, u3;
@@ -157,7 +159,7 @@ layernorm_quantize_kernel(const float* __restrict__ x, int64_t rows, int cols, i
             bits |= __shfl_xor_sync(0xffffffffu, bits, 2) << 16;
         }
         const int word = (v * 32 + lane) / LANES_PER_WORD;
-        if ((lane % LANES_PER_WORD) == 0 && word < words_per_row)
+        if ((lane % LANES_PER_WORD) == 0 && (FULL || word < words_per_row))
             *reinterpret_cast<uint32_t*>(out + row * pitch + (int64_t)word * 4) = bits;
     }
     // row padding beyond the columns the loop above covers
@@ -199,10 +201,15 @@ static int launch_ln(int nv, const float* x, int64_t rows, int cols, int64_t ldx
                      float qn, float qp, cudaStream_t st) {
     const int warps = 4;       // four rows per block: measured best (8: +1 us per call at 25,216 x 768; 16: +3 us)
     dim3 grid((unsigned)((rows + warps - 1) / warps)), block(32 * warps);
+    const bool full = cols == nv * 128 && y == nullptr;
 #define VITINT_LN_CASE(NVV)                                                                                     \
     case NVV:                                                                                                   \
-        launch_kernel(layernorm_quantize_kernel<C, NVV>, dim3(grid), dim3(block), 0, st, x, rows, cols, ldx, gamma, beta, eps, step,   \
-                                                                  out, pitch, y, ld_y, qn, qp);                 \
+        if (full)                                                                                               \
+            launch_kernel(layernorm_quantize_kernel<C, NVV, true>, dim3(grid), dim3(block), 0, st, x, rows, cols, ldx, gamma, beta,    \
+                          eps, step, out, pitch, y, ld_y, qn, qp);                                              \
+        else                                                                                                    \
+            launch_kernel(layernorm_quantize_kernel<C, NVV, false>, dim3(grid), dim3(block), 0, st, x, rows, cols, ldx, gamma, beta,   \
+                          eps, step, out, pitch, y, ld_y, qn, qp);                                              \
         break;
     switch (nv) {
         VITINT_LN_CASE(1) VITINT_LN_CASE(2) VITINT_LN_CASE(3) VITINT_LN_CASE(4) VITINT_LN_CASE(6)

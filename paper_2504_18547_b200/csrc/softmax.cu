@@ -66,9 +66,19 @@ constexpr int SM_TAIL_SLOTS = 4;           // up to 63 columns behind the last w
 // nothing); NTT the compiled number of tail slots.  The loops are straight-line code: loads and stores are
 // predicated, nothing branches per element.  VEC: 16-byte loads are legal; DIV3: the step admits the three-operation
 // exact quotient.
-template <int C, int NVT, int NTT, bool VEC, bool DIV3>
+// TABLE: the scores are known to lie in -smax .. smax and `tab` (shared memory) holds exp(fl32(s * c)) for each of
+// them, tab[s + smax]: e_j is one lookup, no maximum is needed (exp(t_j) / sum_k exp(t_k) is Eq. 3's softmax
+// exactly; the maximum is only subtracted there for range, and the caller has checked smax*|c| <= 80).  A score
+// outside the range reads a clamped entry and sets `bad`.
+template <int C, int NVT, int NTT, bool VEC, bool DIV3, bool TABLE = false>
 __device__ __forceinline__ void softmax_row(const int32_t* __restrict__ sr, int cols, float c, const Divisor dv, float qp,
-                                            uint8_t* crow, float* pr, bool vec_p, int hl) {
+                                            uint8_t* crow, float* pr, bool vec_p, int hl, const float* tab = nullptr,
+                                            int smax = 0, uint32_t* bad = nullptr) {
+    auto lookup = [&](int v) -> float {
+        const uint32_t i = (uint32_t)(v + smax);
+        if (i > (uint32_t)(2 * smax)) *bad = 1u;
+        return tab[min(i, (uint32_t)(2 * smax))];
+    };
     const int nv = cols >> 6;
     const int tail0 = nv << 6, n_tail = cols - tail0;
     const f32x2 c2 = f2_dup(c);
@@ -86,6 +96,13 @@ __device__ __forceinline__ void softmax_row(const int32_t* __restrict__ sr, int 
             if (VEC) a = __ldg(reinterpret_cast<const int4*>(sr + col));
             else a = make_int4(__ldg(sr + col), __ldg(sr + col + 1), __ldg(sr + col + 2), __ldg(sr + col + 3));
         }
+        if (TABLE) {
+            // (a surplus chunk looks up score 0 and discards it: no branch)
+            const float e0 = lookup(a.x), e1 = lookup(a.y), e2 = lookup(a.z), e3 = lookup(a.w);
+            t[2 * j] = have ? f2_pack(e0, e1) : f2_dup(0.0f);
+            t[2 * j + 1] = have ? f2_pack(e2, e3) : f2_dup(0.0f);
+            continue;
+        }
         const f32x2 lo = f2_mul(f2_pack((float)a.x, (float)a.y), c2), hi = f2_mul(f2_pack((float)a.z, (float)a.w), c2);
         t[2 * j] = have ? lo : f2_dup(-INFINITY);
         t[2 * j + 1] = have ? hi : f2_dup(-INFINITY);
@@ -102,21 +119,28 @@ __device__ __forceinline__ void softmax_row(const int32_t* __restrict__ sr, int 
             const int o = q * 16 + hl;
             int v = 0;
             if (o < n_tail) v = __ldg(sr + tail0 + o);
+            if (TABLE) {
+                const float e = lookup(v);
+                x[q] = o < n_tail ? e : 0.0f;
+                continue;
+            }
             x[q] = o < n_tail ? __fmul_rn((float)v, c) : -INFINITY;
             mx = fmaxf(mx, x[q]);
         }
 #pragma unroll
         for (int q = 0; q < NTT; q += 2) t[2 * NVT + q / 2] = f2_pack(x[q], x[q + 1]);
     }
+    if (!TABLE) {
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
 
     // exponentials (kept in the registers of t) and the fp64 row sum
     const f32x2 nmx = f2_dup(-mx);
     double z0 = 0.0, z1 = 0.0;
 #pragma unroll
     for (int i = 0; i < NP; ++i) {
-        t[i] = exp_reduced2(t[i], nmx);
+        if (!TABLE) t[i] = exp_reduced2(t[i], nmx);
         float e0, e1;
         f2_unpack(t[i], e0, e1);
         z0 += (double)e0;
@@ -125,8 +149,9 @@ __device__ __forceinline__ void softmax_row(const int32_t* __restrict__ sr, int 
     double z = z0 + z1;
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-    // 1/Z to about 2^-45 from the fp32 reciprocal and one Newton step in fp64 (Z lies in [1, cols]: no range issue),
-    // then split into two floats
+    // 1/Z to about 2^-45 from the fp32 reciprocal and one Newton step in fp64, then split into two floats (Z lies in
+    // [1, cols]; with the table anywhere in [e^-80, cols e^80] by the caller's bound: 1/Z is still a normal float, and a
+    // low half that has become subnormal only loses bits of a correction that is itself 2^-24 of the result)
     const double r0 = (double)__frcp_rn((float)z);
     const double rz = r0 * (2.0 - z * r0);
     const float rzh = (float)rz, rzl = (float)(rz - (double)(float)rz);

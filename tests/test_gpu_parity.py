@@ -18,7 +18,7 @@ from oracle import pipeline as vp
 pytestmark = pytest.mark.gpu
 
 vt = pytest.importorskip("paper_2504_18547_b200")
-from gpu_util import GELU_TOL_REL, dev, from_codes, padding_is_zero, rand_codes, to_codes, ulp_diff  # noqa: E402
+from gpu_util import GELU_TOL_REL, check_guards, dev, from_codes, guarded_codes, padding_is_zero, rand_codes, to_codes, ulp_diff  # noqa: E402
 
 
 @pytest.fixture(autouse=True)
@@ -299,6 +299,70 @@ def test_softmax_quantize_within_two_ulp_and_band(rows, cols, ld, bits):
     assert np.all(g >= lo) and np.all(g <= hi)
     assert (g != q).mean() < 1e-3
     assert padding_is_zero(got)
+
+
+@pytest.mark.parametrize("bits", [4, 2, 3, 8])
+@pytest.mark.parametrize("rows,cols,ld,bound", [(591, 197, 200, 700), (5000, 197, 200, 4096), (33, 50, 52, 1024), (40, 577, 580, 700),
+                                                (24, 785, 788, 701), (9, 1, 4, 8192), (17, 256, 256, 700), (300, 832, 832, 700),
+                                                (64, 197, 200, 4095)])
+def test_softmax_quantize_bounded_within_two_ulp_and_band(rows, cols, ld, bits, bound):
+    """The table-driven kernel for scores of declared range meets the same contract as the general one: probabilities
+    within 2 ulp of the fp64 softmax, codes inside the oracle's band.  5000 rows exceed one pass of the persistent
+    grid (148 SMs x 4 CTAs x 16 rows would be 9472; with 73 KB of table two CTAs fit: 4736)."""
+    S = np.zeros((rows, ld), np.int32)
+    S[:, :cols] = (si.splitmix64(31 + cols, rows * cols) % np.uint64(1401)).astype(np.int64).reshape(rows, cols) - 700
+    S[0, :cols] = 5
+    if cols > 3:
+        S[1, :cols] = -700
+        S[1, 2] = 700
+    c = np.float32(0.0211 if bound < 2000 else 0.0047)
+    if bound == 4095:
+        # the edge of the no-maximum range: exp arguments reach +-79.9, whole rows near either end (row sums of
+        # about e^79 and e^-79), the two-float 1/Z at the ends of the fp32 range
+        c = np.float32(0.0195)
+        S[:, :cols] = np.clip(S[:, :cols] * 6, -4095, 4095)
+        S[2, :cols] = 4095 - (np.arange(cols) % 7)
+        S[3, :cols] = -4095 + (np.arange(cols) % 5)
+    s_p = np.float32(2.0 / (cols * math.sqrt(si.code_range(bits, False)[1])))
+    got, p = vt.vitint_softmax_quantize_bounded(dev(S), cols, c, s_p, bits, bound, want_p=True)
+    assert vt.vitint_device_status() == 0
+    p_ref, q, lo, hi = vo.softmax_quantize(S[:, :cols], c, s_p, bits)
+    p = p.cpu().numpy()
+    normal = p_ref >= 2.0 ** -126
+    assert ulp_diff(p[normal], p_ref[normal]).max() <= 2
+    assert np.all(np.abs(p[~normal].astype(np.float64) - p_ref[~normal]) <= 2.0 ** -126)
+    g = from_codes(got)
+    assert np.all(g >= lo) and np.all(g <= hi)
+    assert (g != q).mean() < 1e-3
+    assert padding_is_zero(got)
+    # the same table serves a second call
+    ws = torch.empty(vt.vitint_softmax_table_workspace_bytes(bound), dtype=torch.uint8, device="cuda")
+    a = vt.vitint_softmax_quantize_bounded(dev(S), cols, c, s_p, bits, bound, workspace=ws)
+    b = vt.vitint_softmax_quantize_bounded(dev(S), cols, c, s_p, bits, bound, workspace=ws, table_ready=True)
+    assert np.array_equal(from_codes(a), g) and np.array_equal(from_codes(b), g)
+
+
+def test_softmax_quantize_bounded_rejects_and_flags():
+    S = dev(np.zeros((8, 200), np.int32))
+    with pytest.raises(vt.VitintError) as e:
+        vt.vitint_softmax_quantize_bounded(S, 197, 0.02, 0.003, 4, 4097)       # 4096 * 0.02 > 80
+    assert "unsupported" in str(e.value).lower()
+    with pytest.raises(vt.VitintError):
+        vt.vitint_softmax_quantize_bounded(dev(np.zeros((8, 197), np.int32)), 197, 0.002, 0.003, 4, 4096)   # ld % 4 != 0
+    with pytest.raises(vt.VitintError):
+        vt.vitint_softmax_quantize_bounded(S, 197, 0.002, 0.003, 4, 9000)      # no table that large
+    with pytest.raises(vt.VitintError):
+        vt.vitint_softmax_quantize_bounded(S, 197, 0.002, 0.003, 4, 4096,
+                                           workspace=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    # a score outside the declared range reads a clamped table entry (nothing faults) and is reported
+    Sb = np.zeros((8, 200), np.int32)
+    Sb[3, 7] = 5000
+    Sb[4, 9] = -2 ** 31
+    out = guarded_codes(8, 197, 4, False)
+    vt.vitint_softmax_quantize_bounded(dev(Sb), 197, 0.002, 0.003, 4, 4096, out=out)
+    assert vt.vitint_device_status() != 0
+    assert vt.vitint_device_status() == 0
+    check_guards()
 
 
 @pytest.mark.parametrize("bits", [4, 2, 3, 8])
