@@ -112,8 +112,19 @@ extern "C" int vitint_attention_block(const vitint_codes* x, const vitint_attent
         // 3. P = quantize(softmax(c * S)),  c = s_q s_k / sqrt(64)
         const float c = (float)((double)d->q_step * (double)d->k_step / 8.0);
         vitint_codes p{ws + L.off_p, L.n_rows_p, d->tokens, L.pitch_p, d->p_bits, 0, 0, 0};
-        if (int rc = vitint_softmax_quantize(S, L.n_rows_p, d->tokens, L.ld_s, c, d->p_step, &p, nullptr, 0, stream))
-            return rc;
+        // the scores of b-bit codes are bounded by 64 * 2^(b-1) * 2^(b-1) (container width: any bit pattern stays
+        // inside), so the exp table serves whenever one of that size exists and the range allows it
+        const int half = 1 << (cbits - 1);
+        const int32_t bound = 64 * half * half;
+        int sm = VITINT_ERR_UNSUPPORTED;
+        if (L.tab_bytes && vitint_softmax_table_workspace_bytes(bound) != 0 &&
+            vitint_softmax_table_workspace_bytes(bound) <= L.tab_bytes)
+            sm = vitint_softmax_quantize_bounded(S, L.n_rows_p, d->tokens, L.ld_s, c, d->p_step, bound, &p, nullptr, 0,
+                                                 ws + L.off_tab, L.tab_bytes, 0, stream);
+        if (sm != VITINT_OK && sm != VITINT_ERR_UNSUPPORTED) return sm;
+        if (sm == VITINT_ERR_UNSUPPORTED)
+            if (int rc = vitint_softmax_quantize(S, L.n_rows_p, d->tokens, L.ld_s, c, d->p_step, &p, nullptr, 0, stream))
+                return rc;
         if (int rc = copy_codes(dbg_p, p.data, L.pitch_p, L.n_rows_p, row_bytes(d->tokens, d->p_bits), st)) return rc;
 
         // 4. O = P V, requantized to the projection's input step

@@ -70,13 +70,44 @@ constexpr int SM_TAIL_SLOTS = 4;           // up to 63 columns behind the last w
 // them, tab[s + smax]: e_j is one lookup, no maximum is needed (exp(t_j) / sum_k exp(t_k) is Eq. 3's softmax
 // exactly; the maximum is only subtracted there for range, and the caller has checked smax*|c| <= 80).  A score
 // outside the range reads a clamped entry and sets `bad`.
+// The raw scores of a row in the column mapping of softmax_row (zeros where the row has no column): issued as a
+// unit so that a caller can request the next row before it works on the present one.
+template <int NVT, int NTT, bool VEC>
+struct RowScores {
+    int4 a[NVT > 0 ? NVT : 1];
+    int tv[NTT > 0 ? NTT : 1];
+    __device__ __forceinline__ void load(const int32_t* __restrict__ sr, int cols, int hl) {
+        const int nv = cols >> 6;
+        const int tail0 = nv << 6, n_tail = cols - tail0;
+#pragma unroll
+        for (int j = 0; j < NVT; ++j) {
+            const int col = j * 64 + hl * 4;
+            a[j] = make_int4(0, 0, 0, 0);
+            if (j < nv) {
+                if (VEC) a[j] = __ldg(reinterpret_cast<const int4*>(sr + col));
+                else a[j] = make_int4(__ldg(sr + col), __ldg(sr + col + 1), __ldg(sr + col + 2), __ldg(sr + col + 3));
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < NTT; ++q) {
+            const int o = q * 16 + hl;
+            tv[q] = 0;
+            if (o < n_tail) tv[q] = __ldg(sr + tail0 + o);
+        }
+    }
+};
+
 template <int C, int NVT, int NTT, bool VEC, bool DIV3, bool TABLE = false>
-__device__ __forceinline__ void softmax_row(const int32_t* __restrict__ sr, int cols, float c, const Divisor dv, float qp,
+__device__ __forceinline__ void softmax_row(const RowScores<NVT, NTT, VEC>& in, int cols, float c, const Divisor dv, float qp,
                                             uint8_t* crow, float* pr, bool vec_p, int hl, const float* tab = nullptr,
-                                            int smax = 0, uint32_t* bad = nullptr) {
+                                            int smax = 0, uint32_t* worst = nullptr) {
+    // table mode: index v + smax of the score's entry in unsigned arithmetic (a score below -smax wraps to a huge
+    // index, so one comparison covers both ends); one unsigned maximum keeps track of the largest index seen, one
+    // unsigned minimum keeps the load inside the table
+    uint32_t umax = 0u;
     auto lookup = [&](int v) -> float {
-        const uint32_t i = (uint32_t)(v + smax);
-        if (i > (uint32_t)(2 * smax)) *bad = 1u;
+        const uint32_t i = (uint32_t)v + (uint32_t)smax;
+        umax = max(umax, i);
         return tab[min(i, (uint32_t)(2 * smax))];
     };
     const int nv = cols >> 6;
@@ -89,13 +120,8 @@ __device__ __forceinline__ void softmax_row(const int32_t* __restrict__ sr, int 
     // sum and quantize to code 0 without any masking further down.
 #pragma unroll
     for (int j = 0; j < NVT; ++j) {
-        const int col = j * 64 + hl * 4;
         const bool have = j < nv;
-        int4 a = make_int4(0, 0, 0, 0);
-        if (have) {
-            if (VEC) a = __ldg(reinterpret_cast<const int4*>(sr + col));
-            else a = make_int4(__ldg(sr + col), __ldg(sr + col + 1), __ldg(sr + col + 2), __ldg(sr + col + 3));
-        }
+        const int4 a = in.a[j];
         if (TABLE) {
             // (a surplus chunk looks up score 0 and discards it: no branch)
             const float e0 = lookup(a.x), e1 = lookup(a.y), e2 = lookup(a.z), e3 = lookup(a.w);
@@ -117,8 +143,7 @@ __device__ __forceinline__ void softmax_row(const int32_t* __restrict__ sr, int 
 #pragma unroll
         for (int q = 0; q < NTT; ++q) {
             const int o = q * 16 + hl;
-            int v = 0;
-            if (o < n_tail) v = __ldg(sr + tail0 + o);
+            const int v = in.tv[q];
             if (TABLE) {
                 const float e = lookup(v);
                 x[q] = o < n_tail ? e : 0.0f;
@@ -133,6 +158,8 @@ __device__ __forceinline__ void softmax_row(const int32_t* __restrict__ sr, int 
     if (!TABLE) {
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    } else {
+        *worst = max(*worst, umax);
     }
 
     // exponentials (kept in the registers of t) and the fp64 row sum
@@ -250,8 +277,10 @@ softmax_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, i
     __syncwarp();
     float* const pr = (p_out != nullptr && row_ok) ? p_out + row * ld_p : nullptr;
     const Divisor dv = make_divisor(p_step);
-    if (dv.exact) softmax_row<C, NVT, NTT, VEC, true>(s + row * ld_s, cols, c, dv, qp, crow, pr, vec_p != 0, hl);
-    else softmax_row<C, NVT, NTT, VEC, false>(s + row * ld_s, cols, c, dv, qp, crow, pr, vec_p != 0, hl);
+    RowScores<NVT, NTT, VEC> in;
+    in.load(s + row * ld_s, cols, hl);
+    if (dv.exact) softmax_row<C, NVT, NTT, VEC, true>(in, cols, c, dv, qp, crow, pr, vec_p != 0, hl);
+    else softmax_row<C, NVT, NTT, VEC, false>(in, cols, c, dv, qp, crow, pr, vec_p != 0, hl);
     __syncwarp();
     // the finished row leaves in 16-byte pieces
     if (row_ok) {

@@ -15,7 +15,7 @@ namespace vitint {
 namespace {
 
 template <int C, int NVT, int NTT>
-__global__ void __launch_bounds__(32 * SM_ROWS_PER_BLOCK / 2)
+__global__ void __launch_bounds__(32 * SM_ROWS_PER_BLOCK / 2, 4)      // four CTAs fit the shared memory: no use for fewer than 64 registers
 softmax_table_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int cols, int64_t ld_s,
                               const float* __restrict__ table, int smax, float p_step, uint8_t* __restrict__ out,
                               int64_t pitch, float* __restrict__ p_out, int64_t ld_p, float qp, int vec_p) {
@@ -33,15 +33,22 @@ softmax_table_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int c
     for (int o = hl * 16; o < pitch; o += 256) *reinterpret_cast<uint4*>(crow + o) = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     const Divisor dv = make_divisor(p_step);
-    uint32_t bad = 0u;
+    uint32_t worst = 0u;                                               // largest table index any score asked for
     const int64_t groups = (rows + SM_ROWS_PER_BLOCK - 1) / SM_ROWS_PER_BLOCK;
+    auto row_of = [&](int64_t g) -> int64_t {
+        const int64_t r = g * SM_ROWS_PER_BLOCK + hw;
+        return r < rows ? r : rows - 1;                                // a surplus half-warp repeats the last row, stores nothing
+    };
+    // (requesting the next row's scores before working on the present one was measured slower: the second register
+    // set halves the resident CTAs or, capped, spills -- 98 to 108 us against 85)
     for (int64_t g = blockIdx.x; g < groups; g += gridDim.x) {
-        const int64_t row_raw = g * SM_ROWS_PER_BLOCK + hw;
-        const bool row_ok = row_raw < rows;
-        const int64_t row = row_ok ? row_raw : rows - 1;               // a surplus half-warp repeats the last row, stores nothing
+        const bool row_ok = g * SM_ROWS_PER_BLOCK + hw < rows;
+        const int64_t row = row_of(g);
         float* const pr = (p_out != nullptr && row_ok) ? p_out + row * ld_p : nullptr;
-        if (dv.exact) softmax_row<C, NVT, NTT, true, true, true>(s + row * ld_s, cols, 0.0f, dv, qp, crow, pr, vec_p != 0, hl, tab, smax, &bad);
-        else softmax_row<C, NVT, NTT, true, false, true>(s + row * ld_s, cols, 0.0f, dv, qp, crow, pr, vec_p != 0, hl, tab, smax, &bad);
+        RowScores<NVT, NTT, true> in;
+        in.load(s + row * ld_s, cols, hl);
+        if (dv.exact) softmax_row<C, NVT, NTT, true, true, true>(in, cols, 0.0f, dv, qp, crow, pr, vec_p != 0, hl, tab, smax, &worst);
+        else softmax_row<C, NVT, NTT, true, false, true>(in, cols, 0.0f, dv, qp, crow, pr, vec_p != 0, hl, tab, smax, &worst);
         __syncwarp();
         if (row_ok) {
             uint8_t* const orow = out + row * pitch;
@@ -49,8 +56,8 @@ softmax_table_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int c
         }
         __syncwarp();
     }
-    // a score outside the declared range: the row's codes are not to be trusted, say so
-    if (bad) atomicExch(&g_device_status, (int)VITINT_ERR_INVALID_ARG);
+    // a score outside the declared range: that row's codes are not to be trusted, say so
+    if (worst > (uint32_t)(2 * smax)) atomicExch(&g_device_status, (int)VITINT_ERR_INVALID_ARG);
 }
 
 template <int C, int NVT, int NTT>

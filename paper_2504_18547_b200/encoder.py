@@ -85,6 +85,16 @@ class EncoderLayer:
         else:
             self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
             self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
+            # scores of b-bit codes are bounded by 64 * 2^(b-1) * 2^(b-1): where the table-driven softmax takes that
+            # range its exp table is built by the first call and reused afterwards
+            half = 1 << ((4 if bits == 3 else bits) - 1)
+            self.score_bound = 64 * half * half
+            self.sm_table = None
+            if (softmax == "exp" and B.vitint_softmax_table_workspace_bytes(self.score_bound) > 0
+                    and self.score_bound * abs(self.c) <= 80.0 and tokens <= 895):
+                self.sm_table = torch.empty(B.vitint_softmax_table_workspace_bytes(self.score_bound), dtype=torch.uint8,
+                                            device=device)
+                self.sm_table_ready = False
         self.O = B.Codes.empty(M, D, bits, True, device, container=ca)
         self.h = torch.empty((M, D), dtype=torch.float32, device=device)
         self.x2 = B.Codes.empty(M, D, bits, True, device, container=ca)
@@ -122,6 +132,10 @@ class EncoderLayer:
             mark()
             if self.softmax == "shift":
                 B.vitint_softmax_shift_quantize(self.S, t, self.c2, self.s_p, self.bits, out=self.P)
+            elif self.sm_table is not None:
+                B.vitint_softmax_quantize_bounded(self.S, t, self.c, self.s_p, self.bits, self.score_bound, out=self.P,
+                                                  workspace=self.sm_table, table_ready=self.sm_table_ready)
+                self.sm_table_ready = True
             else:
                 B.vitint_softmax_quantize(self.S, t, self.c, self.s_p, self.bits, out=self.P)
             mark()
