@@ -36,7 +36,7 @@ import synth_inputs as si  # noqa: E402
 
 INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor throughput ratio on B200 (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-GEMM_DRAM_BYTES_PER_LAUNCH = 102.5e6   # ncu, ViT-Base layer, batch 128, 4-bit, byte codes: 410 MB over four launches
+GEMM_DRAM_BYTES_PER_LAUNCH = 101.5e6   # ncu, ViT-Base layer, batch 128, 4-bit, byte codes: 405.9 MB (read + write) over four launches
 N_INPUT_BUFFERS = 4           # 4 x 77.5 MB of fp32 activations > 126 MB of L2
 
 

@@ -591,8 +591,8 @@ __device__ __forceinline__ void epilogue_qkv_norm(const GemmParams& P, const Epi
                                                   long long orow, int n_tile, int slice, const float* refs_s, const float* sgn_s) {
     const int tile_col0 = n_tile * P.bn;
     const int valid = P.N - tile_col0 < P.bn ? P.N - tile_col0 : P.bn;      // a multiple of 64
-    const int groups = valid >> 6, half = (groups + 1) >> 1;
-    const int g_begin = slice == 0 ? 0 : half, g_end = slice == 0 ? half : groups;
+    const int groups = valid >> 6, n_slices = P.epi_warps >> 2;
+    const int g_begin = groups * slice / n_slices, g_end = groups * (slice + 1) / n_slices;
     const int v_col0 = 2 * P.norm_dim;
     for (int g = g_begin; g < g_end;) {
         const int col = g << 6, gcol = tile_col0 + col;
@@ -609,7 +609,7 @@ __device__ __forceinline__ void epilogue_qkv_norm(const GemmParams& P, const Epi
         }
     }
     // row padding behind the last column of the matrix
-    if (row_ok && slice == 1 && tile_col0 + valid >= P.N) {
+    if (row_ok && slice == n_slices - 1 && tile_col0 + valid >= P.N) {
         uint8_t* const o_row = (uint8_t*)P.out + orow * P.ld_out;
         for (long long off = ((long long)P.N * P.out_c) >> 3; off + 4 <= P.ld_out; off += 4)
             *reinterpret_cast<uint32_t*>(o_row + off) = 0u;
@@ -1156,6 +1156,9 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     // ... unless the contraction is short (K <= 1024): such a GEMM is bound by its fp32 epilogue, which gains more
     // from twelve warps than the mainloop loses with two ring stages (proj, batch 128: 45 -> 43 us; with the
     // long contraction of fc2 the same choice costs 17 us)
+    // (Sixteen epilogue warps -- four per lane quarter, equal 64-column shares of a tile -- were measured too: the
+    // 576-thread CTA is held to 96 registers a thread, and qkv / fc1 stayed at 57 / 90 us while the fp32 kinds spilled
+    // and lost 10 - 14 us.)
     P.epi_warps = (P.a_direct && P.b_direct && (!staged || K <= 1024)) ? MAX_EPI_WARPS : EPI_WARPS;
     if (P.kind == EK_QKV_NORM) P.epi_warps = EPI_WARPS;        // two warps per lane quarter, each taking whole 64-channel heads
     const uint32_t stage_total = staged ? (uint32_t)(P.epi_warps * STAGE_BYTES) : 0u;
