@@ -789,3 +789,65 @@ def test_softmax_band_is_the_two_ulp_neighbourhood():
     code = lambda v: np.clip(np.rint((v / s_p).astype(np.float32)), 0, 15).astype(np.int16)
     assert np.array_equal(lo, code(dn)) and np.array_equal(hi, code(up)) and np.array_equal(q, code(p))
     assert np.all(hi - lo <= 1) and (hi != lo).mean() < 2e-3
+
+
+def test_o_band_from_p_band_is_the_brute_force_extreme():
+    """Every choice of P codes inside [p_lo, p_hi] is enumerated on a tiny case (3 keys, 2 channels, intervals up to
+    two codes wide): the smallest and largest O codes found are exactly what the helper returns, with V of both
+    signs.  A helper that took the wrong end of the interval for negative V, or transposed V, fails here."""
+    import itertools
+    T, d, n = 3, 2, 2
+    rng = np.random.RandomState(5)
+    p_lo = rng.randint(0, 12, size=(n, T, T)).astype(np.int16)
+    p_hi = (p_lo + rng.randint(0, 3, size=(n, T, T))).astype(np.int16)
+    v = rng.randint(-8, 8, size=(n, T, d)).astype(np.int16)
+    v[0, 0, 0], v[0, 1, 0], v[1, 2, 1] = -7, 6, -8
+    alpha = np.array([0.11, 0.07], np.float32)
+    zero = np.zeros(d, np.float32)
+    lo, hi = vp.o_band_from_p_band(p_lo, p_hi, v, alpha, 4)
+    lo, hi = lo.reshape(n, T, d), hi.reshape(n, T, d)
+    widened = 0
+    for b in range(n):
+        for i in range(T):
+            best_lo, best_hi = np.full(d, 99), np.full(d, -99)
+            for row in itertools.product(*[range(p_lo[b, i, j], p_hi[b, i, j] + 1) for j in range(T)]):
+                acc = np.array([[sum(int(row[j]) * int(v[b, j, c]) for j in range(T)) for c in range(d)]], np.int32)
+                o = vo.epilogue_requant(acc, alpha, zero, 4, True)[0]
+                best_lo, best_hi = np.minimum(best_lo, o), np.maximum(best_hi, o)
+            assert np.array_equal(best_lo, lo[b, i]) and np.array_equal(best_hi, hi[b, i]), (b, i)
+            widened += int((best_hi > best_lo).sum())
+    assert widened > 0                                   # the case is not degenerate
+    # an interval of zero width gives the code itself
+    lo0, hi0 = vp.o_band_from_p_band(p_lo, p_lo, v, alpha, 4)
+    want = vo.epilogue_requant(vo.pv(p_lo, v).reshape(n * T, d), alpha, zero, 4, True)
+    assert np.array_equal(lo0, want) and np.array_equal(hi0, want)
+
+
+def test_stagewise_layer_equals_the_free_running_layer_on_its_own_values():
+    """encoder_layer_stagewise() fed with the free-running oracle's own stage values reproduces every stage of
+    encoder_layer() bit for bit (both softmax forms, both LayerNorm forms); fed with a perturbed upstream stage it
+    follows the perturbation, i.e. it really computes each stage from what it is given."""
+    cfg = si.VIT_TINY_BLOCK.with_(batch=1, tokens=37, mlp_dim=256)
+    T, H, bits = cfg.tokens, cfg.heads, cfg.bits
+    prm = si.layer_parameters(cfg)
+    x = si.activations(cfg)
+    for softmax, layernorm in (("exp", "fp32"), ("shift", "compare")):
+        st = vp.encoder_layer(x, prm, cfg.batch, T, H, bits, softmax=softmax, layernorm=layernorm)
+        att = st["attn"]
+        given = {"x1": st["x1_codes"], "qkv": att["qkv_codes"], "P": att["p_codes"], "O": att["o_codes"], "h": st["h"],
+                 "x2": st["x2_codes"], "g": st["g_codes"]}
+        sw = vp.encoder_layer_stagewise(x, prm, cfg.batch, T, H, bits, given, softmax=softmax, layernorm=layernorm)
+        assert np.array_equal(sw["x1_codes"], st["x1_codes"]) and np.array_equal(sw["qkv_codes"], att["qkv_codes"])
+        assert np.array_equal(sw["p_codes"], att["p_codes"]) and np.array_equal(sw["o_codes"], att["o_codes"])
+        assert np.array_equal(sw["h"].view(np.uint32), st["h"].view(np.uint32))
+        assert np.array_equal(sw["x2_codes"], st["x2_codes"]) and np.array_equal(sw["g_codes"], st["g_codes"])
+        assert np.array_equal(sw["out"].view(np.uint32), st["out"].view(np.uint32))
+        # without given P the O band contains the exact O
+        g2 = dict(given, P=None)
+        sw2 = vp.encoder_layer_stagewise(x, prm, cfg.batch, T, H, bits, g2, softmax=softmax, layernorm=layernorm)
+        assert np.all(sw2["o_lo"] <= att["o_codes"]) and np.all(att["o_codes"] <= sw2["o_hi"])
+        # a changed upstream stage changes what the next stage must be
+        g3 = dict(given, x1=np.where(st["x1_codes"] < 7, st["x1_codes"] + 1, st["x1_codes"]).astype(st["x1_codes"].dtype))
+        sw3 = vp.encoder_layer_stagewise(x, prm, cfg.batch, T, H, bits, g3, softmax=softmax, layernorm=layernorm)
+        assert not np.array_equal(sw3["qkv_codes"], att["qkv_codes"])
+        assert np.array_equal(sw3["x1_codes"], st["x1_codes"])      # LayerNorm 1 still comes from x
