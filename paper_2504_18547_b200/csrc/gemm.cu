@@ -1156,6 +1156,9 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     // ... unless the contraction is short (K <= 1024): such a GEMM is bound by its fp32 epilogue, which gains more
     // from twelve warps than the mainloop loses with two ring stages (proj, batch 128: 45 -> 43 us; with the
     // long contraction of fc2 the same choice costs 17 us)
+    // (An fp32 epilogue without staging -- every thread moving its row's columns as 32-byte sectors, four ring stages and
+    // twelve warps in return -- was measured as well: proj 43 -> 64 us, fc2 67 -> 78 us.  A warp's access to 32 different
+    // rows is served one row at a time, whatever its width.)
     // (Sixteen epilogue warps -- four per lane quarter, equal 64-column shares of a tile -- were measured too: the
     // 576-thread CTA is held to 96 registers a thread, and qkv / fc1 stayed at 57 / 90 us while the fp32 kinds spilled
     // and lost 10 - 14 us.)
