@@ -89,6 +89,7 @@ struct EpiParams {                      // per-column epilogue parameters of the
 #ifdef VITINT_TRACE
 constexpr int TRACE_CTAS = 4, TRACE_ROLES = 4, TRACE_SLOTS = 4096;
 __device__ long long* g_trace_buf = nullptr;
+int g_trace_max_ctas = 0;        // host: when > 0 the persistent grid is capped (how does a CTA run with fewer neighbours?)
 struct Tracer {
     long long* p;
     int n;
@@ -1134,6 +1135,9 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     if ((bound << P.shift) >= (1ll << 31)) return VITINT_ERR_UNSUPPORTED;
     P.small_acc = (bound << P.shift) < (1ll << 22) ? 2 : (bound < (1ll << 22) ? 1 : 0);
     int bn = N >= MAX_BN ? MAX_BN : ((N + 15) / 16) * 16;
+    // (Twelve epilogue warps are three per lane quarter, so a 256-column tile is shared 96 / 96 / 64 and waits for the
+    // 96; 192-column tiles would share evenly but their MMAs stream a sixth more bytes per output and come close to
+    // the issuing thread's rate: fc1 89 -> 101 us, measured.)
     if (b_mn_major) { if (N != 64) return VITINT_ERR_UNSUPPORTED; bn = 64; }
     P.bn = bn;
     P.m_tiles = (M + BM - 1) / BM;
@@ -1208,6 +1212,9 @@ int launch_gemm(const Operand& A, const Operand& B, int M, int N, int K, int n_i
     if (smem < 120 * 1024) smem = 120 * 1024;
     int grid = sm_count();
     if (grid > P.total_tiles) grid = P.total_tiles;
+#ifdef VITINT_TRACE
+    if (g_trace_max_ctas > 0 && grid > g_trace_max_ctas) grid = g_trace_max_ctas;
+#endif
     const int dev = current_device();
     if (dev < 0) return VITINT_ERR_CUDA;
     static bool attr_set_dev[MAX_DEVICES][NUM_KINDS] = {};
@@ -1305,6 +1312,8 @@ extern "C" int vitint_trace_set(long long* buf) {
     return cuda_status(cudaMemcpyToSymbol(g_trace_buf, &buf, sizeof(buf)));
 }
 extern "C" int vitint_trace_words(void) { return TRACE_CTAS * TRACE_ROLES * TRACE_SLOTS; }
+// Diagnostic builds only: cap the persistent grid of the GEMM at n CTAs (0 = one per SM).  Every tile is still computed.
+extern "C" int vitint_trace_max_ctas(int n) { g_trace_max_ctas = n; return VITINT_OK; }
 #endif
 
 extern "C" int vitint_linear(const vitint_codes* x, float x_step, const vitint_codes* w, const float* w_step,

@@ -1,10 +1,12 @@
 """Where the warp roles of the integer GEMM wait: a timeline of the four linear layers of one ViT-Base encoder layer.
 
-    python -m paper_2504_18547_b200.trace_gemm [--batch 128]
+    python -m paper_2504_18547_b200.trace_gemm [--batch 128] [--max-ctas N]
 
 Builds the diagnostic library (-DVITINT_TRACE, a separate .so), runs one encoder-layer pass with the trace buffer
 armed around each vitint_linear call and prints, for the first two CTAs and per role (TMA producer, MMA issuer, two
-epilogue warps), the clock cycles spent blocked on each barrier and per-tile detail.  Diagnostic only.
+epilogue warps), the clock cycles spent blocked on each barrier and per-tile detail.  --max-ctas caps the persistent
+grid (every tile is still computed, by fewer CTAs): comparing cycles per MMA of a CTA with 147 neighbours and with few
+separates what an SM does to itself from what the chip's shared resources (L2, power) do to it.  Diagnostic only.
 """
 from __future__ import annotations
 
@@ -28,6 +30,7 @@ def between(tags, clk, a, b):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--batch", type=int, default=128)
+    ap.add_argument("--max-ctas", type=int, default=0)
     args = ap.parse_args()
     import torch
 
@@ -38,6 +41,7 @@ def main():
     from paper_2504_18547_b200 import encoder
     L = binding.lib()
     L.vitint_trace_set.argtypes = [ctypes.c_void_p]
+    L.vitint_trace_max_ctas(int(args.max_ctas))
     cfg = si.VIT_BASE_LAYER.with_(batch=args.batch)
     prm = si.layer_parameters(cfg)
     dev = torch.device("cuda", 0)
@@ -63,9 +67,10 @@ def main():
     encoder.B.vitint_linear = traced
     layer.forward(x, out)
     torch.cuda.synchronize()
+    k_of = {"qkv": cfg.dim, "proj": cfg.dim, "fc1": cfg.dim, "fc2": cfg.mlp_dim}
     for name, t in zip(("qkv", "proj", "fc1", "fc2"), traces):
         t = t.reshape(CTAS, ROLES, SLOTS)
-        print(f"== {name}")
+        print(f"== {name}" + (f" (grid capped at {args.max_ctas} CTAs)" if args.max_ctas else ""))
         for cta in range(2):
             rec = []
             for role in range(ROLES):
@@ -76,8 +81,11 @@ def main():
             print(f" cta{cta} TMA producer: span {int(clk[-1] - clk[0])} clk, blocked on a free stage {between(tags, clk, WAIT_EMPTY, GOT_EMPTY)}")
             tags, clk = rec[1]
             tiles = int((tags == ISSUED).sum())
-            print(f" cta{cta} MMA issuer: span {int(clk[-1] - clk[0])} clk over {tiles} tiles, blocked on an accumulator buffer "
-                  f"{between(tags, clk, WAIT_EMPTY, GOT_EMPTY)}, on operands {between(tags, clk, WAIT_FULL, GOT_FULL)}")
+            span, b_acc, b_ops = int(clk[-1] - clk[0]), between(tags, clk, WAIT_EMPTY, GOT_EMPTY), between(tags, clk, WAIT_FULL, GOT_FULL)
+            mmas = tiles * (k_of[name] // 32)
+            print(f" cta{cta} MMA issuer: span {span} clk over {tiles} tiles, blocked on an accumulator buffer "
+                  f"{b_acc}, on operands {b_ops}; {mmas} MMAs, {span / max(mmas, 1):.0f} clk per MMA over the span, "
+                  f"{(span - b_acc - b_ops) / max(mmas, 1):.0f} while issuing")
             for role in (2, 3):
                 tags, clk = rec[role]
                 work = [int(clk[i + 1] - clk[i]) for i in range(len(tags) - 1) if tags[i] == GOT_ACC and tags[i + 1] == TILE_DONE]
