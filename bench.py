@@ -410,14 +410,17 @@ def run_ours(args, cfg):
         dx = torch.from_numpy(si.activations(dcfg)).to(device)
         ds_x = float(si.lsq_step(dx[:dcfg.tokens].cpu().numpy(), dcfg.bits, True))
         dxq = vt.vitint_quantize(dx, ds_x, dcfg.bits, True)
-        # fused: the per-head LayerNorm + comparator quantizer runs in the QKV GEMM's epilogue (4 launches);
+        # fused: the per-head LayerNorm + comparator quantizer runs in the QKV GEMM's epilogue and Eq. 4 inside the
+        # attention core (2 launches), or with Q K^T, softmax and P V as three kernels (4 launches);
         # unfused: fp32 Q and K rows through memory and a LayerNorm kernel each (10 launches)
-        for name, fused, launches in (("deit_s_attention_n198_b64", True, 4), ("deit_s_attention_n198_b64_unfused", False, 10)):
-            mod = NormedAttention(dcfg.batch, dcfg.tokens, dcfg.heads, dcfg.bits, dprm, dqkn, device, fused=fused)
+        for name, fused, core, launches in (("deit_s_attention_n198_b64", True, True, 2),
+                                            ("deit_s_attention_n198_b64_three_attention_kernels", True, False, 4),
+                                            ("deit_s_attention_n198_b64_unfused", False, False, 10)):
+            mod = NormedAttention(dcfg.batch, dcfg.tokens, dcfg.heads, dcfg.bits, dprm, dqkn, device, fused=fused, fused_core=core)
             ms = timed(lambda: mod.forward(dxq, ds_x))
             standalone[name] = {"ms": round(ms, 4), "tops": round(mod.ops() / (ms * 1e-3) / 1e12, 1),
                                 "images_per_s": round(dcfg.batch / (ms * 1e-3), 1), "launches": launches}
-            if fused:
+            if fused and core:
                 ms_q = timed(lambda: vt.vitint_linear_qkv_norm(dxq, ds_x, mod.w_qkv, mod.s_w_all, mod.bias_all, mod.refs_all,
                                                                mod.flip_all, mod.n_eps, mod.alpha_v, mod.beta_v, mod.bits,
                                                                out=mod.qkv, stats=mod.stats_all))
@@ -426,15 +429,28 @@ def run_ours(args, cfg):
             del mod
         del dx, dxq
         # the same encoder layer with the paper's own quantizers throughout (Eq. 4 softmax with the division-free
-        # comparator, Eq. 5 statistics with the comparator LayerNorm quantizer): unfused attention, 11 launches
+        # comparator, Eq. 5 statistics with the comparator LayerNorm quantizer), attention fused (Eq. 4 inside the core)
+        # and as three kernels
         from paper_2504_18547_b200.encoder import EncoderLayer as _Layer
-        plain = _Layer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, device, softmax="shift",
-                       layernorm="compare")
-        ms = timed(lambda: plain.forward(xs[0], out), reps=5)
-        standalone["layer_with_comparator_quantizers"] = {"ms": round(ms, 4), "tops": round(ops_step / (ms * 1e-3) / 1e12, 1),
-                                                          "images_per_s": round(cfg.batch / (ms * 1e-3), 1),
-                                                          "launches": len(plain.stages) + 2}
-        del plain
+        for name, fused in (("layer_with_comparator_quantizers", True), ("layer_with_comparator_quantizers_unfused_attention", False)):
+            plain = _Layer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, device, softmax="shift",
+                           layernorm="compare", fused_attention=fused)
+            ms = timed(lambda: plain.forward(xs[0], out), reps=5)
+            standalone[name] = {"ms": round(ms, 4), "tops": round(ops_step / (ms * 1e-3) / 1e12, 1),
+                                "images_per_s": round(cfg.batch / (ms * 1e-3), 1), "launches": len(plain.stages) + 2}
+            if fused:
+                # the fused attention core alone on this layer's QKV codes: Eq. 4 inside against the exp table inside
+                ws4 = torch.empty(vt.vitint_attention_core_shift_workspace_bytes(cfg.bits), dtype=torch.uint8, device=device)
+                args4 = (plain.qkv, cfg.batch, cfg.heads, cfg.tokens, plain.s_q, plain.s_k, plain.s_p, cfg.bits, plain.alpha_o, None)
+                vt.vitint_attention_core_shift(*args4, out=plain.O, workspace=ws4)
+                ms_s = timed(lambda: vt.vitint_attention_core_shift(*args4, out=plain.O, workspace=ws4, table_ready=True))
+                tab = vt.vitint_attention_exp_table(cfg.bits, plain.s_q, plain.s_k, device=device)
+                ms_e = timed(lambda: vt.vitint_attention_core_prepared(*args4, out=plain.O, table=tab))
+                att_ops = 2 * 2 * cfg.batch * cfg.heads * cfg.tokens * cfg.tokens * 64
+                standalone["attention_core_eq4_softmax"] = {"ms": round(ms_s, 4), "tops": round(att_ops / (ms_s * 1e-3) / 1e12, 1)}
+                standalone["attention_core_exp_softmax"] = {"ms": round(ms_e, 4), "tops": round(att_ops / (ms_e * 1e-3) / 1e12, 1)}
+                del ws4, tab
+            del plain
         # the whole DeiT-S-shaped model (patch embedding, 198 tokens, 12 layers, final LayerNorm, two heads), batch 128
         from paper_2504_18547_b200.encoder import DeitModel
         mcfg = si.DEIT_S_MODEL

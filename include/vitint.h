@@ -268,6 +268,22 @@ int vitint_attention_core_prepared(const vitint_codes* qkv, int32_t batch, int32
                                    const float* beta_o, const vitint_codes* o_out, const void* table,
                                    size_t table_bytes, void* stream);
 
+/* The fused attention core with the paper's own softmax (Eq. 4: 2^z with z = S c log2 e split into integer part and
+ *   residual, 2^r ~ 1 + r, integer shifts; the division-free comparator quantizer of Section IV-B whose references are
+ *   scaled by the row sum).  Arguments as vitint_attention_core; the codes of P and O are those of vitint_qk ->
+ *   vitint_softmax_shift_quantize -> vitint_pv bit for bit (every step is an integer or a single fp32 operation).
+ *   The per-score pair (floor z, mantissa of 1 + r) comes from two tables over the bounded score range, built into
+ *   `workspace` (256-byte aligned, at least vitint_attention_core_shift_workspace_bytes(bits) bytes) by one small
+ *   launch, unless table_ready != 0: the workspace then still holds the tables an earlier call with the same bits,
+ *   q_step and k_step wrote.  The row maximum is subtracted (as shift counts), so unlike vitint_attention_core this
+ *   variant has no limit on the size of the logits.
+ *   Errors: as vitint_attention_core; UNSUPPORTED also for codes not stored one per byte (container_bits != 8). */
+size_t vitint_attention_core_shift_workspace_bytes(int32_t bits);
+int vitint_attention_core_shift(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens, float q_step,
+                                float k_step, float p_step, int32_t p_bits, const float* alpha_o, const float* beta_o,
+                                const vitint_codes* o_out, void* workspace, size_t workspace_bytes, int32_t table_ready,
+                                void* stream);
+
 /* vitint_attention_core without caller-provided scratch.  (No counterpart in the paper: this is
  *   a packaging variant, not a step of the method.)
  *   Who needs it: code that is not allowed to obtain device memory when it runs the attention

@@ -77,6 +77,11 @@ def lib():
         L.vitint_attention_core_workspace_bytes.argtypes = [c_int32]
         L.vitint_attention_core.argtypes = [POINTER(_Codes), c_int32, c_int32, c_int32, c_float, c_float, c_float,
                                             c_int32, c_void_p, c_void_p, POINTER(_Codes), c_void_p, c_size_t, c_void_p]
+        L.vitint_attention_core_shift_workspace_bytes.restype = c_size_t
+        L.vitint_attention_core_shift_workspace_bytes.argtypes = [c_int32]
+        L.vitint_attention_core_shift.argtypes = [POINTER(_Codes), c_int32, c_int32, c_int32, c_float, c_float, c_float,
+                                                  c_int32, c_void_p, c_void_p, POINTER(_Codes), c_void_p, c_size_t,
+                                                  c_int32, c_void_p]
         L.vitint_attention_exp_table.argtypes = [c_int32, c_float, c_float, c_void_p, c_size_t, c_void_p]
         L.vitint_attention_core_prepared.argtypes = [POINTER(_Codes), c_int32, c_int32, c_int32, c_float, c_float, c_float,
                                                      c_int32, c_void_p, c_void_p, POINTER(_Codes), c_void_p, c_size_t,
@@ -411,6 +416,28 @@ def vitint_attention_core(qkv: Codes, batch: int, heads: int, tokens: int, q_ste
     _check(lib().vitint_attention_core(byref(dq), batch, heads, tokens, float(q_step), float(k_step), float(p_step),
                                        p_bits, _ptr(alpha_o), _ptr(beta_o), byref(do), workspace.data_ptr(),
                                        workspace.numel(), _stream()), "vitint_attention_core")
+    return out
+
+
+def vitint_attention_core_shift_workspace_bytes(bits: int) -> int:
+    return int(lib().vitint_attention_core_shift_workspace_bytes(int(bits)))
+
+
+def vitint_attention_core_shift(qkv: Codes, batch: int, heads: int, tokens: int, q_step: float, k_step: float,
+                                p_step: float, p_bits: int, alpha_o: torch.Tensor, beta_o: torch.Tensor | None,
+                                out: Codes | None = None, out_bits: int | None = None,
+                                workspace: torch.Tensor | None = None, table_ready: bool = False) -> Codes:
+    """The fused attention core with the Eq. 4 softmax and its division-free comparator quantizer (byte-stored codes).
+    table_ready: `workspace` still holds the table an earlier call with the same bits and steps built."""
+    if out is None:
+        out = Codes.empty(batch * tokens, heads * 64, qkv.bits if out_bits is None else out_bits, True, qkv.data.device)
+    if workspace is None:
+        workspace = torch.empty(vitint_attention_core_shift_workspace_bytes(qkv.bits), dtype=torch.uint8,
+                                device=qkv.data.device)
+    dq, do = qkv.desc(), out.desc()
+    _check(lib().vitint_attention_core_shift(byref(dq), batch, heads, tokens, float(q_step), float(k_step), float(p_step),
+                                             p_bits, _ptr(alpha_o), _ptr(beta_o), byref(do), workspace.data_ptr(),
+                                             workspace.numel(), int(table_ready), _stream()), "vitint_attention_core_shift")
     return out
 
 

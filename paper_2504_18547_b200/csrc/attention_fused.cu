@@ -42,9 +42,10 @@ struct AttnParams {
     int kv_rows;                 // tokens rounded up to 32: K extent of P V, rows of the V tile
     int smax;                    // table covers scores -smax .. smax
     int part_bytes;              // bytes of one of the Q / K / V column blocks in a QKV row
-    uint32_t off_table, off_group, group_bytes;         // shared-memory layout
-    uint32_t off_pq, off_pk, off_pv, off_q, off_k, off_v, off_p, off_col, off_z;   // within a group
+    uint32_t off_table, off_ftab, off_group, group_bytes;         // shared-memory layout
+    uint32_t off_pq, off_pk, off_pv, off_q, off_k, off_v, off_p, off_col, off_z, off_mx;   // within a group
     const float* table;          // global copy of the exp table, 2*smax+1 floats
+    uint32_t ftab_word;          // Eq. 4: word offset of the 16-bit table of integer parts behind the 32-bit table
     float p_step, p_qp;
     const float* alpha_o;        // [D]
     const float* beta_o;         // [D] or null
@@ -58,6 +59,20 @@ struct AttnBars {
     uint64_t packed_full, v_full, ops_ready, s_full, p_ready, o_full, o_done, grp_sync, z_sync;
 };
 
+// Eq. 4's split of every integer score: z = fl32(s * c2), f = floor z (16-bit table behind the 32-bit one),
+// M = trunc((1 + (z - f)) * 2^23), the 24-bit mantissa of 2^r ~ 1 + r (2^24 in the one case where 1 + r rounds to 2).
+__global__ void shift_table_kernel(uint32_t* mtab, short* ftab, int smax, float c2) {
+    grid_dependency_wait();        // an earlier kernel may still read the table
+    grid_dependency_launch();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i > 2 * smax) return;
+    const float z = __fmul_rn((float)(i - smax), c2);
+    const float fl = floorf(z);
+    const float res = __fsub_rn(z, fl);
+    mtab[i] = (uint32_t)__fmul_rn(__fadd_rn(1.0f, res), 8388608.0f);
+    ftab[i] = (short)(int)fl;
+}
+
 // exp(fl32(s * c)) for every integer score, correctly rounded to fp32 (fp64 exp, one rounding).
 __global__ void exp_table_kernel(float* table, int smax, float c) {
     grid_dependency_wait();        // an earlier kernel may still read the table
@@ -68,10 +83,16 @@ __global__ void exp_table_kernel(float* table, int smax, float c) {
     table[i] = (float)exp((double)t);
 }
 
-template <int C>
+// SHIFT: the softmax of Eq. 4 (2^z with z split into integer part and residual, 2^r ~ 1 + r, integer shifts, the
+// division-free comparator quantizer) instead of exp.  With integer scores of bounded range the pair (floor z,
+// mantissa of 1 + r) is one table entry per score, so the arithmetic left per score is the shift, the exact 64-bit
+// row sum and the comparison against references scaled by that sum -- every step an integer or a single fp32
+// operation in the order of the stand-alone kernel, hence the same codes bit for bit.
+template <int C, bool SHIFT>
 __global__ void __launch_bounds__(AT_THREADS, 1)
 attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv,
                        const __grid_constant__ AttnParams P) {
+    static_assert(!SHIFT || C == 8, "the Eq. 4 variant takes byte-stored codes");
     extern __shared__ uint8_t smem_raw[];
     __shared__ AttnBars bars[AT_GROUPS];
     __shared__ uint32_t tmem_base_slot;
@@ -113,6 +134,12 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     {
         float* tab = reinterpret_cast<float*>(smem_gen + P.off_table);
         for (int i = threadIdx.x; i <= 2 * P.smax; i += AT_THREADS) tab[i] = __ldg(P.table + i);
+        if constexpr (SHIFT) {
+            // the 16-bit table of integer parts sits behind the 32-bit one, in the workspace and here
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(P.table) + P.ftab_word;
+            uint32_t* dst = reinterpret_cast<uint32_t*>(smem_gen + P.off_ftab);
+            for (int i = threadIdx.x; i <= P.smax; i += AT_THREADS) dst[i] = __ldg(src + i);
+        }
     }
     if (is_control && lane == 0) { ptx::prefetch_tensormap(&map_q); ptx::prefetch_tensormap(&map_kv); }
     ptx::tc_fence_before();
@@ -263,6 +290,116 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
             w = mbar_wait(ptx::smem_addr(&B.s_full), ph, abort_ptr);
             if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
             ptx::tc_fence_after();
+            if constexpr (SHIFT) {
+                // Two tables over the score range: M[s] = trunc((1 + (z - floor z)) * 2^23) (32-bit) and f[s] = floor z
+                // (16-bit), z = fl32(s * c2).  floor z increases with s, so the row's largest score carries the row's
+                // largest integer part m and pass 0 needs no lookup at all.
+                const int full_chunks = T >> 5;
+                const bool warp_live = qt * 128 + wq * 32 < T;
+                int* const mx = reinterpret_cast<int*>(ggen + P.off_mx);
+                unsigned long long* const sx = reinterpret_cast<unsigned long long*>(ggen + P.off_z);
+                const uint32_t* const mtab = reinterpret_cast<const uint32_t*>(smem_gen + P.off_table);
+                const short* const ftab = reinterpret_cast<const short*>(smem_gen + P.off_ftab);
+                const uint32_t top = (uint32_t)(2 * P.smax);
+                // pass 0: the row's largest score
+                int smx = INT_MIN;
+                for (int ch = hf; warp_live && ch < chunks; ch += 2) {
+                    uint32_t v[32];
+                    ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        smx = max(smx, (ch < full_chunks || ch * 32 + i < T) ? (int)v[i] : INT_MIN);
+                }
+                mx[hf * 128 + row] = smx;
+                ptx::mbar_arrive(ptx::smem_addr(&B.z_sync));
+                w = mbar_wait(ptx::smem_addr(&B.z_sync), 0u, abort_ptr);       // two phases per item: parities 0, 1
+                if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+                smx = max(mx[row], mx[128 + row]);
+                // pass 1: E_j = M_j << (30 + f_j - m) (>> for the few scores more than 30 octaves down), exact 64-bit
+                // row sum, float(E_j) put together from its bits and parked in TMEM over the score
+                const int c0 = 30 - (int)ftab[min((uint32_t)(max(smx, -P.smax) + P.smax), top)];
+                // Straight-line per score (rows with a wide spread of scores take the right-shift form often, so a
+                // branch would mostly run both sides): the 64-bit term is (M * 2^32) >> (32 - sh) with sh kept above
+                // -32 (further down everything is shifted out anyway); float(E) is float(M) * 2^sh put together from
+                // its bits for sh >= 0, and the conversion of the small remainder by the 2^23 trick otherwise.
+                uint32_t sg_lo = 0u, sg_hi = 0u;
+                auto term = [&](uint32_t score, bool valid) -> uint32_t {
+                    const uint32_t idx = min((uint32_t)((int)score + P.smax), top);
+                    const uint32_t m24 = valid ? mtab[idx] : 0u;
+                    const int sh = max((int)ftab[idx] + c0, -31);
+                    const unsigned long long big = ((unsigned long long)m24 << 32) >> (32 - sh);
+                    const uint32_t lo = (uint32_t)big, hi = (uint32_t)(big >> 32);
+                    asm("add.cc.u32 %0, %0, %2;\n\taddc.u32 %1, %1, %3;" : "+r"(sg_lo), "+r"(sg_hi) : "r"(lo), "r"(hi));
+                    const uint32_t up = m24 + 0x4A800000u + ((uint32_t)sh << 23);
+                    const uint32_t dn = __float_as_uint(__fadd_rn(__uint_as_float(0x4B000000u + lo), -8388608.0f));
+                    return m24 == 0u ? 0u : (sh >= 0 ? up : dn);
+                };
+                for (int ch = hf; warp_live && ch < chunks; ch += 2) {
+                    uint32_t v[32];
+                    ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
+                    ptx::tmem_ld_wait();
+                    if (ch < full_chunks) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = term(v[i], true);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = term(v[i], ch * 32 + i < T);      // no score past the last token
+                    }
+                    ptx::tmem_st32(t_row + (uint32_t)(ch * 32), v);
+                }
+                unsigned long long sigma = ((unsigned long long)sg_hi << 32) | sg_lo;
+                ptx::tmem_st_wait();
+                sx[hf * 128 + row] = sigma;
+                ptx::mbar_arrive(ptx::smem_addr(&B.z_sync));
+                w = mbar_wait(ptx::smem_addr(&B.z_sync), 1u, abort_ptr);
+                if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+                sigma = sx[row] + sx[128 + row];
+                const float sig_f = __ull2float_rn(sigma);
+                // pass 2: the code is the number of references fl32(fl32((k - 1/2) s_P) * Sigma) that float(E_j) exceeds.
+                // k0 = rint(E_j / (s_P Sigma)) is at most one off, so the two references around it decide:
+                // code = k0 - 1 + [E > ref(k0)] + [E > ref(k0 + 1)], references formed with the two fp32
+                // multiplications of the definition.
+                const float inv = warp_live ? __frcp_rn(__fmul_rn(P.p_step, sig_f)) : 0.0f;
+                const f32x2 inv2 = f2_dup(inv), qp2 = f2_dup(P.p_qp), magic2 = f2_dup(12582912.0f), nmagic2 = f2_dup(-12582912.0f);
+                const f32x2 half2 = f2_dup(0.5f), nhalf2 = f2_dup(-0.5f), ps2 = f2_dup(P.p_step), sg2 = f2_dup(sig_f);
+                uint8_t* const prow = ggen + P.off_p + row * 128;
+                const int sw = row & 7;
+                for (int ch = hf; warp_live && ch < chunks; ch += 2) {
+                    uint32_t v[32];
+                    ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
+                    ptx::tmem_ld_wait();
+                    uint32_t wd[8];
+#pragma unroll
+                    for (int i4 = 0; i4 < 8; ++i4) {
+                        uint32_t cb[4];
+#pragma unroll
+                        for (int j = 0; j < 4; j += 2) {
+                            const float e0 = __uint_as_float(v[4 * i4 + j]), e1 = __uint_as_float(v[4 * i4 + j + 1]);
+                            const f32x2 e2 = f2_pack(e0, e1);
+                            float u0, u1;
+                            f2_unpack(f2_mul(e2, inv2), u0, u1);
+                            const f32x2 um = f2_add(f2_pack(fminf(u0, P.p_qp), fminf(u1, P.p_qp)), magic2);   // 1.5*2^23 + k0
+                            const f32x2 kf = f2_add(um, nmagic2);
+                            const f32x2 r_lo = f2_mul(f2_mul(f2_add(kf, nhalf2), ps2), sg2);
+                            const f32x2 r_hi = f2_mul(f2_mul(f2_add(kf, half2), ps2), sg2);
+                            float m0, m1, l0, l1, h0, h1, k0f, k1f;
+                            f2_unpack(um, m0, m1);
+                            f2_unpack(r_lo, l0, l1);
+                            f2_unpack(r_hi, h0, h1);
+                            f2_unpack(kf, k0f, k1f);
+                            // (no reference above the last level: the upper test only counts below Qp)
+                            cb[j] = (__float_as_uint(m0) & 0xFFu) - 1u + (e0 > l0 ? 1u : 0u) + ((e0 > h0 && k0f < P.p_qp) ? 1u : 0u);
+                            cb[j + 1] = (__float_as_uint(m1) & 0xFFu) - 1u + (e1 > l1 ? 1u : 0u) + ((e1 > h1 && k1f < P.p_qp) ? 1u : 0u);
+                        }
+                        wd[i4] = cb[0] | (cb[1] << 8) | (cb[2] << 16) | (cb[3] << 24);
+                    }
+                    const int cc = 2 * ch;
+                    uint8_t* const blk = prow + (cc >> 3) * 16384;
+                    *reinterpret_cast<uint4*>(blk + (((cc & 7) ^ sw) << 4)) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                    *reinterpret_cast<uint4*>(blk + ((((cc + 1) & 7) ^ sw) << 4)) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
+                }
+            } else {
             // pass 1: e_j = EXP[S_j] (an integer score is bounded by the code ranges, so the byte offset
             // 4*S always lies inside the table), row sum in fp64, e_j parked in TMEM over S_j
             // four interleaved partial sums: a single fp64 accumulator would chain 32 dependent additions per chunk
@@ -356,6 +493,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 *reinterpret_cast<uint4*>(blk + (((cc & 7) ^ sw) << 4)) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
                 *reinterpret_cast<uint4*>(blk + ((((cc + 1) & 7) ^ sw) << 4)) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
             }
+            }   // exp / Eq. 4
             ptx::fence_proxy_async_smem();
             ptx::tc_fence_before();
             __syncwarp();
@@ -437,6 +575,12 @@ inline uint32_t up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 
 using namespace vitint;
 
+extern "C" size_t vitint_attention_core_shift_workspace_bytes(int32_t bits) {
+    if (bits != 2 && bits != 3 && bits != 4) return 0;
+    const int m = 1 << (container_bits(bits) - 1);
+    return (size_t)(2 * 64 * m * m + 2) * 6 + 256;                   // 32-bit mantissas + 16-bit integer parts
+}
+
 extern "C" size_t vitint_attention_core_workspace_bytes(int32_t bits) {
     if (bits != 2 && bits != 3 && bits != 4) return 0;
     const int m = 1 << (container_bits(bits) - 1);   // sized by the container: any bit pattern indexes inside
@@ -448,7 +592,7 @@ extern "C" size_t vitint_attention_core_workspace_bytes(int32_t bits) {
 static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
                                  float q_step, float k_step, float p_step, int32_t p_bits, const float* alpha_o,
                                  const float* beta_o, const vitint_codes* o_out, void* workspace,
-                                 size_t workspace_bytes, bool build_table, void* stream) {
+                                 size_t workspace_bytes, bool build_table, void* stream, bool shift = false) {
     if (int rc = check_codes(qkv)) return rc;
     if (int rc = check_codes(o_out)) return rc;
     if (batch <= 0 || heads <= 0 || tokens <= 0 || !alpha_o) return VITINT_ERR_INVALID_ARG;
@@ -466,9 +610,14 @@ static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t
     // exp without max subtraction must not overflow for any score the declared code range can produce
     // (the table itself is sized by the container so that any bit pattern indexes inside it)
     const int mq = 1 << (qkv->bits - 1);
-    if (64.0 * mq * mq * (double)cs > 80.0) return VITINT_ERR_UNSUPPORTED;
+    if (!shift && 64.0 * mq * mq * (double)cs > 80.0) return VITINT_ERR_UNSUPPORTED;
+    // Eq. 4: z = S * c2 with c2 = c * log2 e; the row maximum is subtracted (as shifts), so the only range limit is the
+    // 16-bit table of floor z.  Byte-stored codes only.
+    const float c2 = (float)((double)cs * 1.4426950408889634);
+    if (shift && (c != 8 || (double)smax * (double)c2 > 30000.0)) return VITINT_ERR_UNSUPPORTED;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-        workspace_bytes < vitint_attention_core_workspace_bytes(qkv->bits))
+        workspace_bytes < (shift ? vitint_attention_core_shift_workspace_bytes(qkv->bits)
+                                 : vitint_attention_core_workspace_bytes(qkv->bits)))
         return VITINT_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
 
@@ -495,6 +644,12 @@ static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t
     const uint32_t hb = 8u * c;
     P.off_table = 0;
     P.off_group = up((uint32_t)(2 * smax + 1) * 4u, 1024);
+    if (shift) {
+        // 32-bit mantissas, then (from the next whole word on) the 16-bit integer parts
+        P.ftab_word = (uint32_t)(2 * smax + 1);
+        P.off_ftab = (uint32_t)(2 * smax + 1) * 4u;
+        P.off_group = up(P.off_ftab + (uint32_t)(2 * smax + 2) * 2u, 1024);
+    }
     uint32_t o = 0;
     P.off_q = o; o += 128 * 64;
     P.off_k = o; o += up((uint32_t)(c == 8 ? P.kv_rows : P.n_k) * 64, 1024);   // byte codes: the K box is kv_rows high
@@ -507,6 +662,8 @@ static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t
     }
     P.off_col = o; o += 1024;
     P.off_z = o; o += 2 * 128 * 8;
+    P.off_mx = o;
+    if (shift) o += 2 * 128 * 4;                           // partial row maxima of the Eq. 4 variant
     P.group_bytes = up(o, 1024);
     const size_t smem = (size_t)P.off_group + (size_t)AT_GROUPS * P.group_bytes + 1024;
     if (smem > 225 * 1024) return VITINT_ERR_UNSUPPORTED;
@@ -532,7 +689,9 @@ static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t
             return VITINT_ERR_CUDA;
     }
     if (build_table) {
-        launch_kernel(exp_table_kernel, dim3((2 * smax + 1 + 255) / 256), dim3(256), 0, st, (float*)workspace, smax, cs);
+        if (shift) launch_kernel(shift_table_kernel, dim3((2 * smax + 1 + 255) / 256), dim3(256), 0, st, (uint32_t*)workspace,
+                                 reinterpret_cast<short*>((uint32_t*)workspace + (2 * smax + 1)), smax, c2);
+        else launch_kernel(exp_table_kernel, dim3((2 * smax + 1 + 255) / 256), dim3(256), 0, st, (float*)workspace, smax, cs);
         if (cudaGetLastError() != cudaSuccess) return VITINT_ERR_CUDA;
     }
     int grid = sm_count();
@@ -540,21 +699,22 @@ static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t
     if (grid > want) grid = want;
     const int dev = current_device();
     if (dev < 0) return VITINT_ERR_CUDA;
-    static bool attr_set_dev[MAX_DEVICES][3] = {};
+    static bool attr_set_dev[MAX_DEVICES][4] = {};
     bool* const attr_set = attr_set_dev[dev];
-#define VITINT_ATTN_LAUNCH(CC, SLOT)                                                                               \
+#define VITINT_ATTN_LAUNCH(CC, SH, SLOT)                                                                           \
     {                                                                                                              \
         if (!attr_set[SLOT]) {                                                                                     \
-            if (cudaFuncSetAttribute(attention_fused_kernel<CC>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+            if (cudaFuncSetAttribute(attention_fused_kernel<CC, SH>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
                                      225 * 1024) != cudaSuccess)                                                   \
                 return VITINT_ERR_CUDA;                                                                            \
             attr_set[SLOT] = true;                                                                                 \
         }                                                                                                          \
-        launch_kernel(attention_fused_kernel<CC>, dim3(grid), dim3(AT_THREADS), smem, st, map_q, map_kv, P);       \
+        launch_kernel(attention_fused_kernel<CC, SH>, dim3(grid), dim3(AT_THREADS), smem, st, map_q, map_kv, P);   \
     }
-    if (c == 8) VITINT_ATTN_LAUNCH(8, 2)
-    else if (c == 4) VITINT_ATTN_LAUNCH(4, 1)
-    else VITINT_ATTN_LAUNCH(2, 0)
+    if (shift) VITINT_ATTN_LAUNCH(8, true, 3)
+    else if (c == 8) VITINT_ATTN_LAUNCH(8, false, 2)
+    else if (c == 4) VITINT_ATTN_LAUNCH(4, false, 1)
+    else VITINT_ATTN_LAUNCH(2, false, 0)
 #undef VITINT_ATTN_LAUNCH
     return cuda_status(cudaGetLastError());
 }
@@ -565,6 +725,14 @@ extern "C" int vitint_attention_core(const vitint_codes* qkv, int32_t batch, int
                                      size_t workspace_bytes, void* stream) {
     return attention_core_launch(qkv, batch, heads, tokens, q_step, k_step, p_step, p_bits, alpha_o, beta_o, o_out,
                                  workspace, workspace_bytes, true, stream);
+}
+
+extern "C" int vitint_attention_core_shift(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
+                                           float q_step, float k_step, float p_step, int32_t p_bits, const float* alpha_o,
+                                           const float* beta_o, const vitint_codes* o_out, void* workspace,
+                                           size_t workspace_bytes, int32_t table_ready, void* stream) {
+    return attention_core_launch(qkv, batch, heads, tokens, q_step, k_step, p_step, p_bits, alpha_o, beta_o, o_out,
+                                 workspace, workspace_bytes, table_ready == 0, stream, true);
 }
 
 extern "C" int vitint_attention_exp_table(int32_t bits, float q_step, float k_step, void* table, size_t table_bytes,

@@ -39,7 +39,9 @@ class EncoderLayer:
                              "division- and square-root-free comparator quantizer)")
         self.layernorm = layernorm
         # the shift-based softmax is a separate kernel: it runs in the unfused attention pipeline
-        self.fused_attention = fused_attention and bits != 8 and tokens <= 256 and softmax == "exp"
+        # the fused core takes the exp softmax for any container and the Eq. 4 softmax for byte-stored codes
+        self.fused_attention = (fused_attention and bits != 8 and tokens <= 256
+                                and (softmax == "exp" or (softmax == "shift" and wide_activations)))
         self.stages = STAGES_FUSED if self.fused_attention else STAGES_UNFUSED
         d = lambda a: _dev(a, device)
         f = lambda k: float(prm[k])
@@ -79,7 +81,11 @@ class EncoderLayer:
         self.x1 = B.Codes.empty(M, D, bits, True, device, container=ca)
         self.qkv = B.Codes.empty(M, 3 * D, bits, True, device, container=cq)
         self.ld_s = (tokens + 3) // 4 * 4
-        if self.fused_attention:
+        if self.fused_attention and softmax == "shift":
+            # the table of Eq. 4's (integer part, mantissa) pairs is built by the first call and reused
+            self.attn_table = torch.empty(B.vitint_attention_core_shift_workspace_bytes(bits), dtype=torch.uint8, device=device)
+            self.attn_table_ready = False
+        elif self.fused_attention:
             # the exp table of the fused core depends only on the code width and the steps of Q and K: filled once
             self.attn_table = B.vitint_attention_exp_table(bits, self.s_q, self.s_k, device=device)
         else:
@@ -124,7 +130,11 @@ class EncoderLayer:
         mark()
         B.vitint_linear(self.x1, self.s_ln, self.w["qkv"], None, None, self.epi_qkv, out=self.qkv)
         mark()
-        if self.fused_attention:
+        if self.fused_attention and self.softmax == "shift":
+            B.vitint_attention_core_shift(self.qkv, b, h, t, self.s_q, self.s_k, self.s_p, self.bits, self.alpha_o, None,
+                                          out=self.O, workspace=self.attn_table, table_ready=self.attn_table_ready)
+            self.attn_table_ready = True
+        elif self.fused_attention:
             B.vitint_attention_core_prepared(self.qkv, b, h, t, self.s_q, self.s_k, self.s_p, self.bits, self.alpha_o,
                                              None, out=self.O, table=self.attn_table)
         else:
@@ -204,13 +214,16 @@ class NormedAttention:
     Eq. 5, comparator quantizer of Fig. 5(b)), Q K^T, the Eq. 4 softmax with its division-free quantizer, P V.
     A fixed sequence of C-ABI calls over preallocated buffers; `qkn` holds the per-head LayerNorm parameters
     (qn_g, qn_b, kn_g, kn_b over 64 channels) and the steps s_qn, s_kn of the normalised values.
-    fused=True (default): one QKV GEMM whose epilogue normalises and quantizes the Q and K heads and requantizes V
-    (4 launches); fused=False: separate Q, K, V linears with fp32 Q and K rows and a LayerNorm kernel pass each
-    (10 launches, the fp32 rows and their statistics left in `f32` / `stats` for inspection)."""
+    fused=True (default): one QKV GEMM whose epilogue normalises and quantizes the Q and K heads and requantizes V,
+    then the fused attention core with the Eq. 4 softmax inside (2 launches; `fused_core=False` keeps Q K^T, softmax
+    and P V as three kernels with S and P in memory: 4 launches); fused=False: separate Q, K, V linears with fp32 Q
+    and K rows and a LayerNorm kernel pass each (10 launches, the fp32 rows and their statistics left in `f32` /
+    `stats` for inspection)."""
 
     def __init__(self, batch: int, tokens: int, heads: int, bits: int, prm: dict, qkn: dict, device="cuda",
-                 eps: float = 1e-6, fused: bool = True):
+                 eps: float = 1e-6, fused: bool = True, fused_core: bool = True):
         self.fused = fused
+        self.fused_core = fused and fused_core and tokens <= 256 and bits != 8
         self.batch, self.tokens, self.heads, self.bits = batch, tokens, heads, bits
         self.dim = D = heads * 64
         self.rows = M = batch * tokens
@@ -241,7 +254,13 @@ class NormedAttention:
         self.stats_all = torch.empty((2, M * heads, 2), dtype=torch.float32, device=device)
         self.stats = [self.stats_all[0], self.stats_all[1]]
         pitch = D * c_bits // 8
-        if fused:
+        if self.fused_core:
+            # byte-stored QKV codes: the operand form of the fused core
+            self.qkv = B.Codes.empty(M, 3 * D, bits, True, device, container=8)
+            self.core_ws = torch.empty(B.vitint_attention_core_shift_workspace_bytes(bits), dtype=torch.uint8, device=device)
+            self.core_ws_ready = False
+            self.slabs = self.v_slabs = None
+        elif fused:
             self.qkv = B.Codes.empty(M, 3 * D, bits, True, device)
             qp = self.qkv.pitch
             self.slabs = [B.Slabs(self.qkv.data, i * pitch, qp, qp * tokens, 64 * c_bits // 8, bits, True) for i in range(2)]
@@ -253,10 +272,12 @@ class NormedAttention:
             self.v = B.Codes.empty(M, D, bits, True, device)
             self.v_slabs = B.Slabs(self.v.data, 0, self.v.pitch, self.v.pitch * tokens, 64 * c_bits // 8, bits, True)
         self.ld_s = (tokens + 3) // 4 * 4
-        self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
-        self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
+        if not self.fused_core:
+            self.S = torch.empty((batch * heads * tokens, self.ld_s), dtype=torch.int32, device=device)
+            self.P = B.Codes.empty(batch * heads * tokens, tokens, bits, False, device)
         self.O = B.Codes.empty(M, D, bits, True, device)
         self.epi_o = B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_o, out_bits=bits, out_signed=True)
+        self.s_qn, self.s_kn = float(qkn["s_qn"]), float(qkn["s_kn"])
 
     def forward(self, x: "B.Codes", s_x: float) -> "B.Codes":
         """x: codes [batch*tokens, dim] with step s_x.  Returns the O codes [batch*tokens, dim]."""
@@ -277,6 +298,11 @@ class NormedAttention:
             B.vitint_linear(x, s_x, self.w_v, None, None,
                             B.Epilogue(mode=B.EPI_REQUANT, alpha=self.alpha_v, beta=self.beta_v, out_bits=self.bits,
                                        out_signed=True), out=self.v)
+        if self.fused_core:
+            B.vitint_attention_core_shift(self.qkv, b, h, t, self.s_qn, self.s_kn, self.s_p, self.bits, self.alpha_o, None,
+                                          out=self.O, workspace=self.core_ws, table_ready=self.core_ws_ready)
+            self.core_ws_ready = True
+            return self.O
         B.vitint_qk(self.slabs[0], self.slabs[1], b, h, t, out=self.S, ld_s=self.ld_s)
         B.vitint_softmax_shift_quantize(self.S, t, self.c2, self.s_p, self.bits, out=self.P)
         B.vitint_pv(self.P, self.v_slabs, b, h, t, self.s_p, self.s_v, self.epi_o, out=self.O)

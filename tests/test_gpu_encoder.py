@@ -113,23 +113,27 @@ def test_encoder_layer_staged(bits, fused, wide):
     compare_stages(g, x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits, tag=f"{bits}-bit: ")
 
 
+@pytest.mark.parametrize("fused", [True, False], ids=["fused_attention", "unfused_attention"])
 @pytest.mark.parametrize("bits", [4, 3])
-def test_encoder_layer_shift_softmax_attention_bit_exact(bits):
+def test_encoder_layer_shift_softmax_attention_bit_exact(bits, fused):
     """Encoder layer with the Eq. 4 softmax and the comparator quantizer: the attention stage has no fp32 island,
-    so P and O must equal what the oracle computes from the same QKV codes bit for bit, with no band."""
+    so P and O must equal what the oracle computes from the same QKV codes bit for bit, with no band -- as three
+    kernels (P visible) and as the fused core with Eq. 4 inside (P stays on the SM; O is exact)."""
     from paper_2504_18547_b200.encoder import EncoderLayer
     cfg = si.VIT_BASE_LAYER.with_(batch=3, bits=bits)
     prm = si.layer_parameters(cfg)
     x = si.activations(cfg)
-    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, softmax="shift")
-    assert not layer.fused_attention
+    layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, softmax="shift", fused_attention=fused)
+    assert layer.fused_attention == fused
     out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
     layer.forward(dev(x), out)
+    layer.forward(dev(x), out)                      # the second pass reuses the table the first one built
     assert vt.vitint_device_status() == 0
     T, H = cfg.tokens, cfg.heads
     g = gpu_stages(layer, out, range(cfg.batch), T, H)
     st, flips = compare_stages(g, x, prm, cfg.batch, T, H, cfg.bits, softmax="shift")
-    assert flips["P"] == 0.0 and np.array_equal(st["p_lo"], st["p_hi"])
+    assert np.array_equal(st["p_lo"], st["p_hi"])
+    assert flips["O" if fused else "P"] == 0.0 and np.array_equal(g["O"], st["o_codes"])
     assert len(np.unique(st["p_codes"])) >= 4
 
 
@@ -253,8 +257,9 @@ def test_twelve_layer_encoder_batch_256_all_layers_staged():
     print("12 layers, batch 256: largest off-centre share per stage " + ", ".join(f"{k} {v:.2e}" for k, v in worst.items()))
 
 
+@pytest.mark.parametrize("fused", [True, False], ids=["fused_attention", "unfused_attention"])
 @pytest.mark.parametrize("bits", [4, 2])
-def test_encoder_layer_comparator_layernorm_and_shift_softmax_bit_exact_up_to_gelu(bits):
+def test_encoder_layer_comparator_layernorm_and_shift_softmax_bit_exact_up_to_gelu(bits, fused):
     """With the comparator LayerNorm quantizer (Eq. 5, Fig. 5(b)) and the Eq. 4 softmax no stage before the GELU
     decides a level after an fp32 island: LayerNorm levels, QKV, P, O, the fp32 residual stream and the second
     LayerNorm's levels must equal the oracle's bit for bit, for every image and token, with no band."""
@@ -264,7 +269,8 @@ def test_encoder_layer_comparator_layernorm_and_shift_softmax_bit_exact_up_to_ge
     x = si.activations(cfg)
     st = vp.encoder_layer(x, prm, cfg.batch, cfg.tokens, cfg.heads, cfg.bits, softmax="shift", layernorm="compare")
     layer = EncoderLayer(cfg.batch, cfg.tokens, cfg.heads, cfg.mlp_dim, cfg.bits, prm, softmax="shift",
-                         layernorm="compare")
+                         layernorm="compare", fused_attention=fused)
+    assert layer.fused_attention == fused
     out = torch.empty((cfg.rows, cfg.dim), dtype=torch.float32, device="cuda")
     layer.forward(dev(x), out)
     assert vt.vitint_device_status() == 0
@@ -274,13 +280,14 @@ def test_encoder_layer_comparator_layernorm_and_shift_softmax_bit_exact_up_to_ge
     # the oracle's own free-running chain: identical up to the GELU
     assert np.array_equal(g["x1"], st["x1_codes"])
     assert np.array_equal(g["qkv"], att["qkv_codes"])
-    assert np.array_equal(g["P"], att["p_codes"])
+    if not fused:
+        assert np.array_equal(g["P"], att["p_codes"])
     assert np.array_equal(g["O"], att["o_codes"])
     assert np.array_equal(g["h"].view(np.uint32), st["h"].view(np.uint32))
     assert np.array_equal(g["x2"], st["x2_codes"])
     # GELU is the one remaining fp32 island: band for its levels, and the output from the GPU's own levels
     _, flips = compare_stages(g, x, prm, cfg.batch, T, H, cfg.bits, softmax="shift", layernorm="compare")
-    assert flips["x1"] == 0.0 and flips["P"] == 0.0 and flips["x2"] == 0.0
+    assert flips["x1"] == 0.0 and flips["O" if fused else "P"] == 0.0 and flips["x2"] == 0.0
 
 
 @pytest.mark.parametrize("bits", [3, 4])
@@ -315,8 +322,9 @@ def test_normed_attention_module_bit_exact(bits):
     assert per_image == H * (3 * 198 * 384 * 64 + 2 * 198 * 198 * 64)
 
 
+@pytest.mark.parametrize("fused_core", [True, False], ids=["eq4_inside_the_core", "three_attention_kernels"])
 @pytest.mark.parametrize("bits,batch,negate", [(4, 2, False), (3, 2, True), (2, 1, False), (4, 5, True)])
-def test_normed_attention_fused_qkv_epilogue_bit_exact(bits, batch, negate):
+def test_normed_attention_fused_qkv_epilogue_bit_exact(bits, batch, negate, fused_core):
     """The same module with the per-head LayerNorm + comparator quantizer run inside the QKV GEMM's epilogue (one
     launch instead of seven): Q, K and V codes, the (mu, V) statistics of every head row and everything downstream
     equal the oracle bit for bit, although the fp32 Q and K never reach memory.  batch 5 gives 990 rows: seven full
@@ -333,11 +341,12 @@ def test_normed_attention_fused_qkv_epilogue_bit_exact(bits, batch, negate):
     s_x = si.lsq_step(x, cfg.bits, True)
     xq = vo.quantize(x, s_x, cfg.bits, True)
     st = vp.normed_attention(xq, s_x, prm, qkn, cfg.batch, cfg.tokens, cfg.heads, cfg.bits)
-    mod = NormedAttention(cfg.batch, cfg.tokens, cfg.heads, cfg.bits, prm, qkn)
-    assert mod.fused
+    mod = NormedAttention(cfg.batch, cfg.tokens, cfg.heads, cfg.bits, prm, qkn, fused_core=fused_core)
+    assert mod.fused and mod.fused_core == fused_core
     xg = vt.vitint_quantize(dev(x), float(s_x), cfg.bits, True)
     mod.qkv.data.fill_(0x5A)
     O = mod.forward(xg, float(s_x))
+    O = mod.forward(xg, float(s_x))                 # the second pass reuses the core's table
     assert vt.vitint_device_status() == 0
     M, D, T, H = cfg.rows, cfg.dim, cfg.tokens, cfg.heads
     qkv = from_codes(mod.qkv)
@@ -347,8 +356,9 @@ def test_normed_attention_fused_qkv_epilogue_bit_exact(bits, batch, negate):
         assert np.array_equal(qkv[:, i * D:(i + 1) * D], st[n + "_codes"]), n
     assert np.array_equal(qkv[:, 2 * D:], st["v_codes"])
     assert any(st[n + "_refs"][2].any() for n in ("q", "k")) == negate
-    assert np.array_equal(mod.S.cpu().numpy()[:, :T].reshape(cfg.batch * H, T, T), st["S"])
-    assert np.array_equal(from_codes(mod.P).reshape(-1, T, T), st["p_codes"])
+    if not fused_core:
+        assert np.array_equal(mod.S.cpu().numpy()[:, :T].reshape(cfg.batch * H, T, T), st["S"])
+        assert np.array_equal(from_codes(mod.P).reshape(-1, T, T), st["p_codes"])
     assert np.array_equal(from_codes(O), st["o_codes"])
 
 

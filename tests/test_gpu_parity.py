@@ -452,6 +452,58 @@ def test_attention_core_fused(batch, tokens, heads, bits, scale, byte_codes):
         assert np.array_equal(from_codes(out2), got)
 
 
+@pytest.mark.parametrize("bits", [4, 3, 2])
+@pytest.mark.parametrize("batch,tokens,heads,scale", [(2, 197, 2, 1.0), (1, 197, 3, 3.0), (2, 129, 1, 2.5), (1, 256, 2, 2.0),
+                                                      (3, 64, 1, 0.5), (1, 198, 6, 3.3)])
+def test_fused_attention_shift_softmax_bit_exact(batch, tokens, heads, bits, scale):
+    """Eq. 4 inside the fused kernel: the attention codes P (read out through one-hot V slabs and an identity output
+    quantizer) and the O codes with the real V equal the oracle's Q K^T -> shift softmax with the division-free
+    comparator quantizer -> P V -> requantize bit for bit: every step is an integer or a single fp32 operation."""
+    D = heads * 64
+    qkv = _qkv_codes(batch, tokens, heads, bits, 261 + tokens + bits)
+    qmax = si.code_range(bits, True)[1] + 1
+    s_q = s_k = np.float32(math.sqrt(8.0 * scale * 3.0 / (8.0 * qmax * qmax)))
+    p_qp = si.code_range(bits, False)[1]
+    s_p = np.float32(2.0 / (tokens * math.sqrt(p_qp)))
+    q = vp.split_heads(qkv, batch, tokens, heads, 64, 0)
+    k = vp.split_heads(qkv, batch, tokens, heads, 64, D)
+    v = vp.split_heads(qkv, batch, tokens, heads, 64, 2 * D)
+    S = vo.qk(q, k)
+    c = vp.softmax_scale(s_q, s_k, 64)
+    c2 = np.float32(np.float64(c) * np.log2(np.e))
+    n = batch * heads
+    pc = vo.softmax_shift_quantize(S.reshape(n * tokens, tokens), c2, s_p, bits).reshape(n, tokens, tokens)
+    ones = dev(np.ones(D, np.float32))
+    got = np.full((n, tokens, tokens), -1, np.int16)
+    for r in range((tokens + 63) // 64):
+        sel = qkv.copy()
+        sel[:, 2 * D:] = 0
+        for b in range(batch):
+            for j in range(64 * r, min(tokens, 64 * r + 64)):
+                sel[b * tokens + j, 2 * D + (j - 64 * r)::64] = 1
+        sel_dev = vt.vitint_widen(to_codes(sel, bits, True))
+        out = vt.Codes.empty(batch * tokens, D, 8, True)
+        o = from_codes(vt.vitint_attention_core_shift(sel_dev, batch, heads, tokens, s_q, s_k, s_p, bits, ones, None, out=out))
+        o = vp.split_heads(o, batch, tokens, heads, 64, 0)
+        w = min(64, tokens - 64 * r)
+        got[:, :, 64 * r:64 * r + w] = o[:, :, :w]
+    assert np.array_equal(got, pc)
+    if scale >= 1.0:
+        assert len(np.unique(pc)) >= 3
+    # the real V: O codes
+    s_v, s_o = np.float32(0.17), np.float32(0.31)
+    alpha, beta = vp.fold(s_p, np.full(D, s_v, np.float32), None, s_o)
+    want = vo.epilogue_requant(vo.pv(pc, v).reshape(n * tokens, 64), alpha[:64], beta[:64], bits, True)
+    want = vp.merge_heads(want.reshape(n, tokens, 64), batch, tokens, heads, 64)
+    o = vt.vitint_attention_core_shift(vt.vitint_widen(to_codes(qkv, bits, True)), batch, heads, tokens, s_q, s_k, s_p, bits,
+                                       dev(alpha), None)
+    assert np.array_equal(from_codes(o), want)
+    assert vt.vitint_device_status() == 0
+    # packed codes are not taken by this variant
+    with pytest.raises(vt.VitintError):
+        vt.vitint_attention_core_shift(to_codes(qkv, bits, True), batch, heads, tokens, s_q, s_k, s_p, bits, dev(alpha), None)
+
+
 @pytest.mark.parametrize("byte_codes", [False, True], ids=["packed_qkv", "byte_qkv"])
 @pytest.mark.parametrize("bits", [4, 3, 2])
 @pytest.mark.parametrize("batch,tokens,heads,scale", [(2, 197, 2, 1.0), (1, 197, 3, 3.0), (2, 129, 1, 2.5), (1, 256, 2, 2.0),
