@@ -326,7 +326,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 uint32_t sg_lo = 0u, sg_hi = 0u;
                 auto term = [&](uint32_t score, bool valid) -> uint32_t {
                     const uint32_t idx = min((uint32_t)((int)score + P.smax), top);
-                    const uint32_t m24 = valid ? mtab[idx] : 0u;
+                    const uint32_t m24 = valid ? mtab[idx] : 0u;                       // a real entry is at least 2^23
                     const int sh = max((int)ftab[idx] + c0, -31);
                     const unsigned long long big = ((unsigned long long)m24 << 32) >> (32 - sh);
                     const uint32_t lo = (uint32_t)big, hi = (uint32_t)(big >> 32);
@@ -357,11 +357,13 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                 sigma = sx[row] + sx[128 + row];
                 const float sig_f = __ull2float_rn(sigma);
                 // pass 2: the code is the number of references fl32(fl32((k - 1/2) s_P) * Sigma) that float(E_j) exceeds.
-                // k0 = rint(E_j / (s_P Sigma)) is at most one off, so the two references around it decide:
-                // code = k0 - 1 + [E > ref(k0)] + [E > ref(k0 + 1)], references formed with the two fp32
-                // multiplications of the definition.
+                // k0 = rint(min(E_j / (s_P Sigma), Qp - 3/4)) is at most one off and never Qp, so the two references
+                // around it decide: code = k0 - 1 + [E > ref(k0)] + [E > ref(k0 + 1)], references formed with the two
+                // fp32 multiplications of the definition.  The sum is taken in the float that carries k0 in its low
+                // mantissa bits (1.5 * 2^23 - 1 + k0 + the two tests): small integers, exact.
                 const float inv = warp_live ? __frcp_rn(__fmul_rn(P.p_step, sig_f)) : 0.0f;
-                const f32x2 inv2 = f2_dup(inv), qp2 = f2_dup(P.p_qp), magic2 = f2_dup(12582912.0f), nmagic2 = f2_dup(-12582912.0f);
+                const float u_top = P.p_qp - 0.75f;
+                const f32x2 inv2 = f2_dup(inv), magic2 = f2_dup(12582912.0f), nmagic2 = f2_dup(-12582912.0f), neg1 = f2_dup(-1.0f);
                 const f32x2 half2 = f2_dup(0.5f), nhalf2 = f2_dup(-0.5f), ps2 = f2_dup(P.p_step), sg2 = f2_dup(sig_f);
                 uint8_t* const prow = ggen + P.off_p + row * 128;
                 const int sw = row & 7;
@@ -376,23 +378,21 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
 #pragma unroll
                         for (int j = 0; j < 4; j += 2) {
                             const float e0 = __uint_as_float(v[4 * i4 + j]), e1 = __uint_as_float(v[4 * i4 + j + 1]);
-                            const f32x2 e2 = f2_pack(e0, e1);
                             float u0, u1;
-                            f2_unpack(f2_mul(e2, inv2), u0, u1);
-                            const f32x2 um = f2_add(f2_pack(fminf(u0, P.p_qp), fminf(u1, P.p_qp)), magic2);   // 1.5*2^23 + k0
+                            f2_unpack(f2_mul(f2_pack(e0, e1), inv2), u0, u1);
+                            const f32x2 um = f2_add(f2_pack(fminf(u0, u_top), fminf(u1, u_top)), magic2);   // 1.5*2^23 + k0
                             const f32x2 kf = f2_add(um, nmagic2);
-                            const f32x2 r_lo = f2_mul(f2_mul(f2_add(kf, nhalf2), ps2), sg2);
-                            const f32x2 r_hi = f2_mul(f2_mul(f2_add(kf, half2), ps2), sg2);
-                            float m0, m1, l0, l1, h0, h1, k0f, k1f;
-                            f2_unpack(um, m0, m1);
-                            f2_unpack(r_lo, l0, l1);
-                            f2_unpack(r_hi, h0, h1);
-                            f2_unpack(kf, k0f, k1f);
-                            // (no reference above the last level: the upper test only counts below Qp)
-                            cb[j] = (__float_as_uint(m0) & 0xFFu) - 1u + (e0 > l0 ? 1u : 0u) + ((e0 > h0 && k0f < P.p_qp) ? 1u : 0u);
-                            cb[j + 1] = (__float_as_uint(m1) & 0xFFu) - 1u + (e1 > l1 ? 1u : 0u) + ((e1 > h1 && k1f < P.p_qp) ? 1u : 0u);
+                            float l0, l1, h0, h1;
+                            f2_unpack(f2_mul(f2_mul(f2_add(kf, nhalf2), ps2), sg2), l0, l1);
+                            f2_unpack(f2_mul(f2_mul(f2_add(kf, half2), ps2), sg2), h0, h1);
+                            const f32x2 t_lo = f2_pack(e0 > l0 ? 1.0f : 0.0f, e1 > l1 ? 1.0f : 0.0f);
+                            const f32x2 t_hi = f2_pack(e0 > h0 ? 1.0f : 0.0f, e1 > h1 ? 1.0f : 0.0f);
+                            float c0f, c1f;
+                            f2_unpack(f2_add(f2_add(um, neg1), f2_add(t_lo, t_hi)), c0f, c1f);
+                            cb[j] = __float_as_uint(c0f);                                          // code in the low byte
+                            cb[j + 1] = __float_as_uint(c1f);
                         }
-                        wd[i4] = cb[0] | (cb[1] << 8) | (cb[2] << 16) | (cb[3] << 24);
+                        wd[i4] = __byte_perm(__byte_perm(cb[0], cb[1], 0x4040), __byte_perm(cb[2], cb[3], 0x4040), 0x5410);
                     }
                     const int cc = 2 * ch;
                     uint8_t* const blk = prow + (cc >> 3) * 16384;
