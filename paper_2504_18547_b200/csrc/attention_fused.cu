@@ -307,9 +307,13 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     uint32_t v[32];
                     ptx::tmem_ld32(t_row + (uint32_t)(ch * 32), v);
                     ptx::tmem_ld_wait();
+                    if (ch < full_chunks) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        smx = max(smx, (ch < full_chunks || ch * 32 + i < T) ? (int)v[i] : INT_MIN);
+                        for (int i = 0; i < 32; ++i) smx = max(smx, (int)v[i]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) smx = max(smx, ch * 32 + i < T ? (int)v[i] : INT_MIN);
+                    }
                 }
                 mx[hf * 128 + row] = smx;
                 ptx::mbar_arrive(ptx::smem_addr(&B.z_sync));
@@ -333,7 +337,7 @@ attention_fused_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
                     asm("add.cc.u32 %0, %0, %2;\n\taddc.u32 %1, %1, %3;" : "+r"(sg_lo), "+r"(sg_hi) : "r"(lo), "r"(hi));
                     const uint32_t up = m24 + 0x4A800000u + ((uint32_t)sh << 23);
                     const uint32_t dn = __float_as_uint(__fadd_rn(__uint_as_float(0x4B000000u + lo), -8388608.0f));
-                    return m24 == 0u ? 0u : (sh >= 0 ? up : dn);
+                    return valid ? (sh >= 0 ? up : dn) : 0u;
                 };
                 for (int ch = hf; warp_live && ch < chunks; ch += 2) {
                     uint32_t v[32];
