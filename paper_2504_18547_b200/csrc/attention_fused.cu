@@ -591,6 +591,11 @@ extern "C" size_t vitint_attention_core_workspace_bytes(int32_t bits) {
     return (size_t)(2 * 64 * m * m + 1) * sizeof(float) + 256;
 }
 
+namespace vitint {
+int attention_long_launch(const vitint_codes* qkv, int batch, int heads, int tokens, int smax, const float* table, float p_step,
+                          float p_qp, const float* alpha_o, const float* beta_o, const vitint_codes* o_out, cudaStream_t st);
+}
+
 // Shared by the three entry points below.  build_table: fill `workspace` with the exp table first (one more
 // small launch); otherwise the caller has filled it for exactly these steps and bits (vitint_attention_exp_table).
 static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t heads, int32_t tokens,
@@ -606,8 +611,11 @@ static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t
     const float steps[3] = {q_step, k_step, p_step};
     for (float s : steps) if (!(s > 0.0f && s < INFINITY)) return VITINT_ERR_INVALID_ARG;
     if (!valid_bits(p_bits)) return VITINT_ERR_INVALID_ARG;
-    if (qkv->bits == 8 || tokens > 256 || batch > 65535) return VITINT_ERR_UNSUPPORTED;
+    if (qkv->bits == 8 || batch > 65535) return VITINT_ERR_UNSUPPORTED;
     const int c = codes_container(qkv);                  // 2 / 4: packed; 8: one code per byte
+    // beyond 256 tokens S no longer fits tensor memory beside O: the chunked two-pass kernel (byte-stored codes, exp table)
+    const bool long_seq = tokens > 256;
+    if (long_seq && (shift || c != 8 || tokens > 4096)) return VITINT_ERR_UNSUPPORTED;
     const int m = 1 << (container_bits(qkv->bits) - 1);
     const int smax = 64 * m * m;
     const float cs = (float)((double)q_step * (double)k_step / 8.0);
@@ -624,6 +632,16 @@ static int attention_core_launch(const vitint_codes* qkv, int32_t batch, int32_t
                                  : vitint_attention_core_workspace_bytes(qkv->bits)))
         return VITINT_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    if (long_seq) {
+        if (build_table) {
+            launch_kernel(exp_table_kernel, dim3((2 * smax + 1 + 255) / 256), dim3(256), 0, st, (float*)workspace, smax, cs);
+            if (cudaGetLastError() != cudaSuccess) return VITINT_ERR_CUDA;
+        }
+        int pqn, pqp;
+        code_range(p_bits, 0, &pqn, &pqp);
+        return attention_long_launch(qkv, batch, heads, tokens, smax, (const float*)workspace, p_step, (float)pqp, alpha_o,
+                                     beta_o, o_out, st);
+    }
 
     AttnParams P{};
     P.batch = batch; P.heads = heads; P.tokens = tokens;

@@ -40,8 +40,10 @@ class EncoderLayer:
         self.layernorm = layernorm
         # the shift-based softmax is a separate kernel: it runs in the unfused attention pipeline
         # the fused core takes the exp softmax for any container and the Eq. 4 softmax for byte-stored codes
-        self.fused_attention = (fused_attention and bits != 8 and tokens <= 256
-                                and (softmax == "exp" or (softmax == "shift" and wide_activations)))
+        # (beyond 256 tokens the exp core runs its chunked two-pass kernel, which takes byte-stored codes)
+        self.fused_attention = (fused_attention and bits != 8
+                                and ((softmax == "exp" and (tokens <= 256 or (wide_activations and tokens <= 4096)))
+                                     or (softmax == "shift" and wide_activations and tokens <= 256)))
         self.stages = STAGES_FUSED if self.fused_attention else STAGES_UNFUSED
         d = lambda a: _dev(a, device)
         f = lambda k: float(prm[k])

@@ -400,11 +400,18 @@ def test_softmax_error_statistics_on_attention_like_rows():
 @pytest.mark.parametrize("byte_codes", [False, True], ids=["packed_qkv", "byte_qkv"])
 @pytest.mark.parametrize("bits", [4, 2, 3])
 @pytest.mark.parametrize("batch,tokens,heads,scale", [(1, 197, 3, 1.0), (3, 197, 2, 3.0), (2, 50, 1, 3.0), (1, 256, 2, 2.0),
-                                                      (5, 128, 1, 0.3), (2, 129, 2, 2.5)])
+                                                      (5, 128, 1, 0.3), (2, 129, 2, 2.5), (1, 577, 2, 2.0), (2, 785, 1, 2.5),
+                                                      (3, 257, 1, 1.0), (1, 1000, 1, 1.5)])
 def test_attention_core_fused(batch, tokens, heads, bits, scale, byte_codes):
     """Fused Q K^T -> softmax -> P V against the oracle stages; rows whose P codes are unique must be bit-exact.
-    The Q, K, V codes arrive bit-packed (unpacked inside the kernel) or one per byte (the TMA copy is the operand)."""
+    The Q, K, V codes arrive bit-packed (unpacked inside the kernel) or one per byte (the TMA copy is the operand).
+    Beyond 256 tokens the chunked two-pass kernel runs (byte-stored codes; packed codes are declined)."""
     D = heads * 64
+    if tokens > 256 and not byte_codes:
+        with pytest.raises(vt.VitintError):
+            vt.vitint_attention_core(to_codes(_qkv_codes(1, tokens, heads, bits, 3), bits, True), 1, heads, tokens, 0.1, 0.1,
+                                     0.01, bits, dev(np.ones(D, np.float32)), None)
+        return
     qkv = _qkv_codes(batch, tokens, heads, bits, 61 + tokens)
     qmax = si.code_range(bits, True)[1] + 1
     # random codes give scores with spread ~ 8*qmax^2/3; choose the steps so the logits' spread is `scale`
@@ -507,7 +514,7 @@ def test_fused_attention_shift_softmax_bit_exact(batch, tokens, heads, bits, sca
 @pytest.mark.parametrize("byte_codes", [False, True], ids=["packed_qkv", "byte_qkv"])
 @pytest.mark.parametrize("bits", [4, 3, 2])
 @pytest.mark.parametrize("batch,tokens,heads,scale", [(2, 197, 2, 1.0), (1, 197, 3, 3.0), (2, 129, 1, 2.5), (1, 256, 2, 2.0),
-                                                      (3, 64, 1, 0.5)])
+                                                      (3, 64, 1, 0.5), (1, 577, 1, 2.0), (1, 300, 2, 1.0)])
 def test_fused_attention_p_codes(batch, tokens, heads, bits, scale, byte_codes):
     """The attention codes P that the fused kernel forms on the SM (table-driven softmax, no max subtraction,
     two-float reciprocal), read out exactly and compared element by element with the oracle's band.
@@ -515,6 +522,8 @@ def test_fused_attention_p_codes(batch, tokens, heads, bits, scale, byte_codes):
     output quantizer is the identity (alpha 1, beta 0, 8-bit signed output), so O[i][c] = P[i][c + 64 r]; one
     call per r covers every column."""
     D = heads * 64
+    if tokens > 256 and not byte_codes:
+        pytest.skip("the long-sequence kernel takes byte-stored codes")
     qkv = _qkv_codes(batch, tokens, heads, bits, 161 + tokens + bits)
     qmax = si.code_range(bits, True)[1] + 1
     s_q = s_k = np.float32(math.sqrt(8.0 * scale * 3.0 / (8.0 * qmax * qmax)))
