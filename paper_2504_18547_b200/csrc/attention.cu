@@ -11,7 +11,7 @@ namespace {
 
 struct AttnLayout {
     int64_t M, D, n_rows_p;
-    int64_t pitch_qkv, pitch_p, pitch_o, ld_s;
+    int64_t pitch_qkv, pitch_qkv_wide, pitch_p, pitch_o, ld_s;
     size_t off_qkv, off_s, off_p, off_o, off_tab, tab_bytes, total;
 };
 
@@ -28,7 +28,10 @@ int attn_layout(const vitint_attention_desc* d, AttnLayout* L) {
     L->pitch_p = vitint_packed_pitch(d->tokens, d->p_bits);
     L->ld_s = ((int64_t)d->tokens + 3) / 4 * 4;
     size_t off = 0;
-    L->off_qkv = off; off = align256(off + (size_t)(L->M * L->pitch_qkv));
+    // beyond 256 tokens the fused core takes QKV stored one code per byte: room for that form
+    L->pitch_qkv_wide = vitint_packed_pitch(3 * L->D, 8);
+    const int64_t pq = d->tokens > 256 ? L->pitch_qkv_wide : L->pitch_qkv;
+    L->off_qkv = off; off = align256(off + (size_t)(L->M * pq));
     L->off_s = off;   off = align256(off + (size_t)(L->n_rows_p * L->ld_s) * 4);
     L->off_p = off;   off = align256(off + (size_t)(L->n_rows_p * L->pitch_p));
     L->off_o = off;   off = align256(off + (size_t)(L->M * L->pitch_o));
@@ -84,11 +87,16 @@ extern "C" int vitint_attention_block(const vitint_codes* x, const vitint_attent
     uint8_t* ws = (uint8_t*)workspace;
     const int cbits = container_bits(d->bits);
 
-    // 1. QKV linear, requantized per output channel (three per-tensor steps)
-    vitint_codes qkv{ws + L.off_qkv, L.M, 3 * L.D, L.pitch_qkv, d->bits, 1, 0, 0};
+    // 1. QKV linear, requantized per output channel (three per-tensor steps).  Beyond 256 tokens, when no copy of QKV
+    // or P is asked for and the logits' range allows the table-driven core, the codes are stored one per byte: the form
+    // the chunked two-pass core takes (S and P then never reach HBM).
+    const int mq = 1 << (d->bits - 1);
+    const bool wide_qkv = d->tokens > 256 && d->tokens <= 4096 && !dbg_qkv && !dbg_p && L.tab_bytes && d->bits != 8 &&
+                          64.0 * mq * mq * (double)(float)((double)d->q_step * (double)d->k_step / 8.0) <= 80.0;
+    vitint_codes qkv{ws + L.off_qkv, L.M, 3 * L.D, wide_qkv ? L.pitch_qkv_wide : L.pitch_qkv, d->bits, 1, wide_qkv ? 8 : 0, 0};
     vitint_epilogue e1{};
     e1.mode = VITINT_EPI_REQUANT; e1.alpha = d->alpha_qkv; e1.beta = d->beta_qkv;
-    e1.out_bits = d->bits; e1.out_signed = 1;
+    e1.out_bits = d->bits; e1.out_signed = 1; e1.out_container_bits = wide_qkv ? 8 : 0;
     if (int rc = vitint_linear(x, 1.0f, &d->w_qkv, nullptr, nullptr, &e1, qkv.data, qkv.pitch_bytes, stream)) return rc;
     if (int rc = copy_codes(dbg_qkv, qkv.data, L.pitch_qkv, L.M, row_bytes(3 * L.D, d->bits), st)) return rc;
 
@@ -99,6 +107,7 @@ extern "C" int vitint_attention_block(const vitint_codes* x, const vitint_attent
         fused = vitint_attention_core(&qkv, d->batch, d->heads, d->tokens, d->q_step, d->k_step, d->p_step, d->p_bits,
                                       d->alpha_o, d->beta_o, &o, ws + L.off_tab, L.tab_bytes, stream);
     if (fused != VITINT_OK && fused != VITINT_ERR_UNSUPPORTED) return fused;
+    if (fused == VITINT_ERR_UNSUPPORTED && wide_qkv) return fused;      // (the unfused kernels read bit-packed slabs)
     if (fused == VITINT_ERR_UNSUPPORTED) {
         // 2. S = Q K^T per (image, head)
         const int64_t head_bytes = 64 * cbits / 8, seg_bytes = L.D * cbits / 8;

@@ -167,7 +167,7 @@ def test_attention_block_full_size_sampled_images():
     _attention_block_sampled(cfg, [0, 31, 63])
 
 
-def _attention_block_sampled(cfg, images, want_p=False, tag=""):
+def _attention_block_sampled(cfg, images, want_p=False, tag="", fused_core=False):
     prm = si.layer_parameters(cfg)
     x = si.activations(cfg)
     s_x = si.lsq_step(x, cfg.bits, True)
@@ -217,16 +217,64 @@ def _attention_block_sampled(cfg, images, want_p=False, tag=""):
     # projection recomputed from the GPU's own O codes, bit for bit on every element
     want = vo.epilogue_requant(vo.matmul_i32(go, st["w_proj_codes"]), st["alpha_proj"], st["beta_proj"], cfg.bits, True)
     assert np.array_equal(_code_rows(outc, images, T), want)
+    if fused_core:
+        # the same QKV codes, stored one per byte, through the fused core (beyond 256 tokens: keys in chunks, two
+        # passes): O of the sampled images inside the interval that the oracle's P band can reach
+        o2 = vt.vitint_attention_core(vt.vitint_widen(dq), cfg.batch, H, T, float(prm["s_q"]), float(prm["s_k"]),
+                                      float(prm["s_p"]), cfg.bits, dev(np.tile(a_o, H)), None)
+        assert vt.vitint_device_status() == 0
+        g2 = _code_rows(o2, images, T)
+        lo, hi = vp.o_band_from_p_band(st["p_lo"], st["p_hi"], v, a_o, cfg.bits)
+        lo, hi = (vp.merge_heads(a.reshape(n, T, 64), B, T, H, 64) for a in (lo, hi))
+        assert np.all(g2 >= lo) and np.all(g2 <= hi)
+        assert (lo == hi).mean() > 0.9
+        assert float((g2 != st["o_codes"]).mean()) < 0.05
     print(f"{tag}{cfg.name}: off-centre share {'P' if want_p else 'O'} {flip_p:.2e}")
 
 
 @pytest.mark.parametrize("tokens,bits", [(577, 4), (785, 4), (785, 2), (577, 3)])
 def test_attention_block_long_sequences_batch_32(tokens, bits):
     """The token counts of the scaling study beyond one accumulator tile (577 and 785 tokens) at batch 32, through
-    vitint_attention_block (which runs Q K^T, the softmax kernel and P V unfused there): QKV, P (inside the
-    band), O from the GPU's own P codes and the projection, every element of the sampled images."""
+    vitint_attention_block (which runs Q K^T, the softmax kernel and P V unfused there, a copy of P being asked
+    for): QKV, P (inside the band), O from the GPU's own P codes and the projection, every element of the sampled
+    images; and the same QKV codes through the fused core, whose chunked two-pass kernel keeps S and P on the SM."""
     cfg = si.VIT_SMALL_BLOCK.with_(batch=32, tokens=tokens, bits=bits, name=f"vit_small_attn_b32_t{tokens}")
-    _attention_block_sampled(cfg, [0, 31], want_p=True)
+    _attention_block_sampled(cfg, [0, 31], want_p=True, fused_core=True)
+
+
+@pytest.mark.parametrize("tokens", [577, 300])
+def test_attention_block_long_sequences_take_the_fused_core(tokens):
+    """Without a copy of QKV or P asked for, vitint_attention_block beyond 256 tokens stores QKV one code per byte and
+    runs the chunked fused core: O inside the interval the oracle's P band can reach, the projection recomputed from
+    the GPU's own O codes bit for bit."""
+    cfg = si.VIT_SMALL_BLOCK.with_(batch=2, tokens=tokens, name=f"vit_small_attn_b2_t{tokens}")
+    prm = si.layer_parameters(cfg)
+    x = si.activations(cfg)
+    s_x = si.lsq_step(x, cfg.bits, True)
+    T, H, D, B = cfg.tokens, cfg.heads, cfg.dim, cfg.batch
+    xq = vo.quantize(x, s_x, cfg.bits, True)
+    st = vp.attention_block(xq, s_x, prm, B, T, H, cfg.bits, proj="requant")
+    from gpu_util import to_codes
+    aw = vt.AttentionWeights(
+        batch=B, tokens=T, heads=H, bits=cfg.bits, w_qkv=to_codes(st["w_qkv_codes"], cfg.bits, True),
+        alpha_qkv=dev(st["alpha_qkv"]), beta_qkv=dev(st["beta_qkv"]), q_step=float(prm["s_q"]),
+        k_step=float(prm["s_k"]), v_step=float(prm["s_v"]), p_step=float(prm["s_p"]), o_step=float(prm["s_o"]),
+        p_bits=cfg.bits, alpha_o=dev(np.tile(st["alpha_o"], H)), beta_o=None,
+        w_proj=to_codes(st["w_proj_codes"], cfg.bits, True), w_proj_step=dev(prm["s_w_proj"]), b_proj=dev(prm["b_proj"]),
+        proj_epi=vt.Epilogue(mode=vt.EPI_REQUANT, alpha=dev(st["alpha_proj"]), beta=dev(st["beta_proj"]),
+                             out_bits=cfg.bits, out_signed=True))
+    xg = vt.vitint_quantize(dev(x), float(s_x), cfg.bits, True)
+    do = vt.Codes.empty(cfg.rows, D, cfg.bits, True)
+    outc = vt.vitint_attention_block(xg, aw, dbg_o=do)
+    assert vt.vitint_device_status() == 0
+    go = from_codes(do)
+    n = B * H
+    v = vp.split_heads(st["qkv_codes"], B, T, H, 64, 2 * D)
+    lo, hi = vp.o_band_from_p_band(st["p_lo"], st["p_hi"], v, st["alpha_o"], cfg.bits)
+    lo, hi = (vp.merge_heads(a.reshape(n, T, 64), B, T, H, 64) for a in (lo, hi))
+    assert np.all(go >= lo) and np.all(go <= hi) and (lo == hi).mean() > 0.9
+    want = vo.epilogue_requant(vo.matmul_i32(go, st["w_proj_codes"]), st["alpha_proj"], st["beta_proj"], cfg.bits, True)
+    assert np.array_equal(from_codes(outc), want)
 
 
 def test_twelve_layer_encoder_batch_256_all_layers_staged():
