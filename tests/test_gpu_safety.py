@@ -116,6 +116,21 @@ def test_outputs_stay_inside_their_buffers():
                 vt.vitint_attention_core(vt.vitint_widen(c) if wide else c, batch, heads, tokens, 0.2, 0.2, 2.0 / (tokens * 3.8), 4,
                                          alpha, None, out=oo)
                 assert padding_is_zero(oo)
+                if wide:
+                    # the Eq. 4 variant of the core, same buffers
+                    o4 = guarded_codes(batch * tokens, D, ob, True, oc, pitch)
+                    vt.vitint_attention_core_shift(vt.vitint_widen(c), batch, heads, tokens, 0.2, 0.2, 2.0 / (tokens * 3.8), 4,
+                                                   alpha, None, out=o4)
+                    assert padding_is_zero(o4)
+    # the chunked core beyond 256 tokens (byte-stored codes): ragged last chunk and last query tile
+    for batch, tokens, heads in ((1, 300, 2), (2, 257, 1), (1, 577, 1)):
+        D = heads * 64
+        c8 = vt.vitint_widen(to_codes(rand_codes(51 + tokens, (batch * tokens, 3 * D), 4, True), 4, True))
+        alpha = dev(np.full(D, 0.01, np.float32))
+        for ob, oc, pitch in ((4, 0, None), (4, 8, None), (4, 0, D // 2 + 32), (2, 0, None)):
+            oo = guarded_codes(batch * tokens, D, ob, True, oc, pitch)
+            vt.vitint_attention_core(c8, batch, heads, tokens, 0.2, 0.2, 2.0 / (tokens * 3.8), 4, alpha, None, out=oo)
+            assert padding_is_zero(oo)
     # glue
     for rows, cols in ((1, 4), (197, 192), (37, 100)):
         x = si.normal(31 + cols, (rows, cols), 0.5, 1.5)
