@@ -14,6 +14,7 @@
 //                              and false after it: the count is found by bisection (b comparisons for
 //                              2^b - 1 references) with the candidate references kept in registers.
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace vitint {
 namespace {
@@ -21,7 +22,6 @@ namespace {
 constexpr int LNC_ROWS_PER_THREAD = 16;
 constexpr int LNC_BATCH = 4;            // rows whose loads are issued together
 
-constexpr int LNS_PREFETCH_LINES = 6; // 128-byte lines of a row requested into L2 ahead of the register loads
 constexpr int LNS_MAX_COLS = 4096;    // (float(i), RN(1/i)) pairs tabulated in shared memory
 
 // One step of Eq. 5 for element xi, i = fi: every operation a single rounded fp32 one.  The update of S
@@ -42,68 +42,86 @@ __device__ __forceinline__ void running_step(float xi, float fi, float r, float&
     px = xi;
 }
 
+// One warp per 32 rows, a thread walks one row -- but the row reaches the thread through shared memory: the warp
+// copies a 128-column chunk of its 32 rows with coalesced 16-byte asynchronous copies (lane l takes the l-th float4 of
+// every row: 512 contiguous bytes per row) into a [32][132]-float buffer, and each thread then reads its own row from
+// there (132 floats per row: the lanes' 16-byte reads fall on different bank groups).  Read straight from global
+// memory, every load instruction of the warp touched 32 different lines, and the load path took as long as the
+// dependent chain itself.  Two buffers: the next chunk is on its way while this one is walked.
+constexpr int LNS_CHUNK = 128;                 // columns per staged chunk
+constexpr int LNS_ROW_FLOATS = LNS_CHUNK + 4;  // padded row of the staging buffer
 __global__ void __launch_bounds__(32)
 ln_running_stats_kernel(const float* __restrict__ x, int64_t rows, int cols, int64_t ldx, float n_eps,
                         float* __restrict__ stats) {
     // (float(i), RN(1/i)) for every column: one broadcast shared-memory read per element instead of a
     // conversion and a reciprocal (both run on the quarter-rate unit) in front of the dependent chain
-    extern __shared__ float2 inv_tab[];
-    for (int i = threadIdx.x; i < cols; i += 32) {
+    extern __shared__ __align__(16) float2 inv_tab[];
+    float* const stage = reinterpret_cast<float*>(inv_tab + ((cols + 1) & ~1));          // 16-byte aligned behind the table
+    const int lane = threadIdx.x;
+    for (int i = lane; i < cols; i += 32) {
         const float fi = (float)(i + 1);
         inv_tab[i] = make_float2(fi, __frcp_rn(fi));
     }
     __syncwarp();
     grid_dependency_wait();        // x may come from the previous kernel of the stream
     grid_dependency_launch();
-    const int64_t row = (int64_t)blockIdx.x * 32 + threadIdx.x;
-    if (row >= rows) return;
-    const float4* xr = reinterpret_cast<const float4*>(x + row * ldx);
-    const int nv = cols >> 2, nv_full = nv & ~7;
-    float mu = 0.0f, S = 0.0f, pd = 0.0f, px = 0.0f;
-    // With one thread per row only a few megabytes would be in flight; the lines further ahead are therefore
-    // requested into L2 (one prefetch per 128-byte line), so the register loads below find them there.
-#pragma unroll
-    for (int a = 1; a < 1 + LNS_PREFETCH_LINES; ++a)
-        if (8 * a < nv) asm volatile("prefetch.global.L2 [%0];" ::"l"(xr + 8 * a));
-    // whole 128-byte lines: eight 16-byte loads are requested while the previous line is walked
-    float4 cur[8], nxt[8];
-    if (nv_full > 0) {
-#pragma unroll
-        for (int k = 0; k < 8; ++k) cur[k] = __ldg(xr + k);
-    }
-    for (int v0 = 0; v0 < nv_full; v0 += 8) {
-        if (v0 + 8 * (1 + LNS_PREFETCH_LINES) < nv)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(xr + v0 + 8 * (1 + LNS_PREFETCH_LINES)));
-        if (v0 + 8 < nv_full) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) nxt[k] = __ldg(xr + v0 + 8 + k);
-        }
-        const float2* tab = inv_tab + 4 * v0;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const float e[4] = {cur[k].x, cur[k].y, cur[k].z, cur[k].w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float2 t = tab[4 * k + j];
-                running_step(e[j], t.x, t.y, mu, S, pd, px);
+    const int64_t row0 = (int64_t)blockIdx.x * 32;
+    const int n_chunks = (cols + LNS_CHUNK - 1) / LNS_CHUNK;
+    auto request = [&](int c, float* buf) {
+        const int col = c * LNS_CHUNK + lane * 4;
+        if (col < cols) {                                                              // cols is a multiple of 4
+#pragma unroll 8
+            for (int r = 0; r < 32; ++r) {
+                const int64_t row = row0 + r < rows ? row0 + r : rows - 1;             // a surplus row repeats the last one
+                ptx::cp_async16(ptx::smem_addr(buf + r * LNS_ROW_FLOATS + lane * 4), x + row * ldx + col);
             }
         }
-#pragma unroll
-        for (int k = 0; k < 8; ++k) cur[k] = nxt[k];
-    }
-    // the last, partial line
-    for (int v = nv_full; v < nv; ++v) {
-        const float4 c4 = __ldg(xr + v);
-        const float e[4] = {c4.x, c4.y, c4.z, c4.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float2 t = inv_tab[4 * v + j];
-            running_step(e[j], t.x, t.y, mu, S, pd, px);
+        ptx::cp_async_commit();
+    };
+    float mu = 0.0f, S = 0.0f, pd = 0.0f, px = 0.0f;
+    request(0, stage);
+    for (int c = 0; c < n_chunks; ++c) {
+        float* const buf = stage + (c & 1) * 32 * LNS_ROW_FLOATS;
+        if (c + 1 < n_chunks) {
+            request(c + 1, stage + ((c + 1) & 1) * 32 * LNS_ROW_FLOATS);
+            ptx::cp_async_wait<1>();
+        } else {
+            ptx::cp_async_wait<0>();
         }
+        __syncwarp();                                                                  // every lane's copies have landed
+        const float4* mine = reinterpret_cast<const float4*>(buf + lane * LNS_ROW_FLOATS);
+        const float2* tab = inv_tab + c * LNS_CHUNK;
+        const int nv = (cols - c * LNS_CHUNK < LNS_CHUNK ? cols - c * LNS_CHUNK : LNS_CHUNK) >> 2;
+        if (nv == LNS_CHUNK / 4) {
+#pragma unroll 8
+            for (int v = 0; v < LNS_CHUNK / 4; ++v) {
+                const float4 e4 = mine[v];
+                const float e[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float2 t = tab[4 * v + j];
+                    running_step(e[j], t.x, t.y, mu, S, pd, px);
+                }
+            }
+        } else {
+            for (int v = 0; v < nv; ++v) {
+                const float4 e4 = mine[v];
+                const float e[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float2 t = tab[4 * v + j];
+                    running_step(e[j], t.x, t.y, mu, S, pd, px);
+                }
+            }
+        }
+        __syncwarp();                                                                  // the buffer is free for the chunk after next
     }
     S = __fadd_rn(S, __fmul_rn(pd, __fadd_rn(px, -mu)));      // the last element's term
-    stats[2 * row] = mu;
-    stats[2 * row + 1] = __fadd_rn(S, n_eps);
+    const int64_t row = row0 + lane;
+    if (row < rows) {
+        stats[2 * row] = mu;
+        stats[2 * row + 1] = __fadd_rn(S, n_eps);
+    }
 }
 
 // Block (32, 4): lane = four adjacent columns, threadIdx.y = a group of LNC_ROWS_PER_THREAD rows.
@@ -228,7 +246,11 @@ extern "C" int vitint_layernorm_compare_quantize(const float* x, int64_t rows, i
     int qn, qp;
     code_range(out->bits, out->is_signed, &qn, &qp);
     cudaStream_t st = (cudaStream_t)stream;
-    launch_kernel(ln_running_stats_kernel, dim3((unsigned)((rows + 31) / 32)), dim3(32), (size_t)cols * sizeof(float2), st, x, rows, (int)cols, ldx,
+    const size_t stats_smem = (size_t)((cols + 1) & ~(int64_t)1) * sizeof(float2) + 2 * 32 * LNS_ROW_FLOATS * sizeof(float);
+    if (stats_smem > 48 * 1024 &&
+        cudaFuncSetAttribute(ln_running_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stats_smem) != cudaSuccess)
+        return VITINT_ERR_CUDA;
+    launch_kernel(ln_running_stats_kernel, dim3((unsigned)((rows + 31) / 32)), dim3(32), stats_smem, st, x, rows, (int)cols, ldx,
                   n_eps, stats);
     if (int rc = cuda_status(cudaGetLastError())) return rc;
     const int64_t row_groups = (rows + 4 * LNC_ROWS_PER_THREAD - 1) / (4 * LNC_ROWS_PER_THREAD);
