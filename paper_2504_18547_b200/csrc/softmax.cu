@@ -361,7 +361,9 @@ softmax_shift_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int c
             const float z = __fmul_rn((float)sv[i], c2);
             const float fl = floorf(z);
             const float res = __fsub_rn(z, fl);
-            mant[k][i] = (uint32_t)__fmul_rn(__fadd_rn(1.0f, res), 8388608.0f);
+            // trunc((1 + res) * 2^23): 1 + res lies in [1, 2], so this is its mantissa with the hidden bit, read off the
+            // float's bits (2^24 when the sum rounds to 2) -- no conversion instruction
+            mant[k][i] = __float_as_uint(__fadd_rn(1.0f, res)) - 0x3F000000u;
             fi[k][i] = (int)fl;
             if (col + i < cols) m = max(m, fi[k][i]);
             else mant[k][i] = 0u;
@@ -389,12 +391,12 @@ softmax_shift_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int c
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sigma += __shfl_xor_sync(0xffffffffu, sigma, o);
     const float sig_f = __ull2float_rn(sigma);
-    // The comparator references fl32(fl32((t - 1/2) * step) * Sigma), t = 1 .. 2^bits - 1, depend on the row only:
-    // formed once per row and kept in registers (entries past the code range stay +inf and are never exceeded).
-    float thr[16];
-#pragma unroll
-    for (int tcode = 1; tcode < 16; ++tcode)
-        thr[tcode] = tcode < (1 << code_bits) ? __fmul_rn(__fmul_rn(__fsub_rn((float)tcode, 0.5f), p_step), sig_f) : INFINITY;
+    // The code is the number of comparator references fl32(fl32((t - 1/2) * step) * Sigma), t = 1 .. 2^bits - 1, that
+    // float(E) exceeds.  k0 = rint(min(E / (step * Sigma), Qp - 3/4)) is at most one off and never Qp, so the two
+    // references around it decide: code = k0 - 1 + [E > ref(k0)] + [E > ref(k0 + 1)], each reference formed with the
+    // definition's two fp32 multiplications.
+    const float inv = __frcp_rn(__fmul_rn(p_step, sig_f));
+    const float u_top = (float)((1 << code_bits) - 1) - 0.75f;
 
     constexpr uint32_t MASK = (1u << C) - 1u;
     const int chunk_bytes = 32 * C;
@@ -407,31 +409,16 @@ softmax_shift_quantize_kernel(const int32_t* __restrict__ s, int64_t rows, int c
                 if (u == k) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
+                        // float(E): E is a 24-bit mantissa times a power of two, or (shifted right) an integer below
+                        // 2^24 -- both convert exactly (putting the float together from its bits in the loop above
+                        // instead was measured slower: 162 against 149 us)
                         const unsigned long long e = ((unsigned long long)(uint32_t)fi[u][i] << 32) | mant[u][i];
                         const float e_f = __ull2float_rn(e);
-                        // the references ascend, so the number exceeded is found bit by bit; with the candidates in
-                        // registers each step is one comparison and a halving of the candidate list by selects
-                        uint32_t code = 0;
-                        if (code_bits > 4) {
-                            // wide codes: the references are formed on the fly, one comparison per code bit
-                            for (int b = code_bits - 1; b >= 0; --b) {
-                                const uint32_t tc = code | (1u << b);
-                                const float th = __fmul_rn(__fmul_rn(__fsub_rn((float)tc, 0.5f), p_step), sig_f);
-                                code = (e_f > th) ? tc : code;
-                            }
-                        } else {
-                        float cand[7];
-                        const bool p3 = e_f > thr[8];
-#pragma unroll
-                        for (int j = 0; j < 7; ++j) cand[j] = p3 ? thr[9 + j] : thr[1 + j];
-                        const bool p2 = e_f > cand[3];
-#pragma unroll
-                        for (int j = 0; j < 3; ++j) cand[j] = p2 ? cand[4 + j] : cand[j];
-                        const bool p1 = e_f > cand[1];
-                        cand[0] = p1 ? cand[2] : cand[0];
-                        const bool p0 = e_f > cand[0];
-                        code = (p3 ? 8u : 0u) + (p2 ? 4u : 0u) + (p1 ? 2u : 0u) + (p0 ? 1u : 0u);
-                        }
+                        const float um = __fadd_rn(fminf(__fmul_rn(e_f, inv), u_top), 12582912.0f);   // 1.5*2^23 + k0
+                        const float kf = __fadd_rn(um, -12582912.0f);
+                        const float r_lo = __fmul_rn(__fmul_rn(__fadd_rn(kf, -0.5f), p_step), sig_f);
+                        const float r_hi = __fmul_rn(__fmul_rn(__fadd_rn(kf, 0.5f), p_step), sig_f);
+                        uint32_t code = (__float_as_uint(um) & 0xFFu) - 1u + (e_f > r_lo ? 1u : 0u) + (e_f > r_hi ? 1u : 0u);
                         const int col = k * 256 + lane * 8 + i;
                         if (col >= cols) code = 0;
                         if (C == 8) { if (i < 4) w0 |= code << (8 * i); else w1 |= code << (8 * (i - 4)); }
